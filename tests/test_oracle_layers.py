@@ -1,0 +1,184 @@
+"""Pins for the oracle's layer arithmetic and its frame-by-frame cache semantics (Section 5)."""
+import numpy as np
+import pytest
+import torch
+import torch.nn.functional as F
+
+from oracle import deepcache_oracle as orc
+from paper_1712_01670_b200.synth import configs, nets
+
+
+def rng(seed):
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def conv_layer(hi, wi, cin, cout, k, s, p, relu=1):
+    return dict(kind=orc.KIND_CONV, kh=k, kw=k, sh=s, sw=s, ph=p, pw=p, cin=cin, cout=cout, relu=relu,
+                in0=-1, in1=-1, out_h=(hi + 2 * p - k) // s + 1, out_w=(wi + 2 * p - k) // s + 1)
+
+
+@pytest.mark.parametrize("hi,wi,cin,cout,k,s,p,relu", [
+    (13, 17, 3, 5, 3, 1, 1, 1), (23, 19, 4, 6, 11, 4, 0, 0), (16, 16, 8, 4, 5, 1, 2, 1),
+    (15, 14, 6, 7, 1, 2, 0, 0), (20, 21, 3, 4, 7, 2, 3, 1), (9, 9, 2, 3, 3, 2, 1, 0)])
+def test_conv_equals_torch_float64(hi, wi, cin, cout, k, s, p, relu):
+    g = rng(hi * 100 + k)
+    x = g.normal(size=(hi, wi, cin))
+    w = g.normal(size=(cout, k, k, cin))
+    b = g.normal(size=cout)
+    L = conv_layer(hi, wi, cin, cout, k, s, p, relu)
+    out, reused = orc.conv_reuse(x, L, w, b, orc.QUANT_NONE)
+    ref = F.conv2d(torch.from_numpy(x).permute(2, 0, 1)[None], torch.from_numpy(w).permute(0, 3, 1, 2),
+                   torch.from_numpy(b), stride=s, padding=p)
+    if relu:
+        ref = ref.clamp_min(0)
+    ref = ref[0].permute(1, 2, 0).numpy()
+    assert out.shape == ref.shape
+    assert np.abs(out - ref).max() < 1e-12
+    assert not reused.any()
+
+
+@pytest.mark.parametrize("k,s,p", [(2, 2, 0), (3, 2, 0), (3, 2, 1)])
+def test_maxpool_equals_torch(k, s, p):
+    g = rng(k + s)
+    x = g.normal(size=(27, 23, 5))
+    L = dict(kind=orc.KIND_MAXPOOL, kh=k, kw=k, sh=s, sw=s, ph=p, pw=p, cin=5, cout=5, relu=0, in0=-1, in1=-1,
+             out_h=(27 + 2 * p - k) // s + 1, out_w=(23 + 2 * p - k) // s + 1)
+    ref = F.max_pool2d(torch.from_numpy(x).permute(2, 0, 1)[None], k, s, p)[0].permute(1, 2, 0).numpy()
+    assert np.array_equal(orc.maxpool(x, L), ref)
+
+
+@pytest.mark.parametrize("h,w,ho,wo", [(108, 192, 22, 22), (50, 37, 7, 9), (64, 64, 64, 64), (30, 30, 15, 10)])
+def test_resize_area_equals_adaptive_avg_pool(h, w, ho, wo):
+    # adaptive average pooling uses the same spans: [floor(o n/no), ceil((o+1) n/no))
+    f = rng(h).integers(0, 256, size=(h, w, 3), dtype=np.uint8)
+    ref = F.adaptive_avg_pool2d(torch.from_numpy(f.astype(np.float64) / 255.0).permute(2, 0, 1)[None], (ho, wo))
+    ref = ref[0].permute(1, 2, 0).numpy()
+    assert np.abs(orc.resize_area(f, ho, wo, orc.QUANT_NONE) - ref).max() < 1e-14
+
+
+def test_bf16_rounding_equals_torch():
+    g = rng(1)
+    v = np.concatenate([g.normal(size=2000) * 10.0 ** g.integers(-6, 6, size=2000),
+                        [0.0, 1.0, -1.0, 1.00390625, 1.01171875, 255.5, 3.0e-5, 65504.0]])
+    # exact ties: 1 + 2^-8 is halfway between 1 and 1 + 2^-7 -> even (1.0); 1 + 3*2^-8 -> 1 + 2^-6
+    got = orc.quant_array(v, orc.QUANT_BF16)
+    ref = torch.from_numpy(v).to(torch.float64).to(torch.bfloat16).to(torch.float64).numpy()
+    # torch converts double -> float -> bf16; restrict to values where the float step is exact
+    exact = v.astype(np.float32).astype(np.float64) == v
+    assert np.array_equal(got[exact], ref[exact])
+    assert orc.quant_array(np.array([1.00390625]), 1)[0] == 1.0
+    assert orc.quant_array(np.array([1.01171875]), 1)[0] == 1.015625
+    rel = np.abs(got - v) / np.maximum(np.abs(v), 1e-300)
+    assert rel.max() <= 2.0 ** -8
+    assert np.array_equal(orc.quant_array(got, 1), got)                 # idempotent
+
+
+def test_input_map_is_pixel_over_255():
+    f = np.arange(256, dtype=np.uint8).reshape(16, 16, 1).repeat(3, 2)
+    assert np.array_equal(orc.input_map(f, orc.QUANT_NONE), f.astype(np.float64) / 255.0)
+    q = orc.input_map(f, orc.QUANT_BF16)
+    ref = torch.from_numpy(f.astype(np.float32) / np.float32(255.0)).to(torch.bfloat16).to(torch.float64).numpy()
+    assert np.abs(q - ref).max() <= 2.0 ** -8
+
+
+def test_reused_pixels_are_cached_pixels_shifted():
+    g = rng(6)
+    hi, wi = 20, 24
+    L = conv_layer(hi, wi, 3, 4, 3, 1, 1)
+    x = g.normal(size=(hi, wi, 3))
+    w = g.normal(size=(4, 3, 3, 3))
+    b = g.normal(size=4)
+    prev = g.normal(size=(hi, wi, 4))
+    regions = np.zeros(3, orc.REGION_DTYPE)
+    regions[0] = (2, 3, 6, 5, 4, 1)
+    regions[1] = (0, 0, 0, 0, 0, 0)                      # vanished slot: ignored
+    regions[2] = (12, 10, 10, 9, 11, 11)
+    out, reused = orc.conv_reuse(x, L, w, b, orc.QUANT_NONE, prev, regions)
+    full, _ = orc.conv_reuse(x, L, w, b, orc.QUANT_NONE)
+    expect_mask = np.zeros((hi, wi), bool)
+    for r in regions:
+        expect_mask[r["y"]:r["y"] + r["h"], r["x"]:r["x"] + r["w"]] = True
+        d = out[r["y"]:r["y"] + r["h"], r["x"]:r["x"] + r["w"]]
+        s = prev[r["sy"]:r["sy"] + r["h"], r["sx"]:r["sx"] + r["w"]]
+        assert np.array_equal(d, s)                      # bit-equal copies of the cached values
+    assert np.array_equal(reused.astype(bool), expect_mask)
+    assert np.array_equal(out[~expect_mask], full[~expect_mask])      # everything else is fresh
+
+
+def make_cache(w, **kw):
+    ws, bs = w.weights()
+    quant = orc.QUANT_BF16 if w.dtype == configs.DTYPE_BF16 else orc.QUANT_NONE
+    args = dict(block=w.block, search_range=w.range, search_kind=w.search, psnr_db=w.psnr_db,
+                expire_n=w.expire_n, quant=quant)
+    args.update(kw)
+    return orc.OracleCache(w.width, w.height, w.layers, ws, bs, **args)
+
+
+def test_identical_frames_reuse_the_cached_output():
+    w = configs.WORKLOADS[2]()
+    w.layers = nets.small_cnn(96, 80)
+    w.width, w.height = 80, 96
+    f = w.streams(1, 2).frame(0)[0][:96, :80]
+    oc = make_cache(w)
+    a = oc.infer_frame(f)
+    b = oc.infer_frame(f)
+    assert a["refreshed"] and not b["refreshed"]
+    assert b["match"]["M"] == (0, 0) and b["match"]["matched"].all()
+    for i, l in enumerate(w.layers):
+        assert np.array_equal(a["maps"][i], b["maps"][i])
+        if l["kind"] == orc.KIND_CONV:
+            # everything but the border ring that touches padding was copied
+            ring = i + 1 if i < 2 else None
+            assert b["reused"][i][8:-8, 8:-8].all()
+    assert np.array_equal(a["out"], b["out"])
+
+
+def test_all_dirty_equals_full_inference_and_expiry():
+    w = configs.WORKLOADS[2]()
+    w.layers = nets.small_cnn(64, 64)
+    w.width = w.height = 64
+    sb = w.streams(1, 8)
+    frames = [sb.frame(i)[0][:64, :64] for i in range(8)]
+    cached = make_cache(w, expire_n=3)
+    plain = make_cache(w, use_cache=False)
+    noise = rng(1).integers(0, 256, size=(64, 64, 3), dtype=np.uint8)
+    for i, f in enumerate(frames):
+        if i == 4:
+            f = noise                                   # unrelated frame: nothing can match
+        a, b = cached.infer_frame(f), plain.infer_frame(f)
+        assert b["refreshed"]
+        if i % 3 == 0:
+            # cache expiry: every N-th frame is a plain full inference
+            assert a["refreshed"] and np.array_equal(a["out"], b["out"])
+        elif i == 4:
+            assert not a["refreshed"] and a["match"]["K"] == 0 and len(a["match"]["regions"]) == 0
+            assert np.array_equal(a["out"], b["out"])    # all dirty == full fresh inference
+        elif i == 5:
+            assert not a["refreshed"] and len(a["match"]["regions"]) == 0   # its key is the noise frame
+        else:
+            assert not a["refreshed"]
+            assert any(r is not None and r.any() for r in a["reused"])
+
+
+def test_workload_1_end_to_end_reuse():
+    w = configs.WORKLOADS[1]()
+    sp = w.streams()
+    oc = make_cache(w)
+    a = oc.infer_frame(sp.frame(0)[0])
+    b = oc.infer_frame(sp.frame(1)[0])
+    regs = b["regions"][0]
+    assert b["match"]["M"] == (-3, 2)
+    mask = b["reused"][0].astype(bool)
+    assert 0.3 < mask.mean() < 0.9
+    for r in regs:
+        if r["w"] == 0:
+            continue
+        assert r["sx"] - r["x"] == -3 and r["sy"] - r["y"] == 2
+        d = b["out"][r["y"]:r["y"] + r["h"], r["x"]:r["x"] + r["w"]]
+        s = a["out"][r["sy"]:r["sy"] + r["h"], r["sx"]:r["sx"] + r["w"]]
+        assert np.array_equal(d, s)
+    fresh = make_cache(w, use_cache=False).infer_frame(sp.frame(1)[0])["out"]
+    assert np.array_equal(b["out"][~mask], fresh[~mask])
+    # reused values are close to, but not the same as, fresh ones (sigma = 2 pixel noise)
+    diff = np.abs(b["out"][mask] - fresh[mask])
+    assert 0 < diff.max() < 0.2
