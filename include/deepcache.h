@@ -1,0 +1,196 @@
+/*
+ * deepcache.h -- C ABI of the DeepCache hot path for NVIDIA B200 (sm_100a).
+ *
+ * DeepCache (arXiv 1712.01670) speeds up CNN inference on video by reusing,
+ * per convolution layer, the previous frame's outputs wherever the new frame
+ * matches the previous one.  This library implements the per-frame path:
+ *
+ *   Section 4  image block matching     dc_match_blocks
+ *   Section 5  region propagation       dc_propagate_regions   (Table 2)
+ *   Section 5  reuse inside convolution dc_conv_partial        (c_forward of Section 6)
+ *   Sections 3, 5  the whole frame      dc_infer_frame         (with cache expiry)
+ *
+ * General rules
+ *   - Every function returns DC_OK (0) or a negative dc_status; nothing throws
+ *     or aborts across this boundary.  dc_strerror names a status.
+ *   - "_dev" pointers are CUDA device memory owned by the caller; they must stay
+ *     valid until the cache's stream has passed the call.  "_host" pointers are
+ *     ordinary host memory.
+ *   - All work is enqueued on the CUDA stream given to dc_cache_create and is
+ *     asynchronous unless stated otherwise.
+ *   - Frames are uint8, interleaved HWC with 3 channels; n_streams frames are
+ *     stacked, stream s starting at frame + s * height * pitch_bytes.
+ *   - Feature maps are NHWC, N = n_streams, element type float (DC_FP32) or
+ *     bfloat16 (DC_BF16).  Weights are given as float32 [cout][kh][kw][cin] and
+ *     are converted by the library; biases stay float32.
+ *   - A motion vector (dx, dy) points from a block of the current frame to its
+ *     match in the previous frame: previous = current + (dx, dy)
+ *     (Section 4, Step 2: (x'_i - x_i, y'_i - y_i)).
+ *   - Region lists are slot-preserving: slot i of every layer descends from
+ *     matcher rectangle i; a region that has eroded away is all zeros.
+ */
+#ifndef DEEPCACHE_H
+#define DEEPCACHE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DC_MAX_LAYERS 128
+
+typedef enum {
+    DC_OK = 0,
+    DC_ERR_ARG = -1,       /* null or inconsistent argument */
+    DC_ERR_CONFIG = -2,    /* unsupported configuration or layer table */
+    DC_ERR_ALLOC = -3,     /* device or host allocation failed */
+    DC_ERR_CUDA = -4,      /* a CUDA call failed */
+    DC_ERR_OVERFLOW = -5,  /* more rectangles than max_regions (device status word) */
+    DC_ERR_TIMEOUT = -6,   /* a bounded device-side wait ran out (device status word) */
+    DC_ERR_STATE = -7      /* call not valid now (e.g. no cached frame yet) */
+} dc_status;
+
+/* A reusable rectangle (Section 3: "(x, y, w, h) -> (x', y', w, h)").
+ * (x, y, w, h): rectangle in the current frame or map; (sx, sy): origin of the
+ * same-sized rectangle in the previous frame or cached map. */
+typedef struct { int32_t x, y, w, h, sx, sy; } dc_region;
+
+typedef enum {
+    DC_CONV = 0, DC_MAXPOOL = 1, DC_RELU = 2, DC_ADD = 3, DC_CONCAT = 4,
+    DC_RESIZE_AREA = 5, DC_LRN = 6, DC_FC = 7
+} dc_layer_kind;
+
+/* One layer.  in0 / in1: index of the producing layer, -1 = the input frame
+ * (in1 is used by DC_ADD / DC_CONCAT only).  out_h, out_w: output size.
+ * DC_CONV: kh x kw kernel, stride, padding, cin -> cout, optional fused ReLU.
+ * DC_MAXPOOL: floor mode, padded taps ignored.  DC_ADD: element-wise, optional ReLU.
+ * DC_RESIZE_AREA: box average of the input frame (in0 must be -1) to out_h x out_w.
+ * DC_LRN (radius = ph), DC_CONCAT, DC_FC are known to region propagation only;
+ * a cache containing them cannot run dc_infer_frame. */
+typedef struct {
+    int32_t kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w;
+} dc_layer_desc;
+
+typedef enum { DC_SEARCH_EXHAUSTIVE = 0, DC_SEARCH_DIAMOND = 1 } dc_search_kind;
+typedef enum { DC_FP32 = 0, DC_BF16 = 1 } dc_dtype;
+
+/* The developer-facing knobs of Section 6 (threshold, block size, expiry) plus shapes. */
+typedef struct {
+    int32_t width, height, channels;   /* frame size in pixels; channels must be 3 */
+    int32_t n_streams;                 /* independent video streams processed per call */
+    int32_t block;                     /* block edge in pixels (Section 3 default 10), 4..32 */
+    int32_t range;                     /* search range R: |dx|, |dy| <= R, 0..64 */
+    int32_t search;                    /* dc_search_kind */
+    int32_t skip_k;                    /* reserved, must be 1 */
+    int32_t expire_n;                  /* full fresh frame every expire_n frames (default 10) */
+    double  psnr_db;                   /* similarity threshold T in dB (default 20) */
+    int32_t dtype;                     /* dc_dtype of maps and arithmetic inputs */
+    int32_t max_regions;               /* rectangles per stream; 0 = worst case of the grid */
+} dc_config;
+
+/* Per-stream outcome of one dc_infer_frame. */
+typedef struct {
+    int32_t refreshed;                 /* 1: full fresh frame (expiry or empty cache) */
+    int32_t n_blocks, k_passed;        /* grid size; blocks whose best match passed (Step 3's K) */
+    int32_t mvx, mvy;                  /* global motion (Mx, My) */
+    int32_t n_matched, n_regions;      /* Step 4 matches; Step 5 rectangles */
+    float   reuse_ratio[DC_MAX_LAYERS];/* per layer: reused / all output pixels (conv layers) */
+} dc_frame_stats;
+
+typedef struct dc_cache dc_cache;      /* opaque, owned by the library */
+
+/* Builds a cache for one network and one frame geometry: validates, allocates the
+ * key-frame buffer, two maps per convolution (current / cached), one per other layer,
+ * region tables and tile lists, and converts the weights.  weights_dev[i] / bias_dev[i]
+ * are float32 device arrays for DC_CONV layers and ignored (may be NULL) otherwise; they
+ * are read during this call only.  cuda_stream is a cudaStream_t (NULL = default stream).
+ * Synchronous.  Errors: DC_ERR_ARG, DC_ERR_CONFIG, DC_ERR_ALLOC, DC_ERR_CUDA. */
+int dc_cache_create(const dc_config* cfg, const dc_layer_desc* layers, int n_layers,
+                    const void* const* weights_dev, const void* const* bias_dev,
+                    void* cuda_stream, dc_cache** out);
+
+/* Frees everything the cache owns.  Synchronous. */
+int dc_cache_destroy(dc_cache* cache);
+
+/* Empties the cache: the next dc_infer_frame is a full fresh frame (Section 5, expiry). */
+int dc_cache_reset(dc_cache* cache);
+
+/* Device bytes held by the cache (cf. the memory overhead of Section 7.5). */
+int dc_cache_bytes(const dc_cache* cache, size_t* bytes);
+
+/* Stores frame_dev as the cached previous frame (the cache key of Section 3) without
+ * running the network.  Lets dc_match_blocks be used on its own. */
+int dc_cache_set_key(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes);
+
+/* Section 4, Steps 1-5, current frame against the cached previous frame.
+ *   block_mv_dev   int16  [S][Gy][Gx][2]  best (dx, dy) per block (Step 2)
+ *   block_sse_dev  uint32 [S][Gy][Gx]     its sum of squared differences over 3 channels
+ *   matched_dev    uint8  [S][Gy][Gx]     1 = properly matched at the global motion (Step 4)
+ *   global_mv_dev  int32  [S][3]          Mx, My, K (Step 3)
+ *   regions_dev    dc_region [S][max_regions], n_regions_dev int32 [S]   (Step 5)
+ * Gx = ceil(width / block), Gy = ceil(height / block); edge blocks are clipped.
+ * Any output pointer may be NULL (skipped).  Does not change the cache.
+ * Errors: DC_ERR_ARG, DC_ERR_STATE (no cached frame), DC_ERR_CUDA. */
+int dc_match_blocks(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes,
+                    int16_t* block_mv_dev, uint32_t* block_sse_dev, uint8_t* matched_dev,
+                    int32_t* global_mv_dev, dc_region* regions_dev, int32_t* n_regions_dev);
+
+/* Section 5 "Propagation" (Table 2): carries frame-level rectangles through layers
+ * 0 .. layer_end-1 and returns those of layers layer_begin .. layer_end-1.
+ *   in_dev   dc_region [S][max_regions], n_in_dev int32 [S]: rectangles on the input frame
+ *   out_dev  dc_region [layer_end-layer_begin][S][max_regions]
+ *   n_out_dev int32 [layer_end-layer_begin][S] (slot count, equal to n_in; may be NULL)
+ * Errors: DC_ERR_ARG, DC_ERR_CUDA. */
+int dc_propagate_regions(dc_cache* cache, const dc_region* in_dev, const int32_t* n_in_dev,
+                         int layer_begin, int layer_end, dc_region* out_dev, int32_t* n_out_dev);
+
+/* Section 5 "Reuse" for convolution layer `layer` (c_forward(top, bottom, c_blob, c_regions)
+ * of Section 6): output pixels inside a rectangle are copied from prev_out_dev at the mapped
+ * position, all others are convolved (+bias, +ReLU) from in_map_dev.
+ *   in_map_dev    [S][Hi][Wi][cin]   complete input map (bottom blob)
+ *   prev_out_dev  [S][Ho][Wo][cout]  this layer's output for the previous frame (c_blob)
+ *   regions_dev   dc_region [S][max_regions], n_regions_dev int32 [S]: rectangles in output
+ *                 coordinates (c_regions); both NULL = plain full convolution
+ *   out_map_dev   [S][Ho][Wo][cout]  (top blob); must not alias prev_out_dev
+ * Errors: DC_ERR_ARG, DC_ERR_CONFIG (not a convolution), DC_ERR_CUDA. */
+int dc_conv_partial(dc_cache* cache, int layer, const void* in_map_dev, const void* prev_out_dev,
+                    const dc_region* regions_dev, const int32_t* n_regions_dev, void* out_map_dev);
+
+/* One frame per stream through the whole path: expiry check, matching, propagation,
+ * every layer (convolutions partially, the rest in full), then the frame becomes the new
+ * key and the convolution outputs the new cached values (Sections 3 and 5).
+ *   out_map_dev     last layer's map, [S][Ho][Wo][cout]; may be NULL
+ *   stats_host      dc_frame_stats [S] or NULL.  Non-NULL makes the call synchronous.
+ * Errors: DC_ERR_ARG, DC_ERR_STATE (layer table not executable), DC_ERR_CUDA. */
+int dc_infer_frame(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes,
+                   void* out_map_dev, dc_frame_stats* stats_host);
+
+/* Same as dc_infer_frame with HOST buffers: copies the frames to the device, runs the
+ * path, copies the last map back, and waits.  frame_host should be pinned memory for
+ * full copy speed.  out_map_host may be NULL. */
+int dc_infer_frame_host(dc_cache* cache, const uint8_t* frame_host, size_t pitch_bytes,
+                        void* out_map_host, dc_frame_stats* stats_host);
+
+/* Device address and size of the library-owned map of `layer` as of the last
+ * dc_infer_frame (for inspection; valid until the next call on this cache). */
+int dc_cache_layer_map(dc_cache* cache, int layer, void** map_dev, size_t* bytes);
+
+/* Device address of the rectangles dc_infer_frame / dc_propagate_regions last computed for
+ * `layer` ([S][max_regions]) and of their per-stream count ([S]). */
+int dc_cache_layer_regions(dc_cache* cache, int layer, dc_region** regions_dev, int32_t** n_dev);
+
+/* Waits for the stream and returns the device status word: DC_OK, DC_ERR_OVERFLOW or
+ * DC_ERR_TIMEOUT as recorded by a kernel since the last reset.  Synchronous. */
+int dc_get_status(dc_cache* cache, int32_t* status_host);
+
+/* Kernels of this library launched on this cache since creation (for reporting). */
+int dc_cache_launches(const dc_cache* cache, int64_t* launches);
+
+const char* dc_strerror(int status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DEEPCACHE_H */

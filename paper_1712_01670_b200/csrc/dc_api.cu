@@ -1,0 +1,475 @@
+// C ABI of libdeepcache: cache life cycle and the per-frame driver (declared in deepcache.h).
+// Host code only enqueues work; region and tile counts stay on the device.
+#include <math.h>
+#include <stdio.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "dc_common.cuh"
+
+static thread_local char g_last_cuda_error[256];
+
+void dc_note_cuda_error(cudaError_t e, const char* file, int line)
+{
+    snprintf(g_last_cuda_error, sizeof(g_last_cuda_error), "%s at %s:%d", cudaGetErrorString(e), file, line);
+    if (getenv("DC_VERBOSE")) fprintf(stderr, "libdeepcache: CUDA error: %s\n", g_last_cuda_error);
+}
+
+namespace {
+
+// nearest bfloat16 (ties to even) of a double, as its 16 bit pattern
+uint16_t bf16_bits_from_double(double v)
+{
+    if (v == 0.0) return 0;
+    int e = ilogb(v);
+    if (e < -126) e = -126;
+    double q = ldexp(nearbyint(ldexp(v, 7 - e)), e - 7);
+    float f = (float)q;                       // exact: q has at most 8 significant bits
+    uint32_t u; memcpy(&u, &f, 4);
+    return (uint16_t)(u >> 16);
+}
+
+template <typename T>
+int dev_alloc(dc_cache* c, T** p, size_t count)
+{
+    size_t bytes = count * sizeof(T);
+    if (bytes == 0) bytes = sizeof(T);
+    if (cudaMalloc((void**)p, bytes) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
+    c->bytes += bytes;
+    return DC_OK;
+}
+#define DC_TRY(expr) do { int rc__ = (expr); if (rc__ != DC_OK) return rc__; } while (0)
+
+bool kind_executable(int k) { return k == DC_CONV || k == DC_MAXPOOL || k == DC_RELU || k == DC_ADD || k == DC_RESIZE_AREA; }
+
+int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
+{
+    if (cfg->channels != 3 || cfg->width < 1 || cfg->height < 1 || cfg->n_streams < 1) return DC_ERR_CONFIG;
+    if (cfg->block < 4 || cfg->block > 32 || cfg->range < 0 || cfg->range > 64) return DC_ERR_CONFIG;
+    if (cfg->search != DC_SEARCH_EXHAUSTIVE && cfg->search != DC_SEARCH_DIAMOND) return DC_ERR_CONFIG;
+    if (cfg->skip_k != 1 || cfg->expire_n < 1 || cfg->max_regions < 0) return DC_ERR_CONFIG;
+    if (cfg->dtype != DC_FP32 && cfg->dtype != DC_BF16) return DC_ERR_CONFIG;
+    if (!(cfg->psnr_db > 0.0) || !(cfg->psnr_db < 200.0)) return DC_ERR_CONFIG;
+    if (n < 1 || n > DC_MAX_LAYERS) return DC_ERR_CONFIG;
+    const int elt = cfg->dtype == DC_BF16 ? 2 : 4;
+    for (int i = 0; i < n; ++i) {
+        const dc_layer_desc& L = layers[i];
+        if (L.kind < DC_CONV || L.kind > DC_FC) return DC_ERR_CONFIG;
+        if (L.in0 < -1 || L.in0 >= i) return DC_ERR_CONFIG;
+        int ih = L.in0 < 0 ? cfg->height : layers[L.in0].out_h;
+        int iw = L.in0 < 0 ? cfg->width : layers[L.in0].out_w;
+        int ic = L.in0 < 0 ? 3 : layers[L.in0].cout;
+        if (L.out_h < 1 || L.out_w < 1 || L.cout < 1) return DC_ERR_CONFIG;
+        switch (L.kind) {
+        case DC_CONV: case DC_MAXPOOL:
+            if (L.kh < 1 || L.kw < 1 || L.sh < 1 || L.sw < 1 || L.ph < 0 || L.pw < 0) return DC_ERR_CONFIG;
+            if (L.ph >= L.kh || L.pw >= L.kw) return DC_ERR_CONFIG;
+            if ((ih + 2 * L.ph - L.kh) / L.sh + 1 != L.out_h || (iw + 2 * L.pw - L.kw) / L.sw + 1 != L.out_w) return DC_ERR_CONFIG;
+            if (ih + 2 * L.ph < L.kh || iw + 2 * L.pw < L.kw) return DC_ERR_CONFIG;
+            if (L.cin != ic) return DC_ERR_CONFIG;
+            if (L.kind == DC_MAXPOOL && L.cout != ic) return DC_ERR_CONFIG;
+            if (L.kind == DC_CONV && (L.cout * elt) % 16 != 0) return DC_ERR_CONFIG;   // 16-byte pixel vectors
+            break;
+        case DC_ADD: case DC_CONCAT: {
+            if (L.in1 < -1 || L.in1 >= i) return DC_ERR_CONFIG;
+            int jh = L.in1 < 0 ? cfg->height : layers[L.in1].out_h, jw = L.in1 < 0 ? cfg->width : layers[L.in1].out_w;
+            int jc = L.in1 < 0 ? 3 : layers[L.in1].cout;
+            if (jh != ih || jw != iw || L.out_h != ih || L.out_w != iw) return DC_ERR_CONFIG;
+            if (L.kind == DC_ADD && (jc != ic || L.cout != ic)) return DC_ERR_CONFIG;
+            if (L.kind == DC_CONCAT && L.cout != ic + jc) return DC_ERR_CONFIG;
+            break;
+        }
+        case DC_RESIZE_AREA:
+            if (L.in0 != -1 || L.cout != 3 || L.out_h > ih || L.out_w > iw) return DC_ERR_CONFIG;
+            break;
+        case DC_LRN:
+            if (L.ph < 0 || L.out_h != ih || L.out_w != iw || L.cout != ic) return DC_ERR_CONFIG;
+            break;
+        case DC_RELU:
+            if (L.out_h != ih || L.out_w != iw || L.cout != ic) return DC_ERR_CONFIG;
+            break;
+        default: break;
+        }
+    }
+    return DC_OK;
+}
+
+int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_dev, const void* const* bias_dev)
+{
+    const dc_config& cfg = c->cfg;
+    const int S = c->S, n = c->n_layers;
+    // cached key frames: own pitch (16-byte multiple, at least 16 spare bytes per row and a spare
+    // tail) so the matcher may fetch whole aligned words around any candidate
+    c->key_pitch = ((size_t)cfg.width * 3 + 16 + 15) / 16 * 16;
+    DC_TRY(dev_alloc(c, &c->key, c->key_pitch * cfg.height * S + 256));
+    DC_CUDA(cudaMemsetAsync(c->key, 0, c->key_pitch * cfg.height * S + 256, c->stream));
+    const size_t nblk = (size_t)S * c->Gx * c->Gy;
+    DC_TRY(dev_alloc(c, &c->blk_mv, nblk * 2));
+    DC_TRY(dev_alloc(c, &c->blk_sse, nblk));
+    DC_TRY(dev_alloc(c, &c->matched, nblk));
+    DC_TRY(dev_alloc(c, &c->mv_acc, (size_t)S * 4));
+    DC_TRY(dev_alloc(c, &c->gmv, (size_t)S * 3));
+    DC_TRY(dev_alloc(c, &c->regions0, (size_t)S * c->max_regions));
+    DC_TRY(dev_alloc(c, &c->n_regions, (size_t)S));
+    DC_TRY(dev_alloc(c, &c->table, (size_t)n * S * c->max_regions));
+    DC_TRY(dev_alloc(c, &c->layers_dev, (size_t)n));
+    DC_TRY(dev_alloc(c, &c->in_hw_dev, (size_t)n * 2));
+    DC_TRY(dev_alloc(c, &c->dirty_count, (size_t)n));
+    DC_TRY(dev_alloc(c, &c->all_count, (size_t)n));
+    DC_TRY(dev_alloc(c, &c->reuse_px, (size_t)n * S));
+    DC_TRY(dev_alloc(c, &c->status, (size_t)1));
+    DC_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int32_t), c->stream));
+    DC_CUDA(cudaMemsetAsync(c->n_regions, 0, sizeof(int32_t) * S, c->stream));
+    DC_CUDA(cudaMemsetAsync(c->table, 0, sizeof(dc_region) * n * S * c->max_regions, c->stream));
+    DC_CUDA(cudaMemcpyAsync(c->layers_dev, layers, sizeof(dc_layer_desc) * n, cudaMemcpyHostToDevice, c->stream));
+
+    // PSNR > T as an integer bound on the SSE, for the four block shapes of a clipped grid
+    for (int i = 0; i < 4; ++i) {
+        int bw = (i & 1) ? cfg.width - (c->Gx - 1) * cfg.block : cfg.block;
+        int bh = (i & 2) ? cfg.height - (c->Gy - 1) * cfg.block : cfg.block;
+        double q = 65025.0 * (double)(bw * bh * 3) / pow(10.0, cfg.psnr_db / 10.0);
+        double lim = ceil(q) - 1.0;
+        c->sse_limit[i] = lim >= 4294967295.0 ? 4294967295u : (uint32_t)lim;
+    }
+    // pixel -> map element table
+    if (cfg.dtype == DC_BF16) {
+        uint16_t lut[256];
+        for (int i = 0; i < 256; ++i) lut[i] = bf16_bits_from_double((double)i / 255.0);
+        DC_TRY(dev_alloc(c, (uint16_t**)&c->pix_lut, (size_t)256));
+        DC_CUDA(cudaMemcpy(c->pix_lut, lut, sizeof(lut), cudaMemcpyHostToDevice));
+    } else {
+        float lut[256];
+        for (int i = 0; i < 256; ++i) lut[i] = (float)((double)i / 255.0);
+        DC_TRY(dev_alloc(c, (float**)&c->pix_lut, (size_t)256));
+        DC_CUDA(cudaMemcpy(c->pix_lut, lut, sizeof(lut), cudaMemcpyHostToDevice));
+    }
+
+    int32_t in_hw[DC_MAX_LAYERS * 2], all_count[DC_MAX_LAYERS];
+    size_t max_tiles = 1;
+    bool need_input_map = false;
+    for (int i = 0; i < n; ++i) {
+        dc_layer_rt& L = c->L[i];
+        L.d = layers[i];
+        L.in_h = L.d.in0 < 0 ? cfg.height : layers[L.d.in0].out_h;
+        L.in_w = L.d.in0 < 0 ? cfg.width : layers[L.d.in0].out_w;
+        in_hw[2 * i] = L.in_h; in_hw[2 * i + 1] = L.in_w;
+        all_count[i] = 0;
+        if (!c->executable) continue;
+        if (L.d.in0 < 0 && L.d.kind != DC_RESIZE_AREA) need_input_map = true;
+        if (L.d.kind == DC_ADD && L.d.in1 < 0) need_input_map = true;
+        L.map_bytes = (size_t)S * L.d.out_h * L.d.out_w * L.d.cout * c->elt;
+        const int copies = L.d.kind == DC_CONV ? 2 : 1;
+        for (int k = 0; k < copies; ++k) {
+            DC_TRY(dev_alloc(c, (uint8_t**)&L.map[k], L.map_bytes));
+            DC_CUDA(cudaMemsetAsync(L.map[k], 0, L.map_bytes, c->stream));
+        }
+        if (L.d.kind == DC_CONV) {
+            L.tiles_x = dc_div_up(L.d.out_w, DC_TILE_W);
+            L.tiles_y = dc_div_up(L.d.out_h, DC_TILE_H);
+            size_t tiles = (size_t)L.tiles_x * L.tiles_y * S;
+            if (tiles > max_tiles) max_tiles = tiles;
+            all_count[i] = (int32_t)tiles;
+            DC_TRY(dev_alloc(c, &L.masks, tiles * 4));
+            DC_TRY(dev_alloc(c, &L.dirty_list, tiles));
+            DC_TRY(dev_alloc(c, &L.all_list, tiles));
+            int32_t* iota = (int32_t*)malloc(sizeof(int32_t) * tiles);
+            if (!iota) return DC_ERR_ALLOC;
+            for (size_t t = 0; t < tiles; ++t) iota[t] = (int32_t)t;
+            cudaError_t e = cudaMemcpy(L.all_list, iota, sizeof(int32_t) * tiles, cudaMemcpyHostToDevice);
+            free(iota);
+            DC_CUDA(e);
+            if (!weights_dev || !bias_dev || !weights_dev[i] || !bias_dev[i]) return DC_ERR_ARG;
+            DC_TRY(dc_pack_weights(c, i, (const float*)weights_dev[i], (const float*)bias_dev[i]));
+        }
+    }
+    DC_CUDA(cudaMemcpyAsync(c->in_hw_dev, in_hw, sizeof(int32_t) * 2 * n, cudaMemcpyHostToDevice, c->stream));
+    DC_CUDA(cudaMemcpyAsync(c->all_count, all_count, sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream));
+    DC_TRY(dev_alloc(c, &c->zero_masks, max_tiles * 4));
+    DC_CUDA(cudaMemsetAsync(c->zero_masks, 0, max_tiles * 4 * sizeof(uint32_t), c->stream));
+    if (need_input_map)
+        DC_TRY(dev_alloc(c, (uint8_t**)&c->input_map, (size_t)S * cfg.height * cfg.width * 3 * c->elt));
+    size_t stat_ints = (size_t)S * (3 + 4 + 1) + (size_t)n * S;
+    if (cudaMallocHost(&c->stats_pinned, stat_ints * sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
+    DC_CUDA(cudaStreamSynchronize(c->stream));      // layers / in_hw / all_count live on this stack frame
+    return DC_OK;
+}
+
+void release(dc_cache* c)
+{
+    cudaFree(c->key); cudaFree(c->staging); cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched);
+    cudaFree(c->mv_acc); cudaFree(c->gmv); cudaFree(c->regions0); cudaFree(c->n_regions); cudaFree(c->table);
+    cudaFree(c->layers_dev); cudaFree(c->in_hw_dev); cudaFree(c->dirty_count); cudaFree(c->all_count);
+    cudaFree(c->reuse_px); cudaFree(c->zero_masks); cudaFree(c->status); cudaFree(c->input_map); cudaFree(c->pix_lut);
+    if (c->stats_pinned) cudaFreeHost(c->stats_pinned);
+    for (int i = 0; i < c->n_layers; ++i) {
+        dc_layer_rt& L = c->L[i];
+        cudaFree(L.map[0]); cudaFree(L.map[1]); cudaFree(L.weight); cudaFree(L.bias); cudaFree(L.weight_packed);
+        cudaFree(L.masks); cudaFree(L.dirty_list); cudaFree(L.all_list);
+    }
+    cudaGetLastError();
+    delete c;
+}
+
+const void* layer_input(dc_cache* c, int idx)
+{
+    if (idx < 0) return c->input_map;
+    dc_layer_rt& P = c->L[idx];
+    return P.map[P.d.kind == DC_CONV ? P.cur : 0];
+}
+
+int fill_stats(dc_cache* c, bool refreshed, dc_frame_stats* stats)
+{
+    const int S = c->S, n = c->n_layers;
+    int32_t* h = (int32_t*)c->stats_pinned;
+    int32_t* h_gmv = h; int32_t* h_acc = h + 3 * S; int32_t* h_nreg = h + 7 * S; int32_t* h_reuse = h + 8 * S;
+    if (!refreshed) {
+        DC_CUDA(cudaMemcpyAsync(h_gmv, c->gmv, sizeof(int32_t) * 3 * S, cudaMemcpyDeviceToHost, c->stream));
+        DC_CUDA(cudaMemcpyAsync(h_acc, c->mv_acc, sizeof(int32_t) * 4 * S, cudaMemcpyDeviceToHost, c->stream));
+        DC_CUDA(cudaMemcpyAsync(h_nreg, c->n_regions, sizeof(int32_t) * S, cudaMemcpyDeviceToHost, c->stream));
+        DC_CUDA(cudaMemcpyAsync(h_reuse, c->reuse_px, sizeof(int32_t) * n * S, cudaMemcpyDeviceToHost, c->stream));
+    }
+    DC_CUDA(cudaStreamSynchronize(c->stream));
+    for (int s = 0; s < S; ++s) {
+        dc_frame_stats& st = stats[s];
+        memset(&st, 0, sizeof(st));
+        st.refreshed = refreshed ? 1 : 0;
+        st.n_blocks = c->Gx * c->Gy;
+        if (refreshed) continue;
+        st.mvx = h_gmv[3 * s]; st.mvy = h_gmv[3 * s + 1]; st.k_passed = h_gmv[3 * s + 2];
+        st.n_matched = h_acc[4 * s + 3]; st.n_regions = h_nreg[s];
+        for (int l = 0; l < n; ++l)
+            if (c->L[l].d.kind == DC_CONV)
+                st.reuse_ratio[l] = (float)h_reuse[(size_t)l * S + s] / (float)(c->L[l].d.out_h * c->L[l].d.out_w);
+    }
+    return DC_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int dc_cache_create(const dc_config* cfg, const dc_layer_desc* layers, int n_layers,
+                    const void* const* weights_dev, const void* const* bias_dev, void* cuda_stream, dc_cache** out)
+{
+    if (!cfg || !layers || !out) return DC_ERR_ARG;
+    *out = nullptr;
+    int rc = validate(cfg, layers, n_layers);
+    if (rc != DC_OK) return rc;
+    dc_cache* c = new (std::nothrow) dc_cache();
+    if (!c) return DC_ERR_ALLOC;
+    memset((void*)c, 0, sizeof(*c));
+    c->cfg = *cfg; c->n_layers = n_layers; c->stream = (cudaStream_t)cuda_stream;
+    c->S = cfg->n_streams;
+    c->Gx = dc_div_up(cfg->width, cfg->block); c->Gy = dc_div_up(cfg->height, cfg->block);
+    // Step 5 never yields more than ceil(Gx / 2) * Gy rectangles (runs in a row are separated)
+    c->max_regions = cfg->max_regions > 0 ? cfg->max_regions : dc_div_up(c->Gx, 2) * c->Gy;
+    c->elt = cfg->dtype == DC_BF16 ? 2 : 4;
+    c->executable = true;
+    for (int i = 0; i < n_layers; ++i) if (!kind_executable(layers[i].kind)) c->executable = false;
+    rc = build(c, layers, weights_dev, bias_dev);
+    if (rc != DC_OK) { release(c); return rc; }
+    *out = c;
+    return DC_OK;
+}
+
+int dc_cache_destroy(dc_cache* c)
+{
+    if (!c) return DC_ERR_ARG;
+    cudaStreamSynchronize(c->stream);
+    release(c);
+    return DC_OK;
+}
+
+int dc_cache_reset(dc_cache* c)
+{
+    if (!c) return DC_ERR_ARG;
+    c->key_valid = false; c->frame_idx = 0;
+    DC_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int32_t), c->stream));
+    return DC_OK;
+}
+
+int dc_cache_bytes(const dc_cache* c, size_t* bytes)
+{
+    if (!c || !bytes) return DC_ERR_ARG;
+    *bytes = c->bytes;
+    return DC_OK;
+}
+
+int dc_cache_launches(const dc_cache* c, int64_t* launches)
+{
+    if (!c || !launches) return DC_ERR_ARG;
+    *launches = c->launches;
+    return DC_OK;
+}
+
+int dc_cache_set_key(dc_cache* c, const uint8_t* frame_dev, size_t pitch)
+{
+    if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
+    DC_CUDA(cudaMemcpy2DAsync(c->key, c->key_pitch, frame_dev, pitch, (size_t)c->cfg.width * 3,
+                              (size_t)c->cfg.height * c->S, cudaMemcpyDeviceToDevice, c->stream));
+    c->key_valid = true;
+    return DC_OK;
+}
+
+int dc_match_blocks(dc_cache* c, const uint8_t* frame_dev, size_t pitch, int16_t* block_mv_dev,
+                    uint32_t* block_sse_dev, uint8_t* matched_dev, int32_t* global_mv_dev,
+                    dc_region* regions_dev, int32_t* n_regions_dev)
+{
+    if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
+    if (!c->key_valid) return DC_ERR_STATE;
+    DC_TRY(dc_launch_match(c, frame_dev, pitch));
+    const size_t nblk = (size_t)c->S * c->Gx * c->Gy;
+    const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
+    if (block_mv_dev) DC_CUDA(cudaMemcpyAsync(block_mv_dev, c->blk_mv, nblk * 2 * sizeof(int16_t), k, c->stream));
+    if (block_sse_dev) DC_CUDA(cudaMemcpyAsync(block_sse_dev, c->blk_sse, nblk * sizeof(uint32_t), k, c->stream));
+    if (matched_dev) DC_CUDA(cudaMemcpyAsync(matched_dev, c->matched, nblk, k, c->stream));
+    if (global_mv_dev) DC_CUDA(cudaMemcpyAsync(global_mv_dev, c->gmv, sizeof(int32_t) * 3 * c->S, k, c->stream));
+    if (regions_dev) DC_CUDA(cudaMemcpyAsync(regions_dev, c->regions0, sizeof(dc_region) * c->S * c->max_regions, k, c->stream));
+    if (n_regions_dev) DC_CUDA(cudaMemcpyAsync(n_regions_dev, c->n_regions, sizeof(int32_t) * c->S, k, c->stream));
+    return DC_OK;
+}
+
+int dc_propagate_regions(dc_cache* c, const dc_region* in_dev, const int32_t* n_in_dev, int layer_begin,
+                         int layer_end, dc_region* out_dev, int32_t* n_out_dev)
+{
+    if (!c || !in_dev || !n_in_dev || !out_dev) return DC_ERR_ARG;
+    if (layer_begin < 0 || layer_end > c->n_layers || layer_begin >= layer_end) return DC_ERR_ARG;
+    const size_t per_layer = (size_t)c->S * c->max_regions;
+    // slots beyond n_in keep whatever an earlier call left: clear the table first
+    DC_CUDA(cudaMemsetAsync(c->table, 0, sizeof(dc_region) * per_layer * layer_end, c->stream));
+    DC_TRY(dc_launch_propagate(c, in_dev, n_in_dev, layer_end));
+    DC_CUDA(cudaMemcpyAsync(out_dev, c->table + per_layer * layer_begin,
+                            sizeof(dc_region) * per_layer * (layer_end - layer_begin), cudaMemcpyDeviceToDevice, c->stream));
+    if (n_out_dev)
+        for (int l = 0; l < layer_end - layer_begin; ++l)
+            DC_CUDA(cudaMemcpyAsync(n_out_dev + (size_t)l * c->S, n_in_dev, sizeof(int32_t) * c->S,
+                                    cudaMemcpyDeviceToDevice, c->stream));
+    return DC_OK;
+}
+
+int dc_conv_partial(dc_cache* c, int layer, const void* in_map_dev, const void* prev_out_dev,
+                    const dc_region* regions_dev, const int32_t* n_regions_dev, void* out_map_dev)
+{
+    if (!c || !in_map_dev || !out_map_dev || layer < 0 || layer >= c->n_layers) return DC_ERR_ARG;
+    if (!c->executable || c->L[layer].d.kind != DC_CONV) return DC_ERR_CONFIG;
+    dc_layer_rt& L = c->L[layer];
+    const int tiles = L.tiles_x * L.tiles_y * c->S;
+    if (regions_dev || n_regions_dev) {
+        if (!regions_dev || !n_regions_dev || !prev_out_dev || prev_out_dev == out_map_dev) return DC_ERR_ARG;
+        DC_CUDA(cudaMemsetAsync(c->dirty_count + layer, 0, sizeof(int32_t), c->stream));
+        DC_CUDA(cudaMemsetAsync(c->reuse_px + (size_t)layer * c->S, 0, sizeof(int32_t) * c->S, c->stream));
+        DC_TRY(dc_launch_classify_copy(c, layer, regions_dev, n_regions_dev, prev_out_dev, out_map_dev));
+        return dc_launch_conv(c, layer, in_map_dev, out_map_dev, L.dirty_list, c->dirty_count + layer, L.masks, tiles);
+    }
+    return dc_launch_conv(c, layer, in_map_dev, out_map_dev, L.all_list, c->all_count + layer, c->zero_masks, tiles);
+}
+
+int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* out_map_dev, dc_frame_stats* stats)
+{
+    if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
+    if (!c->executable) return DC_ERR_STATE;
+    const int n = c->n_layers, S = c->S;
+    // Section 5: the cache is dropped and a whole new frame computed every N frames
+    const bool refresh = !c->key_valid || (c->frame_idx % c->cfg.expire_n) == 0;
+    if (!refresh) {
+        DC_CUDA(cudaMemsetAsync(c->dirty_count, 0, sizeof(int32_t) * n, c->stream));
+        DC_CUDA(cudaMemsetAsync(c->reuse_px, 0, sizeof(int32_t) * n * S, c->stream));
+        DC_TRY(dc_launch_match(c, frame_dev, pitch));
+        DC_TRY(dc_launch_propagate(c, c->regions0, c->n_regions, n));
+    }
+    if (c->input_map) DC_TRY(dc_launch_input_map(c, frame_dev, pitch));
+    const size_t per_layer = (size_t)S * c->max_regions;
+    for (int i = 0; i < n; ++i) {
+        dc_layer_rt& L = c->L[i];
+        const void* in = layer_input(c, L.d.in0);
+        switch (L.d.kind) {
+        case DC_CONV: {
+            const int tiles = L.tiles_x * L.tiles_y * S;
+            void* prev = L.map[L.cur]; void* out = L.map[L.cur ^ 1];
+            if (!refresh) {
+                DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
+                DC_TRY(dc_launch_conv(c, i, in, out, L.dirty_list, c->dirty_count + i, L.masks, tiles));
+            } else {
+                DC_TRY(dc_launch_conv(c, i, in, out, L.all_list, c->all_count + i, c->zero_masks, tiles));
+            }
+            L.cur ^= 1;          // the newest output is next frame's cached value
+            break;
+        }
+        case DC_MAXPOOL: DC_TRY(dc_launch_maxpool(c, i, in)); break;
+        case DC_ADD: DC_TRY(dc_launch_add(c, i, in, layer_input(c, L.d.in1))); break;
+        case DC_RELU: DC_TRY(dc_launch_relu(c, i, in)); break;
+        case DC_RESIZE_AREA: DC_TRY(dc_launch_resize(c, i, frame_dev, pitch)); break;
+        default: return DC_ERR_STATE;
+        }
+    }
+    // the frame becomes the next cache key (Section 3)
+    DC_CUDA(cudaMemcpy2DAsync(c->key, c->key_pitch, frame_dev, pitch, (size_t)c->cfg.width * 3,
+                              (size_t)c->cfg.height * S, cudaMemcpyDeviceToDevice, c->stream));
+    c->key_valid = true;
+    c->frame_idx += 1;
+    if (out_map_dev)
+        DC_CUDA(cudaMemcpyAsync(out_map_dev, layer_input(c, n - 1), c->L[n - 1].map_bytes, cudaMemcpyDeviceToDevice, c->stream));
+    if (stats) return fill_stats(c, refresh, stats);
+    return DC_OK;
+}
+
+int dc_infer_frame_host(dc_cache* c, const uint8_t* frame_host, size_t pitch, void* out_map_host, dc_frame_stats* stats)
+{
+    if (!c || !frame_host || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
+    const size_t bytes = pitch * (size_t)c->cfg.height * c->S;
+    if (!c->staging) {
+        if (cudaMalloc((void**)&c->staging, bytes + 256) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
+        c->bytes += bytes + 256;
+    }
+    DC_CUDA(cudaMemcpyAsync(c->staging, frame_host, bytes, cudaMemcpyHostToDevice, c->stream));
+    int rc = dc_infer_frame(c, c->staging, pitch, nullptr, stats);
+    if (rc != DC_OK) return rc;
+    if (out_map_host)
+        DC_CUDA(cudaMemcpyAsync(out_map_host, layer_input(c, c->n_layers - 1), c->L[c->n_layers - 1].map_bytes,
+                                cudaMemcpyDeviceToHost, c->stream));
+    DC_CUDA(cudaStreamSynchronize(c->stream));
+    return DC_OK;
+}
+
+int dc_cache_layer_map(dc_cache* c, int layer, void** map_dev, size_t* bytes)
+{
+    if (!c || layer < 0 || layer >= c->n_layers || !map_dev || !c->executable) return DC_ERR_ARG;
+    *map_dev = (void*)layer_input(c, layer);
+    if (bytes) *bytes = c->L[layer].map_bytes;
+    return DC_OK;
+}
+
+int dc_cache_layer_regions(dc_cache* c, int layer, dc_region** regions_dev, int32_t** n_dev)
+{
+    if (!c || layer < -1 || layer >= c->n_layers || !regions_dev) return DC_ERR_ARG;
+    *regions_dev = layer < 0 ? c->regions0 : c->table + (size_t)c->S * c->max_regions * layer;
+    if (n_dev) *n_dev = c->n_regions;
+    return DC_OK;
+}
+
+int dc_get_status(dc_cache* c, int32_t* status_host)
+{
+    if (!c || !status_host) return DC_ERR_ARG;
+    DC_CUDA(cudaStreamSynchronize(c->stream));
+    DC_CUDA(cudaMemcpy(status_host, c->status, sizeof(int32_t), cudaMemcpyDeviceToHost));
+    return DC_OK;
+}
+
+const char* dc_strerror(int status)
+{
+    switch (status) {
+    case DC_OK: return "ok";
+    case DC_ERR_ARG: return "invalid argument";
+    case DC_ERR_CONFIG: return "unsupported configuration";
+    case DC_ERR_ALLOC: return "allocation failed";
+    case DC_ERR_CUDA: return g_last_cuda_error[0] ? g_last_cuda_error : "CUDA call failed";
+    case DC_ERR_OVERFLOW: return "more rectangles than max_regions";
+    case DC_ERR_TIMEOUT: return "device-side wait timed out";
+    case DC_ERR_STATE: return "call not valid in this state";
+    default: return "unknown status";
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,91 @@
+// Internal declarations shared by the translation units of libdeepcache.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "deepcache.h"
+
+#define DC_TILE_H 8          // output tile of the partial convolution: 8 rows x 16 columns
+#define DC_TILE_W 16         // = 128 output pixels = the M dimension of one tensor-core tile
+#define DC_TILE_PX (DC_TILE_H * DC_TILE_W)
+
+#define DC_CUDA(call)                                            \
+    do {                                                         \
+        cudaError_t e__ = (call);                                \
+        if (e__ != cudaSuccess) { dc_note_cuda_error(e__, __FILE__, __LINE__); return DC_ERR_CUDA; } \
+    } while (0)
+
+void dc_note_cuda_error(cudaError_t e, const char* file, int line);
+
+struct dc_layer_rt {
+    dc_layer_desc d;
+    int in_h, in_w;                 // size of the input map (or of the frame)
+    int tiles_x, tiles_y;           // conv only: output tiles per stream
+    void* map[2];                   // conv: current / cached output (ping-pong); others: map[0]
+    int cur;                        // conv: which of map[] holds the newest output
+    size_t map_bytes;               // bytes of one map, all streams
+    void* weight;                   // conv: [cout][kh][kw][cin] in the cache dtype
+    float* bias;                    // conv: [cout]
+    void* weight_packed;            // conv, bf16: K-major tensor-core layout (see dc_conv_bf16.cu)
+    int k_packed;                   // padded reduction length of weight_packed
+    uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
+    int32_t* dirty_list;            // conv: compacted tiles needing computation
+    int32_t* all_list;              // conv: every tile (used by full frames)
+    int32_t* zero_masks_unused;
+};
+
+struct dc_cache {
+    dc_config cfg;
+    int n_layers;
+    dc_layer_rt L[DC_MAX_LAYERS];
+    cudaStream_t stream;
+    int S, Gx, Gy, max_regions;
+    int elt;                        // bytes per map element
+    bool executable;                // every layer kind has an execution kernel
+    bool key_valid;
+    int64_t frame_idx;
+    int64_t launches;
+    size_t bytes;
+
+    uint8_t* key;                   // cached previous frames [S][H][key_pitch]
+    size_t key_pitch;
+    uint8_t* staging;               // device copy of host frames for dc_infer_frame_host
+    uint32_t sse_limit[4];          // PSNR test as an SSE bound, index = 2 * (bottom edge) + (right edge)
+
+    int16_t* blk_mv;                // [S][Gy][Gx][2]
+    uint32_t* blk_sse;              // [S][Gy][Gx]
+    uint8_t* matched;               // [S][Gy][Gx]
+    int32_t* mv_acc;                // [S][4]: sum dx, sum dy, K, n_matched
+    int32_t* gmv;                   // [S][3]: Mx, My, K
+    dc_region* regions0;            // [S][max_regions] rectangles on the frame
+    int32_t* n_regions;             // [S]
+    dc_region* table;               // [n_layers][S][max_regions]
+    dc_layer_desc* layers_dev;      // [n_layers]
+    int32_t* in_hw_dev;             // [n_layers][2]
+    int32_t* dirty_count;           // [n_layers]
+    int32_t* all_count;             // [n_layers]
+    int32_t* reuse_px;              // [n_layers][S]
+    uint32_t* zero_masks;           // all-zero reuse bitmap shared by full frames
+    int32_t* status;                // device status word
+    void* input_map;                // frame / 255 as a map, [S][H][W][3]
+    void* pix_lut;                  // 256 entries: pixel value -> map element
+    void* stats_pinned;             // host staging for statistics
+};
+
+static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }
+
+// ---- kernels' host-side launchers (each returns DC_OK or DC_ERR_CUDA) ----
+int dc_launch_match(dc_cache* c, const uint8_t* frame, size_t pitch);
+int dc_launch_propagate(dc_cache* c, const dc_region* in, const int32_t* n_in, int layer_end);
+int dc_launch_classify_copy(dc_cache* c, int layer, const dc_region* regions, const int32_t* n_regions,
+                            const void* prev_out, void* out);
+int dc_launch_conv(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
+                   const int32_t* tile_count, const uint32_t* masks, int max_tiles);
+int dc_launch_input_map(dc_cache* c, const uint8_t* frame, size_t pitch);
+int dc_launch_resize(dc_cache* c, int layer, const uint8_t* frame, size_t pitch);
+int dc_launch_maxpool(dc_cache* c, int layer, const void* in);
+int dc_launch_add(dc_cache* c, int layer, const void* a, const void* b);
+int dc_launch_relu(dc_cache* c, int layer, const void* a);
+int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_dev);

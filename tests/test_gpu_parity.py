@@ -1,0 +1,272 @@
+"""GPU parity: every C-ABI call against the CPU oracle on the same seeded inputs.
+
+Integer results (motion vectors, SSE, matched maps, rectangles at every layer) must be
+bit-exact; feature maps within 1e-4 max-abs (float32) or 2e-2 relative (bfloat16).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import deepcache_oracle as orc
+from paper_1712_01670_b200 import binding as B
+from paper_1712_01670_b200.engine import DeepCache
+from paper_1712_01670_b200.synth import configs, nets
+
+import parity_util as U
+
+pytestmark = pytest.mark.gpu
+
+
+def rng(seed):
+    return np.random.Generator(np.random.PCG64(seed))
+
+
+def matcher_only(width, height, n_streams, block, R, search, psnr_db=20.0):
+    layers = nets.single_conv(height, width)
+    ws, bs = nets.random_weights(layers, 1)
+    return DeepCache(width, height, layers, ws, bs, n_streams=n_streams, block=block, search_range=R,
+                     search=search, psnr_db=psnr_db)
+
+
+def check_pairs(pairs, block, R, search, psnr_db=20.0):
+    """pairs: list of (prev, cur) frames of equal size, run as one batch of streams."""
+    H, W = pairs[0][0].shape[:2]
+    dc = matcher_only(W, H, len(pairs), block, R, search, psnr_db)
+    try:
+        dc.set_key(np.stack([p for p, _ in pairs]))
+        got = dc.match_blocks(np.stack([c for _, c in pairs]))
+        for s, (prev, cur) in enumerate(pairs):
+            U.assert_match_equal(got, s, orc.match_blocks(cur, prev, block, R, search, psnr_db), f"stream {s}")
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
+
+
+# ------------------------------------------------------------------ dc_match_blocks
+def test_match_workload_1_exhaustive():
+    w = configs.WORKLOADS[1]()
+    sp = w.streams()
+    check_pairs([(sp.frame(0)[0], sp.frame(1)[0])], 8, 8, B.DC_SEARCH_EXHAUSTIVE)
+
+
+@pytest.mark.parametrize("widx,frames", [(2, (1, 2, 5, 9)), (3, (1, 4, 7)), (4, (1, 2, 3))])
+def test_match_diamond_streams(widx, frames):
+    w = configs.WORKLOADS[widx]()
+    sb = w.streams(1, max(frames) + 1)
+    check_pairs([(sb.frame(i - 1)[0], sb.frame(i)[0]) for i in frames], w.block, w.range, B.DC_SEARCH_DIAMOND)
+
+
+@pytest.mark.parametrize("search", [B.DC_SEARCH_EXHAUSTIVE, B.DC_SEARCH_DIAMOND])
+@pytest.mark.parametrize("block,shape", [(8, (40, 56)), (10, (61, 47)), (16, (16, 16)), (16, (90, 131)), (32, (70, 100)), (5, (23, 29))])
+def test_match_edge_geometry(search, block, shape):
+    g = rng(block * 7 + shape[0])
+    H, W = shape
+    prev = g.integers(0, 256, size=(H, W, 3), dtype=np.uint8)
+    moved = np.roll(prev, (2, -3), axis=(0, 1))
+    moved[H // 3:H // 3 + 9, W // 4:W // 4 + 11] = g.integers(0, 256, size=(min(9, H - H // 3), min(11, W - W // 4), 3))
+    smooth = np.clip(prev.astype(np.int32) + g.integers(-6, 7, size=prev.shape), 0, 255).astype(np.uint8)
+    const = np.full_like(prev, 93)
+    pairs = [(prev, moved), (prev, prev), (prev, smooth), (const, const), (const, prev)]
+    check_pairs(pairs, block, 4, search)
+
+
+def test_match_ties_and_thresholds():
+    # periodic pattern: several displacements tie at SSE 0; the smallest motion must win on both sides
+    x = np.arange(64)
+    row = ((x % 4) * 60).astype(np.uint8)
+    prev = np.repeat(np.repeat(row[None, :, None], 48, 0), 3, 2)
+    cur = np.roll(prev, -1, axis=1)
+    for search in (B.DC_SEARCH_EXHAUSTIVE, B.DC_SEARCH_DIAMOND):
+        check_pairs([(prev, cur), (cur, prev)], 8, 6, search)
+    # other thresholds move the integer SSE bound
+    g = rng(3)
+    a = g.integers(0, 256, size=(48, 64, 3), dtype=np.uint8)
+    b = np.clip(a.astype(np.int32) + g.integers(-40, 41, size=a.shape), 0, 255).astype(np.uint8)
+    for T in (12.0, 18.5, 25.0, 33.3):
+        check_pairs([(a, b)], 8, 3, B.DC_SEARCH_DIAMOND, psnr_db=T)
+
+
+def test_match_full_hd_batch():
+    """Workload 5's matcher geometry (1920x1080, block 16, range 32, last block row 8 px) on 2 streams."""
+    w = configs.WORKLOADS[5]()
+    sb = w.streams(2, 3)
+    check_pairs([(sb.frame(1, s), sb.frame(2, s)) for s in range(2)], 16, 32, B.DC_SEARCH_DIAMOND)
+
+
+def test_match_needs_a_key():
+    dc = matcher_only(32, 32, 1, 8, 4, B.DC_SEARCH_DIAMOND)
+    try:
+        with pytest.raises(B.DeepCacheError) as e:
+            dc.match_blocks(np.zeros((32, 32, 3), np.uint8))
+        assert e.value.status == B.DC_ERR_STATE
+    finally:
+        dc.close()
+
+
+# ------------------------------------------------------------------ dc_propagate_regions
+def random_regions(g, n, W, H, max_shift=9):
+    out = np.zeros(n, orc.REGION_DTYPE)
+    for i in range(n):
+        w, h = int(g.integers(1, W // 2)), int(g.integers(1, H // 2))
+        x, y = int(g.integers(0, W - w + 1)), int(g.integers(0, H - h + 1))
+        sx = int(np.clip(x + g.integers(-max_shift, max_shift + 1), 0, W - w))
+        sy = int(np.clip(y + g.integers(-max_shift, max_shift + 1), 0, H - h))
+        out[i] = (x, y, w, h, sx, sy)
+    return out
+
+
+def check_propagation(layers, W, H, n_streams, executable=True):
+    g = rng(len(layers))
+    if executable:
+        ws, bs = nets.random_weights(layers, 2)
+    else:
+        ws, bs = [None] * len(layers), [None] * len(layers)
+    dc = DeepCache(W, H, layers, ws, bs, n_streams=n_streams, block=16, search_range=8, dtype=B.DC_BF16)
+    try:
+        regs = torch.zeros((n_streams, dc.max_regions, 6), dtype=torch.int32)
+        counts, per_stream = [], []
+        for s in range(n_streams):
+            n = int(g.integers(0, min(dc.max_regions, 40) + 1)) if s else min(dc.max_regions, 37)
+            r = random_regions(g, n, W, H)
+            per_stream.append(r)
+            counts.append(n)
+            if n:
+                regs[s, :n] = torch.from_numpy(np.ascontiguousarray(r).view(np.int32).reshape(n, 6))
+        out, n_out = dc.propagate_regions(regs.cuda(), torch.tensor(counts, dtype=torch.int32).cuda())
+        for s in range(n_streams):
+            want = orc.propagate(layers, (H, W), per_stream[s])
+            for li in range(len(layers)):
+                U.assert_regions_equal(U.regions_np(out[li, s, :counts[s]]), want[li], f"layer {li} stream {s}")
+                assert int(n_out[li, s]) == counts[s]
+                assert not out[li, s, counts[s]:].any()
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("net,W,H", [("small", 227, 227), ("alexnet", 227, 227), ("resnet", 224, 224), ("vgg", 1920, 1080)])
+def test_propagate_networks(net, W, H):
+    layers = {"small": lambda: nets.small_cnn(H, W), "alexnet": lambda: nets.alexnet_trunk(H, W),
+              "resnet": lambda: nets.resnet50_trunk(H, W), "vgg": lambda: nets.vgg16_trunk(224, 224, H, W)}[net]()
+    check_propagation(layers, W, H, 3)
+
+
+def test_propagate_table2_rows():
+    """Layer kinds that only region propagation knows (LRN, concat, fully connected)."""
+    b = nets.NetBuilder(96, 96)
+    c1 = b.conv(-1, 16, 11, 2, 5)
+    b.layers.append(dict(kind=B.DC_RELU, kh=1, kw=1, sh=1, sw=1, ph=0, pw=0, cin=16, cout=16, relu=0, in0=c1, in1=-1, out_h=48, out_w=48))
+    b.layers.append(dict(kind=B.DC_LRN, kh=5, kw=5, sh=1, sw=1, ph=2, pw=2, cin=16, cout=16, relu=0, in0=1, in1=-1, out_h=48, out_w=48))
+    p = b.maxpool(2, 3, 2, 1)
+    q = b.conv(2, 16, 3, 2, 1)
+    b.layers.append(dict(kind=B.DC_CONCAT, kh=1, kw=1, sh=1, sw=1, ph=0, pw=0, cin=16, cout=32, relu=0, in0=p, in1=q, out_h=24, out_w=24))
+    b.layers.append(dict(kind=B.DC_FC, kh=1, kw=1, sh=1, sw=1, ph=0, pw=0, cin=32, cout=10, relu=0, in0=5, in1=-1, out_h=1, out_w=1))
+    check_propagation(b.layers, 96, 96, 2, executable=False)
+
+
+# ------------------------------------------------------------------ dc_conv_partial
+@pytest.mark.parametrize("dtype", [B.DC_FP32, B.DC_BF16])
+@pytest.mark.parametrize("hi,wi,cin,cout,k,s,p,relu", [
+    (37, 45, 3, 16, 3, 1, 1, 1), (64, 64, 32, 64, 3, 1, 1, 1), (227, 227, 3, 96, 11, 4, 0, 1),
+    (27, 27, 96, 256, 5, 1, 2, 1), (56, 56, 64, 128, 1, 2, 0, 0), (30, 33, 16, 24, 3, 2, 1, 0),
+    (14, 14, 256, 512, 3, 1, 1, 1), (224, 224, 3, 64, 7, 2, 3, 1)])
+def test_conv_partial(dtype, hi, wi, cin, cout, k, s, p, relu):
+    g = rng(hi + cin + k)
+    bf16 = dtype == B.DC_BF16
+    quant = orc.QUANT_BF16 if bf16 else orc.QUANT_NONE
+    S = 2
+    b = nets.NetBuilder(hi, wi, cin)
+    b.conv(-1, cout, k, s, p, relu)
+    L = b.layers[0]
+    wts = g.normal(0, np.sqrt(2.0 / (k * k * cin)), size=(cout, k, k, cin)).astype(np.float32)
+    bias = g.normal(0, 0.1, size=cout).astype(np.float32)
+    layers = [dict(L)]
+    x = g.normal(size=(S, hi, wi, cin))
+    prev = g.normal(size=(S, L["out_h"], L["out_w"], cout))
+    xq = np.stack([orc.quant_array(v, quant) for v in x])
+    pq = np.stack([orc.quant_array(v, quant) for v in prev])
+    tdt = torch.bfloat16 if bf16 else torch.float32
+    # the library validates cin against the frame's 3 channels for in0 = -1, so give the conv a
+    # producer with the right shape when cin != 3: a 1x1 conv from the frame stands in
+    if cin == 3:
+        net, li, fh, fw = layers, 0, hi, wi
+        ws, bs = [wts], [bias]
+    else:
+        nb = nets.NetBuilder(hi, wi)
+        a = nb.conv(-1, cin, 1, 1, 0)
+        nb.conv(a, cout, k, s, p, relu)
+        net, li, fh, fw = nb.layers, 1, hi, wi
+        ws = [np.zeros((cin, 1, 1, 3), np.float32), wts]
+        bs = [np.zeros(cin, np.float32), bias]
+    dc = DeepCache(fw, fh, net, ws, bs, n_streams=S, block=16, search_range=4, dtype=dtype)
+    try:
+        regs = torch.zeros((S, dc.max_regions, 6), dtype=torch.int32)
+        per_stream, counts = [], []
+        for s_ in range(S):
+            n = min(dc.max_regions, 6)
+            # disjoint rectangles: split the output into a grid of cells, one rectangle inside each
+            r = np.zeros(n, orc.REGION_DTYPE)
+            cw, ch = L["out_w"] // 3, L["out_h"] // 2
+            for i in range(n):
+                cx, cy = (i % 3) * cw, (i // 3) * ch
+                w_ = int(g.integers(1, cw + 1)); h_ = int(g.integers(1, ch + 1))
+                x0 = cx + int(g.integers(0, cw - w_ + 1)); y0 = cy + int(g.integers(0, ch - h_ + 1))
+                sx = int(g.integers(0, L["out_w"] - w_ + 1)); sy = int(g.integers(0, L["out_h"] - h_ + 1))
+                r[i] = (x0, y0, w_, h_, sx, sy)
+            if s_ == 1:
+                r[2] = (0, 0, 0, 0, 0, 0)          # a vanished slot
+            per_stream.append(r); counts.append(n)
+            regs[s_, :n] = torch.from_numpy(np.ascontiguousarray(r).view(np.int32).reshape(n, 6))
+        xin = torch.from_numpy(xq).to(tdt).cuda()
+        pin = torch.from_numpy(pq).to(tdt).cuda()
+        full = dc.conv_partial(li, xin)
+        part = dc.conv_partial(li, xin, pin, regs.cuda(), torch.tensor(counts, dtype=torch.int32).cuda())
+        wq = orc.quant_array(wts, quant)
+        for s_ in range(S):
+            want_full, _ = orc.conv_reuse(xq[s_], L, wq, bias, quant)
+            want, reused = orc.conv_reuse(xq[s_], L, wq, bias, quant, pq[s_], per_stream[s_])
+            U.assert_map_close(full[s_], want_full, bf16, "full")
+            U.assert_map_close(part[s_], want, bf16, "partial")
+            m = reused.astype(bool)
+            got = part[s_].float().cpu().numpy().astype(np.float64)
+            assert np.array_equal(got[m], pq[s_][m]), "reused pixels must be bit-equal copies of the cached map"
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
+
+
+# ------------------------------------------------------------------ dc_infer_frame
+def test_infer_workload_1():
+    U.run_stream_parity(configs.WORKLOADS[1](), 1, [0, 1])
+
+
+def test_infer_workload_2_through_an_expiry():
+    U.run_stream_parity(configs.WORKLOADS[2](), 1, list(range(12)))
+
+
+def test_infer_workload_3_alexnet_bf16():
+    U.run_stream_parity(configs.WORKLOADS[3](), 1, list(range(12)))
+
+
+def test_infer_workload_4_resnet50_bf16():
+    U.run_stream_parity(configs.WORKLOADS[4](), 1, list(range(4)))
+
+
+def test_infer_workload_5_two_streams():
+    """Full-HD matching, area resize to 224x224, VGG-16 trunk; 2 of the 32 streams, frames 0-2."""
+    U.run_stream_parity(configs.WORKLOADS[5](), 2, [0, 1, 2])
+
+
+def test_infer_identical_frames_and_reset():
+    w = configs.WORKLOADS[2]()
+    f = w.streams(1, 1).frame(0)
+    dc = DeepCache.from_workload(w)
+    try:
+        a = dc.infer_frame(f).clone()
+        b, st = dc.infer_frame(f, want_stats=True)
+        assert not st[0].refreshed and (st[0].mvx, st[0].mvy) == (0, 0) and st[0].n_regions == 1
+        assert torch.equal(a, b)                     # everything reusable was copied, the rest recomputed identically
+        dc.reset()
+        c, st = dc.infer_frame(f, want_stats=True)
+        assert st[0].refreshed and torch.equal(a, c)
+    finally:
+        dc.close()
