@@ -1,0 +1,340 @@
+#!/usr/bin/env python
+"""Benchmark of the cache-aware inference hot path: cached frames/s on B200.
+
+A step is one pass of the whole path (matching, propagation, reuse copy, partial
+convolutions, pooling, cache update) over one batch: one new frame for each of the
+workload's independent video streams.  Default workload: "batched_stress" (32 streams of
+1920x1080 video, VGG-16-shaped trunk at 224x224, bf16).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  With --gpus N > 1 it must be started by torchrun; every
+rank then runs its own set of streams (weak scaling, no collective on the data path) and
+the timing is the maximum over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import ctypes
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from concurrent.futures import ThreadPoolExecutor
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+METRIC = "cached_frames_per_sec"
+UNIT = "frames/s"
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", type=int, default=5)
+    ap.add_argument("--streams", type=int, default=0, help="override the number of streams per GPU")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
+                    bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+def workload_config(w, n_streams, n_gpus):
+    return {"workload": w.name, "streams_per_gpu": n_streams, "frame": f"{w.width}x{w.height}x3 uint8",
+            "block": w.block, "range": w.range, "search": "diamond" if w.search == 1 else "exhaustive",
+            "psnr_db": w.psnr_db, "expire_n": w.expire_n, "trunk_layers": len(w.layers),
+            "parallelism": f"streams sharded over {n_gpus} GPU(s), no collective",
+            "l2": "inputs larger than L2 (each step reads a fresh batch of frames)"}
+
+
+def conv_flops_per_pixel(layers):
+    return [2.0 * l["cout"] * l["cin"] * l["kh"] * l["kw"] if l["kind"] == 0 else 0.0 for l in layers]
+
+
+# ---------------------------------------------------------------------------
+# the oracle as CPU baseline / reference arm
+# ---------------------------------------------------------------------------
+def run_oracle_sample(w, n_frames, stream=0):
+    """Times the oracle, as it stands, on frames 0..n_frames-1 of one stream.  Returns
+    (frames/s, seconds, description)."""
+    from oracle import deepcache_oracle as orc
+    ws, bs = w.weights()
+    quant = orc.QUANT_BF16 if w.dtype == 1 else orc.QUANT_NONE
+    oc = orc.OracleCache(w.width, w.height, w.layers, ws, bs, block=w.block, search_range=w.range,
+                         search_kind=w.search, psnr_db=w.psnr_db, expire_n=w.expire_n, quant=quant)
+    sb = w.streams(stream + 1, n_frames)
+    frames = [sb.frame(i, stream) for i in range(n_frames)]
+    orc.lib()
+    t0 = time.perf_counter()
+    for f in frames:
+        oc.infer_frame(f)
+    dt = time.perf_counter() - t0
+    return n_frames / dt, dt, f"stream {stream}, frames 0-{n_frames - 1} (1 full + {n_frames - 1} cached)"
+
+
+def reference_arm(args, w):
+    """The oracle timed on the host cores, per the same metric.  Each step is a bounded
+    sample: one frame of one stream."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import deepcache_oracle as orc
+    ws, bs = w.weights()
+    quant = orc.QUANT_BF16 if w.dtype == 1 else orc.QUANT_NONE
+    oc = orc.OracleCache(w.width, w.height, w.layers, ws, bs, block=w.block, search_range=w.range,
+                         search_kind=w.search, psnr_db=w.psnr_db, expire_n=w.expire_n, quant=quant)
+    total = args.warmup + args.steps
+    sb = w.streams(1, total)
+    frames = [sb.frame(i, 0) for i in range(total)]
+    for f in frames[:args.warmup]:
+        oc.infer_frame(f)
+    t0 = time.perf_counter()
+    for f in frames[args.warmup:]:
+        oc.infer_frame(f)
+    dt = time.perf_counter() - t0
+    fps = args.steps / dt
+    cores = os.cpu_count()
+    sample = f"one stream of the workload, one frame per step ({args.steps} timed frames after {args.warmup})"
+    line = {"impl": "reference", "metric": METRIC, "value": fps, "unit": UNIT, "n_gpus": args.gpus,
+            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "config": workload_config(w, 1, args.gpus),
+            "cpu_baseline": {"value": fps, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": fps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+# ---------------------------------------------------------------------------
+# clocks
+# ---------------------------------------------------------------------------
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.index), "-lms", "100"], stdout=subprocess.PIPE, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.perf_counter(), [v.strip() for v in line.split(",")]))
+
+    def stop(self, t0, t1):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        rows = [r for t, r in self.rows if t0 <= t <= t1] or [r for _, r in self.rows[-3:]]
+        sm, smax, reasons = [], None, set()
+        for r in rows:
+            try:
+                sm.append(float(r[0])); smax = float(r[1])
+            except Exception:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": smax, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+# ---------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------
+def gpu_arm(args, w):
+    import torch
+    import torch.distributed as dist
+    from paper_1712_01670_b200 import binding as B
+    from paper_1712_01670_b200.engine import DeepCache
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus > 1 and world != args.gpus:
+        raise SystemExit("--gpus N > 1 needs torchrun with N ranks")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+
+    S = args.streams or w.n_streams
+    total = args.warmup + args.steps
+    # every rank renders its own streams: global stream index = rank * S + s
+    sb_all = w.streams(S * world, total)
+    my = list(range(rank * S, rank * S + S))
+    frame_bytes = w.height * w.width * 3
+    host = torch.empty((total, S, w.height, w.width, 3), dtype=torch.uint8).pin_memory()
+    host_np = host.numpy()
+
+    def render(job):
+        s, i = job
+        host_np[i, s] = sb_all.streams[my[s]].frame(i)
+    with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 4)) as ex:
+        list(ex.map(render, [(s, i) for s in range(S) for i in range(total)]))
+    dev_frames = host.to(dev, non_blocking=True)
+    torch.cuda.synchronize()
+
+    dc = DeepCache.from_workload(w, n_streams=S, device=f"cuda:{local}")
+    pitch = w.width * 3
+    last = w.layers[-1]
+    out_bytes = S * last["out_h"] * last["out_w"] * last["cout"] * (2 if w.dtype == 1 else 4)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- device-resident timing: value ----
+    for i in range(args.warmup):
+        B.dc_infer_frame(dc.handle, dev_frames[i], pitch)
+    barrier()
+    B.dc_cache_set_profiling(dc.handle, True)
+    B.dc_cache_profile(dc.handle)
+    px0, cached0, full0 = B.dc_cache_counters(dc.handle, len(w.layers))
+    launches0 = dc.launches()
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t0 = time.perf_counter()
+    e0.record()
+    for i in range(args.warmup, total):
+        B.dc_infer_frame(dc.handle, dev_frames[i], pitch)
+    e1.record()
+    barrier()
+    t1 = time.perf_counter()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop(t0, t1)
+    launches = dc.launches() - launches0
+    prof = B.dc_cache_profile(dc.handle)
+    B.dc_cache_set_profiling(dc.handle, False)
+    px1, cached1, full1 = B.dc_cache_counters(dc.handle, len(w.layers))
+    status = dc.status()
+    if status != B.DC_OK:
+        raise SystemExit(f"device status {status}: {B.strerror(status)}")
+    if world > 1:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    value = S * world * args.steps / (ms * 1e-3)
+
+    # ---- end to end through the host-buffer entry point ----
+    e2e = None
+    if not args.no_e2e:
+        dc.reset()
+        out_host = torch.empty(out_bytes, dtype=torch.uint8).pin_memory()
+        for i in range(args.warmup):
+            B.dc_infer_frame_host(dc.handle, host[i].data_ptr(), pitch, out_host.data_ptr())
+        barrier()
+        t0e = time.perf_counter()
+        for i in range(args.warmup, total):
+            B.dc_infer_frame_host(dc.handle, host[i].data_ptr(), pitch, out_host.data_ptr())
+        torch.cuda.synchronize()
+        dte = time.perf_counter() - t0e
+        if world > 1:
+            t = torch.tensor([dte], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            dte = float(t.item())
+        e2e = {"value": S * world * args.steps / dte, "unit": UNIT, "h2d_bytes_per_step": S * frame_bytes,
+               "d2h_bytes_per_step": out_bytes}
+
+    if rank != 0:
+        dc.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
+    # ---- rooflines from the event profile of the timed region ----
+    peaks = measured_peaks()
+    fpp = conv_flops_per_pixel(w.layers)
+    n_cached, n_full = cached1 - cached0, full1 - full0
+    useful_flops = 0.0
+    reuse = {}
+    for li, l in enumerate(w.layers):
+        if l["kind"] != 0:
+            continue
+        all_px = l["out_h"] * l["out_w"] * S * (n_cached + n_full)
+        reused = px1[li] - px0[li]
+        useful_flops += fpp[li] * (all_px - reused)
+        reuse[str(li)] = round(reused / max(1, l["out_h"] * l["out_w"] * S * max(1, n_cached)), 4)
+    conv_ms, conv_n = prof["conv"]
+    stage_ms = {k: round(v[0], 4) for k, v in prof.items()}
+    stage_share = {k: round(v[0] / max(1e-9, sum(x[0] for x in prof.values())), 4) for k, v in prof.items()}
+    bf16 = w.dtype == 1
+    conv_tflops = useful_flops / (conv_ms * 1e-3) / 1e12 if conv_ms > 0 else 0.0
+    conv_peak = peaks["bf16_tflops_sustained"] if bf16 else None
+    roofline = {"kernel": "partial convolution (all conv launches of the timed region)",
+                "bound": "tensor" if bf16 else "alu", "achieved": conv_tflops,
+                "peak": conv_peak, "unit": "TFLOP/s", "frac": (conv_tflops / conv_peak) if conv_peak else None,
+                "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None,
+                "launches": conv_n, "avg_launch_ms": conv_ms / max(1, conv_n),
+                "flops_per_launch": useful_flops / max(1, conv_n)}
+    match_ms = prof["search"][0] + prof["verify"][0]
+    match_bytes = 4.0 * frame_bytes * S * n_cached            # Step 2: cur + prev once; Step 4: both again
+    match_gbs = match_bytes / (match_ms * 1e-3) / 1e9 if match_ms > 0 else 0.0
+    roofline_matcher = {"kernel": "block search + verify", "bound": "hbm", "achieved": match_gbs,
+                        "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": match_gbs / peaks["hbm_gbs"],
+                        "peak_source": f"hbm_gbs, {peaks['source']}", "traffic": None,
+                        "launches": prof["search"][1] + prof["verify"][1],
+                        "bytes_per_frame_batch": 4.0 * frame_bytes * S}
+
+    cpu_baseline = None
+    if not args.no_cpu_baseline:
+        fps, secs, what = run_oracle_sample(w, 3)
+        cpu_baseline = {"value": fps, "unit": UNIT, "cores": os.cpu_count(), "kind": "oracle",
+                        "sample": what + f", {secs:.1f} s"}
+
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
+            "config": workload_config(w, S, world), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "roofline": roofline, "roofline_matcher": roofline_matcher, "cpu_baseline": cpu_baseline,
+            "stage_ms": stage_ms, "stage_share": stage_share, "frames_cached": n_cached, "frames_full": n_full,
+            "reuse_ratio_cached_frames": reuse, "cache_bytes": dc.bytes()}
+    print(json.dumps(line))
+    dc.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    args = parse_args()
+    from paper_1712_01670_b200.synth import configs
+    w = configs.WORKLOADS[args.workload]()
+    if args.impl == "reference":
+        reference_arm(args, w)
+    else:
+        gpu_arm(args, w)
+
+
+if __name__ == "__main__":
+    main()

@@ -188,6 +188,24 @@ int dc_get_status(dc_cache* cache, int32_t* status_host);
 /* Kernels of this library launched on this cache since creation (for reporting). */
 int dc_cache_launches(const dc_cache* cache, int64_t* launches);
 
+/* Optional per-stage timing with CUDA events on the cache's stream.  While enabled, every
+ * kernel launch of the library is bracketed by an event pair.  dc_cache_profile waits for the
+ * stream, adds up the pairs recorded since the last call and clears them.
+ *   ms_host / launches_host: DC_PROFILE_STAGES entries each, indexed by dc_profile_stage. */
+typedef enum {
+    DC_PROF_SEARCH = 0, DC_PROF_VERIFY = 1, DC_PROF_MERGE = 2, DC_PROF_PROPAGATE = 3,
+    DC_PROF_CLASSIFY_COPY = 4, DC_PROF_CONV = 5, DC_PROF_INPUT = 6, DC_PROF_POINTWISE = 7,
+    DC_PROF_KEY_UPDATE = 8
+} dc_profile_stage;
+#define DC_PROFILE_STAGES 9
+int dc_cache_set_profiling(dc_cache* cache, int enable);
+int dc_cache_profile(dc_cache* cache, float* ms_host, int64_t* launches_host);
+
+/* Running totals since creation or the last dc_cache_reset: reused output pixels per layer
+ * (reused_px_host: n_layers entries, summed over streams and frames), frames served from the
+ * cache and full fresh frames (each counts one call, not one stream).  Synchronous. */
+int dc_cache_counters(dc_cache* cache, int64_t* reused_px_host, int64_t* frames_cached, int64_t* frames_full);
+
 const char* dc_strerror(int status);
 
 #ifdef __cplusplus

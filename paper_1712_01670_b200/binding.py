@@ -47,7 +47,9 @@ REGION_DTYPE = np.dtype([(n, "<i4") for n in ("x", "y", "w", "h", "sx", "sy")])
 
 EXPORTS = ["dc_cache_create", "dc_cache_destroy", "dc_cache_reset", "dc_cache_bytes", "dc_cache_set_key",
            "dc_match_blocks", "dc_propagate_regions", "dc_conv_partial", "dc_infer_frame", "dc_infer_frame_host",
-           "dc_cache_layer_map", "dc_cache_layer_regions", "dc_get_status", "dc_cache_launches", "dc_strerror"]
+           "dc_cache_layer_map", "dc_cache_layer_regions", "dc_get_status", "dc_cache_launches",
+           "dc_cache_set_profiling", "dc_cache_profile", "dc_cache_counters", "dc_strerror"]
+PROFILE_STAGES = ["search", "verify", "merge", "propagate", "classify_copy", "conv", "input", "pointwise", "key_update"]
 
 _lib = None
 
@@ -81,6 +83,9 @@ def load():
         L.dc_cache_layer_regions.argtypes = [vp, i, C.POINTER(vp), C.POINTER(vp)]
         L.dc_get_status.argtypes = [vp, C.POINTER(C.c_int32)]
         L.dc_cache_launches.argtypes = [vp, C.POINTER(C.c_int64)]
+        L.dc_cache_set_profiling.argtypes = [vp, i]
+        L.dc_cache_profile.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
+        L.dc_cache_counters.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
         L.dc_strerror.argtypes = [i]
         L.dc_strerror.restype = C.c_char_p
         for name in EXPORTS[:-1]:
@@ -197,3 +202,23 @@ def dc_get_status(cache) -> int:
     v = C.c_int32()
     _check(load().dc_get_status(cache, C.byref(v)), "dc_get_status")
     return v.value
+
+
+def dc_cache_set_profiling(cache, enable: bool):
+    _check(load().dc_cache_set_profiling(cache, int(enable)), "dc_cache_set_profiling")
+
+
+def dc_cache_profile(cache):
+    """{stage: (milliseconds, launches)} recorded since the last call."""
+    ms = (C.c_float * len(PROFILE_STAGES))()
+    n = (C.c_int64 * len(PROFILE_STAGES))()
+    _check(load().dc_cache_profile(cache, ms, n), "dc_cache_profile")
+    return {name: (float(ms[k]), int(n[k])) for k, name in enumerate(PROFILE_STAGES)}
+
+
+def dc_cache_counters(cache, n_layers: int):
+    """(reused pixels per layer, frames served from cache, full fresh frames) since the last reset."""
+    px = (C.c_int64 * n_layers)()
+    a, b = C.c_int64(), C.c_int64()
+    _check(load().dc_cache_counters(cache, px, C.byref(a), C.byref(b)), "dc_cache_counters")
+    return [int(v) for v in px], a.value, b.value

@@ -17,6 +17,8 @@ void dc_note_cuda_error(cudaError_t e, const char* file, int line)
     if (getenv("DC_VERBOSE")) fprintf(stderr, "libdeepcache: CUDA error: %s\n", g_last_cuda_error);
 }
 
+void dc_prof_release(dc_cache* c);
+
 namespace {
 
 // nearest bfloat16 (ties to even) of a double, as its 16 bit pattern
@@ -120,6 +122,8 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     DC_TRY(dev_alloc(c, &c->all_count, (size_t)n));
     DC_TRY(dev_alloc(c, &c->reuse_px, (size_t)n * S));
     DC_TRY(dev_alloc(c, &c->status, (size_t)1));
+    DC_TRY(dev_alloc(c, &c->reused_total, (size_t)n));
+    DC_CUDA(cudaMemsetAsync(c->reused_total, 0, sizeof(unsigned long long) * n, c->stream));
     DC_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int32_t), c->stream));
     DC_CUDA(cudaMemsetAsync(c->n_regions, 0, sizeof(int32_t) * S, c->stream));
     DC_CUDA(cudaMemsetAsync(c->table, 0, sizeof(dc_region) * n * S * c->max_regions, c->stream));
@@ -198,6 +202,8 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
 
 void release(dc_cache* c)
 {
+    dc_prof_release(c);
+    cudaFree(c->reused_total);
     cudaFree(c->key); cudaFree(c->staging); cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched);
     cudaFree(c->mv_acc); cudaFree(c->gmv); cudaFree(c->regions0); cudaFree(c->n_regions); cudaFree(c->table);
     cudaFree(c->layers_dev); cudaFree(c->in_hw_dev); cudaFree(c->dirty_count); cudaFree(c->all_count);
@@ -285,8 +291,9 @@ int dc_cache_destroy(dc_cache* c)
 int dc_cache_reset(dc_cache* c)
 {
     if (!c) return DC_ERR_ARG;
-    c->key_valid = false; c->frame_idx = 0;
+    c->key_valid = false; c->frame_idx = 0; c->frames_cached = 0; c->frames_full = 0;
     DC_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int32_t), c->stream));
+    DC_CUDA(cudaMemsetAsync(c->reused_total, 0, sizeof(unsigned long long) * c->n_layers, c->stream));
     return DC_OK;
 }
 
@@ -405,10 +412,14 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
         }
     }
     // the frame becomes the next cache key (Section 3)
-    DC_CUDA(cudaMemcpy2DAsync(c->key, c->key_pitch, frame_dev, pitch, (size_t)c->cfg.width * 3,
-                              (size_t)c->cfg.height * S, cudaMemcpyDeviceToDevice, c->stream));
+    {
+        dc_prof_scope ps(c, DC_ST_KEY_UPDATE);
+        DC_CUDA(cudaMemcpy2DAsync(c->key, c->key_pitch, frame_dev, pitch, (size_t)c->cfg.width * 3,
+                                  (size_t)c->cfg.height * S, cudaMemcpyDeviceToDevice, c->stream));
+    }
     c->key_valid = true;
     c->frame_idx += 1;
+    if (refresh) c->frames_full += 1; else c->frames_cached += 1;
     if (out_map_dev)
         DC_CUDA(cudaMemcpyAsync(out_map_dev, layer_input(c, n - 1), c->L[n - 1].map_bytes, cudaMemcpyDeviceToDevice, c->stream));
     if (stats) return fill_stats(c, refresh, stats);
@@ -446,6 +457,17 @@ int dc_cache_layer_regions(dc_cache* c, int layer, dc_region** regions_dev, int3
     if (!c || layer < -1 || layer >= c->n_layers || !regions_dev) return DC_ERR_ARG;
     *regions_dev = layer < 0 ? c->regions0 : c->table + (size_t)c->S * c->max_regions * layer;
     if (n_dev) *n_dev = c->n_regions;
+    return DC_OK;
+}
+
+int dc_cache_counters(dc_cache* c, int64_t* reused_px_host, int64_t* frames_cached, int64_t* frames_full)
+{
+    if (!c) return DC_ERR_ARG;
+    DC_CUDA(cudaStreamSynchronize(c->stream));
+    if (reused_px_host)
+        DC_CUDA(cudaMemcpy(reused_px_host, c->reused_total, sizeof(int64_t) * c->n_layers, cudaMemcpyDeviceToHost));
+    if (frames_cached) *frames_cached = c->frames_cached;
+    if (frames_full) *frames_full = c->frames_full;
     return DC_OK;
 }
 

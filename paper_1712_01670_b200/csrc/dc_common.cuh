@@ -19,6 +19,12 @@
 
 void dc_note_cuda_error(cudaError_t e, const char* file, int line);
 
+// Stages timed by the optional event profiler (dc_cache_profile).
+enum dc_stage { DC_ST_SEARCH = 0, DC_ST_VERIFY, DC_ST_MERGE, DC_ST_PROPAGATE, DC_ST_CLASSIFY_COPY, DC_ST_CONV,
+                DC_ST_INPUT, DC_ST_POINTWISE, DC_ST_KEY_UPDATE, DC_ST_COUNT };
+
+struct dc_prof;      // event pool, allocated when profiling is switched on
+
 struct dc_layer_rt {
     dc_layer_desc d;
     int in_h, in_w;                 // size of the input map (or of the frame)
@@ -72,6 +78,16 @@ struct dc_cache {
     void* input_map;                // frame / 255 as a map, [S][H][W][3]
     void* pix_lut;                  // 256 entries: pixel value -> map element
     void* stats_pinned;             // host staging for statistics
+    unsigned long long* reused_total; // [n_layers] reused output pixels summed over all frames so far
+    int64_t frames_cached, frames_full;
+    dc_prof* prof;
+};
+
+// Records a start / stop event pair around the enclosed launches when profiling is on.
+struct dc_prof_scope {
+    dc_cache* c; int stage;
+    dc_prof_scope(dc_cache* cache, int st);
+    ~dc_prof_scope();
 };
 
 static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }

@@ -130,6 +130,7 @@ int dc_launch_conv(dc_cache* c, int layer, const void* in, void* out, const int3
     int cap = dc_div_up(148 * 8, co_groups);
     if (gx > cap) gx = cap;
     dim3 grid(gx, co_groups);
+    dc_prof_scope ps(c, DC_ST_CONV);
     if (c->cfg.dtype == DC_BF16) k_conv_direct<__nv_bfloat16><<<grid, DC_TILE_PX, 0, c->stream>>>(a);
     else k_conv_direct<float><<<grid, DC_TILE_PX, 0, c->stream>>>(a);
     c->launches += 1;

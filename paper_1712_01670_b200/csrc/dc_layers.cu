@@ -120,6 +120,7 @@ int dc_launch_input_map(dc_cache* c, const uint8_t* frame, size_t pitch)
 {
     size_t n = (size_t)c->S * c->cfg.height * c->cfg.width * 3;
     int W = c->cfg.width, H = c->cfg.height;
+    dc_prof_scope ps(c, DC_ST_INPUT);
     DISPATCH(c,
         (k_input_map<float><<<grid_for(n, 256), 256, 0, c->stream>>>(frame, pitch, W, H, c->S, (const float*)c->pix_lut, (float*)c->input_map)),
         (k_input_map<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>(frame, pitch, W, H, c->S, (const __nv_bfloat16*)c->pix_lut, (__nv_bfloat16*)c->input_map)));
@@ -133,6 +134,7 @@ int dc_launch_resize(dc_cache* c, int layer, const uint8_t* frame, size_t pitch)
     dc_layer_rt& L = c->L[layer];
     long long warps = (long long)c->S * L.d.out_h * L.d.out_w;
     int grid = (int)((warps + 7) / 8);
+    dc_prof_scope ps(c, DC_ST_INPUT);
     DISPATCH(c,
         (k_resize_area<float><<<grid, 256, 0, c->stream>>>(frame, pitch, c->cfg.width, c->cfg.height, c->S, L.d.out_w, L.d.out_h, (float*)L.map[0])),
         (k_resize_area<__nv_bfloat16><<<grid, 256, 0, c->stream>>>(frame, pitch, c->cfg.width, c->cfg.height, c->S, L.d.out_w, L.d.out_h, (__nv_bfloat16*)L.map[0])));
@@ -145,6 +147,7 @@ int dc_launch_maxpool(dc_cache* c, int layer, const void* in)
 {
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
+    dc_prof_scope ps(c, DC_ST_POINTWISE);
     DISPATCH(c,
         (k_maxpool<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)L.map[0])),
         (k_maxpool<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)L.map[0])));
@@ -157,6 +160,7 @@ int dc_launch_add(dc_cache* c, int layer, const void* a, const void* b)
 {
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
+    dc_prof_scope ps(c, DC_ST_POINTWISE);
     DISPATCH(c,
         (k_add<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, (const float*)b, n, L.d.relu, (float*)L.map[0])),
         (k_add<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, n, L.d.relu, (__nv_bfloat16*)L.map[0])));
@@ -169,6 +173,7 @@ int dc_launch_relu(dc_cache* c, int layer, const void* a)
 {
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
+    dc_prof_scope ps(c, DC_ST_POINTWISE);
     DISPATCH(c,
         (k_relu<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, n, (float*)L.map[0])),
         (k_relu<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, n, (__nv_bfloat16*)L.map[0])));

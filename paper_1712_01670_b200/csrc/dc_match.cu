@@ -265,8 +265,8 @@ int launch_all(dc_cache* c, MatchArgs& a)
 {
     int warps = a.S * a.Gx * a.Gy;
     int grid = dc_div_up(warps, WARPS);
-    k_search<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a);
-    k_verify<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a);
+    { dc_prof_scope ps(c, DC_ST_SEARCH); k_search<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a); }
+    { dc_prof_scope ps(c, DC_ST_VERIFY); k_verify<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a); }
     return 0;
 }
 
@@ -288,8 +288,11 @@ int dc_launch_match(dc_cache* c, const uint8_t* frame, size_t pitch)
     else if (iters <= 6) launch_all<6>(c, a);
     else if (iters <= 12) launch_all<12>(c, a);
     else launch_all<24>(c, a);
-    k_merge<<<c->S, 256, 0, c->stream>>>(c->matched, c->gmv, a.W, a.H, a.B, a.Gx, a.Gy, c->max_regions,
-                                         c->regions0, c->n_regions, c->status);
+    {
+        dc_prof_scope ps(c, DC_ST_MERGE);
+        k_merge<<<c->S, 256, 0, c->stream>>>(c->matched, c->gmv, a.W, a.H, a.B, a.Gx, a.Gy, c->max_regions,
+                                             c->regions0, c->n_regions, c->status);
+    }
     c->launches += 3;
     DC_CUDA(cudaGetLastError());
     return DC_OK;

@@ -102,6 +102,7 @@ struct ClassifyArgs {
     int Ho, Wo, px_bytes;                        // px_bytes = cout * element size (multiple of 16)
     int tiles_x, tiles_y, S;
     uint32_t* masks; int32_t* dirty_list; int32_t* dirty_count; int32_t* reuse_px;
+    unsigned long long* reused_total;
 };
 
 __global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
@@ -159,7 +160,7 @@ __global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
         mk[0] = m0; mk[1] = m1; mk[2] = m2; mk[3] = m3;
         int covered = __popc(m0) + __popc(m1) + __popc(m2) + __popc(m3);
         int in_tile = (X1 - X0) * (Y1 - Y0);
-        if (covered) atomicAdd(&a.reuse_px[s], covered);
+        if (covered) { atomicAdd(&a.reuse_px[s], covered); atomicAdd(a.reused_total, (unsigned long long)covered); }
         if (covered < in_tile) {
             int slot = atomicAdd(a.dirty_count, 1);
             a.dirty_list[slot] = tile;
@@ -172,8 +173,11 @@ __global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
 int dc_launch_propagate(dc_cache* c, const dc_region* in, const int32_t* n_in, int layer_end)
 {
     dim3 grid(dc_div_up(c->max_regions, 128), c->S);
-    k_propagate<<<grid, 128, 0, c->stream>>>(c->layers_dev, c->in_hw_dev, layer_end, c->S, c->max_regions,
-                                             in, n_in, c->table);
+    {
+        dc_prof_scope ps(c, DC_ST_PROPAGATE);
+        k_propagate<<<grid, 128, 0, c->stream>>>(c->layers_dev, c->in_hw_dev, layer_end, c->S, c->max_regions,
+                                                 in, n_in, c->table);
+    }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -190,9 +194,10 @@ int dc_launch_classify_copy(dc_cache* c, int layer, const dc_region* regions, co
     a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y; a.S = c->S;
     a.masks = L.masks; a.dirty_list = L.dirty_list; a.dirty_count = c->dirty_count + layer;
     a.reuse_px = c->reuse_px + (size_t)layer * c->S;
+    a.reused_total = c->reused_total + layer;
     // the caller has zeroed dirty_count[layer] and reuse_px[layer][*] on the stream
     int tiles = L.tiles_x * L.tiles_y * c->S;
-    k_classify_copy<<<dc_div_up(tiles, 8), 256, 0, c->stream>>>(a);
+    { dc_prof_scope ps(c, DC_ST_CLASSIFY_COPY); k_classify_copy<<<dc_div_up(tiles, 8), 256, 0, c->stream>>>(a); }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
