@@ -1,9 +1,389 @@
-// Tensor-core partial convolution (bf16): placeholder until the tcgen05 kernel lands.
+// Partial convolution on the 5th-generation tensor cores (bf16 in, fp32 accumulate in TMEM).
+//
+// Section 5, "Reuse", third step: convolve only what the cache did not supply.  The unit of
+// work is one dirty 8x16 output tile (128 pixels = the M of one tcgen05.mma) times one block of
+// BN output channels.  It is an implicit GEMM: for every kernel tap (ky, kx) and every chunk of
+// BK input channels, TMA fetches
+//     A: the 8x16 window of the NHWC input map displaced by the tap (a 4-D box; coordinates
+//        outside the map are zero-filled, which is the convolution's padding), 128 rows x BK
+//     B: BN rows x BK of the weights, which are already K-major as [cout][kh][kw][cin]
+// into 128-byte-swizzled shared memory, and one elected thread issues BK/16 tcgen05.mma
+// (M = 128, N = BN, K = 16) accumulating into tensor memory.
+//
+// Warp roles in a CTA of 192 threads (persistent, one CTA per SM):
+//     warp 0      TMA producer             (full/empty mbarrier ring of `stages` slots)
+//     warp 1      TMEM allocation, MMA issue, tcgen05.commit
+//     warps 2-5   epilogue: tcgen05.ld of their 32-lane quadrant, + bias, ReLU, bf16, and a
+//                 store predicated on the tile's reuse bitmap (only non-reused pixels are written)
+// Two accumulators (2 x BN TMEM columns) let the epilogue of one work item overlap the MMAs of
+// the next.  Every mbarrier wait is bounded: on expiry the kernel records DC_ERR_TIMEOUT in the
+// status word, all roles leave their loops, tensor memory is freed and the kernel returns.
+#include <cuda.h>
+#include <stdlib.h>
+
 #include "dc_common.cuh"
 
-int dc_conv_bf16_supported(const dc_cache*, int) { return 0; }
-int dc_launch_conv_bf16(dc_cache*, int, const void*, void*, const int32_t*, const int32_t*, const uint32_t*, int)
+namespace {
+
+constexpr int kThreads = 192;
+constexpr int kMaxStages = 8;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
+
+struct TcArgs {
+    const float* bias; __nv_bfloat16* out;
+    const int32_t* tile_list; const int32_t* tile_count; const uint32_t* masks;
+    int Ho, Wo, Co, Ci, kh, kw, sh, sw, ph, pw, relu, tiles_x, tiles_y;
+    int BN, NB, BK, kchunks, stages, a_bytes, b_bytes;
+    uint32_t idesc, sbo, layout_type;
+    int32_t* status;
+};
+
+struct SmemCtl {
+    unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2];
+    uint32_t tmem_base;
+    volatile int abort_flag;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(void* bar, uint32_t count)
 {
-    return DC_ERR_CONFIG;
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
 }
-int dc_pack_weights_bf16(dc_cache*, int) { return DC_OK; }
+__device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(void* bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(void* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long now_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait.  Returns false (and raises the abort flag + status word) when the limit passes
+// or another role has already given up.
+__device__ __forceinline__ bool mbar_wait(void* bar, uint32_t parity, SmemCtl* ctl, int32_t* status)
+{
+    if (mbar_try(bar, parity)) return true;
+    const unsigned long long t0 = now_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try(bar, parity)) return true;
+        if ((spin & 255u) == 0) {
+            if (ctl->abort_flag) return false;
+            if (now_ns() - t0 > kWaitLimitNs) {
+                ctl->abort_flag = 1;
+                atomicExch(status, (int)DC_ERR_TIMEOUT);
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, void* bar)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int c0, int c1, void* bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
+}
+
+// K-major operand tile in swizzled shared memory: rows of BK bf16, 8-row groups `sbo` bytes apart
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t sbo, uint32_t layout_type)
+{
+    uint32_t lo = ((saddr >> 4) & 0x3FFFu) | (1u << 16);                       // start address, LBO = 16 B (unused)
+    uint32_t hi = ((sbo >> 4) & 0x3FFFu) | (1u << 14) | (layout_type << 29);   // SBO, descriptor version 1, swizzle
+    return ((uint64_t)hi << 32) | lo;
+}
+__device__ __forceinline__ void umma_f16(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(void* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r)
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                 "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+                 "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const int n_items = *a.tile_count * a.NB;
+    if ((int)blockIdx.x >= n_items) return;
+
+    // operand ring at a 1024-byte boundary (the swizzle pattern repeats every 1024 bytes), then control words
+    uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int stage_bytes = a.a_bytes + a.b_bytes;
+    SmemCtl* ctl = (SmemCtl*)(ring + (size_t)a.stages * stage_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per_stream = a.tiles_x * a.tiles_y;
+    const int taps = a.kh * a.kw, kiters = taps * a.kchunks;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < a.stages; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 128); }
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
+    }
+    if (warp == 1) {       // 512 columns: two accumulators of up to 256 columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- TMA producer ----------------
+        uint32_t it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const int tile = a.tile_list[item / a.NB], nb = item % a.NB;
+            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+            const int x_base = tx * DC_TILE_W * a.sw - a.pw, y_base = ty * DC_TILE_H * a.sh - a.ph;
+            for (int k = 0; k < kiters && ok; ++k, ++it) {
+                const int tap = k / a.kchunks, cc = k - tap * a.kchunks, ky = tap / a.kw, kx = tap - ky * a.kw;
+                const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
+                if (lane == 0) {
+                    ok = mbar_wait(&ctl->empty[st], ph ^ 1u, ctl, a.status);
+                    if (ok) {
+                        uint8_t* sa = ring + (size_t)st * stage_bytes;
+                        mbar_expect_tx(&ctl->full[st], (uint32_t)stage_bytes);
+                        tma_load_4d(sa, &tmA, cc * a.BK, x_base + kx, y_base + ky, s, &ctl->full[st]);
+                        tma_load_2d(sa + a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, nb * a.BN, &ctl->full[st]);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+            }
+        }
+        // on an abort: give the copies already issued a bounded chance to land before the CTA exits
+        if (!ok && lane == 0) {
+            const unsigned long long t0 = now_ns();
+            while (now_ns() - t0 < 2000000ull) { }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer ----------------
+        uint32_t it = 0, acc_it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
+            const uint32_t acc = acc_it & 1u, acc_ph = (acc_it >> 1) & 1u;
+            const uint32_t d_tmem = tmem_base + acc * (uint32_t)a.BN;
+            if (lane == 0) {
+                ok = mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1u, ctl, a.status);
+                tc_fence_after();
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            for (int k = 0; k < kiters && ok; ++k, ++it) {
+                const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
+                if (lane == 0) {
+                    ok = mbar_wait(&ctl->full[st], ph, ctl, a.status);
+                    if (ok) {
+                        tc_fence_after();
+                        const uint32_t sa = smem_u32(ring + (size_t)st * stage_bytes);
+                        const uint64_t adesc = umma_desc(sa, a.sbo, a.layout_type);
+                        const uint64_t bdesc = umma_desc(sa + a.a_bytes, a.sbo, a.layout_type);
+                        for (int kk = 0; kk < a.BK / 16; ++kk)       // 16 bf16 = 32 bytes = 2 descriptor units
+                            umma_f16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, a.idesc, (k | kk) != 0);
+                        umma_commit(&ctl->empty[st]);                // frees the slot when these MMAs retire
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+            }
+            if (lane == 0 && ok) umma_commit(&ctl->tmem_full[acc]);
+            __syncwarp();
+        }
+    } else {
+        // ---------------- epilogue ----------------
+        const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
+        const int m = q * 32 + lane, prow = m / DC_TILE_W, pcol = m % DC_TILE_W;
+        uint32_t acc_it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
+            const uint32_t acc = acc_it & 1u, acc_ph = (acc_it >> 1) & 1u;
+            const int tile = a.tile_list[item / a.NB], nb = item % a.NB;
+            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+            const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
+            const uint32_t mword = a.masks[(size_t)tile * 4 + (prow >> 1)];
+            const bool reused = (mword >> ((prow & 1) * 16 + pcol)) & 1u;
+            const bool active = oy < a.Ho && ox < a.Wo && !reused;
+            __nv_bfloat16* op = a.out + (((size_t)s * a.Ho + oy) * a.Wo + ox) * a.Co + nb * a.BN;
+            const float* bias = a.bias + nb * a.BN;
+            ok = mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, a.status);
+            ok = __all_sync(0xffffffffu, ok);
+            if (!ok) break;
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)a.BN;
+            for (int c = 0; c < a.BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(taddr + c * 32, r);
+                tmem_ld_wait();
+                if (active) {
+                    uint4* dst = (uint4*)(op + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 4; ++v) {
+                        float f[8];
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) {
+                            f[j] = __uint_as_float(r[v * 8 + j]) + __ldg(bias + c * 32 + v * 8 + j);
+                            if (a.relu) f[j] = fmaxf(f[j], 0.f);
+                        }
+                        dst[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                    }
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(&ctl->tmem_empty[acc]);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn encode_fn()
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+        cudaGetLastError();
+    }
+    return fn;
+}
+
+struct TcPlan { int BK, BN, NB, stages, a_bytes, b_bytes; CUtensorMapSwizzle swz; uint32_t layout_type, sbo; size_t smem; };
+
+bool make_plan(const dc_layer_desc& d, TcPlan& p)
+{
+    if (d.kind != DC_CONV) return false;
+    if (d.sh != 1 || d.sw != 1) return false;                   // strided layers use the CUDA-core kernel
+    if (d.cin % 64 == 0) { p.BK = 64; p.swz = CU_TENSOR_MAP_SWIZZLE_128B; p.layout_type = 2; }
+    else if (d.cin % 32 == 0) { p.BK = 32; p.swz = CU_TENSOR_MAP_SWIZZLE_64B; p.layout_type = 4; }
+    else if (d.cin % 16 == 0) { p.BK = 16; p.swz = CU_TENSOR_MAP_SWIZZLE_32B; p.layout_type = 6; }
+    else return false;
+    p.BN = 0;
+    for (int bn = 256; bn >= 32; bn -= 32) if (d.cout % bn == 0) { p.BN = bn; break; }
+    if (!p.BN) return false;
+    p.NB = d.cout / p.BN;
+    p.a_bytes = DC_TILE_PX * p.BK * 2;
+    p.b_bytes = p.BN * p.BK * 2;
+    p.sbo = 8 * p.BK * 2;
+    if (p.b_bytes % 1024 != 0) return false;                    // keep every operand tile on a swizzle-pattern boundary
+    int st = (200 * 1024) / (p.a_bytes + p.b_bytes);
+    p.stages = st > kMaxStages ? kMaxStages : st;
+    if (p.stages < 2) return false;
+    p.smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + sizeof(SmemCtl) + 1024;
+    return true;
+}
+
+}  // namespace
+
+int dc_conv_bf16_supported(const dc_cache* c, int layer)
+{
+    TcPlan p;
+    if (getenv("DC_NO_TENSOR_CORES")) return 0;
+    return c->cfg.dtype == DC_BF16 && encode_fn() != nullptr && make_plan(c->L[layer].d, p);
+}
+
+int dc_pack_weights_bf16(dc_cache*, int) { return DC_OK; }       // [cout][kh][kw][cin] is already K-major
+
+int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
+                        const int32_t* tile_count, const uint32_t* masks, int max_tiles)
+{
+    dc_layer_rt& L = c->L[layer];
+    const dc_layer_desc& d = L.d;
+    TcPlan p;
+    if (!make_plan(d, p)) return DC_ERR_CONFIG;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return DC_ERR_CUDA;
+    CUtensorMap tmA, tmB;
+    {   // input map [S][Hi][Wi][Ci] bf16; box = BK channels x 16 columns x 8 rows x 1 stream
+        cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
+        cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
+        cuuint32_t box[4] = {(cuuint32_t)p.BK, DC_TILE_W, DC_TILE_H, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, p.swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return DC_ERR_CUDA;
+    }
+    {   // weights [cout][K] bf16, K = kh * kw * cin
+        const cuuint64_t K = (cuuint64_t)d.kh * d.kw * d.cin;
+        cuuint64_t dims[2] = {K, (cuuint64_t)d.cout};
+        cuuint64_t strides[1] = {K * 2};
+        cuuint32_t box[2] = {(cuuint32_t)p.BK, (cuuint32_t)p.BN};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L.weight, dims, strides, box, estr,
+                CU_TENSOR_MAP_INTERLEAVE_NONE, p.swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return DC_ERR_CUDA;
+    }
+    TcArgs a;
+    a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
+    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = d.sh; a.sw = d.sw;
+    a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
+    a.BN = p.BN; a.NB = p.NB; a.BK = p.BK; a.kchunks = d.cin / p.BK; a.stages = p.stages;
+    a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.sbo = p.sbo; a.layout_type = p.layout_type;
+    // instruction descriptor: D = f32, A = B = bf16, both K-major, N = BN, M = 128
+    a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    a.status = c->status;
+    static bool attr_set = false;
+    if (!attr_set) {
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    long long items = (long long)(max_tiles < 1 ? 1 : max_tiles) * p.NB;
+    int grid = items > 148 ? 148 : (int)items;
+    dc_prof_scope ps(c, DC_ST_CONV);
+    k_conv_tc<<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
+    c->launches += 1;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
