@@ -105,13 +105,22 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     // cached key frames: own pitch (16-byte multiple, at least 16 spare bytes per row and a spare
     // tail) so the matcher may fetch whole aligned words around any candidate
     c->key_pitch = ((size_t)cfg.width * 3 + 16 + 15) / 16 * 16;
-    DC_TRY(dev_alloc(c, &c->key, c->key_pitch * cfg.height * S + 256));
-    DC_CUDA(cudaMemsetAsync(c->key, 0, c->key_pitch * cfg.height * S + 256, c->stream));
+    for (int k = 0; k < 2; ++k) {
+        DC_TRY(dev_alloc(c, &c->key[k], c->key_pitch * cfg.height * S + 256));
+        DC_CUDA(cudaMemsetAsync(c->key[k], 0, c->key_pitch * cfg.height * S + 256, c->stream));
+    }
+    {
+        int dev = 0, sms = 148;
+        DC_CUDA(cudaGetDevice(&dev));
+        DC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+        c->num_sms = sms;
+    }
     const size_t nblk = (size_t)S * c->Gx * c->Gy;
     DC_TRY(dev_alloc(c, &c->blk_mv, nblk * 2));
     DC_TRY(dev_alloc(c, &c->blk_sse, nblk));
     DC_TRY(dev_alloc(c, &c->matched, nblk));
-    DC_TRY(dev_alloc(c, &c->mv_acc, (size_t)S * 4));
+    DC_TRY(dev_alloc(c, &c->mv_acc, (size_t)S * 4 + 4));
+    DC_TRY(dev_alloc(c, &c->long_list, nblk));
     DC_TRY(dev_alloc(c, &c->gmv, (size_t)S * 3));
     DC_TRY(dev_alloc(c, &c->regions0, (size_t)S * c->max_regions));
     DC_TRY(dev_alloc(c, &c->n_regions, (size_t)S));
@@ -204,8 +213,8 @@ void release(dc_cache* c)
 {
     dc_prof_release(c);
     cudaFree(c->reused_total);
-    cudaFree(c->key); cudaFree(c->staging); cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched);
-    cudaFree(c->mv_acc); cudaFree(c->gmv); cudaFree(c->regions0); cudaFree(c->n_regions); cudaFree(c->table);
+    cudaFree(c->key[0]); cudaFree(c->key[1]); cudaFree(c->staging); cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched);
+    cudaFree(c->mv_acc); cudaFree(c->long_list); cudaFree(c->gmv); cudaFree(c->regions0); cudaFree(c->n_regions); cudaFree(c->table);
     cudaFree(c->layers_dev); cudaFree(c->in_hw_dev); cudaFree(c->dirty_count); cudaFree(c->all_count);
     cudaFree(c->reuse_px); cudaFree(c->zero_masks); cudaFree(c->status); cudaFree(c->input_map); cudaFree(c->pix_lut);
     if (c->stats_pinned) cudaFreeHost(c->stats_pinned);
@@ -314,8 +323,7 @@ int dc_cache_launches(const dc_cache* c, int64_t* launches)
 int dc_cache_set_key(dc_cache* c, const uint8_t* frame_dev, size_t pitch)
 {
     if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
-    DC_CUDA(cudaMemcpy2DAsync(c->key, c->key_pitch, frame_dev, pitch, (size_t)c->cfg.width * 3,
-                              (size_t)c->cfg.height * c->S, cudaMemcpyDeviceToDevice, c->stream));
+    DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, c->key[c->key_cur]));
     c->key_valid = true;
     return DC_OK;
 }
@@ -326,7 +334,8 @@ int dc_match_blocks(dc_cache* c, const uint8_t* frame_dev, size_t pitch, int16_t
 {
     if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
     if (!c->key_valid) return DC_ERR_STATE;
-    DC_TRY(dc_launch_match(c, frame_dev, pitch));
+    DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, c->key[c->key_cur ^ 1]));   // scratch copy; the cache key stays
+    DC_TRY(dc_launch_match(c));
     const size_t nblk = (size_t)c->S * c->Gx * c->Gy;
     const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
     if (block_mv_dev) DC_CUDA(cudaMemcpyAsync(block_mv_dev, c->blk_mv, nblk * 2 * sizeof(int16_t), k, c->stream));
@@ -380,13 +389,16 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
     const int n = c->n_layers, S = c->S;
     // Section 5: the cache is dropped and a whole new frame computed every N frames
     const bool refresh = !c->key_valid || (c->frame_idx % c->cfg.expire_n) == 0;
+    // the library's own aligned copy of the frame: matched now, the cache key of the next frame (Section 3)
+    uint8_t* frame_copy = c->key[c->key_cur ^ 1];
+    DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, frame_copy));
     if (!refresh) {
         DC_CUDA(cudaMemsetAsync(c->dirty_count, 0, sizeof(int32_t) * n, c->stream));
         DC_CUDA(cudaMemsetAsync(c->reuse_px, 0, sizeof(int32_t) * n * S, c->stream));
-        DC_TRY(dc_launch_match(c, frame_dev, pitch));
+        DC_TRY(dc_launch_match(c));
         DC_TRY(dc_launch_propagate(c, c->regions0, c->n_regions, n));
     }
-    if (c->input_map) DC_TRY(dc_launch_input_map(c, frame_dev, pitch));
+    if (c->input_map) DC_TRY(dc_launch_input_map(c, frame_copy, c->key_pitch));
     const size_t per_layer = (size_t)S * c->max_regions;
     for (int i = 0; i < n; ++i) {
         dc_layer_rt& L = c->L[i];
@@ -407,16 +419,11 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
         case DC_MAXPOOL: DC_TRY(dc_launch_maxpool(c, i, in)); break;
         case DC_ADD: DC_TRY(dc_launch_add(c, i, in, layer_input(c, L.d.in1))); break;
         case DC_RELU: DC_TRY(dc_launch_relu(c, i, in)); break;
-        case DC_RESIZE_AREA: DC_TRY(dc_launch_resize(c, i, frame_dev, pitch)); break;
+        case DC_RESIZE_AREA: DC_TRY(dc_launch_resize(c, i, frame_copy, c->key_pitch)); break;
         default: return DC_ERR_STATE;
         }
     }
-    // the frame becomes the next cache key (Section 3)
-    {
-        dc_prof_scope ps(c, DC_ST_KEY_UPDATE);
-        DC_CUDA(cudaMemcpy2DAsync(c->key, c->key_pitch, frame_dev, pitch, (size_t)c->cfg.width * 3,
-                                  (size_t)c->cfg.height * S, cudaMemcpyDeviceToDevice, c->stream));
-    }
+    c->key_cur ^= 1;             // the frame becomes the next cache key
     c->key_valid = true;
     c->frame_idx += 1;
     if (refresh) c->frames_full += 1; else c->frames_cached += 1;

@@ -39,7 +39,6 @@ struct dc_layer_rt {
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation
     int32_t* all_list;              // conv: every tile (used by full frames)
-    int32_t* zero_masks_unused;
 };
 
 struct dc_cache {
@@ -55,15 +54,18 @@ struct dc_cache {
     int64_t launches;
     size_t bytes;
 
-    uint8_t* key;                   // cached previous frames [S][H][key_pitch]
+    uint8_t* key[2];                // key frames [S][H][key_pitch]: key[key_cur] is the cached previous
+    int key_cur;                    // frame, the other one receives the frame being processed
     size_t key_pitch;
+    int num_sms;
     uint8_t* staging;               // device copy of host frames for dc_infer_frame_host
     uint32_t sse_limit[4];          // PSNR test as an SSE bound, index = 2 * (bottom edge) + (right edge)
 
     int16_t* blk_mv;                // [S][Gy][Gx][2]
     uint32_t* blk_sse;              // [S][Gy][Gx]
     uint8_t* matched;               // [S][Gy][Gx]
-    int32_t* mv_acc;                // [S][4]: sum dx, sum dy, K, n_matched
+    int32_t* mv_acc;                // [S][4]: sum dx, sum dy, K, n_matched; then 4 words of counters
+    uint4* long_list;               // [S][Gy][Gx] diamond walks handed to the second search phase
     int32_t* gmv;                   // [S][3]: Mx, My, K
     dc_region* regions0;            // [S][max_regions] rectangles on the frame
     int32_t* n_regions;             // [S]
@@ -93,14 +95,15 @@ struct dc_prof_scope {
 static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }
 
 // ---- kernels' host-side launchers (each returns DC_OK or DC_ERR_CUDA) ----
-int dc_launch_match(dc_cache* c, const uint8_t* frame, size_t pitch);
+int dc_launch_copy_frame(dc_cache* c, const uint8_t* frame, size_t pitch, uint8_t* dst);
+int dc_launch_match(dc_cache* c);      // current frame = key[key_cur ^ 1], previous = key[key_cur]
 int dc_launch_propagate(dc_cache* c, const dc_region* in, const int32_t* n_in, int layer_end);
 int dc_launch_classify_copy(dc_cache* c, int layer, const dc_region* regions, const int32_t* n_regions,
                             const void* prev_out, void* out);
 int dc_launch_conv(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
                    const int32_t* tile_count, const uint32_t* masks, int max_tiles);
 int dc_launch_input_map(dc_cache* c, const uint8_t* frame, size_t pitch);
-int dc_launch_resize(dc_cache* c, int layer, const uint8_t* frame, size_t pitch);
+int dc_launch_resize(dc_cache* c, int layer, const uint8_t* frame, size_t pitch);   // frame: 16-byte aligned rows
 int dc_launch_maxpool(dc_cache* c, int layer, const void* in);
 int dc_launch_add(dc_cache* c, int layer, const void* a, const void* b);
 int dc_launch_relu(dc_cache* c, int layer, const void* a);

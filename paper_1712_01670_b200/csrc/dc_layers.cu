@@ -41,33 +41,92 @@ __global__ void k_input_map(const uint8_t* frame, size_t pitch, int W, int H, in
 }
 
 // Box average of the frame: output (oy, ox) is the mean over rows [floor(oy H / Ho),
-// ceil((oy + 1) H / Ho) - 1] and the like columns, divided by 255.  One warp per output pixel;
-// lanes stride over the source bytes of each span row (contiguous), integer sums.
+// ceil((oy + 1) H / Ho) - 1] and the like columns, divided by 255.  One CTA per output row:
+// pass 1 sums the span's source rows column-wise with coalesced 16-byte loads (row starts are
+// 16-byte aligned in the library's frame copy) into shared memory; pass 2 sums each output's
+// column span.  All sums are integers; the one division is done in double.
 template <typename T>
 __global__ void __launch_bounds__(256) k_resize_area(const uint8_t* frame, size_t pitch, int W, int H, int S,
                                                      int Wo, int Ho, T* out)
 {
-    const int lane = threadIdx.x & 31;
-    const long long wid = (long long)blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (wid >= (long long)S * Ho * Wo) return;
-    int ox = (int)(wid % Wo); long long t = wid / Wo; int oy = (int)(t % Ho); int s = (int)(t / Ho);
-    int y0 = (int)((long long)oy * H / Ho), y1 = (int)(((long long)(oy + 1) * H + Ho - 1) / Ho) - 1;
-    int x0 = (int)((long long)ox * W / Wo), x1 = (int)(((long long)(ox + 1) * W + Wo - 1) / Wo) - 1;
-    const uint8_t* base = frame + ((size_t)s * H + y0) * pitch + (size_t)x0 * 3;
-    const int nb = (x1 - x0 + 1) * 3, rows = y1 - y0 + 1;
-    uint32_t c0 = 0, c1 = 0, c2 = 0;
-    for (int i = lane; i < nb * rows; i += 32) {
-        int r = i / nb, b = i - r * nb;
-        uint32_t v = base[(size_t)r * pitch + b];
-        int ch = b % 3;
-        c0 += ch == 0 ? v : 0; c1 += ch == 1 ? v : 0; c2 += ch == 2 ? v : 0;
+    extern __shared__ uint16_t colsum[];                       // [ceil16(W * 3)]
+    const int oy = blockIdx.x % Ho, s = blockIdx.x / Ho;
+    const int y0 = (int)((long long)oy * H / Ho), y1 = (int)(((long long)(oy + 1) * H + Ho - 1) / Ho) - 1;
+    const int row_bytes = W * 3, chunks = (row_bytes + 15) >> 4;
+    const uint8_t* base = frame + ((size_t)s * H + y0) * pitch;
+    for (int c = threadIdx.x; c < chunks; c += blockDim.x) {
+        uint32_t acc[8] = {0, 0, 0, 0, 0, 0, 0, 0};            // 16 byte columns as 8 pairs of 16-bit sums
+        for (int y = 0; y <= y1 - y0; ++y) {
+            const uint4 v = __ldg((const uint4*)(base + (size_t)y * pitch + c * 16));
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                acc[2 * k] += __byte_perm(w[k], 0, 0x4140);    // bytes 0, 1 -> two 16-bit lanes
+                acc[2 * k + 1] += __byte_perm(w[k], 0, 0x4342);
+            }
+        }
+        uint4* dst = (uint4*)(colsum + c * 16);
+        dst[0] = make_uint4(acc[0], acc[1], acc[2], acc[3]);
+        dst[1] = make_uint4(acc[4], acc[5], acc[6], acc[7]);
     }
-    c0 = __reduce_add_sync(0xffffffffu, c0); c1 = __reduce_add_sync(0xffffffffu, c1);
-    c2 = __reduce_add_sync(0xffffffffu, c2);
-    if (lane < 3) {
-        uint32_t sum = lane == 0 ? c0 : (lane == 1 ? c1 : c2);
-        double mean = (double)sum / ((double)(rows * (x1 - x0 + 1)) * 255.0);
-        out[(size_t)wid * 3 + lane] = from_d<T>(mean);
+    __syncthreads();
+    const int rows = y1 - y0 + 1;
+    for (int t = threadIdx.x; t < Wo * 3; t += blockDim.x) {
+        const int ox = t / 3, ch = t - ox * 3;
+        const int x0 = (int)((long long)ox * W / Wo), x1 = (int)(((long long)(ox + 1) * W + Wo - 1) / Wo) - 1;
+        uint32_t sum = 0;
+        for (int x = x0; x <= x1; ++x) sum += colsum[x * 3 + ch];
+        const double mean = (double)sum / ((double)(rows * (x1 - x0 + 1)) * 255.0);
+        out[(((size_t)s * Ho + oy) * Wo + ox) * 3 + ch] = from_d<T>(mean);
+    }
+}
+
+// 8 (bf16) or 4 (float) channels per thread with 16-byte loads; C must be a multiple of that.
+template <typename T> struct Vec16;
+template <> struct Vec16<float> {
+    static constexpr int N = 4;
+    static __device__ __forceinline__ uint4 vmax(uint4 a, uint4 b)
+    {
+        return make_uint4(__float_as_uint(fmaxf(__uint_as_float(a.x), __uint_as_float(b.x))),
+                          __float_as_uint(fmaxf(__uint_as_float(a.y), __uint_as_float(b.y))),
+                          __float_as_uint(fmaxf(__uint_as_float(a.z), __uint_as_float(b.z))),
+                          __float_as_uint(fmaxf(__uint_as_float(a.w), __uint_as_float(b.w))));
+    }
+};
+template <> struct Vec16<__nv_bfloat16> {
+    static constexpr int N = 8;
+    static __device__ __forceinline__ uint32_t m2(uint32_t a, uint32_t b)
+    {
+        __nv_bfloat162 r = __hmax2(*reinterpret_cast<__nv_bfloat162*>(&a), *reinterpret_cast<__nv_bfloat162*>(&b));
+        return *reinterpret_cast<uint32_t*>(&r);
+    }
+    static __device__ __forceinline__ uint4 vmax(uint4 a, uint4 b) { return make_uint4(m2(a.x, b.x), m2(a.y, b.y), m2(a.z, b.z), m2(a.w, b.w)); }
+};
+
+template <typename T>
+__global__ void k_maxpool_vec(const T* in, int Hi, int Wi, int C, int S, dc_layer_desc L, T* out)
+{
+    constexpr int N = Vec16<T>::N;
+    const int cv = C / N;
+    const size_t total = (size_t)S * L.out_h * L.out_w * cv;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        int c = (int)(i % cv); size_t t = i / cv;
+        int ox = (int)(t % L.out_w); t /= L.out_w;
+        int oy = (int)(t % L.out_h); int s = (int)(t / L.out_h);
+        uint4 m = make_uint4(0, 0, 0, 0);
+        bool first = true;
+        for (int ky = 0; ky < L.kh; ++ky) {
+            int iy = oy * L.sh - L.ph + ky;
+            if (iy < 0 || iy >= Hi) continue;
+            for (int kx = 0; kx < L.kw; ++kx) {
+                int ix = ox * L.sw - L.pw + kx;
+                if (ix < 0 || ix >= Wi) continue;
+                uint4 v = __ldg((const uint4*)(in + (((size_t)s * Hi + iy) * Wi + ix) * C) + c);
+                m = first ? v : Vec16<T>::vmax(m, v);
+                first = false;
+            }
+        }
+        *((uint4*)(out + i / cv * C) + c) = m;
     }
 }
 
@@ -132,12 +191,13 @@ int dc_launch_input_map(dc_cache* c, const uint8_t* frame, size_t pitch)
 int dc_launch_resize(dc_cache* c, int layer, const uint8_t* frame, size_t pitch)
 {
     dc_layer_rt& L = c->L[layer];
-    long long warps = (long long)c->S * L.d.out_h * L.d.out_w;
-    int grid = (int)((warps + 7) / 8);
+    int grid = c->S * L.d.out_h;
+    size_t smem = (size_t)((c->cfg.width * 3 + 15) / 16) * 16 * sizeof(uint16_t);
+    if (smem > 48 * 1024 || (size_t)c->cfg.height > 255u * (size_t)L.d.out_h) return DC_ERR_CONFIG;   // 16-bit column sums
     dc_prof_scope ps(c, DC_ST_INPUT);
     DISPATCH(c,
-        (k_resize_area<float><<<grid, 256, 0, c->stream>>>(frame, pitch, c->cfg.width, c->cfg.height, c->S, L.d.out_w, L.d.out_h, (float*)L.map[0])),
-        (k_resize_area<__nv_bfloat16><<<grid, 256, 0, c->stream>>>(frame, pitch, c->cfg.width, c->cfg.height, c->S, L.d.out_w, L.d.out_h, (__nv_bfloat16*)L.map[0])));
+        (k_resize_area<float><<<grid, 256, smem, c->stream>>>(frame, pitch, c->cfg.width, c->cfg.height, c->S, L.d.out_w, L.d.out_h, (float*)L.map[0])),
+        (k_resize_area<__nv_bfloat16><<<grid, 256, smem, c->stream>>>(frame, pitch, c->cfg.width, c->cfg.height, c->S, L.d.out_w, L.d.out_h, (__nv_bfloat16*)L.map[0])));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -148,6 +208,15 @@ int dc_launch_maxpool(dc_cache* c, int layer, const void* in)
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
     dc_prof_scope ps(c, DC_ST_POINTWISE);
+    if ((L.d.cout * c->elt) % 16 == 0) {
+        size_t nv = n * c->elt / 16;
+        DISPATCH(c,
+            (k_maxpool_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)L.map[0])),
+            (k_maxpool_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)L.map[0])));
+        c->launches += 1;
+        DC_CUDA(cudaGetLastError());
+        return DC_OK;
+    }
     DISPATCH(c,
         (k_maxpool<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)L.map[0])),
         (k_maxpool<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)L.map[0])));

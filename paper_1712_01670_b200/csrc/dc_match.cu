@@ -5,7 +5,12 @@
 //              (two aligned loads + funnel shift), |a-b| per byte by vabsdiff4, squares summed
 //              by dp4a, warp-reduced.  Candidates are ordered by (SSE, |dx|+|dy|, dy, dx).
 //              Blocks that pass the PSNR bound add their vector to the Step 3 sums.
-//   k_verify   Steps 3-4: rounds the mean vector M, scores every block at M.
+//   k_search_ds16  Step 2 for 16-pixel blocks with diamond search (the common case): one CTA per strip
+//              of 8 blocks, the previous frame's window (+-10 px) staged once in shared memory,
+//              each lane owns one block row, the two half-warps score two candidates at a time,
+//              and points already scored by the previous diamond are skipped (they cannot win).
+//   k_verify   Steps 3-4: rounds the mean vector M, scores every block at M (reusing the Step 2
+//              score when the block's own best vector is M).
 //   k_merge    Step 5: maximal horizontal runs, merged vertically when spans are identical,
 //              emitted in (y, x) order by a block-wide scan.
 #include "dc_common.cuh"
@@ -194,7 +199,10 @@ __global__ void __launch_bounds__(WARPS * 32) k_verify(MatchArgs a)
     if (K > 0) { Mx = round_mean(a.acc[4 * s + 0], K); My = round_mean(a.acc[4 * s + 1], K); }
     int ok = 0;
     if (K > 0 && c.valid(Mx, My)) {
-        uint32_t v = c.sse(Mx, My);
+        const size_t g = (size_t)s * a.Gx * a.Gy + b;
+        // Section 4: "if the PSNR between (x_i, y_i) and (x_i + M_x, y_i + M_y) is already calculated
+        // in Step 2, we simply reuse the result" -- exact when the block's best vector is M itself
+        uint32_t v = (a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My) ? a.sse[g] : c.sse(Mx, My);
         ok = v <= a.limit[limit_index(a, c.bw, c.bh)];
     }
     if (c.lane == 0) {
@@ -260,34 +268,381 @@ __global__ void __launch_bounds__(256) k_merge(const uint8_t* matched, const int
     if (tid == 0) n_regions[s] = min(base, max_regions);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Fast Steps 2 and 4: 16-pixel blocks, diamond search
+// ---------------------------------------------------------------------------------------------
+constexpr int F_WR = 10;                       // reach of a staged window around a block, pixels
+constexpr int F_ROWS = 16 + 2 * F_WR;          // window rows
+constexpr int F_WORDS = 120;                   // strip window row: (128 + 2 * 10) px * 3 B = 444 B + alignment slack
+constexpr int F_PITCH = 121;                   // odd word pitch: the 16 rows of a half-warp hit 16 banks
+constexpr int L_WORDS = 32;                    // private window row: (16 + 2 * 10) px * 3 B = 108 B + slack
+constexpr int L_PITCH = 33;
+
+// One block row (48 bytes) of the current frame per lane, masked for clipped edge blocks.
+struct RowCtx {
+    uint32_t cw[12], wm[12];
+    bool clipped, row_on;
+    __device__ __forceinline__ void load(const uint8_t* cur_row, int bw, bool on)
+    {
+        row_on = on; clipped = bw < 16;
+        const uint4* p = (const uint4*)cur_row;                // 16-byte aligned in the library's frame copy
+        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0, v2 = v0;
+        if (on) { v0 = __ldg(p); v1 = __ldg(p + 1); v2 = __ldg(p + 2); }
+        cw[0] = v0.x; cw[1] = v0.y; cw[2] = v0.z; cw[3] = v0.w; cw[4] = v1.x; cw[5] = v1.y; cw[6] = v1.z; cw[7] = v1.w;
+        cw[8] = v2.x; cw[9] = v2.y; cw[10] = v2.z; cw[11] = v2.w;
+#pragma unroll
+        for (int j = 0; j < 12; ++j) {
+            int nb = bw * 3 - 4 * j;
+            wm[j] = nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << (8 * nb)) - 1u));
+            cw[j] &= wm[j];
+        }
+    }
+    // partial SSE of this row against 13 consecutive words at q, the row starting sh bits into q[0]
+    template <typename P>
+    __device__ __forceinline__ uint32_t sse(P q, uint32_t sh) const
+    {
+        uint32_t w[13], acc[3] = {0, 0, 0};                     // three chains hide the dp4a latency
+#pragma unroll
+        for (int j = 0; j < 13; ++j) w[j] = q[j];
+        if (!clipped) {
+#pragma unroll
+            for (int j = 0; j < 12; ++j) {
+                uint32_t d = __vabsdiffu4(cw[j], __funnelshift_r(w[j], w[j + 1], sh));
+                acc[j % 3] = __dp4a(d, d, acc[j % 3]);
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 12; ++j) {
+                uint32_t d = __vabsdiffu4(cw[j], __funnelshift_r(w[j], w[j + 1], sh) & wm[j]);
+                acc[j % 3] = __dp4a(d, d, acc[j % 3]);
+            }
+        }
+        return acc[0] + acc[1] + acc[2];
+    }
+};
+
+// Search points relative to a centre, 4 bits per coordinate (value + 2):
+// 0-7 the large diamond, 8 the centre itself, 9-12 the small diamond.
+__device__ __forceinline__ void point_offset(int i, int& dx, int& dy)
+{
+    //            i :  0   1   2   3   4   5   6   7   8   9  10  11  12
+    //           dx :  0  -1   1  -2   2  -1   1   0   0   0  -1   1   0
+    //           dy : -2  -1  -1   0   0   1   1   2   0  -1   0   0   1
+    const unsigned long long X = 0x2312223140312ull;           // nibble i = dx + 2
+    const unsigned long long Y = 0x3221243322110ull;           // nibble i = dy + 2
+    dx = (int)((X >> (4 * i)) & 15) - 2;
+    dy = (int)((Y >> (4 * i)) & 15) - 2;
+}
+
+// The diamond walk of one block by one warp.  `Win` supplies the staged previous-frame pixels:
+//   reach(cx, cy)      true when every point a step around centre (cx, cy) may touch is staged
+//   row(r, dx, dy, sh) pointer to the words holding row r of the candidate displaced by (dx, dy)
+// Returns false when the walk must continue elsewhere (bk then holds the state to resume from).
+template <typename Win>
+__device__ __forceinline__ bool diamond_walk(const MatchArgs& a, const RowCtx& rc, Win& win, int x0, int y0, int bw,
+                                             int bh, int lane, bool resume, unsigned long long& bk)
+{
+    const int r = lane & 15, half = lane >> 4;
+    const unsigned hmask = half ? 0xffff0000u : 0x0000ffffu;
+    // Scores the points of `mask` (bit i = point i around centre (cx, cy)), two per pass: the lower
+    // half-warp takes one, the upper half-warp the next.  One call site keeps the code small.
+    auto score_points = [&](int cx, int cy, unsigned mask) {
+#pragma unroll 1
+        while (mask) {
+            const int i0 = __ffs(mask) - 1; mask &= mask - 1;
+            int i1 = -1;
+            if (mask) { i1 = __ffs(mask) - 1; mask &= mask - 1; }
+            const int i = half ? i1 : i0;
+            int dx = 0, dy = 0;
+            bool ok = i >= 0;
+            if (ok) {
+                point_offset(i, dx, dy);
+                dx += cx; dy += cy;
+                ok = abs(dx) <= a.R && abs(dy) <= a.R && x0 + dx >= 0 && y0 + dy >= 0 && x0 + dx + bw <= a.W && y0 + dy + bh <= a.H;
+            }
+            uint32_t acc = 0;
+            if (ok && rc.row_on) {
+                uint32_t sh;
+                const uint32_t* q = win.row(r, dx, dy, sh);
+                acc = rc.sse(q, sh);
+            }
+            const uint32_t sse = __reduce_add_sync(hmask, acc);
+            unsigned long long key = ok ? cand_key(sse, dx, dy) : ~0ull;
+            const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, 16);
+            key = key < other ? key : other;
+            bk = key < bk ? key : bk;
+        }
+    };
+    int cx, cy;
+    if (!resume) {
+        bk = ~0ull;
+        cx = 0; cy = 0;
+        score_points(0, 0, 0x1ffu);                               // the centre (0, 0) and its large diamond
+    } else {
+        // resumed walk: the best point so far is the centre; score its whole large diamond
+        cx = (int)(bk & 0xff) - 128; cy = (int)((bk >> 8) & 0xff) - 128;
+        if (!win.reach(cx, cy)) return false;
+        score_points(cx, cy, 0xffu);
+    }
+    const int max_steps = (2 * a.R + 1) * (2 * a.R + 1);          // every move strictly lowers the key
+#pragma unroll 1
+    for (int step = 0; step < max_steps; ++step) {
+        const int nx = (int)(bk & 0xff) - 128, ny = (int)((bk >> 8) & 0xff) - 128;
+        if (nx == cx && ny == cy) break;                           // the centre won: large diamond done
+        if (!win.reach(nx, ny)) return false;
+        const int mx = nx - cx, my = ny - cy;
+        cx = nx; cy = ny;
+        // points of the new diamond that the old one already scored lost to the new centre: skip them
+        unsigned mask = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            int qx, qy;
+            point_offset(i, qx, qy);
+            qx += mx; qy += my;                                    // position relative to the old centre
+            const bool known = (abs(qx) + abs(qy) == 2) || (qx == 0 && qy == 0);
+            if (!known) mask |= 1u << i;
+        }
+        score_points(cx, cy, mask);
+    }
+    score_points(cx, cy, 0x1e00u);                                // small diamond around the final centre
+    return true;
+}
+
+__device__ __forceinline__ void publish_block(const MatchArgs& a, int s, size_t g, int bw, int bh, unsigned long long bk)
+{
+    const int fx = (int)(bk & 0xff) - 128, fy = (int)((bk >> 8) & 0xff) - 128;
+    const uint32_t fs = (uint32_t)(bk >> 32);
+    a.mv[2 * g] = (int16_t)fx; a.mv[2 * g + 1] = (int16_t)fy; a.sse[g] = fs;
+    if (fs <= a.limit[limit_index(a, bw, bh)]) {              // PSNR > T: member of Step 3's set S
+        atomicAdd(&a.acc[4 * s + 0], fx);
+        atomicAdd(&a.acc[4 * s + 1], fy);
+        atomicAdd(&a.acc[4 * s + 2], 1);
+    }
+}
+
+// Window shared by the 8 blocks of a strip, centred on zero motion.
+struct StripWin {
+    const uint32_t* win; int x0, wx0;
+    __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx) + 2 <= F_WR && abs(cy) + 2 <= F_WR; }
+    __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
+    {
+        const int off = (x0 + dx) * 3 - wx0;
+        sh = (off & 3) * 8;
+        return win + (r + dy + F_WR) * F_PITCH + (off >> 2);
+    }
+};
+
+// Phase 1: one CTA per strip of 8 blocks.  A walk that leaves the strip window is handed to phase 2.
+__global__ void __launch_bounds__(256, 4) k_search_ds16(MatchArgs a, uint4* long_list, int32_t* long_count)
+{
+    __shared__ uint32_t win[F_ROWS * F_PITCH];
+    const int strips = (a.Gx + 7) >> 3;
+    const int strip = blockIdx.x % strips, by = (blockIdx.x / strips) % a.Gy, s = blockIdx.x / (strips * a.Gy);
+    const int xs = strip * 128, y0 = by * 16;
+    const int wx0 = ((xs - F_WR) * 3) & ~15;                  // byte column of the window origin (may be < 0)
+    const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
+    for (int i = threadIdx.x; i < F_ROWS * F_WORDS; i += 256) {
+        const int row = i / F_WORDS, wi = i - row * F_WORDS;
+        const int gy = y0 - F_WR + row, gb = wx0 + wi * 4;
+        uint32_t v = 0;
+        if (gy >= 0 && gy < a.H && gb >= 0 && gb < (int)a.prev_pitch)
+            v = __ldg((const uint32_t*)(prev + (size_t)gy * a.prev_pitch + gb));
+        win[row * F_PITCH + wi] = v;
+    }
+    __syncthreads();
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int bx = strip * 8 + warp;
+    if (bx >= a.Gx) return;
+    const int x0 = bx * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0), r = lane & 15;
+    RowCtx rc;
+    rc.load(a.cur + (size_t)s * a.cur_stream + (size_t)(y0 + r) * a.cur_pitch + (size_t)x0 * 3, bw, r < bh);
+    StripWin sw = {win, x0, wx0};
+    unsigned long long bk = 0;
+    const bool done = diamond_walk(a, rc, sw, x0, y0, bw, bh, lane, false, bk);
+    if (lane == 0) {
+        const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
+        if (done) publish_block(a, s, g, bw, bh, bk);
+        else long_list[atomicAdd(long_count, 1)] = make_uint4((uint32_t)g, (uint32_t)bk, (uint32_t)(bk >> 32), 0u);
+    }
+}
+
+// Private window of one warp, centred on (wcx, wcy) relative to the block.
+struct WarpWin {
+    uint32_t* win; const uint8_t* prev; size_t pitch; int H, x0, y0, wcx, wcy, wx0, lane;
+    __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx - wcx) + 2 <= F_WR && abs(cy - wcy) + 2 <= F_WR; }
+    __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
+    {
+        const int off = (x0 + dx) * 3 - wx0;
+        sh = (off & 3) * 8;
+        return win + (r + dy - wcy + F_WR) * L_PITCH + (off >> 2);
+    }
+    __device__ __forceinline__ void stage(int cx, int cy)
+    {
+        wcx = cx; wcy = cy;
+        wx0 = ((x0 + cx - F_WR) * 3) & ~15;
+        __syncwarp();
+        for (int row = 0; row < F_ROWS; ++row) {
+            static_assert(L_WORDS == 32, "one lane per window word");
+            const int gy = y0 + cy - F_WR + row, gb = wx0 + lane * 4;
+            uint32_t v = 0;
+            if (gy >= 0 && gy < H && gb >= 0 && gb < (int)pitch) v = __ldg((const uint32_t*)(prev + (size_t)gy * pitch + gb));
+            win[row * L_PITCH + lane] = v;
+        }
+        __syncwarp();
+    }
+};
+
+// Phase 2: the walks that left their strip window, one warp each, re-staging a private window
+// around the walk's centre whenever it nears the window's edge.
+__global__ void __launch_bounds__(256, 4) k_search_ds16_long(MatchArgs a, const uint4* long_list, const int32_t* long_count)
+{
+    __shared__ uint32_t win_all[8][F_ROWS * L_PITCH];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane & 15;
+    const int n = *long_count, per = a.Gx * a.Gy;
+    for (int i = blockIdx.x * 8 + warp; i < n; i += gridDim.x * 8) {
+        const uint4 e = long_list[i];
+        const size_t g = e.x;
+        unsigned long long bk = ((unsigned long long)e.z << 32) | e.y;
+        const int s = (int)(g / per), b = (int)(g - (size_t)s * per), by = b / a.Gx, bx = b - by * a.Gx;
+        const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
+        RowCtx rc;
+        rc.load(a.cur + (size_t)s * a.cur_stream + (size_t)(y0 + r) * a.cur_pitch + (size_t)x0 * 3, bw, r < bh);
+        WarpWin ww = {win_all[warp], a.prev + (size_t)s * a.prev_stream, a.prev_pitch, a.H, x0, y0, 0, 0, 0, lane};
+        const int limit = 4 * a.R + 8;                           // each re-staging moves the centre >= 8 px
+        bool done = false;
+        for (int round = 0; round < limit && !done; ++round) {
+            ww.stage((int)(bk & 0xff) - 128, (int)((bk >> 8) & 0xff) - 128);
+            done = diamond_walk(a, rc, ww, x0, y0, bw, bh, lane, true, bk);
+        }
+        __syncwarp();
+        if (lane == 0) publish_block(a, s, g, bw, bh, bk);
+    }
+}
+
+// Step 4 for 16-pixel blocks: one half-warp per block, one lane per block row.
+__global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
+{
+    const int lane = threadIdx.x & 31, r = lane & 15, half = lane >> 4;
+    const int per = a.Gx * a.Gy;
+    const long long gi = ((long long)blockIdx.x * 8 + (threadIdx.x >> 5)) * 2 + half;
+    const bool in_grid = gi < (long long)per * a.S;
+    const int s = in_grid ? (int)(gi / per) : 0, b = in_grid ? (int)(gi - (long long)s * per) : 0;
+    const int by = b / a.Gx, bx = b - by * a.Gx;
+    const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
+    const int K = a.acc[4 * s + 2];
+    int Mx = 0, My = 0;
+    if (K > 0) { Mx = round_mean(a.acc[4 * s + 0], K); My = round_mean(a.acc[4 * s + 1], K); }
+    const bool cand_ok = in_grid && K > 0 && abs(Mx) <= a.R && abs(My) <= a.R && x0 + Mx >= 0 && y0 + My >= 0 &&
+                         x0 + Mx + bw <= a.W && y0 + My + bh <= a.H;
+    const size_t g = (size_t)s * per + b;
+    // Section 4: reuse the Step 2 score when that step already scored this pair (best vector == M)
+    const bool known = cand_ok && a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My;
+    uint32_t acc = 0;
+    if (cand_ok && !known && r < bh) {
+        RowCtx rc;
+        rc.load(a.cur + (size_t)s * a.cur_stream + (size_t)(y0 + r) * a.cur_pitch + (size_t)x0 * 3, bw, true);
+        const uint8_t* p = a.prev + (size_t)s * a.prev_stream + (size_t)(y0 + My + r) * a.prev_pitch + (size_t)(x0 + Mx) * 3;
+        acc = rc.sse((const uint32_t*)((uintptr_t)p & ~(uintptr_t)3), ((uint32_t)(uintptr_t)p & 3u) * 8u);
+    }
+    const uint32_t sse = __reduce_add_sync(half ? 0xffff0000u : 0x0000ffffu, acc);
+    if (r == 0 && in_grid) {
+        const uint32_t v = known ? a.sse[g] : sse;
+        const int ok = cand_ok && v <= a.limit[limit_index(a, bw, bh)];
+        a.matched[g] = (uint8_t)ok;
+        if (ok) atomicAdd(&a.acc[4 * s + 3], 1);
+        if (b == 0) { a.gmv[3 * s] = Mx; a.gmv[3 * s + 1] = My; a.gmv[3 * s + 2] = K; }
+    }
+}
+
+// Frame -> the library's aligned copy.  16-byte vectors when the source rows are aligned.
+__global__ void k_copy_frame(const uint8_t* src, size_t src_pitch, uint8_t* dst, size_t dst_pitch, int row_bytes,
+                             int rows, int vec)
+{
+    if (vec) {
+        const int chunks = (row_bytes + 15) >> 4;             // the last chunk may read source padding? no: see below
+        const size_t total = (size_t)rows * chunks;
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+            const size_t row = i / chunks; const int c = (int)(i - row * chunks);
+            if (c * 16 + 16 <= row_bytes) {
+                *(uint4*)(dst + row * dst_pitch + c * 16) = __ldg((const uint4*)(src + row * src_pitch + c * 16));
+            } else {                                          // ragged tail of the row: byte by byte
+                for (int k = c * 16; k < row_bytes; ++k) dst[row * dst_pitch + k] = src[row * src_pitch + k];
+            }
+        }
+    } else {
+        const size_t total = (size_t)rows * row_bytes;
+        for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+            const size_t row = i / row_bytes; const int k = (int)(i - row * row_bytes);
+            dst[row * dst_pitch + k] = src[row * src_pitch + k];
+        }
+    }
+}
+
 template <int ITERS>
-int launch_all(dc_cache* c, MatchArgs& a)
+void launch_generic(dc_cache* c, MatchArgs& a, bool search)
 {
     int warps = a.S * a.Gx * a.Gy;
     int grid = dc_div_up(warps, WARPS);
-    { dc_prof_scope ps(c, DC_ST_SEARCH); k_search<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a); }
-    { dc_prof_scope ps(c, DC_ST_VERIFY); k_verify<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a); }
-    return 0;
+    if (search) { dc_prof_scope ps(c, DC_ST_SEARCH); k_search<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a); }
+    else { dc_prof_scope ps(c, DC_ST_VERIFY); k_verify<ITERS><<<grid, WARPS * 32, 0, c->stream>>>(a); }
+}
+
+void launch_by_block(dc_cache* c, MatchArgs& a, bool search)
+{
+    int row_words = (a.B * 3 + 3) / 4, iters = dc_div_up(a.B * row_words, 32);
+    if (iters <= 2) launch_generic<2>(c, a, search);
+    else if (iters <= 3) launch_generic<3>(c, a, search);
+    else if (iters <= 6) launch_generic<6>(c, a, search);
+    else if (iters <= 12) launch_generic<12>(c, a, search);
+    else launch_generic<24>(c, a, search);
 }
 
 }  // namespace
 
-int dc_launch_match(dc_cache* c, const uint8_t* frame, size_t pitch)
+int dc_launch_copy_frame(dc_cache* c, const uint8_t* frame, size_t pitch, uint8_t* dst)
+{
+    const int row_bytes = c->cfg.width * 3, rows = c->cfg.height * c->S;
+    const int vec = ((uintptr_t)frame % 16 == 0) && (pitch % 16 == 0);
+    size_t work = vec ? (size_t)rows * ((row_bytes + 15) / 16) : (size_t)rows * row_bytes;
+    int grid = (int)((work + 255) / 256);
+    if (grid > c->num_sms * 16) grid = c->num_sms * 16;
+    if (grid < 1) grid = 1;
+    dc_prof_scope ps(c, DC_ST_KEY_UPDATE);
+    k_copy_frame<<<grid, 256, 0, c->stream>>>(frame, pitch, dst, c->key_pitch, row_bytes, rows, vec);
+    c->launches += 1;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
+
+int dc_launch_match(dc_cache* c)
 {
     MatchArgs a;
-    a.cur = frame; a.cur_pitch = pitch; a.cur_stream = pitch * (size_t)c->cfg.height;
-    a.prev = c->key; a.prev_pitch = c->key_pitch; a.prev_stream = c->key_pitch * (size_t)c->cfg.height;
+    a.cur = c->key[c->key_cur ^ 1]; a.cur_pitch = c->key_pitch; a.cur_stream = c->key_pitch * (size_t)c->cfg.height;
+    a.prev = c->key[c->key_cur]; a.prev_pitch = c->key_pitch; a.prev_stream = c->key_pitch * (size_t)c->cfg.height;
     a.W = c->cfg.width; a.H = c->cfg.height; a.B = c->cfg.block; a.R = c->cfg.range;
     a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search;
     for (int i = 0; i < 4; ++i) a.limit[i] = c->sse_limit[i];
     a.mv = c->blk_mv; a.sse = c->blk_sse; a.matched = c->matched; a.acc = c->mv_acc; a.gmv = c->gmv;
-    DC_CUDA(cudaMemsetAsync(c->mv_acc, 0, sizeof(int32_t) * 4 * c->S, c->stream));
-    int row_words = (a.B * 3 + 3) / 4, iters = dc_div_up(a.B * row_words, 32);
-    if (iters <= 2) launch_all<2>(c, a);
-    else if (iters <= 3) launch_all<3>(c, a);
-    else if (iters <= 6) launch_all<6>(c, a);
-    else if (iters <= 12) launch_all<12>(c, a);
-    else launch_all<24>(c, a);
+    // Step 3 sums and, behind them, the counter of walks handed to the second search phase
+    DC_CUDA(cudaMemsetAsync(c->mv_acc, 0, sizeof(int32_t) * (4 * c->S + 4), c->stream));
+    int32_t* long_count = c->mv_acc + 4 * c->S;
+    if (a.B == 16 && a.search == DC_SEARCH_DIAMOND) {
+        dc_prof_scope ps(c, DC_ST_SEARCH);
+        k_search_ds16<<<((a.Gx + 7) / 8) * a.Gy * a.S, 256, 0, c->stream>>>(a, c->long_list, long_count);
+        int blocks = a.S * a.Gx * a.Gy;
+        int grid = dc_div_up(blocks, 8);
+        if (grid > c->num_sms * 4) grid = c->num_sms * 4;
+        k_search_ds16_long<<<grid, 256, 0, c->stream>>>(a, c->long_list, long_count);
+        c->launches += 1;
+    } else {
+        launch_by_block(c, a, true);
+    }
+    if (a.B == 16) {
+        dc_prof_scope ps(c, DC_ST_VERIFY);
+        k_verify16<<<dc_div_up(a.S * a.Gx * a.Gy, 16), 256, 0, c->stream>>>(a);
+    } else {
+        launch_by_block(c, a, false);
+    }
     {
         dc_prof_scope ps(c, DC_ST_MERGE);
         k_merge<<<c->S, 256, 0, c->stream>>>(c->matched, c->gmv, a.W, a.H, a.B, a.Gx, a.Gy, c->max_regions,
