@@ -36,6 +36,7 @@ struct dc_layer_rt {
     float* bias;                    // conv: [cout]
     void* weight_packed;            // conv, bf16: K-major tensor-core layout (see dc_conv_bf16.cu)
     int k_packed;                   // padded reduction length of weight_packed
+    void* in_padded;                // conv, bf16, cin <= 8: input with channels padded to 8
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation
     int32_t* all_list;              // conv: every tile (used by full frames)

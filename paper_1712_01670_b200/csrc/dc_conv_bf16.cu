@@ -101,10 +101,12 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, in
                  ::"r"(smem_u32(dst)), "l"(tm), "r"(smem_u32(bar)), "r"(c0), "r"(c1) : "memory");
 }
 
-// K-major operand tile in swizzled shared memory: rows of BK bf16, 8-row groups `sbo` bytes apart
-__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t sbo, uint32_t layout_type)
+// K-major operand tile in shared memory.  Swizzled layouts: rows of BK bf16, 8-row groups `sbo`
+// bytes apart (lbo unused, 16).  Unswizzled layout (layout_type 0): 8-row x 16-byte core matrices,
+// `sbo` bytes apart along M/N and `lbo` bytes apart along K.
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t sbo, uint32_t layout_type, uint32_t lbo = 16)
 {
-    uint32_t lo = ((saddr >> 4) & 0x3FFFu) | (1u << 16);                       // start address, LBO = 16 B (unused)
+    uint32_t lo = ((saddr >> 4) & 0x3FFFu) | (((lbo >> 4) & 0x3FFFu) << 16);   // start address, LBO
     uint32_t hi = ((sbo >> 4) & 0x3FFFu) | (1u << 14) | (layout_type << 29);   // SBO, descriptor version 1, swizzle
     return ((uint64_t)hi << 32) | lo;
 }
@@ -138,6 +140,54 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 {
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
+}
+
+// Epilogue warps (4 warps = 128 TMEM lanes = the 128 pixels of a tile): for every work item wait
+// for its accumulator, read it 32 columns at a time, add the bias, apply ReLU, round to bf16 and
+// store the pixel's channels unless the reuse bitmap says the pixel was filled from the cache.
+__device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uint32_t tmem_base, int n_items, int warp, int lane)
+{
+    const int per_stream = a.tiles_x * a.tiles_y;
+    const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
+    const int m = q * 32 + lane, prow = m / DC_TILE_W, pcol = m % DC_TILE_W;
+    uint32_t acc_it = 0;
+    bool ok = true;
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
+        const uint32_t acc = acc_it & 1u, acc_ph = (acc_it >> 1) & 1u;
+        const int tile = a.tile_list[item / a.NB], nb = item % a.NB;
+        const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+        const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
+        const uint32_t mword = a.masks[(size_t)tile * 4 + (prow >> 1)];
+        const bool reused = (mword >> ((prow & 1) * 16 + pcol)) & 1u;
+        const bool active = oy < a.Ho && ox < a.Wo && !reused;
+        __nv_bfloat16* op = a.out + (((size_t)s * a.Ho + oy) * a.Wo + ox) * a.Co + nb * a.BN;
+        const float* bias = a.bias + nb * a.BN;
+        ok = mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, a.status);
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)a.BN;
+        for (int c = 0; c < a.BN / 32; ++c) {
+            uint32_t r[32];
+            tmem_ld32(taddr + c * 32, r);
+            tmem_ld_wait();
+            if (active) {
+                uint4* dst = (uint4*)(op + c * 32);
+#pragma unroll
+                for (int v = 0; v < 4; ++v) {
+                    float f[8];
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) {
+                        f[j] = __uint_as_float(r[v * 8 + j]) + __ldg(bias + c * 32 + v * 8 + j);
+                        if (a.relu) f[j] = fmaxf(f[j], 0.f);
+                    }
+                    dst[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                }
+            }
+        }
+        tc_fence_before();
+        mbar_arrive(&ctl->tmem_empty[acc]);
+    }
 }
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -233,52 +283,146 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         }
     } else {
         // ---------------- epilogue ----------------
-        const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
-        const int m = q * 32 + lane, prow = m / DC_TILE_W, pcol = m % DC_TILE_W;
-        uint32_t acc_it = 0;
-        bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
-            const uint32_t acc = acc_it & 1u, acc_ph = (acc_it >> 1) & 1u;
-            const int tile = a.tile_list[item / a.NB], nb = item % a.NB;
-            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
-            const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
-            const uint32_t mword = a.masks[(size_t)tile * 4 + (prow >> 1)];
-            const bool reused = (mword >> ((prow & 1) * 16 + pcol)) & 1u;
-            const bool active = oy < a.Ho && ox < a.Wo && !reused;
-            __nv_bfloat16* op = a.out + (((size_t)s * a.Ho + oy) * a.Wo + ox) * a.Co + nb * a.BN;
-            const float* bias = a.bias + nb * a.BN;
-            ok = mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, a.status);
-            ok = __all_sync(0xffffffffu, ok);
-            if (!ok) break;
-            tc_fence_after();
-            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)a.BN;
-            for (int c = 0; c < a.BN / 32; ++c) {
-                uint32_t r[32];
-                tmem_ld32(taddr + c * 32, r);
-                tmem_ld_wait();
-                if (active) {
-                    uint4* dst = (uint4*)(op + c * 32);
-#pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        float f[8];
-#pragma unroll
-                        for (int j = 0; j < 8; ++j) {
-                            f[j] = __uint_as_float(r[v * 8 + j]) + __ldg(bias + c * 32 + v * 8 + j);
-                            if (a.relu) f[j] = fmaxf(f[j], 0.f);
-                        }
-                        dst[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
-                    }
-                }
-            }
-            tc_fence_before();
-            mbar_arrive(&ctl->tmem_empty[acc]);
-        }
+        epilogue_loop(a, ctl, tmem_base, n_items, warp, lane);
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Few input channels (cin <= 8, e.g. the first layer on RGB): the channels are padded to 8
+// (16 bytes per pixel) and the kernel taps are laid side by side along K: K = taps * 8, padded to
+// a multiple of 16.  Operands use the unswizzled core-matrix layout: per tap one TMA box lands as
+// 128 rows x 16 bytes (= 16 core matrices 128 bytes apart), consecutive taps 2048 bytes apart,
+// so one tcgen05.mma (K = 16) consumes two taps.  The packed weights ([K/8][cout][8]) stay in
+// shared memory for the whole kernel.  A whole work item is one pipeline stage.
+// ---------------------------------------------------------------------------------------------
+struct TcSmallArgs {
+    TcArgs t;                     // shared fields (BN = cout, NB = 1)
+    const __nv_bfloat16* wpacked; // [kblocks][cout][8]
+    int kblocks;                  // K / 8 (even); taps = kh * kw real ones, the rest zero
+    int w_bytes;                  // kblocks * cout * 16
+};
+
+__global__ void __launch_bounds__(kThreads, 1)
+k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const TcArgs& a = sa.t;
+    const int n_items = *a.tile_count;
+    if ((int)blockIdx.x >= n_items) return;
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    uint8_t* wsm = base;                                        // packed weights
+    const int stage_bytes = sa.kblocks * 2048;
+    uint8_t* ring = wsm + ((sa.w_bytes + 127) & ~127);
+    SmemCtl* ctl = (SmemCtl*)(ring + (size_t)a.stages * stage_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per_stream = a.tiles_x * a.tiles_y;
+    const int taps = a.kh * a.kw;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < a.stages; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 128); }
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+    }
+    // weights into shared memory; zero the tap slots no TMA box ever fills (their weights are zero too,
+    // but 0 x garbage could be NaN)
+    for (int i = threadIdx.x; i < sa.w_bytes / 16; i += kThreads)
+        ((uint4*)wsm)[i] = __ldg((const uint4*)sa.wpacked + i);
+    for (int st = 0; st < a.stages; ++st)
+        for (int i = threadIdx.x; i < (sa.kblocks - taps) * 128; i += kThreads)
+            ((uint4*)(ring + (size_t)st * stage_bytes + taps * 2048))[i] = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        uint32_t it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            const int tile = a.tile_list[item];
+            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+            const int x_base = tx * DC_TILE_W - a.pw, y_base = ty * DC_TILE_H - a.ph;
+            const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
+            if (lane == 0) {
+                ok = mbar_wait(&ctl->empty[st], ph ^ 1u, ctl, a.status);
+                if (ok) {
+                    uint8_t* dst = ring + (size_t)st * stage_bytes;
+                    mbar_expect_tx(&ctl->full[st], (uint32_t)(taps * 2048));
+                    for (int tap = 0; tap < taps; ++tap)
+                        tma_load_4d(dst + tap * 2048, &tmA, 0, x_base + tap % a.kw, y_base + tap / a.kw, s, &ctl->full[st]);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
+        if (!ok && lane == 0) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) { } }
+    } else if (warp == 1) {
+        uint32_t it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
+            const uint32_t acc = it & 1u, acc_ph = (it >> 1) & 1u;
+            const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
+            if (lane == 0) {
+                ok = mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1u, ctl, a.status);
+                if (ok) ok = mbar_wait(&ctl->full[st], ph, ctl, a.status);
+                if (ok) {
+                    tc_fence_after();
+                    const uint32_t d_tmem = tmem_base + acc * (uint32_t)a.BN;
+                    const uint32_t sa_addr = smem_u32(ring + (size_t)st * stage_bytes), sb_addr = smem_u32(wsm);
+                    const uint32_t b_lbo = (uint32_t)a.Co * 16u;
+                    for (int kk = 0; kk < sa.kblocks / 2; ++kk) {
+                        const uint64_t adesc = umma_desc(sa_addr + kk * 4096, 128, 0, 2048);
+                        const uint64_t bdesc = umma_desc(sb_addr + kk * 2 * b_lbo, 128, 0, b_lbo);
+                        umma_f16(d_tmem, adesc, bdesc, a.idesc, kk != 0);
+                    }
+                    umma_commit(&ctl->empty[st]);
+                    umma_commit(&ctl->tmem_full[acc]);
+                }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+        }
+    } else {
+        epilogue_loop(a, ctl, tmem_base, n_items, warp, lane);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// [S][H][W][C] -> [S][H][W][8] with zero padding, C <= 8
+__global__ void k_pad_channels8(const __nv_bfloat16* in, size_t pixels, int C, __nv_bfloat16* out)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < pixels; i += (size_t)gridDim.x * blockDim.x) {
+        unsigned short v[8] = {0, 0, 0, 0, 0, 0, 0, 0};
+        const unsigned short* p = (const unsigned short*)in + i * C;
+        for (int c = 0; c < C; ++c) v[c] = p[c];
+        ((uint4*)out)[i] = make_uint4(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16),
+                                      v[4] | ((uint32_t)v[5] << 16), v[6] | ((uint32_t)v[7] << 16));
+    }
+}
+
+// weights [cout][taps][cin] -> [kblocks][cout][8]: block j holds tap j (cin real channels, rest zero)
+__global__ void k_pack_smallc(const __nv_bfloat16* w, int cout, int taps, int cin, int kblocks, __nv_bfloat16* out)
+{
+    const int total = kblocks * cout * 8;
+    for (int i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const int e = i & 7, n = (i >> 3) % cout, j = (i >> 3) / cout;
+        out[i] = (j < taps && e < cin) ? w[((size_t)n * taps + j) * cin + e] : __float2bfloat16_rn(0.f);
     }
 }
 
@@ -325,16 +469,88 @@ bool make_plan(const dc_layer_desc& d, TcPlan& p)
     return true;
 }
 
+bool smallc_ok(const dc_layer_desc& d)
+{
+    return d.kind == DC_CONV && d.sh == 1 && d.sw == 1 && d.cin <= 8 && d.cout % 32 == 0 && d.cout <= 256 &&
+           d.kh * d.kw <= 64;
+}
+
 }  // namespace
 
 int dc_conv_bf16_supported(const dc_cache* c, int layer)
 {
     TcPlan p;
     if (getenv("DC_NO_TENSOR_CORES")) return 0;
-    return c->cfg.dtype == DC_BF16 && encode_fn() != nullptr && make_plan(c->L[layer].d, p);
+    if (c->cfg.dtype != DC_BF16 || encode_fn() == nullptr) return 0;
+    return make_plan(c->L[layer].d, p) || smallc_ok(c->L[layer].d);
 }
 
-int dc_pack_weights_bf16(dc_cache*, int) { return DC_OK; }       // [cout][kh][kw][cin] is already K-major
+// Normal layers need no repacking ([cout][kh][kw][cin] is already K-major); few-channel layers
+// get their tap-major packed copy and a buffer for the channel-padded input.
+int dc_pack_weights_bf16(dc_cache* c, int layer)
+{
+    dc_layer_rt& L = c->L[layer];
+    TcPlan p;
+    if (make_plan(L.d, p) || !smallc_ok(L.d)) return DC_OK;
+    const int taps = L.d.kh * L.d.kw, kblocks = (taps + 1) / 2 * 2;
+    const size_t wbytes = (size_t)kblocks * L.d.cout * 16, pbytes = (size_t)c->S * L.in_h * L.in_w * 16;
+    DC_CUDA(cudaMalloc(&L.weight_packed, wbytes));
+    DC_CUDA(cudaMalloc(&L.in_padded, pbytes));
+    c->bytes += wbytes + pbytes;
+    L.k_packed = kblocks * 8;
+    k_pack_smallc<<<dc_div_up(kblocks * L.d.cout * 8, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, L.d.cout, taps,
+                                                                               L.d.cin, kblocks, (__nv_bfloat16*)L.weight_packed);
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
+
+static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
+                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
+{
+    dc_layer_rt& L = c->L[layer];
+    const dc_layer_desc& d = L.d;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc || !L.weight_packed) return DC_ERR_CUDA;
+    const size_t pixels = (size_t)c->S * L.in_h * L.in_w;
+    CUtensorMap tmA;
+    cuuint64_t dims[4] = {8, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
+    cuuint64_t strides[3] = {16, (cuuint64_t)L.in_w * 16, (cuuint64_t)L.in_h * L.in_w * 16};
+    cuuint32_t box[4] = {8, DC_TILE_W, DC_TILE_H, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (enc(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, L.in_padded, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+        return DC_ERR_CUDA;
+    TcSmallArgs sa;
+    TcArgs& a = sa.t;
+    a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
+    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
+    a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
+    a.BN = d.cout; a.NB = 1; a.BK = 16; a.kchunks = 1; a.a_bytes = 0; a.b_bytes = 0; a.sbo = 128; a.layout_type = 0;
+    a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(d.cout >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    a.status = c->status;
+    sa.wpacked = (const __nv_bfloat16*)L.weight_packed;
+    sa.kblocks = L.k_packed / 8;
+    sa.w_bytes = sa.kblocks * d.cout * 16;
+    const int stage_bytes = sa.kblocks * 2048;
+    int st = (200 * 1024 - sa.w_bytes) / stage_bytes;
+    a.stages = st > kMaxStages ? kMaxStages : st;
+    if (a.stages < 2) return DC_ERR_CONFIG;
+    const size_t smem = (size_t)a.stages * stage_bytes + ((sa.w_bytes + 127) & ~127) + sizeof(SmemCtl) + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_smallc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    int grid_pad = (int)((pixels + 255) / 256); if (grid_pad > c->num_sms * 8) grid_pad = c->num_sms * 8;
+    int items = max_tiles < 1 ? 1 : max_tiles;
+    int grid = items > c->num_sms ? c->num_sms : items;
+    dc_prof_scope ps(c, DC_ST_CONV);
+    k_pad_channels8<<<grid_pad, 256, 0, c->stream>>>((const __nv_bfloat16*)in, pixels, d.cin, (__nv_bfloat16*)L.in_padded);
+    k_conv_tc_smallc<<<grid, kThreads, smem, c->stream>>>(tmA, sa);
+    c->launches += 2;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
 
 int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
@@ -342,7 +558,10 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     dc_layer_rt& L = c->L[layer];
     const dc_layer_desc& d = L.d;
     TcPlan p;
-    if (!make_plan(d, p)) return DC_ERR_CONFIG;
+    if (!make_plan(d, p)) {
+        if (smallc_ok(d)) return launch_smallc(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
+        return DC_ERR_CONFIG;
+    }
     EncodeTiledFn enc = encode_fn();
     if (!enc) return DC_ERR_CUDA;
     CUtensorMap tmA, tmB;
@@ -380,7 +599,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
         attr_set = true;
     }
     long long items = (long long)(max_tiles < 1 ? 1 : max_tiles) * p.NB;
-    int grid = items > 148 ? 148 : (int)items;
+    int grid = items > c->num_sms ? c->num_sms : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
     k_conv_tc<<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
     c->launches += 1;
