@@ -49,7 +49,8 @@ typedef enum {
     DC_ERR_CUDA = -4,      /* a CUDA call failed */
     DC_ERR_OVERFLOW = -5,  /* more rectangles than max_regions (device status word) */
     DC_ERR_TIMEOUT = -6,   /* a bounded device-side wait ran out (device status word) */
-    DC_ERR_STATE = -7      /* call not valid now (e.g. no cached frame yet) */
+    DC_ERR_STATE = -7,     /* call not valid now (e.g. no cached frame yet) */
+    DC_ERR_LIMIT = -8      /* size beyond a fixed built-in limit (dc_search_blocks_noalloc) */
 } dc_status;
 
 /* A reusable rectangle (Section 3: "(x, y, w, h) -> (x', y', w, h)").
@@ -205,6 +206,32 @@ int dc_cache_profile(dc_cache* cache, float* ms_host, int64_t* launches_host);
  * (reused_px_host: n_layers entries, summed over streams and frames), frames served from the
  * cache and full fresh frames (each counts one call, not one stream).  Synchronous. */
 int dc_cache_counters(dc_cache* cache, int64_t* reused_px_host, int64_t* frames_cached, int64_t* frames_full);
+
+/* Block search without any allocation.  (The paper has no counterpart: this entry point exists
+ * for callers that must not allocate device memory, so cannot create a dc_cache -- code running
+ * where cudaMalloc is not allowed or not affordable, such as a processing loop whose memory was
+ * fixed at start-up, or a plug-in whose host forbids allocation after initialisation.)
+ *
+ * Runs Steps 2 and 3 of the matcher on caller-owned frames: for each block of frame_dev the best
+ * motion vector into prev_dev and its SSE, and per stream the rounded mean vector of the blocks
+ * that pass the PSNR test.  Same definitions, candidate order and outputs as dc_match_blocks.
+ *   frame_dev, prev_dev   uint8 HWC frames, n_streams stacked, any alignment, row pitch pitch_bytes
+ *   block_mv_dev   int16  [S][Gy][Gx][2],  block_sse_dev uint32 [S][Gy][Gx],  global_mv_dev int32 [S][3]
+ *   cuda_stream    cudaStream_t the work is enqueued on (asynchronous)
+ * Its only scratch memory is a fixed array inside the library (DC_NOALLOC_MAX_STREAMS x 16 bytes
+ * = 1 KiB per GPU, held from library load to process exit).  The call never calls cudaMalloc,
+ * cudaFree or any allocating routine.  All calls on one GPU share that array: each call clears what
+ * it uses first, so calls must not overlap on the GPU (run them on one stream, or order them with
+ * events); overlapping calls race and return wrong mean vectors.  The first call on a device looks
+ * up the array's device address (cudaGetSymbolAddress); make that first call outside any stream
+ * capture.
+ * Errors: DC_ERR_ARG, DC_ERR_CONFIG (block, range, search, threshold out of range),
+ * DC_ERR_LIMIT (n_streams > DC_NOALLOC_MAX_STREAMS, or device ordinal >= 64), DC_ERR_CUDA. */
+#define DC_NOALLOC_MAX_STREAMS 64
+int dc_search_blocks_noalloc(const uint8_t* frame_dev, const uint8_t* prev_dev, size_t pitch_bytes,
+                             int32_t width, int32_t height, int32_t n_streams, int32_t block, int32_t range,
+                             int32_t search, double psnr_db, int16_t* block_mv_dev, uint32_t* block_sse_dev,
+                             int32_t* global_mv_dev, void* cuda_stream);
 
 const char* dc_strerror(int status);
 

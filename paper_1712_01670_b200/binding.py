@@ -14,7 +14,8 @@ import torch
 
 DC_MAX_LAYERS = 128
 DC_OK = 0
-DC_ERR_ARG, DC_ERR_CONFIG, DC_ERR_ALLOC, DC_ERR_CUDA, DC_ERR_OVERFLOW, DC_ERR_TIMEOUT, DC_ERR_STATE = range(-1, -8, -1)
+DC_ERR_ARG, DC_ERR_CONFIG, DC_ERR_ALLOC, DC_ERR_CUDA, DC_ERR_OVERFLOW, DC_ERR_TIMEOUT, DC_ERR_STATE, DC_ERR_LIMIT = range(-1, -9, -1)
+DC_NOALLOC_MAX_STREAMS = 64
 DC_CONV, DC_MAXPOOL, DC_RELU, DC_ADD, DC_CONCAT, DC_RESIZE_AREA, DC_LRN, DC_FC = range(8)
 DC_SEARCH_EXHAUSTIVE, DC_SEARCH_DIAMOND = 0, 1
 DC_FP32, DC_BF16 = 0, 1
@@ -48,7 +49,7 @@ REGION_DTYPE = np.dtype([(n, "<i4") for n in ("x", "y", "w", "h", "sx", "sy")])
 EXPORTS = ["dc_cache_create", "dc_cache_destroy", "dc_cache_reset", "dc_cache_bytes", "dc_cache_set_key",
            "dc_match_blocks", "dc_propagate_regions", "dc_conv_partial", "dc_infer_frame", "dc_infer_frame_host",
            "dc_cache_layer_map", "dc_cache_layer_regions", "dc_get_status", "dc_cache_launches",
-           "dc_cache_set_profiling", "dc_cache_profile", "dc_cache_counters", "dc_strerror"]
+           "dc_cache_set_profiling", "dc_cache_profile", "dc_cache_counters", "dc_search_blocks_noalloc", "dc_strerror"]
 PROFILE_STAGES = ["search", "verify", "merge", "propagate", "classify_copy", "conv", "input", "pointwise", "key_update"]
 
 _lib = None
@@ -86,6 +87,8 @@ def load():
         L.dc_cache_set_profiling.argtypes = [vp, i]
         L.dc_cache_profile.argtypes = [vp, C.POINTER(C.c_float), C.POINTER(C.c_int64)]
         L.dc_cache_counters.argtypes = [vp, C.POINTER(C.c_int64), C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+        L.dc_search_blocks_noalloc.argtypes = [vp, vp, sz, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.c_int32,
+                                               C.c_int32, C.c_double, vp, vp, vp, vp]
         L.dc_strerror.argtypes = [i]
         L.dc_strerror.restype = C.c_char_p
         for name in EXPORTS[:-1]:
@@ -222,3 +225,13 @@ def dc_cache_counters(cache, n_layers: int):
     a, b = C.c_int64(), C.c_int64()
     _check(load().dc_cache_counters(cache, px, C.byref(a), C.byref(b)), "dc_cache_counters")
     return [int(v) for v in px], a.value, b.value
+
+
+def dc_search_blocks_noalloc(frame, prev, pitch, width, height, n_streams, block, search_range, search, psnr_db,
+                             block_mv, block_sse, global_mv, stream=None):
+    """Block search for callers that cannot allocate device memory: no cache handle, the only scratch
+    is a fixed array inside the library.  Calls on one GPU must not overlap (they share that array)."""
+    st = stream if stream is not None else torch.cuda.current_stream().cuda_stream
+    _check(load().dc_search_blocks_noalloc(_ptr(frame), _ptr(prev), pitch, width, height, n_streams, block,
+                                           search_range, search, psnr_db, _ptr(block_mv), _ptr(block_sse),
+                                           _ptr(global_mv), C.c_void_p(st)), "dc_search_blocks_noalloc")

@@ -497,6 +497,7 @@ const char* dc_strerror(int status)
     case DC_ERR_OVERFLOW: return "more rectangles than max_regions";
     case DC_ERR_TIMEOUT: return "device-side wait timed out";
     case DC_ERR_STATE: return "call not valid in this state";
+    case DC_ERR_LIMIT: return "size beyond a fixed built-in limit (dc_search_blocks_noalloc: at most 64 streams)";
     default: return "unknown status";
     }
 }
