@@ -173,6 +173,7 @@ def gpu_arm(args, w):
     import torch
     import torch.distributed as dist
     from paper_1712_01670_b200 import binding as B
+    from paper_1712_01670_b200 import sharding
     from paper_1712_01670_b200.engine import DeepCache
 
     rank = int(os.environ.get("RANK", "0"))
@@ -188,15 +189,15 @@ def gpu_arm(args, w):
     S = args.streams or w.n_streams
     total = args.warmup + args.steps
     # every rank renders its own streams: global stream index = rank * S + s
-    sb_all = w.streams(S * world, total)
-    my = list(range(rank * S, rank * S + S))
+    my = sharding.shard_streams(rank, world, S)
+    sb_mine = w.streams(S, total, first=my[0]) if world > 1 else w.streams(S, total)
     frame_bytes = w.height * w.width * 3
     host = torch.empty((total, S, w.height, w.width, 3), dtype=torch.uint8).pin_memory()
     host_np = host.numpy()
 
     def render(job):
         s, i = job
-        host_np[i, s] = sb_all.streams[my[s]].frame(i)
+        host_np[i, s] = sb_mine.streams[s].frame(i)
     with ThreadPoolExecutor(max_workers=min(16, os.cpu_count() or 4)) as ex:
         list(ex.map(render, [(s, i) for s in range(S) for i in range(total)]))
     dev_frames = host.to(dev, non_blocking=True)
@@ -241,11 +242,8 @@ def gpu_arm(args, w):
     status = dc.status()
     if status != B.DC_OK:
         raise SystemExit(f"device status {status}: {B.strerror(status)}")
-    if world > 1:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
-    value = S * world * args.steps / (ms * 1e-3)
+    ms = sharding.max_over_ranks(ms, dev)
+    value = sharding.aggregate_rate(S * args.steps, world, ms * 1e-3)
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
@@ -260,11 +258,8 @@ def gpu_arm(args, w):
             B.dc_infer_frame_host(dc.handle, host[i].data_ptr(), pitch, out_host.data_ptr())
         torch.cuda.synchronize()
         dte = time.perf_counter() - t0e
-        if world > 1:
-            t = torch.tensor([dte], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            dte = float(t.item())
-        e2e = {"value": S * world * args.steps / dte, "unit": UNIT, "h2d_bytes_per_step": S * frame_bytes,
+        dte = sharding.max_over_ranks(dte, dev)
+        e2e = {"value": sharding.aggregate_rate(S * args.steps, world, dte), "unit": UNIT, "h2d_bytes_per_step": S * frame_bytes,
                "d2h_bytes_per_step": out_bytes}
 
     if rank != 0:

@@ -36,7 +36,11 @@ class Workload:
     def weights(self):
         return nets.random_weights(self.layers, self.seed, std=self.weight_std, bias_std=self.bias_std)
 
-    def streams(self, n_streams: int | None = None, n_frames: int | None = None) -> streams.StreamBatch:
+    def streams(self, n_streams: int | None = None, n_frames: int | None = None, first: int = 0) -> streams.StreamBatch:
+        """``n_streams`` streams starting at global stream index ``first`` (a stream's pixels depend
+        only on its global index, so ranks can render disjoint subsets)."""
+        if first:
+            return self.make_streams(n_streams or self.n_streams, n_frames or self.n_frames, first)
         return self.make_streams(n_streams or self.n_streams, n_frames or self.n_frames)
 
 
@@ -86,11 +90,11 @@ def batched_stress(width: int = 1920, height: int = 1080, canvas: int = 2048) ->
     sd = _seed(5)
     n_patches = int(np.ceil(0.20 * width * height / (64 * 64)))
 
-    def make(s, f):
+    def make(s, f, first=0):
         return streams.StreamBatch(
             [streams.PannedStream(width, height, f, sd + 1000 * k, canvas=canvas, max_pan=8,
                                   disturbance="patches", patch=64, n_patches=n_patches)
-             for k in range(s)])
+             for k in range(first, first + s)])
 
     return Workload("batched_stress", 5, width, height, 32, 60, 16, 32, SEARCH_DS, DTYPE_BF16,
                     nets.vgg16_trunk(224, 224, height, width), make, seed=sd)
