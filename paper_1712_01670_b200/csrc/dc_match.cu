@@ -277,29 +277,53 @@ constexpr int F_WORDS = 120;                   // strip window row: (128 + 2 * 1
 constexpr int F_PITCH = 121;                   // odd word pitch: the 16 rows of a half-warp hit 16 banks
 constexpr int L_WORDS = 32;                    // private window row: (16 + 2 * 10) px * 3 B = 108 B + slack
 constexpr int L_PITCH = 33;
+constexpr int F_CANDS = 2;                     // candidates scored per pass (2: half-warp each, 4: quarter-warp each)
+constexpr int F_LPC = 32 / F_CANDS;            // lanes per candidate
+constexpr int F_NR = 16 / F_LPC;               // block rows per lane
 
-// One block row (48 bytes) of the current frame per lane, masked for clipped edge blocks.
+// NR rows (48 bytes each) of the current block per lane, masked for clipped edge blocks.
+template <int NR>
 struct RowCtx {
-    uint32_t cw[12], wm[12];
-    bool clipped, row_on;
-    __device__ __forceinline__ void load(const uint8_t* cur_row, int bw, bool on)
+    uint32_t cw[NR][12], wm[12];
+    bool clipped, row_on[NR];
+    // cur_rows[k]: address of row k of this lane (16-byte aligned in the library's frame copy)
+    __device__ __forceinline__ void load(const uint8_t* const* cur_rows, int bw, const bool* on)
     {
-        row_on = on; clipped = bw < 16;
-        const uint4* p = (const uint4*)cur_row;                // 16-byte aligned in the library's frame copy
-        uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0, v2 = v0;
-        if (on) { v0 = __ldg(p); v1 = __ldg(p + 1); v2 = __ldg(p + 2); }
-        cw[0] = v0.x; cw[1] = v0.y; cw[2] = v0.z; cw[3] = v0.w; cw[4] = v1.x; cw[5] = v1.y; cw[6] = v1.z; cw[7] = v1.w;
-        cw[8] = v2.x; cw[9] = v2.y; cw[10] = v2.z; cw[11] = v2.w;
+        clipped = bw < 16;
 #pragma unroll
-        for (int j = 0; j < 12; ++j) {
-            int nb = bw * 3 - 4 * j;
-            wm[j] = nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << (8 * nb)) - 1u));
-            cw[j] &= wm[j];
+        for (int j = 0; j < 12; ++j) wm[j] = 0xffffffffu;
+        if (clipped) {                                             // only the frame's last block column
+#pragma unroll
+            for (int j = 0; j < 12; ++j) {
+                int nb = bw * 3 - 4 * j;
+                wm[j] = nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << (8 * nb)) - 1u));
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < NR; ++k) {
+            row_on[k] = on[k];
+            const uint4* p = (const uint4*)cur_rows[k];
+            uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0, v2 = v0;
+            if (on[k]) { v0 = __ldg(p); v1 = __ldg(p + 1); v2 = __ldg(p + 2); }
+            cw[k][0] = v0.x; cw[k][1] = v0.y; cw[k][2] = v0.z; cw[k][3] = v0.w; cw[k][4] = v1.x; cw[k][5] = v1.y;
+            cw[k][6] = v1.z; cw[k][7] = v1.w; cw[k][8] = v2.x; cw[k][9] = v2.y; cw[k][10] = v2.z; cw[k][11] = v2.w;
+            if (clipped) {
+#pragma unroll
+                for (int j = 0; j < 12; ++j) cw[k][j] &= wm[j];
+            }
         }
     }
-    // partial SSE of this row against 13 consecutive words at q, the row starting sh bits into q[0]
+    // rows r, r + step, ... of the block whose top-left byte is `base`
+    __device__ __forceinline__ void load_block(const uint8_t* base, size_t pitch, int r, int step, int bw, int bh)
+    {
+        const uint8_t* rows[NR]; bool on[NR];
+#pragma unroll
+        for (int k = 0; k < NR; ++k) { rows[k] = base + (size_t)(r + k * step) * pitch; on[k] = r + k * step < bh; }
+        load(rows, bw, on);
+    }
+    // partial SSE of row k against 13 consecutive words at q, the row starting sh bits into q[0]
     template <typename P>
-    __device__ __forceinline__ uint32_t sse(P q, uint32_t sh) const
+    __device__ __forceinline__ uint32_t sse(int k, P q, uint32_t sh) const
     {
         uint32_t w[13], acc[3] = {0, 0, 0};                     // three chains hide the dp4a latency
 #pragma unroll
@@ -307,13 +331,13 @@ struct RowCtx {
         if (!clipped) {
 #pragma unroll
             for (int j = 0; j < 12; ++j) {
-                uint32_t d = __vabsdiffu4(cw[j], __funnelshift_r(w[j], w[j + 1], sh));
+                uint32_t d = __vabsdiffu4(cw[k][j], __funnelshift_r(w[j], w[j + 1], sh));
                 acc[j % 3] = __dp4a(d, d, acc[j % 3]);
             }
         } else {
 #pragma unroll
             for (int j = 0; j < 12; ++j) {
-                uint32_t d = __vabsdiffu4(cw[j], __funnelshift_r(w[j], w[j + 1], sh) & wm[j]);
+                uint32_t d = __vabsdiffu4(cw[k][j], __funnelshift_r(w[j], w[j + 1], sh) & wm[j]);
                 acc[j % 3] = __dp4a(d, d, acc[j % 3]);
             }
         }
@@ -321,55 +345,59 @@ struct RowCtx {
     }
 };
 
-// Search points relative to a centre, 4 bits per coordinate (value + 2):
-// 0-7 the large diamond, 8 the centre itself, 9-12 the small diamond.
-__device__ __forceinline__ void point_offset(int i, int& dx, int& dy)
-{
-    //            i :  0   1   2   3   4   5   6   7   8   9  10  11  12
-    //           dx :  0  -1   1  -2   2  -1   1   0   0   0  -1   1   0
-    //           dy : -2  -1  -1   0   0   1   1   2   0  -1   0   0   1
-    const unsigned long long X = 0x2312223140312ull;           // nibble i = dx + 2
-    const unsigned long long Y = 0x3221243322110ull;           // nibble i = dy + 2
-    dx = (int)((X >> (4 * i)) & 15) - 2;
-    dy = (int)((Y >> (4 * i)) & 15) - 2;
-}
+// Search points relative to a centre: 0-7 the large diamond, 8 the centre itself, 9-12 the small diamond.
+__constant__ signed char kPointX[13] = {0, -1, 1, -2, 2, -1, 1, 0, 0, 0, -1, 1, 0};
+__constant__ signed char kPointY[13] = {-2, -1, -1, 0, 0, 1, 1, 2, 0, -1, 0, 0, 1};
+// After a move by (mx, my) (one of the 8 large-diamond offsets) the new large diamond overlaps the old
+// one; entry (my + 2) * 5 + (mx + 2) has bit j set for every point j of the new diamond that the old
+// diamond (its 8 points and its centre) did not contain.
+__constant__ unsigned char kNewPoints[25] = {0, 0, 31, 0, 0, 0, 11, 0, 21, 0, 171, 0, 0, 0, 213, 0, 168, 0, 208, 0, 0, 0, 248, 0, 0};
 
 // The diamond walk of one block by one warp.  `Win` supplies the staged previous-frame pixels:
 //   reach(cx, cy)      true when every point a step around centre (cx, cy) may touch is staged
 //   row(r, dx, dy, sh) pointer to the words holding row r of the candidate displaced by (dx, dy)
 // Returns false when the walk must continue elsewhere (bk then holds the state to resume from).
 template <typename Win>
-__device__ __forceinline__ bool diamond_walk(const MatchArgs& a, const RowCtx& rc, Win& win, int x0, int y0, int bw,
+__device__ __forceinline__ bool diamond_walk(const MatchArgs& a, const RowCtx<F_NR>& rc, Win& win, int x0, int y0, int bw,
                                              int bh, int lane, bool resume, unsigned long long& bk)
 {
-    const int r = lane & 15, half = lane >> 4;
-    const unsigned hmask = half ? 0xffff0000u : 0x0000ffffu;
-    // Scores the points of `mask` (bit i = point i around centre (cx, cy)), two per pass: the lower
-    // half-warp takes one, the upper half-warp the next.  One call site keeps the code small.
+    const int r = lane & (F_LPC - 1), group = lane / F_LPC;       // lane owns block rows r, r + F_LPC, ...
+    const unsigned qmask = (F_LPC == 32 ? 0xffffffffu : ((1u << F_LPC) - 1u)) << (F_LPC * group);
+    // displacements that keep the block inside the previous frame and within the search range
+    const int dx_lo = max(-a.R, -x0), dy_lo = max(-a.R, -y0);
+    const unsigned dx_span = (unsigned)(min(a.R, a.W - bw - x0) - dx_lo), dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
+    // Scores the points of `mask` (bit i = point i around centre (cx, cy)), F_CANDS per pass: each
+    // group of F_LPC lanes takes one candidate, each lane F_NR block rows.  One call site keeps
+    // the code small.
     auto score_points = [&](int cx, int cy, unsigned mask) {
 #pragma unroll 1
         while (mask) {
-            const int i0 = __ffs(mask) - 1; mask &= mask - 1;
-            int i1 = -1;
-            if (mask) { i1 = __ffs(mask) - 1; mask &= mask - 1; }
-            const int i = half ? i1 : i0;
-            int dx = 0, dy = 0;
-            bool ok = i >= 0;
-            if (ok) {
-                point_offset(i, dx, dy);
-                dx += cx; dy += cy;
-                ok = abs(dx) <= a.R && abs(dy) <= a.R && x0 + dx >= 0 && y0 + dy >= 0 && x0 + dx + bw <= a.W && y0 + dy + bh <= a.H;
+            int i = -1;
+#pragma unroll
+            for (int k = 0; k < F_CANDS; ++k) {
+                if (mask) {
+                    const int b = __ffs(mask) - 1; mask &= mask - 1;
+                    if (group == k) i = b;
+                }
             }
+            const int ii = i < 0 ? 8 : i;
+            const int dx = cx + kPointX[ii], dy = cy + kPointY[ii];
+            // inside the frame and the range: one unsigned compare per axis against the block's valid span
+            const bool ok = i >= 0 && (unsigned)(dx - dx_lo) <= dx_span && (unsigned)(dy - dy_lo) <= dy_span;
             uint32_t acc = 0;
-            if (ok && rc.row_on) {
+            if (ok) {
                 uint32_t sh;
-                const uint32_t* q = win.row(r, dx, dy, sh);
-                acc = rc.sse(q, sh);
+#pragma unroll
+                for (int k = 0; k < F_NR; ++k)
+                    if (rc.row_on[k]) { const uint32_t* q = win.row(r + k * F_LPC, dx, dy, sh); acc += rc.sse(k, q, sh); }
             }
-            const uint32_t sse = __reduce_add_sync(hmask, acc);
+            const uint32_t sse = __reduce_add_sync(qmask, acc);
             unsigned long long key = ok ? cand_key(sse, dx, dy) : ~0ull;
-            const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, 16);
-            key = key < other ? key : other;
+#pragma unroll
+            for (int off = F_LPC; off < 32; off <<= 1) {
+                const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, off);
+                key = key < other ? key : other;
+            }
             bk = key < bk ? key : bk;
         }
     };
@@ -393,16 +421,7 @@ __device__ __forceinline__ bool diamond_walk(const MatchArgs& a, const RowCtx& r
         const int mx = nx - cx, my = ny - cy;
         cx = nx; cy = ny;
         // points of the new diamond that the old one already scored lost to the new centre: skip them
-        unsigned mask = 0;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            int qx, qy;
-            point_offset(i, qx, qy);
-            qx += mx; qy += my;                                    // position relative to the old centre
-            const bool known = (abs(qx) + abs(qy) == 2) || (qx == 0 && qy == 0);
-            if (!known) mask |= 1u << i;
-        }
-        score_points(cx, cy, mask);
+        score_points(cx, cy, kNewPoints[(my + 2) * 5 + (mx + 2)]);
     }
     score_points(cx, cy, 0x1e00u);                                // small diamond around the final centre
     return true;
@@ -441,21 +460,22 @@ __global__ void __launch_bounds__(256, 4) k_search_ds16(MatchArgs a, uint4* long
     const int xs = strip * 128, y0 = by * 16;
     const int wx0 = ((xs - F_WR) * 3) & ~15;                  // byte column of the window origin (may be < 0)
     const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
-    for (int i = threadIdx.x; i < F_ROWS * F_WORDS; i += 256) {
-        const int row = i / F_WORDS, wi = i - row * F_WORDS;
-        const int gy = y0 - F_WR + row, gb = wx0 + wi * 4;
-        uint32_t v = 0;
-        if (gy >= 0 && gy < a.H && gb >= 0 && gb < (int)a.prev_pitch)
-            v = __ldg((const uint32_t*)(prev + (size_t)gy * a.prev_pitch + gb));
-        win[row * F_PITCH + wi] = v;
+    for (int i = threadIdx.x; i < F_ROWS * (F_WORDS / 4); i += 256) {   // 16-byte chunks; wx0 and the pitch are 16-byte multiples
+        const int row = i / (F_WORDS / 4), ci = i - row * (F_WORDS / 4);
+        const int gy = y0 - F_WR + row, gb = wx0 + ci * 16;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (gy >= 0 && gy < a.H && gb >= 0 && gb + 16 <= (int)a.prev_pitch)
+            v = __ldg((const uint4*)(prev + (size_t)gy * a.prev_pitch + gb));
+        uint32_t* d = win + row * F_PITCH + ci * 4;
+        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
     }
     __syncthreads();
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bx = strip * 8 + warp;
     if (bx >= a.Gx) return;
-    const int x0 = bx * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0), r = lane & 15;
-    RowCtx rc;
-    rc.load(a.cur + (size_t)s * a.cur_stream + (size_t)(y0 + r) * a.cur_pitch + (size_t)x0 * 3, bw, r < bh);
+    const int x0 = bx * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
+    RowCtx<F_NR> rc;
+    rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, lane & (F_LPC - 1), F_LPC, bw, bh);
     StripWin sw = {win, x0, wx0};
     unsigned long long bk = 0;
     const bool done = diamond_walk(a, rc, sw, x0, y0, bw, bh, lane, false, bk);
@@ -497,7 +517,7 @@ struct WarpWin {
 __global__ void __launch_bounds__(256, 4) k_search_ds16_long(MatchArgs a, const uint4* long_list, const int32_t* long_count)
 {
     __shared__ uint32_t win_all[8][F_ROWS * L_PITCH];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane & 15;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int n = *long_count, per = a.Gx * a.Gy;
     for (int i = blockIdx.x * 8 + warp; i < n; i += gridDim.x * 8) {
         const uint4 e = long_list[i];
@@ -505,8 +525,8 @@ __global__ void __launch_bounds__(256, 4) k_search_ds16_long(MatchArgs a, const 
         unsigned long long bk = ((unsigned long long)e.z << 32) | e.y;
         const int s = (int)(g / per), b = (int)(g - (size_t)s * per), by = b / a.Gx, bx = b - by * a.Gx;
         const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
-        RowCtx rc;
-        rc.load(a.cur + (size_t)s * a.cur_stream + (size_t)(y0 + r) * a.cur_pitch + (size_t)x0 * 3, bw, r < bh);
+        RowCtx<F_NR> rc;
+        rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, lane & (F_LPC - 1), F_LPC, bw, bh);
         WarpWin ww = {win_all[warp], a.prev + (size_t)s * a.prev_stream, a.prev_pitch, a.H, x0, y0, 0, 0, 0, lane};
         const int limit = 4 * a.R + 8;                           // each re-staging moves the centre >= 8 px
         bool done = false;
@@ -524,9 +544,9 @@ __global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
 {
     const int lane = threadIdx.x & 31, r = lane & 15, half = lane >> 4;
     const int per = a.Gx * a.Gy;
-    const long long gi = ((long long)blockIdx.x * 8 + (threadIdx.x >> 5)) * 2 + half;
-    const bool in_grid = gi < (long long)per * a.S;
-    const int s = in_grid ? (int)(gi / per) : 0, b = in_grid ? (int)(gi - (long long)s * per) : 0;
+    const unsigned gi = (blockIdx.x * 8u + (threadIdx.x >> 5)) * 2u + half;     // S * Gx * Gy < 2^31
+    const bool in_grid = gi < (unsigned)(per * a.S);
+    const int s = in_grid ? (int)(gi / (unsigned)per) : 0, b = in_grid ? (int)(gi - (unsigned)s * per) : 0;
     const int by = b / a.Gx, bx = b - by * a.Gx;
     const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
     const int K = a.acc[4 * s + 2];
@@ -539,10 +559,10 @@ __global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
     const bool known = cand_ok && a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My;
     uint32_t acc = 0;
     if (cand_ok && !known && r < bh) {
-        RowCtx rc;
-        rc.load(a.cur + (size_t)s * a.cur_stream + (size_t)(y0 + r) * a.cur_pitch + (size_t)x0 * 3, bw, true);
+        RowCtx<1> rc;
+        rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, r, 16, bw, bh);
         const uint8_t* p = a.prev + (size_t)s * a.prev_stream + (size_t)(y0 + My + r) * a.prev_pitch + (size_t)(x0 + Mx) * 3;
-        acc = rc.sse((const uint32_t*)((uintptr_t)p & ~(uintptr_t)3), ((uint32_t)(uintptr_t)p & 3u) * 8u);
+        acc = rc.sse(0, (const uint32_t*)((uintptr_t)p & ~(uintptr_t)3), ((uint32_t)(uintptr_t)p & 3u) * 8u);
     }
     const uint32_t sse = __reduce_add_sync(half ? 0xffff0000u : 0x0000ffffu, acc);
     if (r == 0 && in_grid) {
