@@ -362,10 +362,10 @@ __device__ __forceinline__ bool diamond_walk(const MatchArgs& a, const RowCtx<F_
                                              int bh, int lane, bool resume, unsigned long long& bk)
 {
     const int r = lane & (F_LPC - 1), group = lane / F_LPC;       // lane owns block rows r, r + F_LPC, ...
-    const unsigned qmask = (F_LPC == 32 ? 0xffffffffu : ((1u << F_LPC) - 1u)) << (F_LPC * group);
     // displacements that keep the block inside the previous frame and within the search range
     const int dx_lo = max(-a.R, -x0), dy_lo = max(-a.R, -y0);
     const unsigned dx_span = (unsigned)(min(a.R, a.W - bw - x0) - dx_lo), dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
+    uint32_t bs = (uint32_t)(bk >> 32), bt = (uint32_t)bk;        // best so far: SSE and tie-break word
     // Scores the points of `mask` (bit i = point i around centre (cx, cy)), F_CANDS per pass: each
     // group of F_LPC lanes takes one candidate, each lane F_NR block rows.  One call site keeps
     // the code small.
@@ -391,39 +391,44 @@ __device__ __forceinline__ bool diamond_walk(const MatchArgs& a, const RowCtx<F_
                 for (int k = 0; k < F_NR; ++k)
                     if (rc.row_on[k]) { const uint32_t* q = win.row(r + k * F_LPC, dx, dy, sh); acc += rc.sse(k, q, sh); }
             }
-            const uint32_t sse = __reduce_add_sync(qmask, acc);
-            unsigned long long key = ok ? cand_key(sse, dx, dy) : ~0ull;
+            uint32_t ks = acc;                                     // sum over the candidate's lanes
+#pragma unroll
+            for (int off = F_LPC / 2; off > 0; off >>= 1) ks += __shfl_xor_sync(0xffffffffu, ks, off);
+            // candidate order (SSE, |dx| + |dy|, dy, dx) as two 32-bit words; all-ones = no candidate
+            uint32_t kt = ((uint32_t)(abs(dx) + abs(dy)) << 16) | ((uint32_t)(dy + 128) << 8) | (uint32_t)(dx + 128);
+            if (!ok) { ks = 0xffffffffu; kt = 0xffffffffu; }
 #pragma unroll
             for (int off = F_LPC; off < 32; off <<= 1) {
-                const unsigned long long other = __shfl_xor_sync(0xffffffffu, key, off);
-                key = key < other ? key : other;
+                const uint32_t os = __shfl_xor_sync(0xffffffffu, ks, off), ot = __shfl_xor_sync(0xffffffffu, kt, off);
+                if (os < ks || (os == ks && ot < kt)) { ks = os; kt = ot; }
             }
-            bk = key < bk ? key : bk;
+            if (ks < bs || (ks == bs && kt < bt)) { bs = ks; bt = kt; }
         }
     };
     int cx, cy;
     if (!resume) {
-        bk = ~0ull;
+        bs = 0xffffffffu; bt = 0xffffffffu;
         cx = 0; cy = 0;
         score_points(0, 0, 0x1ffu);                               // the centre (0, 0) and its large diamond
     } else {
         // resumed walk: the best point so far is the centre; score its whole large diamond
-        cx = (int)(bk & 0xff) - 128; cy = (int)((bk >> 8) & 0xff) - 128;
+        cx = (int)(bt & 0xff) - 128; cy = (int)((bt >> 8) & 0xff) - 128;
         if (!win.reach(cx, cy)) return false;
         score_points(cx, cy, 0xffu);
     }
     const int max_steps = (2 * a.R + 1) * (2 * a.R + 1);          // every move strictly lowers the key
 #pragma unroll 1
     for (int step = 0; step < max_steps; ++step) {
-        const int nx = (int)(bk & 0xff) - 128, ny = (int)((bk >> 8) & 0xff) - 128;
+        const int nx = (int)(bt & 0xff) - 128, ny = (int)((bt >> 8) & 0xff) - 128;
         if (nx == cx && ny == cy) break;                           // the centre won: large diamond done
-        if (!win.reach(nx, ny)) return false;
+        if (!win.reach(nx, ny)) { bk = ((unsigned long long)bs << 32) | bt; return false; }
         const int mx = nx - cx, my = ny - cy;
         cx = nx; cy = ny;
         // points of the new diamond that the old one already scored lost to the new centre: skip them
         score_points(cx, cy, kNewPoints[(my + 2) * 5 + (mx + 2)]);
     }
     score_points(cx, cy, 0x1e00u);                                // small diamond around the final centre
+    bk = ((unsigned long long)bs << 32) | bt;
     return true;
 }
 
@@ -501,12 +506,14 @@ struct WarpWin {
         wcx = cx; wcy = cy;
         wx0 = ((x0 + cx - F_WR) * 3) & ~15;
         __syncwarp();
-        for (int row = 0; row < F_ROWS; ++row) {
-            static_assert(L_WORDS == 32, "one lane per window word");
-            const int gy = y0 + cy - F_WR + row, gb = wx0 + lane * 4;
-            uint32_t v = 0;
-            if (gy >= 0 && gy < H && gb >= 0 && gb < (int)pitch) v = __ldg((const uint32_t*)(prev + (size_t)gy * pitch + gb));
-            win[row * L_PITCH + lane] = v;
+        static_assert(L_WORDS == 32, "8 chunks of 16 bytes per window row");
+        for (int i = lane; i < F_ROWS * 8; i += 32) {                 // wx0 and the pitch are 16-byte multiples
+            const int row = i >> 3, ci = i & 7;
+            const int gy = y0 + cy - F_WR + row, gb = wx0 + ci * 16;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (gy >= 0 && gy < H && gb >= 0 && gb + 16 <= (int)pitch) v = __ldg((const uint4*)(prev + (size_t)gy * pitch + gb));
+            uint32_t* d = win + row * L_PITCH + ci * 4;
+            d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
         }
         __syncwarp();
     }
@@ -514,7 +521,7 @@ struct WarpWin {
 
 // Phase 2: the walks that left their strip window, one warp each, re-staging a private window
 // around the walk's centre whenever it nears the window's edge.
-__global__ void __launch_bounds__(256, 4) k_search_ds16_long(MatchArgs a, const uint4* long_list, const int32_t* long_count)
+__global__ void __launch_bounds__(256, 3) k_search_ds16_long(MatchArgs a, const uint4* long_list, const int32_t* long_count)
 {
     __shared__ uint32_t win_all[8][F_ROWS * L_PITCH];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
