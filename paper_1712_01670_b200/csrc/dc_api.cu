@@ -206,6 +206,12 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     size_t stat_ints = (size_t)S * (3 + 4 + 1) + (size_t)n * S;
     if (cudaMallocHost(&c->stats_pinned, stat_ints * sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
     DC_CUDA(cudaStreamSynchronize(c->stream));      // layers / in_hw / all_count live on this stack frame
+    for (int i = 0; i < n; ++i)
+        if (c->executable && c->L[i].d.kind == DC_CONV) {
+            const void* in = c->L[i].d.in0 < 0 ? c->input_map : c->L[c->L[i].d.in0].map[0];
+            DC_TRY(dc_conv_bf16_autotune(c, i, in));
+        }
+    DC_CUDA(cudaStreamSynchronize(c->stream));
     return DC_OK;
 }
 

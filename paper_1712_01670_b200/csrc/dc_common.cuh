@@ -36,6 +36,7 @@ struct dc_layer_rt {
     float* bias;                    // conv: [cout]
     void* weight_packed;            // conv, bf16: K-major tensor-core layout (see dc_conv_bf16.cu)
     int k_packed;                   // padded reduction length of weight_packed
+    int tc_mt, tc_bn;               // conv, bf16: tuned tiles per work item and channels per block (0 = default)
     void* in_padded;                // conv, bf16, cin <= 8: input with channels padded to 8
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation
@@ -109,3 +110,4 @@ int dc_launch_maxpool(dc_cache* c, int layer, const void* in);
 int dc_launch_add(dc_cache* c, int layer, const void* a, const void* b);
 int dc_launch_relu(dc_cache* c, int layer, const void* a);
 int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_dev);
+int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in);

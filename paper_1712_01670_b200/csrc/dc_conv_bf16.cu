@@ -19,6 +19,7 @@
 // the next.  Every mbarrier wait is bounded: on expiry the kernel records DC_ERR_TIMEOUT in the
 // status word, all roles leave their loops, tensor memory is freed and the kernel returns.
 #include <cuda.h>
+#include <stdio.h>
 #include <stdlib.h>
 
 #include "dc_common.cuh"
@@ -34,6 +35,7 @@ struct TcArgs {
     const int32_t* tile_list; const int32_t* tile_count; const uint32_t* masks;
     int Ho, Wo, Co, Ci, kh, kw, sh, sw, ph, pw, relu, tiles_x, tiles_y;
     int BN, NB, BK, kchunks, stages, a_bytes, b_bytes;
+    int MT, nbuf;                 // tiles per work item (1 or 2, sharing one B tile); TMEM accumulator sets (2, or 1 when MT * BN = 512)
     uint32_t idesc, sbo, layout_type;
     int32_t* status;
 };
@@ -145,7 +147,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 // Epilogue warps (4 warps = 128 TMEM lanes = the 128 pixels of a tile): for every work item wait
 // for its accumulator, read it 32 columns at a time, add the bias, apply ReLU, round to bf16 and
 // store the pixel's channels unless the reuse bitmap says the pixel was filled from the cache.
-__device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uint32_t tmem_base, int n_items, int warp, int lane)
+__device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uint32_t tmem_base, int n_items, int n_tiles, int warp, int lane)
 {
     const int per_stream = a.tiles_x * a.tiles_y;
     const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
@@ -153,35 +155,39 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
     uint32_t acc_it = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
-        const uint32_t acc = acc_it & 1u, acc_ph = (acc_it >> 1) & 1u;
-        const int tile = a.tile_list[item / a.NB], nb = item % a.NB;
-        const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
-        const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
-        const uint32_t mword = a.masks[(size_t)tile * 4 + (prow >> 1)];
-        const bool reused = (mword >> ((prow & 1) * 16 + pcol)) & 1u;
-        const bool active = oy < a.Ho && ox < a.Wo && !reused;
-        __nv_bfloat16* op = a.out + (((size_t)s * a.Ho + oy) * a.Wo + ox) * a.Co + nb * a.BN;
-        const float* bias = a.bias + nb * a.BN;
+        const uint32_t acc = acc_it % (uint32_t)a.nbuf, acc_ph = (acc_it / (uint32_t)a.nbuf) & 1u;
+        const int group = item / a.NB, nb = item % a.NB;
         ok = mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, a.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + acc * (uint32_t)a.BN;
-        for (int c = 0; c < a.BN / 32; ++c) {
-            uint32_t r[32];
-            tmem_ld32(taddr + c * 32, r);
-            tmem_ld_wait();
-            if (active) {
-                uint4* dst = (uint4*)(op + c * 32);
+        const float* bias = a.bias + nb * a.BN;
+        for (int j = 0; j < a.MT; ++j) {
+            if (group * a.MT + j >= n_tiles) break;             // odd tile count: the last item has one tile
+            const int tile = a.tile_list[group * a.MT + j];
+            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+            const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
+            const uint32_t mword = a.masks[(size_t)tile * 4 + (prow >> 1)];
+            const bool reused = (mword >> ((prow & 1) * 16 + pcol)) & 1u;
+            const bool active = oy < a.Ho && ox < a.Wo && !reused;
+            __nv_bfloat16* op = a.out + (((size_t)s * a.Ho + oy) * a.Wo + ox) * a.Co + nb * a.BN;
+            const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (acc * (uint32_t)a.MT + (uint32_t)j) * (uint32_t)a.BN;
+            for (int c = 0; c < a.BN / 32; ++c) {
+                uint32_t r[32];
+                tmem_ld32(taddr + c * 32, r);
+                tmem_ld_wait();
+                if (active) {
+                    uint4* dst = (uint4*)(op + c * 32);
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    float f[8];
+                    for (int v = 0; v < 4; ++v) {
+                        float f[8];
 #pragma unroll
-                    for (int j = 0; j < 8; ++j) {
-                        f[j] = __uint_as_float(r[v * 8 + j]) + __ldg(bias + c * 32 + v * 8 + j);
-                        if (a.relu) f[j] = fmaxf(f[j], 0.f);
+                        for (int jj = 0; jj < 8; ++jj) {
+                            f[jj] = __uint_as_float(r[v * 8 + jj]) + __ldg(bias + c * 32 + v * 8 + jj);
+                            if (a.relu) f[jj] = fmaxf(f[jj], 0.f);
+                        }
+                        dst[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
                     }
-                    dst[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
                 }
             }
         }
@@ -190,16 +196,18 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
     }
 }
 
+template <int MT>
 __global__ void __launch_bounds__(kThreads, 1)
 k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
-    const int n_items = *a.tile_count * a.NB;
+    const int n_tiles = *a.tile_count;
+    const int n_items = (n_tiles + MT - 1) / MT * a.NB;     // an item: MT tiles x one block of BN channels
     if ((int)blockIdx.x >= n_items) return;
 
     // operand ring at a 1024-byte boundary (the swizzle pattern repeats every 1024 bytes), then control words
     uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
-    const int stage_bytes = a.a_bytes + a.b_bytes;
+    const int stage_bytes = MT * a.a_bytes + a.b_bytes;
     SmemCtl* ctl = (SmemCtl*)(ring + (size_t)a.stages * stage_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per_stream = a.tiles_x * a.tiles_y;
@@ -227,9 +235,15 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         uint32_t it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
-            const int tile = a.tile_list[item / a.NB], nb = item % a.NB;
-            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
-            const int x_base = tx * DC_TILE_W * a.sw - a.pw, y_base = ty * DC_TILE_H * a.sh - a.ph;
+            const int group = item / a.NB, nb = item % a.NB;
+            int sN[MT], xb[MT], yb[MT];
+#pragma unroll
+            for (int j = 0; j < MT; ++j) {                      // an absent second tile repeats the first (never stored)
+                const int idx = group * MT + j;
+                const int tile = a.tile_list[idx < n_tiles ? idx : group * MT];
+                const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+                sN[j] = s; xb[j] = tx * DC_TILE_W * a.sw - a.pw; yb[j] = ty * DC_TILE_H * a.sh - a.ph;
+            }
             for (int k = 0; k < kiters && ok; ++k, ++it) {
                 const int tap = k / a.kchunks, cc = k - tap * a.kchunks, ky = tap / a.kw, kx = tap - ky * a.kw;
                 const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
@@ -238,8 +252,10 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     if (ok) {
                         uint8_t* sa = ring + (size_t)st * stage_bytes;
                         mbar_expect_tx(&ctl->full[st], (uint32_t)stage_bytes);
-                        tma_load_4d(sa, &tmA, cc * a.BK, x_base + kx, y_base + ky, s, &ctl->full[st]);
-                        tma_load_2d(sa + a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, nb * a.BN, &ctl->full[st]);
+#pragma unroll
+                        for (int j = 0; j < MT; ++j)
+                            tma_load_4d(sa + j * a.a_bytes, &tmA, cc * a.BK, xb[j] + kx, yb[j] + ky, sN[j], &ctl->full[st]);
+                        tma_load_2d(sa + MT * a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, nb * a.BN, &ctl->full[st]);
                     }
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -255,8 +271,8 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         uint32_t it = 0, acc_it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
-            const uint32_t acc = acc_it & 1u, acc_ph = (acc_it >> 1) & 1u;
-            const uint32_t d_tmem = tmem_base + acc * (uint32_t)a.BN;
+            const uint32_t acc = acc_it % (uint32_t)a.nbuf, acc_ph = (acc_it / (uint32_t)a.nbuf) & 1u;
+            const uint32_t d_tmem = tmem_base + acc * (uint32_t)(MT * a.BN);
             if (lane == 0) {
                 ok = mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1u, ctl, a.status);
                 tc_fence_after();
@@ -269,10 +285,13 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                     if (ok) {
                         tc_fence_after();
                         const uint32_t sa = smem_u32(ring + (size_t)st * stage_bytes);
-                        const uint64_t adesc = umma_desc(sa, a.sbo, a.layout_type);
-                        const uint64_t bdesc = umma_desc(sa + a.a_bytes, a.sbo, a.layout_type);
-                        for (int kk = 0; kk < a.BK / 16; ++kk)       // 16 bf16 = 32 bytes = 2 descriptor units
-                            umma_f16(d_tmem, adesc + 2 * kk, bdesc + 2 * kk, a.idesc, (k | kk) != 0);
+                        const uint64_t bdesc = umma_desc(sa + MT * a.a_bytes, a.sbo, a.layout_type);
+#pragma unroll
+                        for (int j = 0; j < MT; ++j) {
+                            const uint64_t adesc = umma_desc(sa + j * a.a_bytes, a.sbo, a.layout_type);
+                            for (int kk = 0; kk < a.BK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor units
+                                umma_f16(d_tmem + j * a.BN, adesc + 2 * kk, bdesc + 2 * kk, a.idesc, (k | kk) != 0);
+                        }
                         umma_commit(&ctl->empty[st]);                // frees the slot when these MMAs retire
                     }
                 }
@@ -283,7 +302,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         }
     } else {
         // ---------------- epilogue ----------------
-        epilogue_loop(a, ctl, tmem_base, n_items, warp, lane);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane);
     }
     tc_fence_before();
     __syncthreads();
@@ -394,7 +413,7 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
             ok = __shfl_sync(0xffffffffu, ok, 0);
         }
     } else {
-        epilogue_loop(a, ctl, tmem_base, n_items, warp, lane);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_items, warp, lane);
     }
     tc_fence_before();
     __syncthreads();
@@ -444,9 +463,9 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
-struct TcPlan { int BK, BN, NB, stages, a_bytes, b_bytes; CUtensorMapSwizzle swz; uint32_t layout_type, sbo; size_t smem; };
+struct TcPlan { int BK, BN, NB, MT, nbuf, stages, a_bytes, b_bytes; CUtensorMapSwizzle swz; uint32_t layout_type, sbo; size_t smem; };
 
-bool make_plan(const dc_layer_desc& d, TcPlan& p)
+bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn = 0)
 {
     if (d.kind != DC_CONV) return false;
     if (d.sh != 1 || d.sw != 1) return false;                   // strided layers use the CUDA-core kernel
@@ -457,15 +476,23 @@ bool make_plan(const dc_layer_desc& d, TcPlan& p)
     p.BN = 0;
     for (int bn = 256; bn >= 32; bn -= 32) if (d.cout % bn == 0) { p.BN = bn; break; }
     if (!p.BN) return false;
+    if (want_bn > 0) {                                           // a tuned choice: must divide cout like the default
+        if (want_bn % 32 != 0 || want_bn > 256 || d.cout % want_bn != 0) return false;
+        p.BN = want_bn;
+    }
     p.NB = d.cout / p.BN;
     p.a_bytes = DC_TILE_PX * p.BK * 2;
     p.b_bytes = p.BN * p.BK * 2;
     p.sbo = 8 * p.BK * 2;
     if (p.b_bytes % 1024 != 0) return false;                    // keep every operand tile on a swizzle-pattern boundary
-    int st = (200 * 1024) / (p.a_bytes + p.b_bytes);
+    // two tiles share each B tile: halves the weight traffic per FLOP; 512 TMEM columns hold
+    // MT * BN * nbuf accumulator columns
+    p.MT = want_mt > 0 ? want_mt : 1;
+    p.nbuf = p.MT * p.BN * 2 <= 512 ? 2 : 1;
+    int st = (200 * 1024) / (p.MT * p.a_bytes + p.b_bytes);
     p.stages = st > kMaxStages ? kMaxStages : st;
     if (p.stages < 2) return false;
-    p.smem = (size_t)p.stages * (p.a_bytes + p.b_bytes) + sizeof(SmemCtl) + 1024;
+    p.smem = (size_t)p.stages * (p.MT * p.a_bytes + p.b_bytes) + sizeof(SmemCtl) + 1024;
     return true;
 }
 
@@ -525,7 +552,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
     a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
     a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
-    a.BN = d.cout; a.NB = 1; a.BK = 16; a.kchunks = 1; a.a_bytes = 0; a.b_bytes = 0; a.sbo = 128; a.layout_type = 0;
+    a.BN = d.cout; a.NB = 1; a.MT = 1; a.nbuf = 2; a.BK = 16; a.kchunks = 1; a.a_bytes = 0; a.b_bytes = 0; a.sbo = 128; a.layout_type = 0;
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(d.cout >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
     sa.wpacked = (const __nv_bfloat16*)L.weight_packed;
@@ -558,7 +585,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     dc_layer_rt& L = c->L[layer];
     const dc_layer_desc& d = L.d;
     TcPlan p;
-    if (!make_plan(d, p)) {
+    if (!make_plan(d, p, L.tc_mt, L.tc_bn)) {
         if (smallc_ok(d)) return launch_smallc(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
         return DC_ERR_CONFIG;
     }
@@ -588,21 +615,64 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
     a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = d.sh; a.sw = d.sw;
     a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
-    a.BN = p.BN; a.NB = p.NB; a.BK = p.BK; a.kchunks = d.cin / p.BK; a.stages = p.stages;
+    a.BN = p.BN; a.NB = p.NB; a.BK = p.BK; a.kchunks = d.cin / p.BK; a.stages = p.stages; a.MT = p.MT; a.nbuf = p.nbuf;
     a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.sbo = p.sbo; a.layout_type = p.layout_type;
     // instruction descriptor: D = f32, A = B = bf16, both K-major, N = BN, M = 128
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
     static bool attr_set = false;
     if (!attr_set) {
-        DC_CUDA(cudaFuncSetAttribute(k_conv_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
-    long long items = (long long)(max_tiles < 1 ? 1 : max_tiles) * p.NB;
+    long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + p.MT - 1) / p.MT) * p.NB;
     int grid = items > c->num_sms ? c->num_sms : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
-    k_conv_tc<<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
+    if (p.MT == 2) k_conv_tc<2><<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
+    else k_conv_tc<1><<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
+
+// Picks, per convolution layer, the work-item shape (tiles per item x channels per block) by timing
+// the candidates once on the layer's own buffers with every tile dirty.  The choice changes only how
+// the work is cut: each output element is accumulated over K in the same order, so results do not
+// depend on it.  Called by dc_cache_create (which may synchronise).
+int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
+{
+    dc_layer_rt& L = c->L[layer];
+    TcPlan p;
+    if (c->cfg.dtype != DC_BF16 || !encode_fn() || !make_plan(L.d, p) || getenv("DC_NO_TENSOR_CORES")) return DC_OK;
+    if (getenv("DC_CONV_NO_TUNE")) return DC_OK;
+    const int tiles = L.tiles_x * L.tiles_y * c->S;
+    cudaEvent_t e0, e1;
+    DC_CUDA(cudaEventCreate(&e0));
+    DC_CUDA(cudaEventCreate(&e1));
+    float best = 1e30f; int best_mt = 1, best_bn = p.BN;
+    const int default_bn = p.BN;
+    for (int bn = default_bn; bn >= 64 && bn >= default_bn / 2; bn -= 32) {
+        if (L.d.cout % bn != 0) continue;
+        for (int mt = 1; mt <= 2; ++mt) {
+            TcPlan q;
+            if (!make_plan(L.d, q, mt, bn)) continue;
+            L.tc_mt = mt; L.tc_bn = bn;
+            int rc = DC_OK;
+            for (int rep = 0; rep < 3 && rc == DC_OK; ++rep) {
+                if (rep == 1) cudaEventRecord(e0, c->stream);
+                rc = dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles);
+            }
+            cudaEventRecord(e1, c->stream);
+            if (rc != DC_OK || cudaEventSynchronize(e1) != cudaSuccess) { cudaGetLastError(); continue; }
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, e0, e1);
+            if (ms < best) { best = ms; best_mt = mt; best_bn = bn; }
+        }
+    }
+    L.tc_mt = best_mt; L.tc_bn = best_bn;
+    cudaEventDestroy(e0); cudaEventDestroy(e1);
+    c->launches = 0;
+    if (getenv("DC_VERBOSE")) fprintf(stderr, "libdeepcache: layer %d: %d tile(s) per item, %d channels per block (%.3f ms)\n", layer, best_mt, best_bn, best / 2);
     return DC_OK;
 }
