@@ -7,9 +7,11 @@
 
 #include "deepcache.h"
 
-#define DC_TILE_H 8          // output tile of the partial convolution: 8 rows x 16 columns
-#define DC_TILE_W 16         // = 128 output pixels = the M dimension of one tensor-core tile
-#define DC_TILE_PX (DC_TILE_H * DC_TILE_W)
+#define DC_TILE_H 16         // output tile of the partial convolution: 16 rows x 8 columns
+#define DC_TILE_W 8          // = 128 output pixels = the M dimension of one tensor-core tile; 8 columns = one
+#define DC_TILE_PX (DC_TILE_H * DC_TILE_W)   // 8-row operand group per image row (see dc_conv_bf16.cu)
+// Reuse bitmap of a tile: 128 bits, bit (row * DC_TILE_W + col), in four 32-bit words.
+#define DC_TILE_BIT(row, col) ((row) * DC_TILE_W + (col))
 
 #define DC_CUDA(call)                                            \
     do {                                                         \

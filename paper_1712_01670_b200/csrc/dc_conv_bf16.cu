@@ -1,10 +1,10 @@
 // Partial convolution on the 5th-generation tensor cores (bf16 in, fp32 accumulate in TMEM).
 //
 // Section 5, "Reuse", third step: convolve only what the cache did not supply.  The unit of
-// work is one dirty 8x16 output tile (128 pixels = the M of one tcgen05.mma) times one block of
+// work is one dirty 16x8 output tile (128 pixels = the M of one tcgen05.mma) times one block of
 // BN output channels.  It is an implicit GEMM: for every kernel tap (ky, kx) and every chunk of
 // BK input channels, TMA fetches
-//     A: the 8x16 window of the NHWC input map displaced by the tap (a 4-D box; coordinates
+//     A: the 16x8 window of the NHWC input map displaced by the tap (a 4-D box; coordinates
 //        outside the map are zero-filled, which is the convolution's padding), 128 rows x BK
 //     B: BN rows x BK of the weights, which are already K-major as [cout][kh][kw][cin]
 // into 128-byte-swizzled shared memory, and one elected thread issues BK/16 tcgen05.mma
@@ -167,8 +167,8 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
             const int tile = a.tile_list[group * a.MT + j];
             const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
             const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
-            const uint32_t mword = a.masks[(size_t)tile * 4 + (prow >> 1)];
-            const bool reused = (mword >> ((prow & 1) * 16 + pcol)) & 1u;
+            const uint32_t mword = a.masks[(size_t)tile * 4 + (DC_TILE_BIT(prow, pcol) >> 5)];
+            const bool reused = (mword >> (DC_TILE_BIT(prow, pcol) & 31)) & 1u;
             const bool active = oy < a.Ho && ox < a.Wo && !reused;
             __nv_bfloat16* op = a.out + (((size_t)s * a.Ho + oy) * a.Wo + ox) * a.Co + nb * a.BN;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (acc * (uint32_t)a.MT + (uint32_t)j) * (uint32_t)a.BN;

@@ -3,7 +3,7 @@
 //
 // Used for float32 networks, whose 1e-4 accuracy bound rules out tensor-core input formats,
 // and for layer shapes the tensor-core kernel does not take.  One CTA of 128 threads owns one
-// dirty 8x16 output tile and a group of 32 output channels; thread t owns pixel t and keeps 32
+// dirty 16x8 output tile and a group of 32 output channels; thread t owns pixel t and keeps 32
 // float accumulators.  Weights for one kernel row and 8 input channels are staged in shared
 // memory as floats [kx][ci][co] and read as broadcast float4; inputs come straight from the
 // NHWC map (8 consecutive channels per load).  The epilogue adds the bias, applies ReLU and
@@ -43,8 +43,8 @@ __global__ void __launch_bounds__(DC_TILE_PX) k_conv_direct(ConvArgs a)
         const int s = tile / per, t = tile - s * per, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
         const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
         const bool in_map = oy < a.Ho && ox < a.Wo;
-        const uint32_t mword = a.masks[(size_t)tile * 4 + (prow >> 1)];
-        const bool reused = (mword >> ((prow & 1) * 16 + pcol)) & 1u;
+        const uint32_t mword = a.masks[(size_t)tile * 4 + (DC_TILE_BIT(prow, pcol) >> 5)];
+        const bool reused = (mword >> (DC_TILE_BIT(prow, pcol) & 31)) & 1u;
         const bool active = in_map && !reused;
         float acc[CO_T];
 #pragma unroll

@@ -4,7 +4,7 @@
 //   k_propagate      one thread per (stream, rectangle slot) walks the layer table in order and
 //                    writes the rectangle's image after every layer.  Slots are independent,
 //                    so no synchronisation is needed; a vanished rectangle is all zeros.
-//   k_classify_copy  one warp per 8x16 output tile: lanes test the stream's rectangles against
+//   k_classify_copy  one warp per 16x8 output tile: lanes test the stream's rectangles against
 //                    the tile, OR their coverage into a 128-bit bitmap, the warp copies each
 //                    covered span from the cached map with 16-byte vectors, and tiles that
 //                    still hold uncovered pixels are appended to the layer's dirty list.
@@ -117,7 +117,7 @@ __global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
     const dc_region* regs = a.regions + (size_t)s * a.max_regions;
     const int n = a.n_regions[s];
     const size_t map_base = (size_t)s * a.Ho * a.Wo * a.px_bytes;
-    uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;      // bit (row * 16 + col) of the tile, row-major
+    uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;      // bit (row * DC_TILE_W + col) of the tile, row-major
     for (int base = 0; base < n; base += 32) {
         int i = base + lane;
         dc_region r = empty_region();
@@ -129,11 +129,11 @@ __global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
         }
         bool hit = ix1 > ix0 && iy1 > iy0;
         if (hit) {
-            uint32_t rowbits = ((1u << (ix1 - X0)) - 1u) & ~((1u << (ix0 - X0)) - 1u);   // 16-bit row pattern
+            const uint32_t rowbits = ((1u << (ix1 - X0)) - 1u) & ~((1u << (ix0 - X0)) - 1u);   // DC_TILE_W-bit row pattern
             for (int y = iy0; y < iy1; ++y) {
-                int row = y - Y0;
-                uint32_t v = rowbits << ((row & 1) * 16);
-                switch (row >> 1) { case 0: m0 |= v; break; case 1: m1 |= v; break; case 2: m2 |= v; break; default: m3 |= v; }
+                const int bit = DC_TILE_BIT(y - Y0, 0);
+                const uint32_t v = rowbits << (bit & 31);
+                switch (bit >> 5) { case 0: m0 |= v; break; case 1: m1 |= v; break; case 2: m2 |= v; break; default: m3 |= v; }
             }
         }
         // the warp copies every hit span together: rows of (ix1 - ix0) pixels, px_bytes each
