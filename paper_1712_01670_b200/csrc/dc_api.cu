@@ -226,7 +226,7 @@ void release(dc_cache* c)
     if (c->stats_pinned) cudaFreeHost(c->stats_pinned);
     for (int i = 0; i < c->n_layers; ++i) {
         dc_layer_rt& L = c->L[i];
-        cudaFree(L.map[0]); cudaFree(L.map[1]); cudaFree(L.weight); cudaFree(L.bias); cudaFree(L.weight_packed); cudaFree(L.in_padded);
+        cudaFree(L.map[0]); cudaFree(L.map[1]); cudaFree(L.weight); cudaFree(L.bias); cudaFree(L.weight_packed); cudaFree(L.in_padded); cudaFree(L.weight_halo);
         cudaFree(L.masks); cudaFree(L.dirty_list); cudaFree(L.all_list);
     }
     cudaGetLastError();

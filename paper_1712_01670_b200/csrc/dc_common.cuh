@@ -38,7 +38,9 @@ struct dc_layer_rt {
     float* bias;                    // conv: [cout]
     void* weight_packed;            // conv, bf16: K-major tensor-core layout (see dc_conv_bf16.cu)
     int k_packed;                   // padded reduction length of weight_packed
-    int tc_mt, tc_bn;               // conv, bf16: tuned tiles per work item and channels per block (0 = default)
+    int tc_mt, tc_bn;               // conv, bf16: tuned tiles per work item (3, 4: patch-reuse kernel with 1, 2) and
+                                    // channels per block (0 = default)
+    void* weight_halo;              // conv, bf16: weights packed for the patch-reuse kernel
     void* in_padded;                // conv, bf16, cin <= 8: input with channels padded to 8
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation

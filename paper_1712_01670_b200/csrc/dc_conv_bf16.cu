@@ -42,6 +42,7 @@ struct TcArgs {
 
 struct SmemCtl {
     unsigned long long full[kMaxStages], empty[kMaxStages], tmem_full[2], tmem_empty[2];
+    unsigned long long a_full[4], a_empty[4];     // halo kernel: ring of input patches
     uint32_t tmem_base;
     volatile int abort_flag;
 };
@@ -232,7 +233,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
-        uint32_t it = 0;
+        int st = 0; uint32_t ph = 0;                              // ring slot and its phase
         bool ok = true;
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const int group = item / a.NB, nb = item % a.NB;
@@ -244,21 +245,23 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                 const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
                 sN[j] = s; xb[j] = tx * DC_TILE_W * a.sw - a.pw; yb[j] = ty * DC_TILE_H * a.sh - a.ph;
             }
-            for (int k = 0; k < kiters && ok; ++k, ++it) {
-                const int tap = k / a.kchunks, cc = k - tap * a.kchunks, ky = tap / a.kw, kx = tap - ky * a.kw;
-                const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
-                if (lane == 0) {
-                    ok = mbar_wait(&ctl->empty[st], ph ^ 1u, ctl, a.status);
-                    if (ok) {
-                        uint8_t* sa = ring + (size_t)st * stage_bytes;
-                        mbar_expect_tx(&ctl->full[st], (uint32_t)stage_bytes);
+            for (int tap = 0; tap < taps && ok; ++tap) {
+                const int ky = tap / a.kw, kx = tap - ky * a.kw;
+                for (int cc = 0; cc < a.kchunks && ok; ++cc) {
+                    if (lane == 0) {
+                        ok = mbar_wait(&ctl->empty[st], ph ^ 1u, ctl, a.status);
+                        if (ok) {
+                            uint8_t* sa = ring + (size_t)st * stage_bytes;
+                            mbar_expect_tx(&ctl->full[st], (uint32_t)stage_bytes);
 #pragma unroll
-                        for (int j = 0; j < MT; ++j)
-                            tma_load_4d(sa + j * a.a_bytes, &tmA, cc * a.BK, xb[j] + kx, yb[j] + ky, sN[j], &ctl->full[st]);
-                        tma_load_2d(sa + MT * a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, nb * a.BN, &ctl->full[st]);
+                            for (int j = 0; j < MT; ++j)
+                                tma_load_4d(sa + j * a.a_bytes, &tmA, cc * a.BK, xb[j] + kx, yb[j] + ky, sN[j], &ctl->full[st]);
+                            tma_load_2d(sa + MT * a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, nb * a.BN, &ctl->full[st]);
+                        }
                     }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (++st == a.stages) { st = 0; ph ^= 1u; }
                 }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
             }
         }
         // on an abort: give the copies already issued a bounded chance to land before the CTA exits
@@ -268,38 +271,42 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         }
     } else if (warp == 1) {
         // ---------------- MMA issuer ----------------
-        uint32_t it = 0, acc_it = 0;
-        bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
-            const uint32_t acc = acc_it % (uint32_t)a.nbuf, acc_ph = (acc_it / (uint32_t)a.nbuf) & 1u;
-            const uint32_t d_tmem = tmem_base + acc * (uint32_t)(MT * a.BN);
-            if (lane == 0) {
+        // Only lane 0 works; descriptors differ from slot to slot in their address bits alone, so the
+        // constant upper half is built once and the loop adds (address >> 4).
+        if (lane == 0) {
+            const uint64_t dconst = umma_desc(0, a.sbo, a.layout_type);
+            const uint32_t ring_lo = smem_u32(ring) >> 4, stage_lo = (uint32_t)stage_bytes >> 4, a_lo = (uint32_t)a.a_bytes >> 4;
+            const int ksteps = a.BK / 16;
+            int st = 0; uint32_t ph = 0, acc = 0, acc_ph = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)(MT * a.BN);
                 ok = mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1u, ctl, a.status);
                 tc_fence_after();
-            }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            for (int k = 0; k < kiters && ok; ++k, ++it) {
-                const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
-                if (lane == 0) {
+                uint32_t accumulate = 0;
+                for (int k = 0; k < kiters && ok; ++k) {
                     ok = mbar_wait(&ctl->full[st], ph, ctl, a.status);
-                    if (ok) {
-                        tc_fence_after();
-                        const uint32_t sa = smem_u32(ring + (size_t)st * stage_bytes);
-                        const uint64_t bdesc = umma_desc(sa + MT * a.a_bytes, a.sbo, a.layout_type);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t adesc0 = dconst + (ring_lo + (uint32_t)st * stage_lo);
+                    const uint64_t bdesc = adesc0 + MT * a_lo;
 #pragma unroll
-                        for (int j = 0; j < MT; ++j) {
-                            const uint64_t adesc = umma_desc(sa + j * a.a_bytes, a.sbo, a.layout_type);
-                            for (int kk = 0; kk < a.BK / 16; ++kk)   // 16 bf16 = 32 bytes = 2 descriptor units
-                                umma_f16(d_tmem + j * a.BN, adesc + 2 * kk, bdesc + 2 * kk, a.idesc, (k | kk) != 0);
+                    for (int j = 0; j < MT; ++j) {
+                        uint32_t acc_j = accumulate;
+                        for (int kk = 0; kk < ksteps; ++kk) {          // 16 bf16 = 32 bytes = 2 descriptor units
+                            umma_f16(d_tmem + j * a.BN, adesc0 + j * a_lo + 2 * kk, bdesc + 2 * kk, a.idesc, acc_j);
+                            acc_j = 1;
                         }
-                        umma_commit(&ctl->empty[st]);                // frees the slot when these MMAs retire
                     }
+                    accumulate = 1;
+                    umma_commit(&ctl->empty[st]);                      // frees the slot when these MMAs retire
+                    if (++st == a.stages) { st = 0; ph ^= 1u; }
                 }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (ok) umma_commit(&ctl->tmem_full[acc]);
+                if (++acc == (uint32_t)a.nbuf) { acc = 0; acc_ph ^= 1u; }
             }
-            if (lane == 0 && ok) umma_commit(&ctl->tmem_full[acc]);
-            __syncwarp();
         }
+        __syncwarp();
     } else {
         // ---------------- epilogue ----------------
         epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane);
@@ -423,6 +430,183 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Input-patch reuse ("halo") variant for stride-1 k x k convolutions with cin a multiple of 64.
+// k_conv_tc fetches the 16x8 input window once per kernel tap (9 x 16 KB for 3x3); here the
+// (16 + kh - 1) x (8 + kw - 1) patch is fetched ONCE per 64-channel chunk and every tap reads it
+// in place.  That needs an operand layout whose rows may start at any patch pixel: the
+// unswizzled core-matrix layout with the patch stored as 8 planes (one per 8 channels = 16
+// bytes) of [patch row][patch column] pixels.  A tile is 8 pixels wide, so the 8 rows of one
+// operand group are the 8 consecutive pixels of one image row, and groups are one patch row
+// (PW x 16 bytes) apart: SBO = PW * 16, LBO = plane size, start = plane + (ky * PW + kx) * 16.
+// Weights are pre-packed per (channel block, tap, chunk) as [k/8][BN][8] and arrive with one
+// plain bulk copy each.
+// ---------------------------------------------------------------------------------------------
+struct TcHaloArgs {
+    TcArgs t;
+    const __nv_bfloat16* wpacked;    // [NB][taps][kchunks][8][BN][8]
+    int PW, PH, plane_bytes, patch_bytes, a_stages;
+};
+
+__device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32_t bytes, void* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+
+template <int MT>
+__global__ void __launch_bounds__(kThreads, 1)
+k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const TcArgs& a = ha.t;
+    const int n_tiles = *a.tile_count;
+    const int n_items = (n_tiles + MT - 1) / MT * a.NB;
+    if ((int)blockIdx.x >= n_items) return;
+    uint8_t* aring = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    const int a_slot = MT * ha.patch_bytes;
+    uint8_t* bring = aring + (size_t)ha.a_stages * a_slot;
+    SmemCtl* ctl = (SmemCtl*)(bring + (size_t)a.stages * a.b_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per_stream = a.tiles_x * a.tiles_y;
+    const int taps = a.kh * a.kw;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < a.stages; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 128); }
+        for (int i = 0; i < 4; ++i) { mbar_init(&ctl->a_full[i], 1); mbar_init(&ctl->a_empty[i], 1); }
+        ctl->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- producer: patches by TMA, weights by bulk copy ----------------
+        int sa = 0, sb = 0; uint32_t pa = 0, pb = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+            const int group = item / a.NB, nb = item % a.NB;
+            int sN[MT], xb[MT], yb[MT];
+#pragma unroll
+            for (int j = 0; j < MT; ++j) {
+                const int idx = group * MT + j;
+                const int tile = a.tile_list[idx < n_tiles ? idx : group * MT];
+                const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+                sN[j] = s; xb[j] = tx * DC_TILE_W - a.pw; yb[j] = ty * DC_TILE_H - a.ph;
+            }
+            for (int cc = 0; cc < a.kchunks && ok; ++cc) {
+                if (lane == 0) {
+                    ok = mbar_wait(&ctl->a_empty[sa], pa ^ 1u, ctl, a.status);
+                    if (ok) {
+                        mbar_expect_tx(&ctl->a_full[sa], (uint32_t)(MT * 8 * ha.PW * ha.PH * 16));
+#pragma unroll
+                        for (int j = 0; j < MT; ++j)
+                            for (int g = 0; g < 8; ++g)
+                                tma_load_4d(aring + (size_t)sa * a_slot + j * ha.patch_bytes + g * ha.plane_bytes, &tmA,
+                                            cc * 64 + g * 8, xb[j], yb[j], sN[j], &ctl->a_full[sa]);
+                    }
+                }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
+                for (int tap = 0; tap < taps && ok; ++tap) {
+                    if (lane == 0) {
+                        ok = mbar_wait(&ctl->empty[sb], pb ^ 1u, ctl, a.status);
+                        if (ok) {
+                            mbar_expect_tx(&ctl->full[sb], (uint32_t)a.b_bytes);
+                            const uint8_t* src = (const uint8_t*)ha.wpacked + ((size_t)(nb * taps + tap) * a.kchunks + cc) * a.b_bytes;
+                            bulk_copy_g2s(bring + (size_t)sb * a.b_bytes, src, (uint32_t)a.b_bytes, &ctl->full[sb]);
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (++sb == a.stages) { sb = 0; pb ^= 1u; }
+                }
+            }
+        }
+        if (!ok && lane == 0) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) { } }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (lane 0 only) ----------------
+        if (lane == 0) {
+            const uint32_t b_lbo = (uint32_t)a.BN * 16u;
+            const uint64_t aconst = umma_desc(0, (uint32_t)ha.PW * 16u, 0, (uint32_t)ha.plane_bytes);
+            const uint64_t bconst = umma_desc(0, 128, 0, b_lbo);
+            const uint32_t aring_lo = smem_u32(aring) >> 4, bring_lo = smem_u32(bring) >> 4;
+            const uint32_t a_slot_lo = (uint32_t)a_slot >> 4, patch_lo = (uint32_t)ha.patch_bytes >> 4;
+            const uint32_t a_kstep = (uint32_t)(2 * ha.plane_bytes) >> 4, b_kstep = (2 * b_lbo) >> 4, b_lo = (uint32_t)a.b_bytes >> 4;
+            int sa = 0, sb = 0; uint32_t pa = 0, pb = 0, acc = 0, acc_ph = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)(MT * a.BN);
+                ok = mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1u, ctl, a.status);
+                tc_fence_after();
+                uint32_t accumulate = 0;
+                for (int cc = 0; cc < a.kchunks && ok; ++cc) {
+                    ok = mbar_wait(&ctl->a_full[sa], pa, ctl, a.status);
+                    const uint64_t apatch = aconst + (aring_lo + (uint32_t)sa * a_slot_lo);
+                    uint32_t tap_lo = 0;                                // (ky * PW + kx) * 16 bytes, in 16-byte units
+                    for (int ky = 0; ky < a.kh && ok; ++ky, tap_lo += (uint32_t)(ha.PW - a.kw)) {
+                        for (int kx = 0; kx < a.kw && ok; ++kx, ++tap_lo) {
+                            ok = mbar_wait(&ctl->full[sb], pb, ctl, a.status);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint64_t bdesc = bconst + (bring_lo + (uint32_t)sb * b_lo);
+#pragma unroll
+                            for (int j = 0; j < MT; ++j) {
+                                const uint64_t adesc = apatch + j * patch_lo + tap_lo;
+                                uint32_t acc_j = accumulate;
+#pragma unroll
+                                for (int kk = 0; kk < 4; ++kk) {        // K = 16: two 8-channel planes
+                                    umma_f16(d_tmem + j * a.BN, adesc + kk * a_kstep, bdesc + kk * b_kstep, a.idesc, acc_j);
+                                    acc_j = 1;
+                                }
+                            }
+                            accumulate = 1;
+                            umma_commit(&ctl->empty[sb]);
+                            if (++sb == a.stages) { sb = 0; pb ^= 1u; }
+                        }
+                    }
+                    if (ok) umma_commit(&ctl->a_empty[sa]);             // the patch is free once its taps retire
+                    if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
+                }
+                if (ok) umma_commit(&ctl->tmem_full[acc]);
+                if (++acc == (uint32_t)a.nbuf) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else {
+        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+    }
+}
+
+// weights [cout][taps][cin] -> [NB][taps][kchunks][8][BN][8]
+__global__ void k_pack_halo(const __nv_bfloat16* w, int cout, int taps, int cin, int BN, __nv_bfloat16* out)
+{
+    const int kchunks = cin / 64;
+    const size_t total = (size_t)cout * taps * cin;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        size_t r = i;
+        const int e = (int)(r & 7); r >>= 3;
+        const int n = (int)(r % BN); r /= BN;
+        const int k8 = (int)(r & 7); r >>= 3;
+        const int cc = (int)(r % kchunks); r /= kchunks;
+        const int tap = (int)(r % taps); const int nb = (int)(r / taps);
+        out[i] = w[((size_t)(nb * BN + n) * taps + tap) * cin + cc * 64 + k8 * 8 + e];
+    }
+}
+
 // [S][H][W][C] -> [S][H][W][8] with zero padding, C <= 8
 __global__ void k_pad_channels8(const __nv_bfloat16* in, size_t pixels, int C, __nv_bfloat16* out)
 {
@@ -496,6 +680,22 @@ bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn =
     return true;
 }
 
+struct HaloPlan { int BN, NB, PW, PH, plane_bytes, patch_bytes, b_bytes; };
+
+bool halo_ok(const dc_layer_desc& d, HaloPlan& h)
+{
+    if (d.kind != DC_CONV || d.sh != 1 || d.sw != 1 || d.cin % 64 != 0 || d.kh * d.kw < 2 || d.kh > 5 || d.kw > 5) return false;
+    h.BN = 0;
+    for (int bn = 256; bn >= 32; bn -= 32) if (d.cout % bn == 0) { h.BN = bn; break; }
+    if (!h.BN) return false;
+    h.NB = d.cout / h.BN;
+    h.PW = DC_TILE_W + d.kw - 1; h.PH = DC_TILE_H + d.kh - 1;
+    h.plane_bytes = (h.PW * h.PH * 16 + 127) & ~127;       // TMA destinations are 128-byte aligned
+    h.patch_bytes = 8 * h.plane_bytes;
+    h.b_bytes = h.BN * 128;
+    return true;
+}
+
 bool smallc_ok(const dc_layer_desc& d)
 {
     return d.kind == DC_CONV && d.sh == 1 && d.sw == 1 && d.cin <= 8 && d.cout % 32 == 0 && d.cout <= 256 &&
@@ -518,6 +718,16 @@ int dc_pack_weights_bf16(dc_cache* c, int layer)
 {
     dc_layer_rt& L = c->L[layer];
     TcPlan p;
+    HaloPlan h;
+    if (halo_ok(L.d, h) && !getenv("DC_CONV_NO_HALO")) {
+        const size_t n = (size_t)L.d.cout * L.d.kh * L.d.kw * L.d.cin;
+        DC_CUDA(cudaMalloc(&L.weight_halo, n * 2));
+        c->bytes += n * 2;
+        int grid = (int)((n + 255) / 256); if (grid > c->num_sms * 8) grid = c->num_sms * 8;
+        k_pack_halo<<<grid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, L.d.cout, L.d.kh * L.d.kw, L.d.cin, h.BN,
+                                                 (__nv_bfloat16*)L.weight_halo);
+        DC_CUDA(cudaGetLastError());
+    }
     if (make_plan(L.d, p) || !smallc_ok(L.d)) return DC_OK;
     const int taps = L.d.kh * L.d.kw, kblocks = (taps + 1) / 2 * 2;
     const size_t wbytes = (size_t)kblocks * L.d.cout * 16, pbytes = (size_t)c->S * L.in_h * L.in_w * 16;
@@ -579,11 +789,65 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     return DC_OK;
 }
 
+static int launch_halo(dc_cache* c, int layer, int mt, const void* in, void* out, const int32_t* tile_list,
+                       const int32_t* tile_count, const uint32_t* masks, int max_tiles)
+{
+    dc_layer_rt& L = c->L[layer];
+    const dc_layer_desc& d = L.d;
+    HaloPlan h;
+    EncodeTiledFn enc = encode_fn();
+    if (!enc || !L.weight_halo || !halo_ok(d, h)) return DC_ERR_CONFIG;
+    CUtensorMap tmA;
+    cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
+    cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
+    cuuint32_t box[4] = {8, (cuuint32_t)h.PW, (cuuint32_t)h.PH, 1};
+    cuuint32_t estr[4] = {1, 1, 1, 1};
+    if (enc(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return DC_ERR_CUDA;
+    TcHaloArgs ha;
+    TcArgs& a = ha.t;
+    a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
+    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
+    a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
+    a.BN = h.BN; a.NB = h.NB; a.BK = 64; a.kchunks = d.cin / 64; a.MT = mt; a.nbuf = mt * h.BN * 2 <= 512 ? 2 : 1;
+    a.a_bytes = 0; a.b_bytes = h.b_bytes; a.sbo = 128; a.layout_type = 0;
+    a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(h.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+    a.status = c->status;
+    ha.wpacked = (const __nv_bfloat16*)L.weight_halo;
+    ha.PW = h.PW; ha.PH = h.PH; ha.plane_bytes = h.plane_bytes; ha.patch_bytes = h.patch_bytes;
+    // patch ring: as deep as leaves at least 3 weight stages (a small-K item is one patch, so depth = items in flight)
+    ha.a_stages = 2;
+    for (int as = 4; as > 2; --as)
+        if (200 * 1024 - as * mt * h.patch_bytes >= 3 * h.b_bytes) { ha.a_stages = as; break; }
+    if (getenv("DC_HALO_ASTAGES")) ha.a_stages = atoi(getenv("DC_HALO_ASTAGES"));
+    const int a_total = ha.a_stages * mt * h.patch_bytes;
+    int st = (200 * 1024 - a_total) / h.b_bytes;
+    a.stages = st > kMaxStages ? kMaxStages : st;
+    if (a.stages < 2) return DC_ERR_CONFIG;
+    const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + sizeof(SmemCtl) + 256;
+    static bool attr_set = false;
+    if (!attr_set) {
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        attr_set = true;
+    }
+    long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + mt - 1) / mt) * h.NB;
+    int grid = items > c->num_sms ? c->num_sms : (int)items;
+    dc_prof_scope ps(c, DC_ST_CONV);
+    if (mt == 2) k_conv_tc_halo<2><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+    else k_conv_tc_halo<1><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+    c->launches += 1;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
+
 int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
     const dc_layer_desc& d = L.d;
+    if (L.tc_mt >= 3) return launch_halo(c, layer, L.tc_mt - 2, in, out, tile_list, tile_count, masks, max_tiles);
     TcPlan p;
     if (!make_plan(d, p, L.tc_mt, L.tc_bn)) {
         if (smallc_ok(d)) return launch_smallc(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
@@ -670,6 +934,24 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
             if (ms < best) { best = ms; best_mt = mt; best_bn = bn; }
         }
     }
+    HaloPlan h;
+    if (L.weight_halo && halo_ok(L.d, h)) {
+        for (int mt = 1; mt <= 2; ++mt) {                          // tc_mt 3 / 4: patch-reuse kernel with 1 / 2 tiles per item
+            L.tc_mt = mt + 2; L.tc_bn = 0;
+            int rc = DC_OK;
+            for (int rep = 0; rep < 3 && rc == DC_OK; ++rep) {
+                if (rep == 1) cudaEventRecord(e0, c->stream);
+                rc = dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles);
+            }
+            cudaEventRecord(e1, c->stream);
+            if (rc != DC_OK || cudaEventSynchronize(e1) != cudaSuccess) { cudaGetLastError(); continue; }
+            float ms = 0.f;
+            cudaEventElapsedTime(&ms, e0, e1);
+            if (getenv("DC_VERBOSE")) fprintf(stderr, "libdeepcache: layer %d: patch-reuse kernel, %d tile(s) per item: %.3f ms\n", layer, mt, ms / 2);
+            if (ms < best) { best = ms; best_mt = mt + 2; best_bn = 0; }
+        }
+    }
+    if (getenv("DC_CONV_FORCE_HALO") && L.weight_halo) { best_mt = atoi(getenv("DC_CONV_FORCE_HALO")) + 2; best_bn = 0; }
     L.tc_mt = best_mt; L.tc_bn = best_bn;
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     c->launches = 0;
