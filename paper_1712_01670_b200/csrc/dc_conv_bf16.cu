@@ -45,6 +45,9 @@ struct SmemCtl {
     unsigned long long a_full[4], a_empty[4];     // halo kernel: ring of input patches
     uint32_t tmem_base;
     volatile int abort_flag;
+    // epilogue staging: per warp 32 pixels x 64 bytes (32 bf16 channels), rows padded to 80 bytes so
+    // 16-byte accesses of neighbouring lanes fall in different banks
+    __align__(16) uint8_t stage[4][32 * 80];
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -60,6 +63,12 @@ __device__ __forceinline__ void mbar_expect_tx(void* bar, uint32_t bytes)
 __device__ __forceinline__ void mbar_arrive(void* bar)
 {
     asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+// Arrival that orders nothing but the barrier itself: used to hand a TMEM accumulator back (its reads are
+// ordered by tcgen05.wait::ld + tcgen05.fence), so the arrival need not wait for the epilogue's global stores.
+__device__ __forceinline__ void mbar_arrive_relaxed(void* bar)
+{
+    asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ bool mbar_try(void* bar, uint32_t parity)
 {
@@ -153,47 +162,81 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
     const int per_stream = a.tiles_x * a.tiles_y;
     const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
     const int m = q * 32 + lane, prow = m / DC_TILE_W, pcol = m % DC_TILE_W;
-    uint32_t acc_it = 0;
+    const int mword_i = DC_TILE_BIT(prow, pcol) >> 5, mbit = DC_TILE_BIT(prow, pcol) & 31;
+    uint32_t acc = 0, acc_ph = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++acc_it) {
-        const uint32_t acc = acc_it % (uint32_t)a.nbuf, acc_ph = (acc_it / (uint32_t)a.nbuf) & 1u;
-        const int group = item / a.NB, nb = item % a.NB;
+    // the tile index and this pixel's bitmap word of the NEXT item are fetched while the current one is
+    // processed: two dependent global loads would otherwise sit on every item's critical path
+    int tile_n[2] = {-1, -1}; uint32_t mask_n[2] = {0, 0};
+    auto fetch = [&](int item) {
+        if (item >= n_items) return;
+        const int group = item / a.NB;
+        for (int j = 0; j < a.MT; ++j) {
+            const int idx = group * a.MT + j;
+            tile_n[j] = idx < n_tiles ? a.tile_list[idx] : -1;   // odd tile count: the last item has one tile
+            mask_n[j] = tile_n[j] >= 0 ? a.masks[(size_t)tile_n[j] * 4 + mword_i] : 0u;
+        }
+    };
+    fetch(blockIdx.x);
+    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+        const int nb = item % a.NB;
+        const int tile_c[2] = {tile_n[0], tile_n[1]};
+        const uint32_t mask_c[2] = {mask_n[0], mask_n[1]};
+        fetch(item + gridDim.x);
         ok = mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, a.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
         const float* bias = a.bias + nb * a.BN;
         for (int j = 0; j < a.MT; ++j) {
-            if (group * a.MT + j >= n_tiles) break;             // odd tile count: the last item has one tile
-            const int tile = a.tile_list[group * a.MT + j];
+            const int tile = tile_c[j];
+            if (tile < 0) break;
             const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
             const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
-            const uint32_t mword = a.masks[(size_t)tile * 4 + (DC_TILE_BIT(prow, pcol) >> 5)];
-            const bool reused = (mword >> (DC_TILE_BIT(prow, pcol) & 31)) & 1u;
+            const bool reused = (mask_c[j] >> mbit) & 1u;
             const bool active = oy < a.Ho && ox < a.Wo && !reused;
-            __nv_bfloat16* op = a.out + (((size_t)s * a.Ho + oy) * a.Wo + ox) * a.Co + nb * a.BN;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (acc * (uint32_t)a.MT + (uint32_t)j) * (uint32_t)a.BN;
+            // Each lane owns one pixel (TMEM lane) and gets 32 channels = 64 bytes per step.  Storing them
+            // directly would make every warp store touch 32 different lines 16 bytes at a time (half-written
+            // sectors); instead the warp stages its 32 x 64 bytes in shared memory and writes them back with
+            // 4 lanes per pixel, so each pixel's 64 bytes leave as two whole sectors.
+            const unsigned act_mask = __ballot_sync(0xffffffffu, active);
+            uint8_t* stg = ctl->stage[q];
             for (int c = 0; c < a.BN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld32(taddr + c * 32, r);
                 tmem_ld_wait();
-                if (active) {
-                    uint4* dst = (uint4*)(op + c * 32);
+                const float4* b4 = (const float4*)(bias + c * 32);
+                uint4* mine = (uint4*)(stg + lane * 80);
 #pragma unroll
-                    for (int v = 0; v < 4; ++v) {
-                        float f[8];
+                for (int v = 0; v < 4; ++v) {
+                    const float4 ba = __ldg(b4 + 2 * v), bb = __ldg(b4 + 2 * v + 1);
+                    float f[8] = {__uint_as_float(r[v * 8 + 0]) + ba.x, __uint_as_float(r[v * 8 + 1]) + ba.y,
+                                  __uint_as_float(r[v * 8 + 2]) + ba.z, __uint_as_float(r[v * 8 + 3]) + ba.w,
+                                  __uint_as_float(r[v * 8 + 4]) + bb.x, __uint_as_float(r[v * 8 + 5]) + bb.y,
+                                  __uint_as_float(r[v * 8 + 6]) + bb.z, __uint_as_float(r[v * 8 + 7]) + bb.w};
+                    if (a.relu) {
 #pragma unroll
-                        for (int jj = 0; jj < 8; ++jj) {
-                            f[jj] = __uint_as_float(r[v * 8 + jj]) + __ldg(bias + c * 32 + v * 8 + jj);
-                            if (a.relu) f[jj] = fmaxf(f[jj], 0.f);
-                        }
-                        dst[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                        for (int jj = 0; jj < 8; ++jj) f[jj] = fmaxf(f[jj], 0.f);
+                    }
+                    mine[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                }
+                __syncwarp();
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int piece = lane + 32 * k, pl = piece >> 2, part = piece & 3;    // pixel (lane) pl of this warp, 16-byte part
+                    if ((act_mask >> pl) & 1u) {
+                        const int mm = q * 32 + pl, pr = mm / DC_TILE_W, pc = mm % DC_TILE_W;
+                        __nv_bfloat16* o2 = a.out + (((size_t)s * a.Ho + ty * DC_TILE_H + pr) * a.Wo + tx * DC_TILE_W + pc) * a.Co + nb * a.BN + c * 32;
+                        ((uint4*)o2)[part] = *(const uint4*)(stg + pl * 80 + part * 16);
                     }
                 }
+                __syncwarp();
             }
         }
         tc_fence_before();
-        mbar_arrive(&ctl->tmem_empty[acc]);
+        mbar_arrive_relaxed(&ctl->tmem_empty[acc]);
+        if (++acc == (uint32_t)a.nbuf) { acc = 0; acc_ph ^= 1u; }
     }
 }
 
@@ -322,16 +365,19 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 // ---------------------------------------------------------------------------------------------
 // Few input channels (cin <= 8, e.g. the first layer on RGB): the channels are padded to 8
 // (16 bytes per pixel) and the kernel taps are laid side by side along K: K = taps * 8, padded to
-// a multiple of 16.  Operands use the unswizzled core-matrix layout: per tap one TMA box lands as
-// 128 rows x 16 bytes (= 16 core matrices 128 bytes apart), consecutive taps 2048 bytes apart,
-// so one tcgen05.mma (K = 16) consumes two taps.  The packed weights ([K/8][cout][8]) stay in
-// shared memory for the whole kernel.  A whole work item is one pipeline stage.
+// a multiple of 16.  Operands use the unswizzled core-matrix layout.  ONE TMA box per tile brings the
+// (16 + kh - 1) x (8 + kw - 1) input patch as pixels of 16 bytes; the rows of tap (ky, kx) are the
+// patch pixels starting at (ky * PW + kx), one patch row (PW x 16 bytes) between 8-row groups, so
+// every tap is read in place, and one tcgen05.mma (K = 16) consumes two taps whose pixel offsets
+// differ by the descriptor's leading-dimension offset.  The packed weights ([K/8][cout][8]) stay
+// in shared memory for the whole kernel.  A whole work item is one pipeline stage.
 // ---------------------------------------------------------------------------------------------
 struct TcSmallArgs {
     TcArgs t;                     // shared fields (BN = cout, NB = 1)
     const __nv_bfloat16* wpacked; // [kblocks][cout][8]
     int kblocks;                  // K / 8 (even); taps = kh * kw real ones, the rest zero
     int w_bytes;                  // kblocks * cout * 16
+    int PW, PH, stage_bytes;      // input patch per tile: (8 + kw - 1) x (16 + kh - 1) pixels of 16 bytes, + pad
 };
 
 __global__ void __launch_bounds__(kThreads, 1)
@@ -343,9 +389,8 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
     if ((int)blockIdx.x >= n_items) return;
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     uint8_t* wsm = base;                                        // packed weights
-    const int stage_bytes = sa.kblocks * 2048;
     uint8_t* ring = wsm + ((sa.w_bytes + 127) & ~127);
-    SmemCtl* ctl = (SmemCtl*)(ring + (size_t)a.stages * stage_bytes);
+    SmemCtl* ctl = (SmemCtl*)(ring + (size_t)a.stages * sa.stage_bytes);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int per_stream = a.tiles_x * a.tiles_y;
     const int taps = a.kh * a.kw;
@@ -357,14 +402,13 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     }
-    // weights into shared memory; zero the tap slots no TMA box ever fills (their weights are zero too,
-    // but 0 x garbage could be NaN)
+    // weights into shared memory; zero the ring once: each slot ends in a pad that no TMA box fills but
+    // the last (zero-weight) K block reads, and 0 x garbage could be NaN
     for (int i = threadIdx.x; i < sa.w_bytes / 16; i += kThreads)
         ((uint4*)wsm)[i] = __ldg((const uint4*)sa.wpacked + i);
-    for (int st = 0; st < a.stages; ++st)
-        for (int i = threadIdx.x; i < (sa.kblocks - taps) * 128; i += kThreads)
-            ((uint4*)(ring + (size_t)st * stage_bytes + taps * 2048))[i] = make_uint4(0, 0, 0, 0);
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to the MMA
+    for (int i = threadIdx.x; i < a.stages * sa.stage_bytes / 16; i += kThreads)
+        ((uint4*)ring)[i] = make_uint4(0, 0, 0, 0);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to TMA / MMA
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -375,50 +419,57 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
     const uint32_t tmem_base = ctl->tmem_base;
 
     if (warp == 0) {
-        uint32_t it = 0;
-        bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
-            const int tile = a.tile_list[item];
-            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
-            const int x_base = tx * DC_TILE_W - a.pw, y_base = ty * DC_TILE_H - a.ph;
-            const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
-            if (lane == 0) {
+        if (lane == 0) {                                        // producer: one patch per item
+            int st = 0; uint32_t ph = 0;
+            bool ok = true;
+            int tile_next = a.tile_list[blockIdx.x];            // fetched one item ahead: off the critical path
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+                const int tile = tile_next;
+                if (item + (int)gridDim.x < n_items) tile_next = a.tile_list[item + gridDim.x];
+                const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
                 ok = mbar_wait(&ctl->empty[st], ph ^ 1u, ctl, a.status);
-                if (ok) {
-                    uint8_t* dst = ring + (size_t)st * stage_bytes;
-                    mbar_expect_tx(&ctl->full[st], (uint32_t)(taps * 2048));
-                    for (int tap = 0; tap < taps; ++tap)
-                        tma_load_4d(dst + tap * 2048, &tmA, 0, x_base + tap % a.kw, y_base + tap / a.kw, s, &ctl->full[st]);
-                }
+                if (!ok) break;
+                mbar_expect_tx(&ctl->full[st], (uint32_t)(sa.PW * sa.PH * 16));
+                tma_load_4d(ring + (size_t)st * sa.stage_bytes, &tmA, 0, tx * DC_TILE_W - a.pw, ty * DC_TILE_H - a.ph, s, &ctl->full[st]);
+                if (++st == a.stages) { st = 0; ph ^= 1u; }
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
+            if (!ok) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) { } }
         }
-        if (!ok && lane == 0) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) { } }
+        __syncwarp();
     } else if (warp == 1) {
-        uint32_t it = 0;
-        bool ok = true;
-        for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++it) {
-            const uint32_t acc = it & 1u, acc_ph = (it >> 1) & 1u;
-            const int st = it % a.stages; const uint32_t ph = (it / a.stages) & 1u;
-            if (lane == 0) {
+        if (lane == 0) {                                        // MMA issuer
+            const uint32_t b_lbo = (uint32_t)a.Co * 16u;
+            const uint64_t bconst = umma_desc(smem_u32(wsm), 128, 0, b_lbo);
+            const uint32_t ring_lo = smem_u32(ring) >> 4, stage_lo = (uint32_t)sa.stage_bytes >> 4;
+            const uint64_t hi = umma_desc(0, (uint32_t)sa.PW * 16u, 0, 0);     // SBO = one patch row; LBO added per K step
+            int st = 0; uint32_t ph = 0, acc = 0, acc_ph = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
                 ok = mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1u, ctl, a.status);
                 if (ok) ok = mbar_wait(&ctl->full[st], ph, ctl, a.status);
-                if (ok) {
-                    tc_fence_after();
-                    const uint32_t d_tmem = tmem_base + acc * (uint32_t)a.BN;
-                    const uint32_t sa_addr = smem_u32(ring + (size_t)st * stage_bytes), sb_addr = smem_u32(wsm);
-                    const uint32_t b_lbo = (uint32_t)a.Co * 16u;
-                    for (int kk = 0; kk < sa.kblocks / 2; ++kk) {
-                        const uint64_t adesc = umma_desc(sa_addr + kk * 4096, 128, 0, 2048);
-                        const uint64_t bdesc = umma_desc(sb_addr + kk * 2 * b_lbo, 128, 0, b_lbo);
-                        umma_f16(d_tmem, adesc, bdesc, a.idesc, kk != 0);
-                    }
-                    umma_commit(&ctl->empty[st]);
-                    umma_commit(&ctl->tmem_full[acc]);
+                if (!ok) break;
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)a.BN;
+                const uint32_t patch_lo = ring_lo + (uint32_t)st * stage_lo;
+                // K step kk covers taps 2kk and 2kk+1: two 16-byte pixel columns of the patch, `lbo` apart
+                int tap = 0, ky = 0, kx = 0;
+                for (int kk = 0; kk < sa.kblocks / 2; ++kk) {
+                    const uint32_t off0 = (uint32_t)(ky * sa.PW + kx);
+                    if (++kx == a.kw) { kx = 0; ++ky; }
+                    ++tap;
+                    uint32_t off1 = off0 + 1;                      // past the last tap: any finite data (its weights are zero)
+                    if (tap < taps) { off1 = (uint32_t)(ky * sa.PW + kx); if (++kx == a.kw) { kx = 0; ++ky; } }
+                    ++tap;
+                    const uint64_t adesc = hi + (patch_lo + off0) + ((uint64_t)(off1 - off0) << 16);
+                    umma_f16(d_tmem, adesc, bconst + (uint64_t)(kk * ((2 * b_lbo) >> 4)), a.idesc, kk != 0);
                 }
+                umma_commit(&ctl->empty[st]);
+                umma_commit(&ctl->tmem_full[acc]);
+                if (++st == a.stages) { st = 0; ph ^= 1u; }
+                if (++acc == 2u) { acc = 0; acc_ph ^= 1u; }
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
         }
+        __syncwarp();
     } else {
         epilogue_loop(a, ctl, tmem_base, n_items, n_items, warp, lane);
     }
@@ -752,7 +803,8 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     CUtensorMap tmA;
     cuuint64_t dims[4] = {8, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
     cuuint64_t strides[3] = {16, (cuuint64_t)L.in_w * 16, (cuuint64_t)L.in_h * L.in_w * 16};
-    cuuint32_t box[4] = {8, DC_TILE_W, DC_TILE_H, 1};
+    const int PW = DC_TILE_W + d.kw - 1, PH = DC_TILE_H + d.kh - 1;
+    cuuint32_t box[4] = {8, (cuuint32_t)PW, (cuuint32_t)PH, 1};
     cuuint32_t estr[4] = {1, 1, 1, 1};
     if (enc(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, L.in_padded, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
             CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
@@ -768,7 +820,9 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     sa.wpacked = (const __nv_bfloat16*)L.weight_packed;
     sa.kblocks = L.k_packed / 8;
     sa.w_bytes = sa.kblocks * d.cout * 16;
-    const int stage_bytes = sa.kblocks * 2048;
+    sa.PW = PW; sa.PH = PH;
+    sa.stage_bytes = (PW * PH * 16 + 128 + 127) & ~127;          // patch + a readable pad behind its last pixel
+    const int stage_bytes = sa.stage_bytes;
     int st = (200 * 1024 - sa.w_bytes) / stage_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
