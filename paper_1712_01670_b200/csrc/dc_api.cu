@@ -119,6 +119,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     DC_TRY(dev_alloc(c, &c->blk_mv, nblk * 2));
     DC_TRY(dev_alloc(c, &c->blk_sse, nblk));
     DC_TRY(dev_alloc(c, &c->matched, nblk));
+    DC_TRY(dev_alloc(c, &c->run_end, nblk));
     DC_TRY(dev_alloc(c, &c->mv_acc, (size_t)S * 4 + 4));
     DC_TRY(dev_alloc(c, &c->long_list, nblk));
     DC_TRY(dev_alloc(c, &c->gmv, (size_t)S * 3));
@@ -129,7 +130,8 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     DC_TRY(dev_alloc(c, &c->in_hw_dev, (size_t)n * 2));
     DC_TRY(dev_alloc(c, &c->dirty_count, (size_t)n));
     DC_TRY(dev_alloc(c, &c->all_count, (size_t)n));
-    DC_TRY(dev_alloc(c, &c->reuse_px, (size_t)n * S));
+    DC_TRY(dev_alloc(c, &c->reuse_px, (size_t)n * S * 2));
+    c->alive = c->reuse_px + (size_t)n * S;
     DC_TRY(dev_alloc(c, &c->status, (size_t)1));
     DC_TRY(dev_alloc(c, &c->reused_total, (size_t)n));
     DC_CUDA(cudaMemsetAsync(c->reused_total, 0, sizeof(unsigned long long) * n, c->stream));
@@ -219,7 +221,7 @@ void release(dc_cache* c)
 {
     dc_prof_release(c);
     cudaFree(c->reused_total);
-    cudaFree(c->key[0]); cudaFree(c->key[1]); cudaFree(c->staging); cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched);
+    cudaFree(c->key[0]); cudaFree(c->key[1]); cudaFree(c->staging); cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched); cudaFree(c->run_end);
     cudaFree(c->mv_acc); cudaFree(c->long_list); cudaFree(c->gmv); cudaFree(c->regions0); cudaFree(c->n_regions); cudaFree(c->table);
     cudaFree(c->layers_dev); cudaFree(c->in_hw_dev); cudaFree(c->dirty_count); cudaFree(c->all_count);
     cudaFree(c->reuse_px); cudaFree(c->zero_masks); cudaFree(c->status); cudaFree(c->input_map); cudaFree(c->pix_lut);
@@ -361,6 +363,7 @@ int dc_propagate_regions(dc_cache* c, const dc_region* in_dev, const int32_t* n_
     const size_t per_layer = (size_t)c->S * c->max_regions;
     // slots beyond n_in keep whatever an earlier call left: clear the table first
     DC_CUDA(cudaMemsetAsync(c->table, 0, sizeof(dc_region) * per_layer * layer_end, c->stream));
+    DC_CUDA(cudaMemsetAsync(c->alive, 0, sizeof(int32_t) * c->n_layers * c->S, c->stream));
     DC_TRY(dc_launch_propagate(c, in_dev, n_in_dev, layer_end));
     DC_CUDA(cudaMemcpyAsync(out_dev, c->table + per_layer * layer_begin,
                             sizeof(dc_region) * per_layer * (layer_end - layer_begin), cudaMemcpyDeviceToDevice, c->stream));
@@ -400,7 +403,7 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
     DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, frame_copy));
     if (!refresh) {
         DC_CUDA(cudaMemsetAsync(c->dirty_count, 0, sizeof(int32_t) * n, c->stream));
-        DC_CUDA(cudaMemsetAsync(c->reuse_px, 0, sizeof(int32_t) * n * S, c->stream));
+        DC_CUDA(cudaMemsetAsync(c->reuse_px, 0, sizeof(int32_t) * n * S * 2, c->stream));     // and `alive` behind it
         DC_TRY(dc_launch_match(c));
         DC_TRY(dc_launch_propagate(c, c->regions0, c->n_regions, n));
     }

@@ -70,6 +70,7 @@ struct dc_cache {
     int16_t* blk_mv;                // [S][Gy][Gx][2]
     uint32_t* blk_sse;              // [S][Gy][Gx]
     uint8_t* matched;               // [S][Gy][Gx]
+    uint16_t* run_end;              // [S][Gy][Gx] Step 5: end column of the run starting at each block, else 0
     int32_t* mv_acc;                // [S][4]: sum dx, sum dy, K, n_matched; then 4 words of counters
     uint4* long_list;               // [S][Gy][Gx] diamond walks handed to the second search phase
     int32_t* gmv;                   // [S][3]: Mx, My, K
@@ -81,6 +82,7 @@ struct dc_cache {
     int32_t* dirty_count;           // [n_layers]
     int32_t* all_count;             // [n_layers]
     int32_t* reuse_px;              // [n_layers][S]
+    int32_t* alive;                 // [n_layers][S] rectangles not yet eroded away (directly behind reuse_px)
     uint32_t* zero_masks;           // all-zero reuse bitmap shared by full frames
     int32_t* status;                // device status word
     void* input_map;                // frame / 255 as a map, [S][H][W][3]

@@ -11,8 +11,8 @@
 //              and points already scored by the previous diamond are skipped (they cannot win).
 //   k_verify   Steps 3-4: rounds the mean vector M, scores every block at M (reusing the Step 2
 //              score when the block's own best vector is M).
-//   k_merge    Step 5: maximal horizontal runs, merged vertically when spans are identical,
-//              emitted in (y, x) order by a block-wide scan.
+//   k_merge_runs, k_merge   Step 5: maximal horizontal runs per block row, merged vertically when the
+//              spans are identical, emitted in (y, x) order by a CTA-wide ordered compaction.
 #include "dc_common.cuh"
 
 namespace {
@@ -212,49 +212,61 @@ __global__ void __launch_bounds__(WARPS * 32) k_verify(MatchArgs a)
     }
 }
 
-// Step 5.  One CTA per stream.
-__global__ void __launch_bounds__(256) k_merge(const uint8_t* matched, const int32_t* gmv, int W, int H, int B,
-                                               int Gx, int Gy, int max_regions, dc_region* regions,
-                                               int32_t* n_regions, int32_t* status)
+// Step 5, part 1: for every block that starts a maximal horizontal run of matched blocks, the column
+// where the run ends; 0 for every other block (an end is never 0).  One thread per block; the forward
+// scan of a run start stays inside one row of bytes (cache hits after the first touch).
+__global__ void k_merge_runs(const uint8_t* matched, int Gx, int total, uint16_t* run_end)
 {
-    __shared__ int warp_sums[8];
+    const int b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b >= total) return;
+    const int c = b % Gx;
+    uint16_t e = 0;
+    if (matched[b] && (c == 0 || !matched[b - 1])) {
+        int j = c + 1;
+        while (j < Gx && matched[b - c + j]) ++j;
+        e = (uint16_t)j;
+    }
+    run_end[b] = e;
+}
+
+// Step 5, part 2: a run continues the rectangle above it only when the run directly above starts and
+// ends at the same columns; every other run heads a rectangle that extends down while that holds.
+// One CTA per stream; heads are emitted in (y, x) order by a CTA-wide ordered compaction.
+__global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const int32_t* gmv, int W, int H, int B,
+                                                int Gx, int Gy, int max_regions, dc_region* regions,
+                                                int32_t* n_regions, int32_t* status)
+{
+    __shared__ int warp_sums[32];
     __shared__ int base;
     const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
-    const uint8_t* m = matched + (size_t)s * Gx * Gy;
+    const uint16_t* e = run_end + (size_t)s * Gx * Gy;
     dc_region* out = regions + (size_t)s * max_regions;
     const int Mx = gmv[3 * s], My = gmv[3 * s + 1];
     if (tid == 0) base = 0;
     __syncthreads();
-    auto same_run = [&](int r, int c0, int c1) {      // row r has a maximal run exactly [c0, c1)
-        if (c0 > 0 && m[r * Gx + c0 - 1]) return false;
-        if (c1 < Gx && m[r * Gx + c1]) return false;
-        for (int c = c0; c < c1; ++c) if (!m[r * Gx + c]) return false;
-        return true;
-    };
-    for (int start = 0; start < Gx * Gy; start += 256) {
-        int b = start + tid, head = 0, c1 = 0, h = 0, r = 0, c0 = 0;
+    for (int start = 0; start < Gx * Gy; start += 1024) {
+        const int b = start + tid;
+        int head = 0, c1 = 0, h = 0, r = 0, c0 = 0;
         if (b < Gx * Gy) {
             r = b / Gx; c0 = b - r * Gx;
-            if (m[b] && (c0 == 0 || !m[b - 1])) {
-                c1 = c0; while (c1 < Gx && m[r * Gx + c1]) ++c1;
-                if (!(r > 0 && same_run(r - 1, c0, c1))) {
-                    head = 1; h = 1;
-                    while (r + h < Gy && same_run(r + h, c0, c1)) ++h;
-                }
+            c1 = e[b];
+            if (c1 != 0 && !(r > 0 && e[b - Gx] == c1)) {
+                head = 1; h = 1;
+                while (r + h < Gy && e[b + h * Gx] == c1) ++h;
             }
         }
-        // ordered compaction: exclusive scan of `head` over the 256 threads
-        unsigned bal = __ballot_sync(0xffffffffu, head);
-        int pre = __popc(bal & ((1u << lane) - 1u));
+        // ordered compaction: exclusive scan of `head` over the 1024 threads
+        const unsigned bal = __ballot_sync(0xffffffffu, head);
+        const int pre = __popc(bal & ((1u << lane) - 1u));
         if (lane == 0) warp_sums[wid] = __popc(bal);
         __syncthreads();
         int woff = 0, total = 0;
-        for (int i = 0; i < 8; ++i) { if (i < wid) woff += warp_sums[i]; total += warp_sums[i]; }
-        int idx = base + woff + pre;
+        for (int i = 0; i < 32; ++i) { const int v = warp_sums[i]; if (i < wid) woff += v; total += v; }
+        const int idx = base + woff + pre;
         if (head) {
             if (idx < max_regions) {
-                int x = c0 * B, y = r * B;
-                int x1 = min(c1 * B, W), y1 = min((r + h) * B, H);
+                const int x = c0 * B, y = r * B;
+                const int x1 = min(c1 * B, W), y1 = min((r + h) * B, H);
                 dc_region g = { x, y, x1 - x, y1 - y, x + Mx, y + My };
                 out[idx] = g;
             } else {
@@ -672,10 +684,11 @@ int dc_launch_match(dc_cache* c)
     }
     {
         dc_prof_scope ps(c, DC_ST_MERGE);
-        k_merge<<<c->S, 256, 0, c->stream>>>(c->matched, c->gmv, a.W, a.H, a.B, a.Gx, a.Gy, c->max_regions,
-                                             c->regions0, c->n_regions, c->status);
+        k_merge_runs<<<dc_div_up(c->S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(c->matched, a.Gx, c->S * a.Gx * a.Gy, c->run_end);
+        k_merge<<<c->S, 1024, 0, c->stream>>>(c->run_end, c->gmv, a.W, a.H, a.B, a.Gx, a.Gy, c->max_regions,
+                                              c->regions0, c->n_regions, c->status);
     }
-    c->launches += 3;
+    c->launches += 4;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
 }

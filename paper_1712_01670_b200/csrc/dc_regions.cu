@@ -79,7 +79,7 @@ __device__ dc_region apply_layer(const dc_layer_desc& L, int in_h, int in_w, dc_
 }
 
 __global__ void k_propagate(const dc_layer_desc* layers, const int32_t* in_hw, int layer_end, int S, int max_regions,
-                            const dc_region* in, const int32_t* n_in, dc_region* table)
+                            const dc_region* in, const int32_t* n_in, dc_region* table, int32_t* alive)
 {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     int s = blockIdx.y;
@@ -92,7 +92,9 @@ __global__ void k_propagate(const dc_layer_desc* layers, const int32_t* in_hw, i
         dc_region a = L.in0 < 0 ? r0 : table[L.in0 * layer_stride + slot];
         dc_region b = a;
         if (L.kind == DC_ADD || L.kind == DC_CONCAT) b = L.in1 < 0 ? r0 : table[L.in1 * layer_stride + slot];
-        table[l * layer_stride + slot] = apply_layer(L, in_hw[2 * l], in_hw[2 * l + 1], a, b);
+        const dc_region o = apply_layer(L, in_hw[2 * l], in_hw[2 * l + 1], a, b);
+        table[l * layer_stride + slot] = o;
+        if (o.w > 0 && alive) atomicAdd(&alive[l * S + s], 1);     // rectangles still alive at this layer
     }
 }
 
@@ -102,6 +104,7 @@ struct ClassifyArgs {
     int Ho, Wo, px_bytes;                        // px_bytes = cout * element size (multiple of 16)
     int tiles_x, tiles_y, S;
     uint32_t* masks; int32_t* dirty_list; int32_t* dirty_count; int32_t* reuse_px;
+    const int32_t* alive;                        // per stream: rectangles alive at this layer, or NULL (unknown)
     unsigned long long* reused_total;
 };
 
@@ -115,7 +118,8 @@ __global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
     const int X0 = tx * DC_TILE_W, Y0 = ty * DC_TILE_H;
     const int X1 = min(X0 + DC_TILE_W, a.Wo), Y1 = min(Y0 + DC_TILE_H, a.Ho);
     const dc_region* regs = a.regions + (size_t)s * a.max_regions;
-    const int n = a.n_regions[s];
+    // every rectangle of this stream has eroded away before this layer: nothing to test or copy
+    const int n = (a.alive && a.alive[s] == 0) ? 0 : a.n_regions[s];
     const size_t map_base = (size_t)s * a.Ho * a.Wo * a.px_bytes;
     uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;      // bit (row * DC_TILE_W + col) of the tile, row-major
     for (int base = 0; base < n; base += 32) {
@@ -176,7 +180,7 @@ int dc_launch_propagate(dc_cache* c, const dc_region* in, const int32_t* n_in, i
     {
         dc_prof_scope ps(c, DC_ST_PROPAGATE);
         k_propagate<<<grid, 128, 0, c->stream>>>(c->layers_dev, c->in_hw_dev, layer_end, c->S, c->max_regions,
-                                                 in, n_in, c->table);
+                                                 in, n_in, c->table, c->alive);
     }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
@@ -195,6 +199,7 @@ int dc_launch_classify_copy(dc_cache* c, int layer, const dc_region* regions, co
     a.masks = L.masks; a.dirty_list = L.dirty_list; a.dirty_count = c->dirty_count + layer;
     a.reuse_px = c->reuse_px + (size_t)layer * c->S;
     a.reused_total = c->reused_total + layer;
+    a.alive = (regions == c->table + (size_t)layer * c->S * c->max_regions) ? c->alive + (size_t)layer * c->S : nullptr;
     // the caller has zeroed dirty_count[layer] and reuse_px[layer][*] on the stream
     int tiles = L.tiles_x * L.tiles_y * c->S;
     { dc_prof_scope ps(c, DC_ST_CLASSIFY_COPY); k_classify_copy<<<dc_div_up(tiles, 8), 256, 0, c->stream>>>(a); }
