@@ -118,7 +118,7 @@ int dc_cache_destroy(dc_cache* cache);
 /* Empties the cache: the next dc_infer_frame is a full fresh frame (Section 5, expiry). */
 int dc_cache_reset(dc_cache* cache);
 
-/* Device bytes held by the cache (cf. the memory overhead of Section 7.5). */
+/* Device bytes held by the cache (cf. the memory overhead of Section 7.7). */
 int dc_cache_bytes(const dc_cache* cache, size_t* bytes);
 
 /* Stores frame_dev as the cached previous frame (the cache key of Section 3) without
@@ -173,6 +173,14 @@ int dc_infer_frame(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes
  * full copy speed.  out_map_host may be NULL. */
 int dc_infer_frame_host(dc_cache* cache, const uint8_t* frame_host, size_t pitch_bytes,
                         void* out_map_host, dc_frame_stats* stats_host);
+
+/* Starts the host-to-device copy of the NEXT frame on a separate stream, so it overlaps the frame being
+ * computed (Section 7.6 notes that matching one image and inferring another can run at the same time).
+ * A later dc_infer_frame_host with the same frame_host and pitch_bytes uses that copy instead of copying
+ * again.  Typical loop: prefetch(frame t+1), infer(frame t), prefetch(frame t+2), infer(frame t+1), ...
+ * At most two frames can be pending (DC_ERR_STATE otherwise).  frame_host must stay unchanged until that call and should be
+ * pinned memory (a pageable buffer makes the copy synchronous).  Errors: DC_ERR_ARG, DC_ERR_ALLOC, DC_ERR_CUDA. */
+int dc_prefetch_frame_host(dc_cache* cache, const uint8_t* frame_host, size_t pitch_bytes);
 
 /* Device address and size of the library-owned map of `layer` as of the last
  * dc_infer_frame (for inspection; valid until the next call on this cache). */

@@ -221,7 +221,8 @@ void release(dc_cache* c)
 {
     dc_prof_release(c);
     cudaFree(c->reused_total);
-    cudaFree(c->key[0]); cudaFree(c->key[1]); cudaFree(c->staging); cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched); cudaFree(c->run_end);
+    cudaFree(c->key[0]); cudaFree(c->key[1]); cudaFree(c->staging[0]); cudaFree(c->staging[1]);
+    if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaEventDestroy(c->copied[0]); cudaEventDestroy(c->copied[1]); cudaStreamDestroy(c->copy_stream); } cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched); cudaFree(c->run_end);
     cudaFree(c->mv_acc); cudaFree(c->long_list); cudaFree(c->gmv); cudaFree(c->regions0); cudaFree(c->n_regions); cudaFree(c->table);
     cudaFree(c->layers_dev); cudaFree(c->in_hw_dev); cudaFree(c->dirty_count); cudaFree(c->all_count);
     cudaFree(c->reuse_px); cudaFree(c->zero_masks); cudaFree(c->status); cudaFree(c->input_map); cudaFree(c->pix_lut);
@@ -442,16 +443,56 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
     return DC_OK;
 }
 
+static int ensure_staging(dc_cache* c, size_t bytes)
+{
+    for (int k = 0; k < 2; ++k)
+        if (!c->staging[k]) {
+            if (cudaMalloc((void**)&c->staging[k], bytes + 256) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
+            c->bytes += bytes + 256;
+        }
+    return DC_OK;
+}
+
+int dc_prefetch_frame_host(dc_cache* c, const uint8_t* frame_host, size_t pitch)
+{
+    if (!c || !frame_host || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
+    const size_t bytes = pitch * (size_t)c->cfg.height * c->S;
+    DC_TRY(ensure_staging(c, bytes));
+    if (!c->copy_stream) {
+        DC_CUDA(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+        for (int k = 0; k < 2; ++k) DC_CUDA(cudaEventCreateWithFlags(&c->copied[k], cudaEventDisableTiming));
+    }
+    // a staging buffer that holds no pending prefetch; dc_infer_frame_host waits for its own work before it
+    // returns, so such a buffer is idle
+    int slot = -1;
+    for (int k = 0; k < 2; ++k) if (!c->prefetched[k]) { slot = k; break; }
+    if (slot < 0) return DC_ERR_STATE;                           // two frames are already on their way
+    DC_CUDA(cudaMemcpyAsync(c->staging[slot], frame_host, bytes, cudaMemcpyHostToDevice, c->copy_stream));
+    DC_CUDA(cudaEventRecord(c->copied[slot], c->copy_stream));
+    c->prefetched[slot] = frame_host; c->prefetched_pitch[slot] = pitch;
+    return DC_OK;
+}
+
 int dc_infer_frame_host(dc_cache* c, const uint8_t* frame_host, size_t pitch, void* out_map_host, dc_frame_stats* stats)
 {
     if (!c || !frame_host || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
     const size_t bytes = pitch * (size_t)c->cfg.height * c->S;
-    if (!c->staging) {
-        if (cudaMalloc((void**)&c->staging, bytes + 256) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
-        c->bytes += bytes + 256;
+    DC_TRY(ensure_staging(c, bytes));
+    int slot = -1;
+    for (int k = 0; k < 2; ++k)
+        if (c->prefetched[k] == frame_host && c->prefetched_pitch[k] == pitch) slot = k;
+    if (slot >= 0) {
+        DC_CUDA(cudaStreamWaitEvent(c->stream, c->copied[slot], 0));     // the copy is already on its way
+    } else {
+        for (int k = 0; k < 2; ++k) if (!c->prefetched[k]) { slot = k; break; }
+        if (slot < 0) {                                           // both buffers hold prefetches of other frames: drop one
+            DC_CUDA(cudaStreamSynchronize(c->copy_stream));
+            slot = 0;
+        }
+        DC_CUDA(cudaMemcpyAsync(c->staging[slot], frame_host, bytes, cudaMemcpyHostToDevice, c->stream));
     }
-    DC_CUDA(cudaMemcpyAsync(c->staging, frame_host, bytes, cudaMemcpyHostToDevice, c->stream));
-    int rc = dc_infer_frame(c, c->staging, pitch, nullptr, stats);
+    c->prefetched[slot] = nullptr;
+    int rc = dc_infer_frame(c, c->staging[slot], pitch, nullptr, stats);
     if (rc != DC_OK) return rc;
     if (out_map_host)
         DC_CUDA(cudaMemcpyAsync(out_map_host, layer_input(c, c->n_layers - 1), c->L[c->n_layers - 1].map_bytes,

@@ -64,7 +64,10 @@ struct dc_cache {
     int key_cur;                    // frame, the other one receives the frame being processed
     size_t key_pitch;
     int num_sms;
-    uint8_t* staging;               // device copy of host frames for dc_infer_frame_host
+    uint8_t* staging[2];            // device copies of host frames for dc_infer_frame_host (one in use, one prefetching)
+    cudaStream_t copy_stream;       // dc_prefetch_frame_host copies on its own stream
+    cudaEvent_t copied[2];
+    const uint8_t* prefetched[2]; size_t prefetched_pitch[2];   // host frame whose copy each buffer holds, or NULL
     uint32_t sse_limit[4];          // PSNR test as an SSE bound, index = 2 * (bottom edge) + (right edge)
 
     int16_t* blk_mv;                // [S][Gy][Gx][2]

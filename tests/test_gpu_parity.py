@@ -273,3 +273,32 @@ def test_infer_identical_frames_and_reset():
         assert st[0].refreshed and torch.equal(a, c)
     finally:
         dc.close()
+
+
+def test_infer_host_buffers_with_and_without_prefetch():
+    """dc_infer_frame_host (host frames in, last map out) with the next frame prefetched, without, and with a
+    prefetch that is then not used: all equal dc_infer_frame on device buffers, bit for bit."""
+    w = configs.WORKLOADS[2]()
+    sb = w.streams(1, 6)
+    frames = [torch.from_numpy(np.ascontiguousarray(sb.frame(i))).pin_memory() for i in range(6)]
+    ref = DeepCache.from_workload(w)
+    dc = DeepCache.from_workload(w)
+    try:
+        pitch = w.width * 3
+        out_host = torch.empty(ref.out_shape(-1), dtype=torch.float32).pin_memory()
+        B.dc_prefetch_frame_host(dc.handle, frames[0].data_ptr(), pitch)
+        for i in range(6):
+            want = ref.infer_frame(frames[i].cuda())
+            if i in (0, 1, 3):                        # the usual loop: prefetch the next frame, then compute this one
+                B.dc_prefetch_frame_host(dc.handle, frames[i + 1].data_ptr(), pitch)
+            B.dc_infer_frame_host(dc.handle, frames[i].data_ptr(), pitch, out_host.data_ptr())
+            assert torch.equal(out_host, want.cpu()), f"frame {i}"
+        # a third pending prefetch is refused
+        B.dc_prefetch_frame_host(dc.handle, frames[0].data_ptr(), pitch)
+        B.dc_prefetch_frame_host(dc.handle, frames[1].data_ptr(), pitch)
+        with pytest.raises(B.DeepCacheError) as e:
+            B.dc_prefetch_frame_host(dc.handle, frames[2].data_ptr(), pitch)
+        assert e.value.status == B.DC_ERR_STATE
+        assert dc.status() == B.DC_OK
+    finally:
+        ref.close(); dc.close()
