@@ -145,20 +145,32 @@ static void search_ds(const uint8_t* cur, const uint8_t* prev, int W, int H, int
     *bdx = nx; *bdy = ny; *bsse = ns;
 }
 
-/* Step 2 for every block of the grid.  kind: 0 exhaustive, 1 diamond.
- * mv is [Gy][Gx][2] = (dx, dy); sse is [Gy][Gx]. */
-void orc_search(const uint8_t* cur, const uint8_t* prev, int W, int H, int64_t pitch,
-                int B, int R, int kind, int16_t* mv, uint32_t* sse)
+#define ORC_NOT_SEARCHED UINT32_MAX
+
+/* Step 2 for the blocks of the grid.  kind: 0 exhaustive, 1 diamond.
+ * mv is [Gy][Gx][2] = (dx, dy); sse is [Gy][Gx].
+ * skip_k (Section 4, "skipping some blocks"): only blocks whose row and column index are
+ * multiples of skip_k are searched; the others get mv = (0, 0), sse = ORC_NOT_SEARCHED and take
+ * no part in Step 3.  skip_k = 1 searches every block. */
+void orc_search_k(const uint8_t* cur, const uint8_t* prev, int W, int H, int64_t pitch,
+                  int B, int R, int kind, int skip_k, int16_t* mv, uint32_t* sse)
 {
     int Gx = (W + B - 1) / B, Gy = (H + B - 1) / B;
     #pragma omp parallel for schedule(dynamic, 4)
     for (int b = 0; b < Gx * Gy; ++b) {
         int bx = b % Gx, by = b / Gx, x0, y0, bw, bh, dx, dy; uint64_t s;
+        if (bx % skip_k != 0 || by % skip_k != 0) { mv[2 * b] = 0; mv[2 * b + 1] = 0; sse[b] = ORC_NOT_SEARCHED; continue; }
         block_geom(W, H, B, bx, by, &x0, &y0, &bw, &bh);
         if (kind == 0) search_es(cur, prev, W, H, pitch, x0, y0, bw, bh, R, &dx, &dy, &s);
         else           search_ds(cur, prev, W, H, pitch, x0, y0, bw, bh, R, &dx, &dy, &s);
         mv[2 * b] = (int16_t)dx; mv[2 * b + 1] = (int16_t)dy; sse[b] = (uint32_t)s;
     }
+}
+
+void orc_search(const uint8_t* cur, const uint8_t* prev, int W, int H, int64_t pitch,
+                int B, int R, int kind, int16_t* mv, uint32_t* sse)
+{
+    orc_search_k(cur, prev, W, H, pitch, B, R, kind, 1, mv, sse);
 }
 
 /* Step 3: mean motion of the blocks whose best match passes the PSNR test.
@@ -171,6 +183,7 @@ void orc_mean_mv(const int16_t* mv, const uint32_t* sse, int W, int H, int B, do
     for (int b = 0; b < Gx * Gy; ++b) {
         int x0, y0, bw, bh;
         block_geom(W, H, B, b % Gx, b / Gx, &x0, &y0, &bw, &bh);
+        if (sse[b] == ORC_NOT_SEARCHED) continue;                 /* skipped by k-skip */
         if (orc_psnr_pass(sse[b], (int64_t)bw * bh * 3, T)) { sx += mv[2 * b]; sy += mv[2 * b + 1]; ++K; }
     }
     out[0] = out[1] = 0; out[2] = (int32_t)K;

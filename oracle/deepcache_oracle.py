@@ -66,6 +66,8 @@ def lib():
         L.orc_psnr_pass.argtypes = [C.c_uint64, i64, d]
         L.orc_search.restype = None
         L.orc_search.argtypes = [u8p, u8p, i, i, i64, i, i, i, i16p, u32p]
+        L.orc_search_k.restype = None
+        L.orc_search_k.argtypes = [u8p, u8p, i, i, i64, i, i, i, i, i16p, u32p]
         L.orc_mean_mv.restype = None
         L.orc_mean_mv.argtypes = [i16p, u32p, i, i, i, d, i32p]
         L.orc_verify.restype = None
@@ -122,15 +124,16 @@ def psnr_limit(n: int, T: float) -> int:
     return int(lib().orc_psnr_limit(n, T))
 
 
-def search(cur, prev, B, R, kind):
-    """Section 4 Step 2.  Returns mv int16 [Gy, Gx, 2] as (dx, dy) and sse uint32 [Gy, Gx]."""
+def search(cur, prev, B, R, kind, skip_k=1):
+    """Section 4 Step 2.  Returns mv int16 [Gy, Gx, 2] as (dx, dy) and sse uint32 [Gy, Gx].
+    skip_k > 1: only blocks on every skip_k-th row and column are searched (the rest: sse = 2^32 - 1)."""
     cur, prev = _u8(cur), _u8(prev)
     H, W = cur.shape[:2]
     Gx, Gy = -(-W // B), -(-H // B)
     mv = np.zeros((Gy, Gx, 2), np.int16)
     sse = np.zeros((Gy, Gx), np.uint32)
-    lib().orc_search(_p(cur, C.c_uint8), _p(prev, C.c_uint8), W, H, W * 3, B, R, kind,
-                     _p(mv, C.c_int16), _p(sse, C.c_uint32))
+    lib().orc_search_k(_p(cur, C.c_uint8), _p(prev, C.c_uint8), W, H, W * 3, B, R, kind, skip_k,
+                       _p(mv, C.c_int16), _p(sse, C.c_uint32))
     return mv, sse
 
 
@@ -160,10 +163,10 @@ def merge(matched, W, H, B, Mx, My):
     return out[:n].copy()
 
 
-def match_blocks(cur, prev, B, R, kind, T):
+def match_blocks(cur, prev, B, R, kind, T, skip_k=1):
     """Steps 1-5 in order.  Returns dict(mv, sse, M, K, matched, regions)."""
     H, W = cur.shape[:2]
-    mv, sse = search(cur, prev, B, R, kind)
+    mv, sse = search(cur, prev, B, R, kind, skip_k)
     Mx, My, K = mean_mv(mv, sse, W, H, B, T)
     matched = verify(cur, prev, B, Mx, My, K, T)
     regions = merge(matched, W, H, B, Mx, My)
@@ -271,11 +274,12 @@ class OracleCache:
     """
 
     def __init__(self, width, height, layers, weights, biases, *, block=10, search_range=8,
-                 search_kind=SEARCH_DS, psnr_db=20.0, expire_n=10, quant=QUANT_NONE, use_cache=True):
+                 search_kind=SEARCH_DS, psnr_db=20.0, expire_n=10, quant=QUANT_NONE, use_cache=True, skip_k=1):
         self.W, self.H = width, height
         self.layers = layers
         self.block, self.R, self.kind = block, search_range, search_kind
         self.T, self.N, self.quant, self.use_cache = psnr_db, expire_n, quant, use_cache
+        self.skip_k = skip_k
         # weights are stored at the storage precision (bf16 workloads round them once)
         self.weights = [None if w is None else quant_array(w, quant) for w in weights]
         self.biases = [None if b is None else np.asarray(b, np.float64) for b in biases]
@@ -295,7 +299,7 @@ class OracleCache:
         info = dict(refreshed=bool(refresh), match=None, regions=None, reused=[None] * len(layers))
         per_layer_regions = None
         if not refresh:
-            m = match_blocks(frame, self.prev_frame, self.block, self.R, self.kind, self.T)
+            m = match_blocks(frame, self.prev_frame, self.block, self.R, self.kind, self.T, self.skip_k)
             per_layer_regions = propagate(layers, (self.H, self.W), m["regions"])
             info["match"], info["regions"] = m, per_layer_regions
         maps = []

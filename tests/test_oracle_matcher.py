@@ -296,3 +296,36 @@ def test_merge_covers_exactly_the_matched_blocks():
         c = cover(r, W, H)
         expect = np.kron(m, np.ones((B, B), np.int32))[:H, :W]
         assert np.array_equal(c, expect)             # disjoint (no pixel counted twice) and complete
+
+
+def test_k_skip_searches_every_kth_block_only():
+    """Section 4: with k-skip only blocks on every k-th row and column are searched; k = 2 leaves a quarter."""
+    w = configs.WORKLOADS[2]()
+    sb = w.streams(1, 3)
+    cur, prev = sb.frame(2)[0], sb.frame(1)[0]
+    mv1, sse1 = orc.search(cur, prev, 16, 8, orc.SEARCH_DS)
+    for k in (2, 3):
+        mvk, ssek = orc.search(cur, prev, 16, 8, orc.SEARCH_DS, skip_k=k)
+        Gy, Gx = sse1.shape
+        on = np.zeros((Gy, Gx), bool)
+        on[::k, ::k] = True
+        assert np.array_equal(mvk[on], mv1[on]) and np.array_equal(ssek[on], sse1[on])     # searched blocks: unchanged
+        assert (ssek[~on] == 2 ** 32 - 1).all() and not mvk[~on].any()                     # the rest: not searched
+        if k == 2:
+            assert on.sum() == -(-Gy // 2) * -(-Gx // 2)                                   # about a quarter of the blocks
+        # Step 3 averages the searched blocks only
+        lim = orc.psnr_limit(16 * 16 * 3, 20.0)
+        full = (np.arange(Gy)[:, None] < Gy - 1) & (np.arange(Gx)[None, :] < Gx - 1)      # unclipped blocks share one bound
+        sel = on & full & (sse1 <= lim)
+        Mx, My, K = orc.mean_mv(mvk, ssek, 227, 227, 16, 20.0)
+        edge_pass = 0
+        for by in range(Gy):
+            for bx in range(Gx):
+                if on[by, bx] and not full[by, bx]:
+                    bw, bh = min(16, 227 - bx * 16), min(16, 227 - by * 16)
+                    edge_pass += int(ssek[by, bx] <= orc.psnr_limit(bw * bh * 3, 20.0))
+        assert K == int(sel.sum()) + edge_pass
+    # k-skip changes Step 2 and 3 only: Step 4 still scores every block at M
+    m = orc.match_blocks(cur, prev, 16, 8, orc.SEARCH_DS, 20.0, skip_k=2)
+    want = orc.verify(cur, prev, 16, m["M"][0], m["M"][1], m["K"], 20.0)
+    assert np.array_equal(m["matched"], want)
