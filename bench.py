@@ -42,6 +42,7 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", type=int, default=5)
     ap.add_argument("--streams", type=int, default=0, help="override the number of streams per GPU")
+    ap.add_argument("--skip-k", type=int, default=1, help="Step 2 on every k-th block row / column only (Section 4); default 1 = all blocks")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -203,7 +204,7 @@ def gpu_arm(args, w):
     dev_frames = host.to(dev, non_blocking=True)
     torch.cuda.synchronize()
 
-    dc = DeepCache.from_workload(w, n_streams=S, device=f"cuda:{local}")
+    dc = DeepCache.from_workload(w, n_streams=S, device=f"cuda:{local}", skip_k=args.skip_k)
     pitch = w.width * 3
     last = w.layers[-1]
     out_bytes = S * last["out_h"] * last["out_w"] * last["cout"] * (2 if w.dtype == 1 else 4)
@@ -313,7 +314,7 @@ def gpu_arm(args, w):
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
-            "config": workload_config(w, S, world), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "config": dict(workload_config(w, S, world), skip_k=args.skip_k), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "roofline_matcher": roofline_matcher, "cpu_baseline": cpu_baseline,
             "stage_ms": stage_ms, "stage_share": stage_share, "frames_cached": n_cached, "frames_full": n_full,
             "reuse_ratio_cached_frames": reuse, "cache_bytes": dc.bytes()}

@@ -84,7 +84,8 @@ typedef struct {
     int32_t block;                     /* block edge in pixels (Section 3 default 10), 4..32 */
     int32_t range;                     /* search range R: |dx|, |dy| <= R, 0..64 */
     int32_t search;                    /* dc_search_kind */
-    int32_t skip_k;                    /* reserved, must be 1 */
+    int32_t skip_k;                    /* Step 2 searches only blocks on every skip_k-th row and column (Section 4,
+                                          "k-skip"); 1 = every block; 1..16 */
     int32_t expire_n;                  /* full fresh frame every expire_n frames (default 10) */
     double  psnr_db;                   /* similarity threshold T in dB (default 20) */
     int32_t dtype;                     /* dc_dtype of maps and arithmetic inputs */
@@ -128,6 +129,7 @@ int dc_cache_set_key(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_byt
 /* Section 4, Steps 1-5, current frame against the cached previous frame.
  *   block_mv_dev   int16  [S][Gy][Gx][2]  best (dx, dy) per block (Step 2)
  *   block_sse_dev  uint32 [S][Gy][Gx]     its sum of squared differences over 3 channels
+ *                                         (blocks skipped by skip_k: vector (0, 0), SSE 0xFFFFFFFF)
  *   matched_dev    uint8  [S][Gy][Gx]     1 = properly matched at the global motion (Step 4)
  *   global_mv_dev  int32  [S][3]          Mx, My, K (Step 3)
  *   regions_dev    dc_region [S][max_regions], n_regions_dev int32 [S]   (Step 5)

@@ -23,7 +23,7 @@ constexpr int MAX_ROW_WORDS = 24;       // block <= 32 px -> 96 bytes per row
 struct MatchArgs {
     const uint8_t* cur;  size_t cur_pitch;  size_t cur_stream;
     const uint8_t* prev; size_t prev_pitch; size_t prev_stream;
-    int W, H, B, R, Gx, Gy, S, search;
+    int W, H, B, R, Gx, Gy, S, search, skip_k;
     uint32_t limit[4];
     int16_t* mv; uint32_t* sse; uint8_t* matched; int32_t* acc; int32_t* gmv;
 };
@@ -131,6 +131,14 @@ __global__ void __launch_bounds__(WARPS * 32) k_search(MatchArgs a)
     __shared__ uint32_t sm_all[WARPS][32 * MAX_ROW_WORDS];
     BlockCtx<ITERS> c; int s, b;
     if (!load_block<ITERS>(a, sm_all[threadIdx.x >> 5], c, s, b)) return;
+    if (a.skip_k > 1 && ((b % a.Gx) % a.skip_k != 0 || (b / a.Gx) % a.skip_k != 0)) {
+        // Section 4, k-skip: this block is not searched and takes no part in Step 3
+        if (c.lane == 0) {
+            size_t g = (size_t)s * a.Gx * a.Gy + b;
+            a.mv[2 * g] = 0; a.mv[2 * g + 1] = 0; a.sse[g] = 0xffffffffu;
+        }
+        return;
+    }
 
     int bx_ = 0, by_ = 0;
     uint32_t bs = c.sse(0, 0);                         // the zero vector is always a candidate
@@ -202,7 +210,7 @@ __global__ void __launch_bounds__(WARPS * 32) k_verify(MatchArgs a)
         const size_t g = (size_t)s * a.Gx * a.Gy + b;
         // Section 4: "if the PSNR between (x_i, y_i) and (x_i + M_x, y_i + M_y) is already calculated
         // in Step 2, we simply reuse the result" -- exact when the block's best vector is M itself
-        uint32_t v = (a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My) ? a.sse[g] : c.sse(Mx, My);
+        uint32_t v = (a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My && a.sse[g] != 0xffffffffu) ? a.sse[g] : c.sse(Mx, My);
         ok = v <= a.limit[limit_index(a, c.bw, c.bh)];
     }
     if (c.lane == 0) {
@@ -477,7 +485,8 @@ __global__ void __launch_bounds__(256, 4) k_search_ds16(MatchArgs a, uint4* long
     const int xs = strip * 128, y0 = by * 16;
     const int wx0 = ((xs - F_WR) * 3) & ~15;                  // byte column of the window origin (may be < 0)
     const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
-    for (int i = threadIdx.x; i < F_ROWS * (F_WORDS / 4); i += 256) {   // 16-byte chunks; wx0 and the pitch are 16-byte multiples
+    const bool row_searched = a.skip_k <= 1 || by % a.skip_k == 0;
+    for (int i = threadIdx.x; row_searched && i < F_ROWS * (F_WORDS / 4); i += 256) {   // 16-byte chunks; wx0 and the pitch are 16-byte multiples
         const int row = i / (F_WORDS / 4), ci = i - row * (F_WORDS / 4);
         const int gy = y0 - F_WR + row, gb = wx0 + ci * 16;
         uint4 v = make_uint4(0, 0, 0, 0);
@@ -490,6 +499,13 @@ __global__ void __launch_bounds__(256, 4) k_search_ds16(MatchArgs a, uint4* long
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int bx = strip * 8 + warp;
     if (bx >= a.Gx) return;
+    if (a.skip_k > 1 && (bx % a.skip_k != 0 || by % a.skip_k != 0)) {      // Section 4, k-skip: not searched
+        if (lane == 0) {
+            const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
+            a.mv[2 * g] = 0; a.mv[2 * g + 1] = 0; a.sse[g] = 0xffffffffu;
+        }
+        return;
+    }
     const int x0 = bx * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
     RowCtx<F_NR> rc;
     rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, lane & (F_LPC - 1), F_LPC, bw, bh);
@@ -575,7 +591,7 @@ __global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
                          x0 + Mx + bw <= a.W && y0 + My + bh <= a.H;
     const size_t g = (size_t)s * per + b;
     // Section 4: reuse the Step 2 score when that step already scored this pair (best vector == M)
-    const bool known = cand_ok && a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My;
+    const bool known = cand_ok && a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My && a.sse[g] != 0xffffffffu;
     uint32_t acc = 0;
     if (cand_ok && !known && r < bh) {
         RowCtx<1> rc;
@@ -659,7 +675,7 @@ int dc_launch_match(dc_cache* c)
     a.cur = c->key[c->key_cur ^ 1]; a.cur_pitch = c->key_pitch; a.cur_stream = c->key_pitch * (size_t)c->cfg.height;
     a.prev = c->key[c->key_cur]; a.prev_pitch = c->key_pitch; a.prev_stream = c->key_pitch * (size_t)c->cfg.height;
     a.W = c->cfg.width; a.H = c->cfg.height; a.B = c->cfg.block; a.R = c->cfg.range;
-    a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search;
+    a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search; a.skip_k = c->cfg.skip_k;
     for (int i = 0; i < 4; ++i) a.limit[i] = c->sse_limit[i];
     a.mv = c->blk_mv; a.sse = c->blk_sse; a.matched = c->matched; a.acc = c->mv_acc; a.gmv = c->gmv;
     // Step 3 sums and, behind them, the counter of walks handed to the second search phase

@@ -29,7 +29,7 @@ def device_view(ptr: int, shape, dtype: torch.dtype, device) -> torch.Tensor:
 
 class DeepCache:
     def __init__(self, width, height, layers, weights, biases, *, n_streams=1, block=10, search_range=8,
-                 search=B.DC_SEARCH_DIAMOND, psnr_db=20.0, expire_n=10, dtype=B.DC_FP32, max_regions=0,
+                 search=B.DC_SEARCH_DIAMOND, psnr_db=20.0, expire_n=10, dtype=B.DC_FP32, max_regions=0, skip_k=1,
                  device="cuda:0"):
         if not torch.cuda.is_available():
             raise RuntimeError("DeepCache needs a CUDA device; there is no CPU fallback")
@@ -37,7 +37,7 @@ class DeepCache:
         torch.cuda.set_device(self.device)
         self.layers = [dict(l) for l in layers]
         self.cfg = B.dc_config(width=width, height=height, channels=3, n_streams=n_streams, block=block,
-                               range=search_range, search=search, skip_k=1, expire_n=expire_n, psnr_db=psnr_db,
+                               range=search_range, search=search, skip_k=skip_k, expire_n=expire_n, psnr_db=psnr_db,
                                dtype=dtype, max_regions=max_regions)
         self.S, self.W, self.H = n_streams, width, height
         self.Gx, self.Gy = -(-width // block), -(-height // block)

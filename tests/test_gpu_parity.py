@@ -21,22 +21,22 @@ def rng(seed):
     return np.random.Generator(np.random.PCG64(seed))
 
 
-def matcher_only(width, height, n_streams, block, R, search, psnr_db=20.0):
+def matcher_only(width, height, n_streams, block, R, search, psnr_db=20.0, skip_k=1):
     layers = nets.single_conv(height, width)
     ws, bs = nets.random_weights(layers, 1)
     return DeepCache(width, height, layers, ws, bs, n_streams=n_streams, block=block, search_range=R,
-                     search=search, psnr_db=psnr_db)
+                     search=search, psnr_db=psnr_db, skip_k=skip_k)
 
 
-def check_pairs(pairs, block, R, search, psnr_db=20.0):
+def check_pairs(pairs, block, R, search, psnr_db=20.0, skip_k=1):
     """pairs: list of (prev, cur) frames of equal size, run as one batch of streams."""
     H, W = pairs[0][0].shape[:2]
-    dc = matcher_only(W, H, len(pairs), block, R, search, psnr_db)
+    dc = matcher_only(W, H, len(pairs), block, R, search, psnr_db, skip_k)
     try:
         dc.set_key(np.stack([p for p, _ in pairs]))
         got = dc.match_blocks(np.stack([c for _, c in pairs]))
         for s, (prev, cur) in enumerate(pairs):
-            U.assert_match_equal(got, s, orc.match_blocks(cur, prev, block, R, search, psnr_db), f"stream {s}")
+            U.assert_match_equal(got, s, orc.match_blocks(cur, prev, block, R, search, psnr_db, skip_k), f"stream {s}")
         assert dc.status() == B.DC_OK
     finally:
         dc.close()
@@ -91,6 +91,21 @@ def test_match_full_hd_batch():
     w = configs.WORKLOADS[5]()
     sb = w.streams(2, 3)
     check_pairs([(sb.frame(1, s), sb.frame(2, s)) for s in range(2)], 16, 32, B.DC_SEARCH_DIAMOND)
+
+
+@pytest.mark.parametrize("k", [2, 3])
+def test_match_k_skip(k):
+    """Section 4's k-skip: Step 2 on every k-th block row and column only (16-px fast path and generic path)."""
+    w = configs.WORKLOADS[2]()
+    sb = w.streams(1, 4)
+    pairs = [(sb.frame(i - 1)[0], sb.frame(i)[0]) for i in (1, 2, 3)]
+    check_pairs(pairs, 16, 16, B.DC_SEARCH_DIAMOND, skip_k=k)
+    check_pairs(pairs, 10, 6, B.DC_SEARCH_DIAMOND, skip_k=k)
+    check_pairs([(p[:96, :96], c[:96, :96]) for p, c in pairs], 8, 3, B.DC_SEARCH_EXHAUSTIVE, skip_k=k)
+
+
+def test_infer_with_k_skip():
+    U.run_stream_parity(configs.WORKLOADS[3](), 1, list(range(5)), skip_k=2)
 
 
 def test_match_needs_a_key():
