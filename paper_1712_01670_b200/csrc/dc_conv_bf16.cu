@@ -703,7 +703,7 @@ struct TcPlan { int BK, BN, NB, MT, nbuf, stages, a_bytes, b_bytes; CUtensorMapS
 bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn = 0)
 {
     if (d.kind != DC_CONV) return false;
-    if (d.sh != 1 || d.sw != 1) return false;                   // strided layers use the CUDA-core kernel
+    if (d.sh < 1 || d.sw < 1 || DC_TILE_W * d.sw > 256 || DC_TILE_H * d.sh > 256) return false;   // TMA box limit
     if (d.cin % 64 == 0) { p.BK = 64; p.swz = CU_TENSOR_MAP_SWIZZLE_128B; p.layout_type = 2; }
     else if (d.cin % 32 == 0) { p.BK = 32; p.swz = CU_TENSOR_MAP_SWIZZLE_64B; p.layout_type = 4; }
     else if (d.cin % 16 == 0) { p.BK = 16; p.swz = CU_TENSOR_MAP_SWIZZLE_32B; p.layout_type = 6; }
@@ -913,8 +913,10 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     {   // input map [S][Hi][Wi][Ci] bf16; box = BK channels x 16 columns x 8 rows x 1 stream
         cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
         cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
-        cuuint32_t box[4] = {(cuuint32_t)p.BK, DC_TILE_W, DC_TILE_H, 1};
-        cuuint32_t estr[4] = {1, 1, 1, 1};
+        // a strided convolution reads every sw-th column / sh-th row: the box spans TW * sw x TH * sh input
+        // pixels and the traversal strides pick TW x TH of them
+        cuuint32_t box[4] = {(cuuint32_t)p.BK, (cuuint32_t)(DC_TILE_W * d.sw), (cuuint32_t)(DC_TILE_H * d.sh), 1};
+        cuuint32_t estr[4] = {1, (cuuint32_t)d.sw, (cuuint32_t)d.sh, 1};
         if (enc(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, p.swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return DC_ERR_CUDA;

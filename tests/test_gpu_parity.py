@@ -184,7 +184,8 @@ def test_propagate_table2_rows():
     (37, 45, 3, 16, 3, 1, 1, 1), (64, 64, 32, 64, 3, 1, 1, 1), (227, 227, 3, 96, 11, 4, 0, 1),
     (27, 27, 96, 256, 5, 1, 2, 1), (56, 56, 64, 128, 1, 2, 0, 0), (30, 33, 16, 24, 3, 2, 1, 0),
     (14, 14, 256, 512, 3, 1, 1, 1), (224, 224, 3, 64, 7, 2, 3, 1), (40, 52, 3, 64, 3, 1, 1, 1),
-    (33, 35, 3, 32, 5, 1, 2, 0), (28, 28, 32, 96, 3, 1, 1, 1), (20, 24, 16, 64, 1, 1, 0, 1)])
+    (33, 35, 3, 32, 5, 1, 2, 0), (28, 28, 32, 96, 3, 1, 1, 1), (20, 24, 16, 64, 1, 1, 0, 1),
+    (28, 28, 64, 64, 3, 2, 1, 1), (31, 29, 128, 64, 3, 2, 1, 0), (40, 40, 32, 32, 5, 3, 2, 1)])
 def test_conv_partial(dtype, hi, wi, cin, cout, k, s, p, relu):
     g = rng(hi + cin + k)
     bf16 = dtype == B.DC_BF16
