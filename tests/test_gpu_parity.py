@@ -318,3 +318,26 @@ def test_infer_host_buffers_with_and_without_prefetch():
         assert dc.status() == B.DC_OK
     finally:
         ref.close(); dc.close()
+
+
+def test_region_overflow_sets_the_status_word():
+    """More rectangles than max_regions: the extra ones are dropped and the device status word says so."""
+    prev = rng(2).integers(0, 256, size=(64, 64, 3), dtype=np.uint8)
+    cur = prev.copy()
+    cur[::16, :] = 255 - cur[::16, :]                 # ruin every other 8-px block row: matched rows alternate
+    cur[:, 24:32] = 255 - cur[:, 24:32]               # and one block column: two runs per matched row
+    layers = nets.single_conv(64, 64)
+    ws, bs = nets.random_weights(layers, 1)
+    want = orc.match_blocks(cur, prev, 8, 2, orc.SEARCH_DS, 20.0)
+    assert len(want["regions"]) > 2
+    dc = DeepCache(64, 64, layers, ws, bs, block=8, search_range=2, max_regions=2)
+    try:
+        dc.set_key(prev)
+        got = dc.match_blocks(cur)
+        assert int(got["n_regions"][0]) == 2
+        U.assert_regions_equal(U.regions_np(got["regions"][0, :2]), want["regions"][:2], "kept rectangles")
+        assert dc.status() == B.DC_ERR_OVERFLOW
+        dc.reset()
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
