@@ -265,8 +265,26 @@ def gpu_arm(args, w):
         e2e = {"value": sharding.aggregate_rate(S * args.steps, world, dte), "unit": UNIT, "h2d_bytes_per_step": S * frame_bytes,
                "d2h_bytes_per_step": out_bytes}
 
+    # ---- the same frames with the cache switched off (every frame computed in full): the paper's "no-cache" arm ----
+    dc.close()
+    nc = DeepCache.from_workload(w, n_streams=S, device=f"cuda:{local}", expire_n=1)
+    for i in range(args.warmup):
+        B.dc_infer_frame(nc.handle, dev_frames[i], pitch)
+    barrier()
+    n0, n1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    n0.record()
+    for i in range(args.warmup, total):
+        B.dc_infer_frame(nc.handle, dev_frames[i], pitch)
+    n1.record()
+    barrier()
+    no_cache_ms = sharding.max_over_ranks(n0.elapsed_time(n1), dev)
+    no_cache = {"value": sharding.aggregate_rate(S * args.steps, world, no_cache_ms * 1e-3), "unit": UNIT,
+                "ms_per_step": no_cache_ms / args.steps,
+                "note": "same kernels, expire_n = 1: no matching, no reuse, every tile computed"}
+    cache_bytes = nc.bytes()
+    nc.close()
+
     if rank != 0:
-        dc.close()
         if world > 1:
             dist.destroy_process_group()
         return
@@ -317,9 +335,8 @@ def gpu_arm(args, w):
             "config": dict(workload_config(w, S, world), skip_k=args.skip_k), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "roofline_matcher": roofline_matcher, "cpu_baseline": cpu_baseline,
             "stage_ms": stage_ms, "stage_share": stage_share, "frames_cached": n_cached, "frames_full": n_full,
-            "reuse_ratio_cached_frames": reuse, "cache_bytes": dc.bytes()}
+            "reuse_ratio_cached_frames": reuse, "cache_bytes": cache_bytes, "no_cache": no_cache}
     print(json.dumps(line))
-    dc.close()
     if world > 1:
         dist.destroy_process_group()
 

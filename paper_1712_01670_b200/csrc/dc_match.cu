@@ -304,21 +304,20 @@ constexpr int F_NR = 16 / F_LPC;               // block rows per lane
 // NR rows (48 bytes each) of the current block per lane, masked for clipped edge blocks.
 template <int NR>
 struct RowCtx {
-    uint32_t cw[NR][12], wm[12];
+    uint32_t cw[NR][12];
+    int row_bytes;                                                 // bw * 3: bytes of a block row (48 unless clipped)
+    // mask of the valid bytes of word j of a clipped row
+    __device__ __forceinline__ uint32_t word_mask(int j) const
+    {
+        const int nb = row_bytes - 4 * j;
+        return nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << (8 * nb)) - 1u));
+    }
     bool clipped, row_on[NR];
     // cur_rows[k]: address of row k of this lane (16-byte aligned in the library's frame copy)
     __device__ __forceinline__ void load(const uint8_t* const* cur_rows, int bw, const bool* on)
     {
         clipped = bw < 16;
-#pragma unroll
-        for (int j = 0; j < 12; ++j) wm[j] = 0xffffffffu;
-        if (clipped) {                                             // only the frame's last block column
-#pragma unroll
-            for (int j = 0; j < 12; ++j) {
-                int nb = bw * 3 - 4 * j;
-                wm[j] = nb >= 4 ? 0xffffffffu : (nb <= 0 ? 0u : ((1u << (8 * nb)) - 1u));
-            }
-        }
+        row_bytes = bw * 3;
 #pragma unroll
         for (int k = 0; k < NR; ++k) {
             row_on[k] = on[k];
@@ -329,7 +328,7 @@ struct RowCtx {
             cw[k][6] = v1.z; cw[k][7] = v1.w; cw[k][8] = v2.x; cw[k][9] = v2.y; cw[k][10] = v2.z; cw[k][11] = v2.w;
             if (clipped) {
 #pragma unroll
-                for (int j = 0; j < 12; ++j) cw[k][j] &= wm[j];
+                for (int j = 0; j < 12; ++j) cw[k][j] &= word_mask(j);
             }
         }
     }
@@ -357,7 +356,7 @@ struct RowCtx {
         } else {
 #pragma unroll
             for (int j = 0; j < 12; ++j) {
-                uint32_t d = __vabsdiffu4(cw[k][j], __funnelshift_r(w[j], w[j + 1], sh) & wm[j]);
+                uint32_t d = __vabsdiffu4(cw[k][j], __funnelshift_r(w[j], w[j + 1], sh) & word_mask(j));
                 acc[j % 3] = __dp4a(d, d, acc[j % 3]);
             }
         }
@@ -477,7 +476,7 @@ struct StripWin {
 };
 
 // Phase 1: one CTA per strip of 8 blocks.  A walk that leaves the strip window is handed to phase 2.
-__global__ void __launch_bounds__(256, 4) k_search_ds16(MatchArgs a, uint4* long_list, int32_t* long_count)
+__global__ void __launch_bounds__(256, 5) k_search_ds16(MatchArgs a, uint4* long_list, int32_t* long_count)
 {
     __shared__ uint32_t win[F_ROWS * F_PITCH];
     const int strips = (a.Gx + 7) >> 3;
@@ -549,7 +548,7 @@ struct WarpWin {
 
 // Phase 2: the walks that left their strip window, one warp each, re-staging a private window
 // around the walk's centre whenever it nears the window's edge.
-__global__ void __launch_bounds__(256, 3) k_search_ds16_long(MatchArgs a, const uint4* long_list, const int32_t* long_count)
+__global__ void __launch_bounds__(256, 4) k_search_ds16_long(MatchArgs a, const uint4* long_list, const int32_t* long_count)
 {
     __shared__ uint32_t win_all[8][F_ROWS * L_PITCH];
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
