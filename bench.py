@@ -43,6 +43,7 @@ def parse_args():
     ap.add_argument("--workload", type=int, default=5)
     ap.add_argument("--streams", type=int, default=0, help="override the number of streams per GPU")
     ap.add_argument("--skip-k", type=int, default=1, help="Step 2 on every k-th block row / column only (Section 4); default 1 = all blocks")
+    ap.add_argument("--no-lookahead", action="store_true", help="do not overlap the next frame's matching with this frame's inference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -215,12 +216,18 @@ def gpu_arm(args, w):
         torch.cuda.synchronize()
 
     # ---- device-resident timing: value ----
-    for i in range(args.warmup):
+    # The loop a user runs: infer frame t, then announce frame t+1 so that its matching runs on a side stream
+    # beside the convolutions of frame t (dc_lookahead_frame; results are identical without it).
+    overlap = not args.no_lookahead
+
+    def step(i):
         B.dc_infer_frame(dc.handle, dev_frames[i], pitch)
+        if overlap and i + 1 < total:
+            B.dc_lookahead_frame(dc.handle, dev_frames[i + 1], pitch)
+
+    for i in range(args.warmup):
+        step(i)
     barrier()
-    B.dc_cache_set_profiling(dc.handle, True)
-    B.dc_cache_profile(dc.handle)
-    px0, cached0, full0 = B.dc_cache_counters(dc.handle, len(w.layers))
     launches0 = dc.launches()
     sampler = ClockSampler(local)
     sampler.start()
@@ -230,21 +237,38 @@ def gpu_arm(args, w):
     t0 = time.perf_counter()
     e0.record()
     for i in range(args.warmup, total):
-        B.dc_infer_frame(dc.handle, dev_frames[i], pitch)
+        step(i)
     e1.record()
     barrier()
     t1 = time.perf_counter()
     ms = e0.elapsed_time(e1)
     clocks = sampler.stop(t0, t1)
     launches = dc.launches() - launches0
-    prof = B.dc_cache_profile(dc.handle)
-    B.dc_cache_set_profiling(dc.handle, False)
-    px1, cached1, full1 = B.dc_cache_counters(dc.handle, len(w.layers))
     status = dc.status()
     if status != B.DC_OK:
         raise SystemExit(f"device status {status}: {B.strerror(status)}")
     ms = sharding.max_over_ranks(ms, dev)
     value = sharding.aggregate_rate(S * args.steps, world, ms * 1e-3)
+
+    # ---- the same K steps once more, one stream only and every launch bracketed by events: per-kernel
+    #      durations for the rooflines are taken here, where kernels do not share the SMs ----
+    dc.reset()
+    for i in range(args.warmup):
+        B.dc_infer_frame(dc.handle, dev_frames[i], pitch)
+    barrier()
+    B.dc_cache_set_profiling(dc.handle, True)
+    B.dc_cache_profile(dc.handle)
+    px0, cached0, full0 = B.dc_cache_counters(dc.handle, len(w.layers))
+    s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    s0.record()
+    for i in range(args.warmup, total):
+        B.dc_infer_frame(dc.handle, dev_frames[i], pitch)
+    s1.record()
+    barrier()
+    serial_ms = sharding.max_over_ranks(s0.elapsed_time(s1), dev)
+    prof = B.dc_cache_profile(dc.handle)
+    B.dc_cache_set_profiling(dc.handle, False)
+    px1, cached1, full1 = B.dc_cache_counters(dc.handle, len(w.layers))
 
     # ---- end to end through the host-buffer entry point ----
     e2e = None
@@ -335,7 +359,11 @@ def gpu_arm(args, w):
             "config": dict(workload_config(w, S, world), skip_k=args.skip_k), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "roofline_matcher": roofline_matcher, "cpu_baseline": cpu_baseline,
             "stage_ms": stage_ms, "stage_share": stage_share, "frames_cached": n_cached, "frames_full": n_full,
-            "reuse_ratio_cached_frames": reuse, "cache_bytes": cache_bytes, "no_cache": no_cache}
+            "reuse_ratio_cached_frames": reuse, "cache_bytes": cache_bytes, "no_cache": no_cache,
+            "serial": {"value": sharding.aggregate_rate(S * args.steps, world, serial_ms * 1e-3), "unit": UNIT,
+                       "ms_per_step": serial_ms / args.steps,
+                       "note": "same steps without dc_lookahead_frame and with per-launch events: source of stage_ms and the rooflines"},
+            "lookahead": overlap}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

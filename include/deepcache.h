@@ -170,6 +170,15 @@ int dc_conv_partial(dc_cache* cache, int layer, const void* in_map_dev, const vo
 int dc_infer_frame(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes,
                    void* out_map_dev, dc_frame_stats* stats_host);
 
+/* Announces the frame that the NEXT dc_infer_frame will get, so that its matching (Steps 1-5) runs on a
+ * side stream while the convolutions of the current frame are still running: Section 7.6 points out that
+ * matching one image and inferring another can proceed at the same time.  Call it after dc_infer_frame
+ * for frame t, with frame t+1; the next dc_infer_frame must then be given the same frame_dev and
+ * pitch_bytes (any other frame simply discards the lookahead).  frame_dev must stay unchanged until that
+ * call.  Results are identical with and without it.
+ * Errors: DC_ERR_ARG, DC_ERR_STATE (no frame inferred yet, or layer table not executable), DC_ERR_CUDA. */
+int dc_lookahead_frame(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes);
+
 /* Same as dc_infer_frame with HOST buffers: copies the frames to the device, runs the
  * path, copies the last map back, and waits.  frame_host should be pinned memory for
  * full copy speed.  out_map_host may be NULL. */
@@ -179,7 +188,8 @@ int dc_infer_frame_host(dc_cache* cache, const uint8_t* frame_host, size_t pitch
 /* Starts the host-to-device copy of the NEXT frame on a separate stream, so it overlaps the frame being
  * computed (Section 7.6 notes that matching one image and inferring another can run at the same time).
  * A later dc_infer_frame_host with the same frame_host and pitch_bytes uses that copy instead of copying
- * again.  Typical loop: prefetch(frame t+1), infer(frame t), prefetch(frame t+2), infer(frame t+1), ...
+ * again, and matches the prefetched frame on a side stream while the current one is computed (as
+ * dc_lookahead_frame does).  Typical loop: prefetch(frame t+1), infer(frame t), prefetch(frame t+2), infer(frame t+1), ...
  * At most two frames can be pending (DC_ERR_STATE otherwise).  frame_host must stay unchanged until that call and should be
  * pinned memory (a pageable buffer makes the copy synchronous).  Errors: DC_ERR_ARG, DC_ERR_ALLOC, DC_ERR_CUDA. */
 int dc_prefetch_frame_host(dc_cache* cache, const uint8_t* frame_host, size_t pitch_bytes);

@@ -48,7 +48,7 @@ REGION_DTYPE = np.dtype([(n, "<i4") for n in ("x", "y", "w", "h", "sx", "sy")])
 
 EXPORTS = ["dc_cache_create", "dc_cache_destroy", "dc_cache_reset", "dc_cache_bytes", "dc_cache_set_key",
            "dc_match_blocks", "dc_propagate_regions", "dc_conv_partial", "dc_infer_frame", "dc_infer_frame_host",
-           "dc_prefetch_frame_host",
+           "dc_prefetch_frame_host", "dc_lookahead_frame",
            "dc_cache_layer_map", "dc_cache_layer_regions", "dc_get_status", "dc_cache_launches",
            "dc_cache_set_profiling", "dc_cache_profile", "dc_cache_counters", "dc_search_blocks_noalloc", "dc_strerror"]
 PROFILE_STAGES = ["search", "verify", "merge", "propagate", "classify_copy", "conv", "input", "pointwise", "key_update"]
@@ -82,6 +82,7 @@ def load():
         L.dc_infer_frame.argtypes = [vp, vp, sz, vp, C.POINTER(dc_frame_stats)]
         L.dc_infer_frame_host.argtypes = [vp, vp, sz, vp, C.POINTER(dc_frame_stats)]
         L.dc_prefetch_frame_host.argtypes = [vp, vp, sz]
+        L.dc_lookahead_frame.argtypes = [vp, vp, sz]
         L.dc_cache_layer_map.argtypes = [vp, i, C.POINTER(vp), C.POINTER(sz)]
         L.dc_cache_layer_regions.argtypes = [vp, i, C.POINTER(vp), C.POINTER(vp)]
         L.dc_get_status.argtypes = [vp, C.POINTER(C.c_int32)]
@@ -189,6 +190,10 @@ def dc_infer_frame(cache, frame, pitch, out_map=None, stats=None):
 def dc_infer_frame_host(cache, frame_host_ptr, pitch, out_host_ptr=None, stats=None):
     _check(load().dc_infer_frame_host(cache, C.c_void_p(frame_host_ptr), pitch,
                                       C.c_void_p(out_host_ptr) if out_host_ptr else None, stats), "dc_infer_frame_host")
+
+
+def dc_lookahead_frame(cache, frame, pitch):
+    _check(load().dc_lookahead_frame(cache, _ptr(frame), pitch), "dc_lookahead_frame")
 
 
 def dc_prefetch_frame_host(cache, frame_host_ptr, pitch):

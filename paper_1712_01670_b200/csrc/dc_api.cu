@@ -19,6 +19,14 @@ void dc_note_cuda_error(cudaError_t e, const char* file, int line)
 
 void dc_prof_release(dc_cache* c);
 
+void dc_use_match_set(dc_cache* c, int k)
+{
+    const dc_match_set& m = c->mset[k];
+    c->mset_cur = k;
+    c->blk_mv = m.blk_mv; c->blk_sse = m.blk_sse; c->matched = m.matched; c->run_end = m.run_end; c->mv_acc = m.mv_acc;
+    c->long_list = m.long_list; c->gmv = m.gmv; c->regions0 = m.regions0; c->n_regions = m.n_regions;
+}
+
 namespace {
 
 // nearest bfloat16 (ties to even) of a double, as its 16 bit pattern
@@ -105,7 +113,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     // cached key frames: own pitch (16-byte multiple, at least 16 spare bytes per row and a spare
     // tail) so the matcher may fetch whole aligned words around any candidate
     c->key_pitch = ((size_t)cfg.width * 3 + 16 + 15) / 16 * 16;
-    for (int k = 0; k < 2; ++k) {
+    for (int k = 0; k < 3; ++k) {
         DC_TRY(dev_alloc(c, &c->key[k], c->key_pitch * cfg.height * S + 256));
         DC_CUDA(cudaMemsetAsync(c->key[k], 0, c->key_pitch * cfg.height * S + 256, c->stream));
     }
@@ -116,15 +124,20 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
         c->num_sms = sms;
     }
     const size_t nblk = (size_t)S * c->Gx * c->Gy;
-    DC_TRY(dev_alloc(c, &c->blk_mv, nblk * 2));
-    DC_TRY(dev_alloc(c, &c->blk_sse, nblk));
-    DC_TRY(dev_alloc(c, &c->matched, nblk));
-    DC_TRY(dev_alloc(c, &c->run_end, nblk));
-    DC_TRY(dev_alloc(c, &c->mv_acc, (size_t)S * 4 + 4));
-    DC_TRY(dev_alloc(c, &c->long_list, nblk));
-    DC_TRY(dev_alloc(c, &c->gmv, (size_t)S * 3));
-    DC_TRY(dev_alloc(c, &c->regions0, (size_t)S * c->max_regions));
-    DC_TRY(dev_alloc(c, &c->n_regions, (size_t)S));
+    for (int k = 0; k < 2; ++k) {
+        dc_match_set& m = c->mset[k];
+        DC_TRY(dev_alloc(c, &m.blk_mv, nblk * 2));
+        DC_TRY(dev_alloc(c, &m.blk_sse, nblk));
+        DC_TRY(dev_alloc(c, &m.matched, nblk));
+        DC_TRY(dev_alloc(c, &m.run_end, nblk));
+        DC_TRY(dev_alloc(c, &m.mv_acc, (size_t)S * 4 + 4));
+        DC_TRY(dev_alloc(c, &m.long_list, nblk));
+        DC_TRY(dev_alloc(c, &m.gmv, (size_t)S * 3));
+        DC_TRY(dev_alloc(c, &m.regions0, (size_t)S * c->max_regions));
+        DC_TRY(dev_alloc(c, &m.n_regions, (size_t)S));
+        DC_CUDA(cudaMemsetAsync(m.n_regions, 0, sizeof(int32_t) * S, c->stream));
+    }
+    dc_use_match_set(c, 0);
     DC_TRY(dev_alloc(c, &c->table, (size_t)n * S * c->max_regions));
     DC_TRY(dev_alloc(c, &c->layers_dev, (size_t)n));
     DC_TRY(dev_alloc(c, &c->in_hw_dev, (size_t)n * 2));
@@ -136,7 +149,6 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     DC_TRY(dev_alloc(c, &c->reused_total, (size_t)n));
     DC_CUDA(cudaMemsetAsync(c->reused_total, 0, sizeof(unsigned long long) * n, c->stream));
     DC_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int32_t), c->stream));
-    DC_CUDA(cudaMemsetAsync(c->n_regions, 0, sizeof(int32_t) * S, c->stream));
     DC_CUDA(cudaMemsetAsync(c->table, 0, sizeof(dc_region) * n * S * c->max_regions, c->stream));
     DC_CUDA(cudaMemcpyAsync(c->layers_dev, layers, sizeof(dc_layer_desc) * n, cudaMemcpyHostToDevice, c->stream));
 
@@ -221,9 +233,16 @@ void release(dc_cache* c)
 {
     dc_prof_release(c);
     cudaFree(c->reused_total);
-    cudaFree(c->key[0]); cudaFree(c->key[1]); cudaFree(c->staging[0]); cudaFree(c->staging[1]);
-    if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaEventDestroy(c->copied[0]); cudaEventDestroy(c->copied[1]); cudaStreamDestroy(c->copy_stream); } cudaFree(c->blk_mv); cudaFree(c->blk_sse); cudaFree(c->matched); cudaFree(c->run_end);
-    cudaFree(c->mv_acc); cudaFree(c->long_list); cudaFree(c->gmv); cudaFree(c->regions0); cudaFree(c->n_regions); cudaFree(c->table);
+    if (c->la_stream) { cudaStreamSynchronize(c->la_stream); cudaEventDestroy(c->ev_key); cudaEventDestroy(c->ev_match); cudaStreamDestroy(c->la_stream); }
+    if (c->copy_stream) { cudaStreamSynchronize(c->copy_stream); cudaEventDestroy(c->copied[0]); cudaEventDestroy(c->copied[1]); cudaStreamDestroy(c->copy_stream); }
+    for (int k = 0; k < 3; ++k) cudaFree(c->key[k]);
+    cudaFree(c->staging[0]); cudaFree(c->staging[1]);
+    for (int k = 0; k < 2; ++k) {
+        dc_match_set& m = c->mset[k];
+        cudaFree(m.blk_mv); cudaFree(m.blk_sse); cudaFree(m.matched); cudaFree(m.run_end); cudaFree(m.mv_acc);
+        cudaFree(m.long_list); cudaFree(m.gmv); cudaFree(m.regions0); cudaFree(m.n_regions);
+    }
+    cudaFree(c->table);
     cudaFree(c->layers_dev); cudaFree(c->in_hw_dev); cudaFree(c->dirty_count); cudaFree(c->all_count);
     cudaFree(c->reuse_px); cudaFree(c->zero_masks); cudaFree(c->status); cudaFree(c->input_map); cudaFree(c->pix_lut);
     if (c->stats_pinned) cudaFreeHost(c->stats_pinned);
@@ -241,6 +260,16 @@ const void* layer_input(dc_cache* c, int idx)
     if (idx < 0) return c->input_map;
     dc_layer_rt& P = c->L[idx];
     return P.map[P.d.kind == DC_CONV ? P.cur : 0];
+}
+
+// Drops a pending lookahead: the main stream first waits for it, so nothing it wrote is still in flight.
+int cancel_lookahead(dc_cache* c)
+{
+    if (c->la_frame) {
+        DC_CUDA(cudaStreamWaitEvent(c->stream, c->ev_match, 0));
+        c->la_frame = nullptr;
+    }
+    return DC_OK;
 }
 
 int fill_stats(dc_cache* c, bool refreshed, dc_frame_stats* stats)
@@ -309,6 +338,7 @@ int dc_cache_destroy(dc_cache* c)
 int dc_cache_reset(dc_cache* c)
 {
     if (!c) return DC_ERR_ARG;
+    DC_TRY(cancel_lookahead(c));
     c->key_valid = false; c->frame_idx = 0; c->frames_cached = 0; c->frames_full = 0;
     DC_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int32_t), c->stream));
     DC_CUDA(cudaMemsetAsync(c->reused_total, 0, sizeof(unsigned long long) * c->n_layers, c->stream));
@@ -332,6 +362,7 @@ int dc_cache_launches(const dc_cache* c, int64_t* launches)
 int dc_cache_set_key(dc_cache* c, const uint8_t* frame_dev, size_t pitch)
 {
     if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
+    DC_TRY(cancel_lookahead(c));
     DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, c->key[c->key_cur]));
     c->key_valid = true;
     return DC_OK;
@@ -343,8 +374,10 @@ int dc_match_blocks(dc_cache* c, const uint8_t* frame_dev, size_t pitch, int16_t
 {
     if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
     if (!c->key_valid) return DC_ERR_STATE;
-    DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, c->key[c->key_cur ^ 1]));   // scratch copy; the cache key stays
-    DC_TRY(dc_launch_match(c));
+    DC_TRY(cancel_lookahead(c));
+    uint8_t* scratch = c->key[(c->key_cur + 1) % 3];                             // scratch copy; the cache key stays
+    DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, scratch));
+    DC_TRY(dc_launch_match(c, scratch, c->key[c->key_cur]));
     const size_t nblk = (size_t)c->S * c->Gx * c->Gy;
     const cudaMemcpyKind k = cudaMemcpyDeviceToDevice;
     if (block_mv_dev) DC_CUDA(cudaMemcpyAsync(block_mv_dev, c->blk_mv, nblk * 2 * sizeof(int16_t), k, c->stream));
@@ -400,12 +433,22 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
     // Section 5: the cache is dropped and a whole new frame computed every N frames
     const bool refresh = !c->key_valid || (c->frame_idx % c->cfg.expire_n) == 0;
     // the library's own aligned copy of the frame: matched now, the cache key of the next frame (Section 3)
-    uint8_t* frame_copy = c->key[c->key_cur ^ 1];
-    DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, frame_copy));
+    uint8_t* frame_copy = c->key[(c->key_cur + 1) % 3];
+    const bool looked_ahead = c->la_frame == frame_dev && c->la_pitch == pitch && c->key_valid;
+    if (looked_ahead) {
+        // dc_lookahead_frame already copied this frame in and (unless it is a full frame) matched it
+        DC_CUDA(cudaStreamWaitEvent(c->stream, c->ev_match, 0));
+        c->la_frame = nullptr;
+    } else {
+        DC_TRY(cancel_lookahead(c));
+        DC_TRY(dc_launch_copy_frame(c, frame_dev, pitch, frame_copy));
+    }
+    if (c->la_stream) DC_CUDA(cudaEventRecord(c->ev_key, c->stream));   // a later lookahead may start from here
     if (!refresh) {
         DC_CUDA(cudaMemsetAsync(c->dirty_count, 0, sizeof(int32_t) * n, c->stream));
         DC_CUDA(cudaMemsetAsync(c->reuse_px, 0, sizeof(int32_t) * n * S * 2, c->stream));     // and `alive` behind it
-        DC_TRY(dc_launch_match(c));
+        if (looked_ahead && c->la_matched) dc_use_match_set(c, c->mset_cur ^ 1);              // results are waiting there
+        else DC_TRY(dc_launch_match(c, frame_copy, c->key[c->key_cur]));
         DC_TRY(dc_launch_propagate(c, c->regions0, c->n_regions, n));
     }
     if (c->input_map) DC_TRY(dc_launch_input_map(c, frame_copy, c->key_pitch));
@@ -433,13 +476,53 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
         default: return DC_ERR_STATE;
         }
     }
-    c->key_cur ^= 1;             // the frame becomes the next cache key
+    c->key_cur = (c->key_cur + 1) % 3;      // the frame becomes the next cache key
     c->key_valid = true;
     c->frame_idx += 1;
     if (refresh) c->frames_full += 1; else c->frames_cached += 1;
+    c->last_refreshed = refresh;
     if (out_map_dev)
         DC_CUDA(cudaMemcpyAsync(out_map_dev, layer_input(c, n - 1), c->L[n - 1].map_bytes, cudaMemcpyDeviceToDevice, c->stream));
     if (stats) return fill_stats(c, refresh, stats);
+    return DC_OK;
+}
+
+static int ensure_lookahead_stream(dc_cache* c)
+{
+    if (c->la_stream) return DC_OK;
+    DC_CUDA(cudaStreamCreateWithFlags(&c->la_stream, cudaStreamNonBlocking));
+    DC_CUDA(cudaEventCreateWithFlags(&c->ev_key, cudaEventDisableTiming));
+    DC_CUDA(cudaEventCreateWithFlags(&c->ev_match, cudaEventDisableTiming));
+    DC_CUDA(cudaEventRecord(c->ev_key, c->stream));     // first use: everything enqueued so far
+    return DC_OK;
+}
+
+int dc_lookahead_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch)
+{
+    if (!c || !frame_dev || pitch < (size_t)c->cfg.width * 3) return DC_ERR_ARG;
+    if (!c->executable || !c->key_valid) return DC_ERR_STATE;       // needs a frame to match against
+    DC_TRY(ensure_lookahead_stream(c));
+    DC_TRY(cancel_lookahead(c));
+    // Everything the side stream touches is free once the main stream has passed the frame copy of the last
+    // dc_infer_frame (where ev_key was recorded): the third key buffer was last read two frames ago, and the
+    // match set that the current inference does not read was last read by the frame before it.  Waiting for
+    // that point only -- not for the end of the current inference -- is what lets the two overlap.
+    DC_CUDA(cudaStreamWaitEvent(c->la_stream, c->ev_key, 0));
+    const bool next_is_full = (c->frame_idx % c->cfg.expire_n) == 0;
+    cudaStream_t main_stream = c->stream;
+    const int main_set = c->mset_cur;
+    c->stream = c->la_stream;                                       // the launchers enqueue on c->stream
+    uint8_t* next_copy = c->key[(c->key_cur + 1) % 3];
+    int rc = dc_launch_copy_frame(c, frame_dev, pitch, next_copy);
+    if (rc == DC_OK && !next_is_full) {
+        dc_use_match_set(c, main_set ^ 1);
+        rc = dc_launch_match(c, next_copy, c->key[c->key_cur]);
+        dc_use_match_set(c, main_set);
+    }
+    c->stream = main_stream;
+    if (rc != DC_OK) return rc;
+    DC_CUDA(cudaEventRecord(c->ev_match, c->la_stream));
+    c->la_frame = frame_dev; c->la_pitch = pitch; c->la_matched = !next_is_full;
     return DC_OK;
 }
 
@@ -492,8 +575,17 @@ int dc_infer_frame_host(dc_cache* c, const uint8_t* frame_host, size_t pitch, vo
         DC_CUDA(cudaMemcpyAsync(c->staging[slot], frame_host, bytes, cudaMemcpyHostToDevice, c->stream));
     }
     c->prefetched[slot] = nullptr;
-    int rc = dc_infer_frame(c, c->staging[slot], pitch, nullptr, stats);
+    int rc = dc_infer_frame(c, c->staging[slot], pitch, nullptr, nullptr);
     if (rc != DC_OK) return rc;
+    // a frame that is already prefetched can be matched on the side stream while this one is computed
+    const int other = slot ^ 1;
+    if (c->prefetched[other] && c->prefetched_pitch[other] == pitch && c->executable) {
+        DC_TRY(ensure_lookahead_stream(c));
+        DC_CUDA(cudaStreamWaitEvent(c->la_stream, c->copied[other], 0));
+        rc = dc_lookahead_frame(c, c->staging[other], pitch);
+        if (rc != DC_OK) return rc;
+    }
+    if (stats) { rc = fill_stats(c, c->last_refreshed, stats); if (rc != DC_OK) return rc; }
     if (out_map_host)
         DC_CUDA(cudaMemcpyAsync(out_map_host, layer_input(c, c->n_layers - 1), c->L[c->n_layers - 1].map_bytes,
                                 cudaMemcpyDeviceToHost, c->stream));

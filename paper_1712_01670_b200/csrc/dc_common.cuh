@@ -47,6 +47,13 @@ struct dc_layer_rt {
     int32_t* all_list;              // conv: every tile (used by full frames)
 };
 
+// Everything one run of the matcher writes.  Two sets exist so that the matcher may already work on the
+// next frame (dc_lookahead_frame) while inference of the current frame still reads its own set.
+struct dc_match_set {
+    int16_t* blk_mv; uint32_t* blk_sse; uint8_t* matched; uint16_t* run_end; int32_t* mv_acc; uint4* long_list;
+    int32_t* gmv; dc_region* regions0; int32_t* n_regions;
+};
+
 struct dc_cache {
     dc_config cfg;
     int n_layers;
@@ -60,8 +67,14 @@ struct dc_cache {
     int64_t launches;
     size_t bytes;
 
-    uint8_t* key[2];                // key frames [S][H][key_pitch]: key[key_cur] is the cached previous
-    int key_cur;                    // frame, the other one receives the frame being processed
+    uint8_t* key[3];                // key frames [S][H][key_pitch]: key[key_cur] is the cached previous frame,
+    int key_cur;                    // key[(key_cur + 1) % 3] receives the frame being processed or looked ahead
+    dc_match_set mset[2];           // the members blk_mv ... n_regions below alias mset[mset_cur]
+    int mset_cur;
+    cudaStream_t la_stream;         // dc_lookahead_frame: matcher of the next frame beside the current inference
+    cudaEvent_t ev_key, ev_match;   // main stream: frame copied in; side stream: lookahead finished
+    const uint8_t* la_frame; size_t la_pitch; bool la_matched;
+    bool last_refreshed;
     size_t key_pitch;
     int num_sms;
     uint8_t* staging[2];            // device copies of host frames for dc_infer_frame_host (one in use, one prefetching)
@@ -107,7 +120,8 @@ static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }
 
 // ---- kernels' host-side launchers (each returns DC_OK or DC_ERR_CUDA) ----
 int dc_launch_copy_frame(dc_cache* c, const uint8_t* frame, size_t pitch, uint8_t* dst);
-int dc_launch_match(dc_cache* c);      // current frame = key[key_cur ^ 1], previous = key[key_cur]
+int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key);   // both in key-frame layout
+void dc_use_match_set(dc_cache* c, int k);
 int dc_launch_propagate(dc_cache* c, const dc_region* in, const int32_t* n_in, int layer_end);
 int dc_launch_classify_copy(dc_cache* c, int layer, const dc_region* regions, const int32_t* n_regions,
                             const void* prev_out, void* out);

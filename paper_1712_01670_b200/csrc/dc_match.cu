@@ -668,11 +668,11 @@ int dc_launch_copy_frame(dc_cache* c, const uint8_t* frame, size_t pitch, uint8_
     return DC_OK;
 }
 
-int dc_launch_match(dc_cache* c)
+int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key)
 {
     MatchArgs a;
-    a.cur = c->key[c->key_cur ^ 1]; a.cur_pitch = c->key_pitch; a.cur_stream = c->key_pitch * (size_t)c->cfg.height;
-    a.prev = c->key[c->key_cur]; a.prev_pitch = c->key_pitch; a.prev_stream = c->key_pitch * (size_t)c->cfg.height;
+    a.cur = cur_key; a.cur_pitch = c->key_pitch; a.cur_stream = c->key_pitch * (size_t)c->cfg.height;
+    a.prev = prev_key; a.prev_pitch = c->key_pitch; a.prev_stream = c->key_pitch * (size_t)c->cfg.height;
     a.W = c->cfg.width; a.H = c->cfg.height; a.B = c->cfg.block; a.R = c->cfg.range;
     a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search; a.skip_k = c->cfg.skip_k;
     for (int i = 0; i < 4; ++i) a.limit[i] = c->sse_limit[i];

@@ -341,3 +341,42 @@ def test_region_overflow_sets_the_status_word():
         assert dc.status() == B.DC_OK
     finally:
         dc.close()
+
+
+def test_lookahead_gives_identical_results():
+    """dc_lookahead_frame moves the matching of frame t+1 beside the inference of frame t; outputs, motion
+    vectors and rectangles must not change.  Also: a lookahead for a frame that is then not used.
+    One cache runs the sequence twice (plain, then with lookahead) so that both passes use the same kernels."""
+    w = configs.WORKLOADS[3]()
+    sb = w.streams(1, 13)
+    frames = [torch.from_numpy(np.ascontiguousarray(sb.frame(i))).cuda() for i in range(13)]
+    dc = DeepCache.from_workload(w)
+    try:
+        pitch = w.width * 3
+
+        def run(lookahead):
+            rec = []
+            dc.reset()
+            for i in range(12):
+                out, st = dc.infer_frame(frames[i], want_stats=True)
+                out = out.clone()
+                if lookahead:
+                    if i == 5:
+                        B.dc_lookahead_frame(dc.handle, frames[0], pitch)        # announced, but frame 6 comes next
+                    elif i != 7:
+                        B.dc_lookahead_frame(dc.handle, frames[i + 1], pitch)    # crosses the expiry at frame 10
+                regs, _ = dc.layer_regions(-1)
+                key = (st[0].refreshed, st[0].mvx, st[0].mvy, st[0].k_passed, st[0].n_matched, st[0].n_regions)
+                rec.append((out, key, regs[0, :st[0].n_regions].clone()))
+            return rec
+
+        plain, ahead = run(False), run(True)
+        assert any(not k[0] and k[4] > 0 for _, k, _ in plain)
+        for i, ((o0, k0, r0), (o1, k1, r1)) in enumerate(zip(plain, ahead)):
+            assert k0 == k1, f"frame {i}: {k0} vs {k1}"
+            if not k0[0]:
+                assert torch.equal(r0, r1), f"frame {i} rectangles"
+            assert torch.equal(o0, o1), f"frame {i} output"
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
