@@ -187,7 +187,14 @@ def gpu_arm(args, w):
     dev = torch.device("cuda", local)
     if world > 1:
         dist.init_process_group("nccl", device_id=dev)
+    # The cache works on the stream that is current when it is created.  A stream of raised priority lets the
+    # inference kernels take the SMs ahead of the looked-ahead matcher, which runs on a lowest-priority stream.
+    with torch.cuda.stream(torch.cuda.Stream(dev, priority=-1)):
+        gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local, dev)
 
+
+def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local, dev):
+    import torch
     S = args.streams or w.n_streams
     total = args.warmup + args.steps
     # every rank renders its own streams: global stream index = rank * S + s
@@ -363,7 +370,7 @@ def gpu_arm(args, w):
             "serial": {"value": sharding.aggregate_rate(S * args.steps, world, serial_ms * 1e-3), "unit": UNIT,
                        "ms_per_step": serial_ms / args.steps,
                        "note": "same steps without dc_lookahead_frame and with per-launch events: source of stage_ms and the rooflines"},
-            "lookahead": overlap}
+            "lookahead": {"enabled": overlap, "main_stream_priority": -1, "side_stream_priority": 0}}
     print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()

@@ -175,7 +175,9 @@ int dc_infer_frame(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes
  * matching one image and inferring another can proceed at the same time.  Call it after dc_infer_frame
  * for frame t, with frame t+1; the next dc_infer_frame must then be given the same frame_dev and
  * pitch_bytes (any other frame simply discards the lookahead).  frame_dev must stay unchanged until that
- * call.  Results are identical with and without it.
+ * call.  Results are identical with and without it.  The side stream has the lowest priority; when the
+ * stream given to dc_cache_create has a higher one, the convolution kernels get the SMs first and the
+ * matcher fills what they leave, which shortens the overlapped step further.
  * Errors: DC_ERR_ARG, DC_ERR_STATE (no frame inferred yet, or layer table not executable), DC_ERR_CUDA. */
 int dc_lookahead_frame(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_bytes);
 

@@ -490,7 +490,9 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
 static int ensure_lookahead_stream(dc_cache* c)
 {
     if (c->la_stream) return DC_OK;
-    DC_CUDA(cudaStreamCreateWithFlags(&c->la_stream, cudaStreamNonBlocking));
+    int least = 0, greatest = 0;
+    DC_CUDA(cudaDeviceGetStreamPriorityRange(&least, &greatest));
+    DC_CUDA(cudaStreamCreateWithPriority(&c->la_stream, cudaStreamNonBlocking, least));
     DC_CUDA(cudaEventCreateWithFlags(&c->ev_key, cudaEventDisableTiming));
     DC_CUDA(cudaEventCreateWithFlags(&c->ev_match, cudaEventDisableTiming));
     DC_CUDA(cudaEventRecord(c->ev_key, c->stream));     // first use: everything enqueued so far
