@@ -145,9 +145,40 @@ static void search_ds(const uint8_t* cur, const uint8_t* prev, int W, int H, int
     *bdx = nx; *bdy = ny; *bsse = ns;
 }
 
+/* Three step search (named in Section 7.5 as an alternative unit for Step 2; its definition is the
+ * classic one from the block-matching literature the paper cites).  Around the current centre the
+ * eight points at (+-S, 0), (0, +-S), (+-S, +-S) are scored; the best of the nine becomes the centre;
+ * S halves; the pass with S = 1 gives the result.  The first step is the largest power of two S0
+ * with 2 S0 - 1 <= R (R = 7 gives the textbook 4, 2, 1), so no visited point lies beyond +-R by
+ * construction of the sum S0 + S0/2 + ... + 1; points outside the frame are skipped, and the bound
+ * on |d| is still checked for R that are not of the form 2^n - 1. */
+static void search_tss(const uint8_t* cur, const uint8_t* prev, int W, int H, int64_t pitch,
+                       int x0, int y0, int bw, int bh, int R, int* bdx, int* bdy, uint64_t* bsse)
+{
+    int S = 1;
+    while (2 * (2 * S) - 1 <= R) S *= 2;
+    if (R < 1) S = 0;
+    int cx = 0, cy = 0;
+    uint64_t cs = orc_block_sse(cur, prev, W, H, pitch, x0, y0, bw, bh, 0, 0);
+    for (; S >= 1; S /= 2) {
+        int nx = cx, ny = cy; uint64_t ns = cs;
+        for (int j = -1; j <= 1; ++j)
+            for (int i = -1; i <= 1; ++i) {
+                if (i == 0 && j == 0) continue;
+                int dx = cx + i * S, dy = cy + j * S;
+                if (abs(dx) > R || abs(dy) > R) continue;
+                uint64_t s = orc_block_sse(cur, prev, W, H, pitch, x0, y0, bw, bh, dx, dy);
+                if (s == ORC_INVALID) continue;
+                if (key_less(s, dx, dy, ns, nx, ny)) { ns = s; nx = dx; ny = dy; }
+            }
+        cx = nx; cy = ny; cs = ns;
+    }
+    *bdx = cx; *bdy = cy; *bsse = cs;
+}
+
 #define ORC_NOT_SEARCHED UINT32_MAX
 
-/* Step 2 for the blocks of the grid.  kind: 0 exhaustive, 1 diamond.
+/* Step 2 for the blocks of the grid.  kind: 0 exhaustive, 1 diamond, 2 three step.
  * mv is [Gy][Gx][2] = (dx, dy); sse is [Gy][Gx].
  * skip_k (Section 4, "skipping some blocks"): only blocks whose row and column index are
  * multiples of skip_k are searched; the others get mv = (0, 0), sse = ORC_NOT_SEARCHED and take
@@ -162,6 +193,7 @@ void orc_search_k(const uint8_t* cur, const uint8_t* prev, int W, int H, int64_t
         if (bx % skip_k != 0 || by % skip_k != 0) { mv[2 * b] = 0; mv[2 * b + 1] = 0; sse[b] = ORC_NOT_SEARCHED; continue; }
         block_geom(W, H, B, bx, by, &x0, &y0, &bw, &bh);
         if (kind == 0) search_es(cur, prev, W, H, pitch, x0, y0, bw, bh, R, &dx, &dy, &s);
+        else if (kind == 2) search_tss(cur, prev, W, H, pitch, x0, y0, bw, bh, R, &dx, &dy, &s);
         else           search_ds(cur, prev, W, H, pitch, x0, y0, bw, bh, R, &dx, &dy, &s);
         mv[2 * b] = (int16_t)dx; mv[2 * b + 1] = (int16_t)dy; sse[b] = (uint32_t)s;
     }

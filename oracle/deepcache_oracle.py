@@ -25,7 +25,7 @@ _SRC = os.path.join(_HERE, "deepcache_oracle.c")
 _LIB = os.path.join(_HERE, "libdeepcache_oracle.so")
 
 KIND_CONV, KIND_MAXPOOL, KIND_RELU, KIND_ADD, KIND_CONCAT, KIND_RESIZE_AREA, KIND_LRN, KIND_FC = range(8)
-SEARCH_ES, SEARCH_DS = 0, 1
+SEARCH_ES, SEARCH_DS, SEARCH_TSS = 0, 1, 2
 QUANT_NONE, QUANT_BF16 = 0, 1
 
 

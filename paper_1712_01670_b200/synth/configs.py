@@ -8,7 +8,7 @@ import numpy as np
 
 from . import nets, streams
 
-SEARCH_ES, SEARCH_DS = 0, 1
+SEARCH_ES, SEARCH_DS, SEARCH_TSS = 0, 1, 2
 DTYPE_FP32, DTYPE_BF16 = 0, 1
 
 

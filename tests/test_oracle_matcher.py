@@ -329,3 +329,92 @@ def test_k_skip_searches_every_kth_block_only():
     m = orc.match_blocks(cur, prev, 16, 8, orc.SEARCH_DS, 20.0, skip_k=2)
     want = orc.verify(cur, prev, 16, m["M"][0], m["M"][1], m["K"], 20.0)
     assert np.array_equal(m["matched"], want)
+
+
+# ---------------------------------------------------------------------------
+# three step search (Section 7.5 names it as an alternative unit for Step 2)
+# ---------------------------------------------------------------------------
+def smooth_pair(shift, size=96):
+    """prev = sin(x) + sin(y) with period 16; cur[y][x] = prev[y + sy][x + sx] (see the diamond pin above)."""
+    y, x = np.mgrid[0:size, 0:size].astype(np.float64)
+    v = 127.0 + 60.0 * np.sin(2 * np.pi * x / 16.0) + 60.0 * np.sin(2 * np.pi * y / 16.0)
+    prev = np.repeat(np.rint(v).astype(np.uint8)[:, :, None], 3, 2)
+    return np.roll(prev, (-shift[1], -shift[0]), axis=(0, 1)), prev
+
+
+def test_three_step_with_range_1_is_the_exhaustive_search():
+    # R = 1: the only pass has S = 1, and the centre plus its eight neighbours are the whole +-1 window
+    g = rng(41)
+    prev = g.integers(0, 256, size=(37, 45, 3), dtype=np.uint8)
+    cur = g.integers(0, 256, size=(37, 45, 3), dtype=np.uint8)
+    cur[5:30, 4:40] = prev[6:31, 3:39]                       # part of the frame moved by (-1, +1)
+    for B in (8, 10, 16):
+        tss, sse_tss = orc.search(cur, prev, B, 1, orc.SEARCH_TSS)
+        es, sse_es = orc.search(cur, prev, B, 1, orc.SEARCH_ES)
+        assert np.array_equal(tss, es) and np.array_equal(sse_tss, sse_es)
+
+
+@pytest.mark.parametrize("shift", [(3, -2), (-5, 4), (0, 6), (7, 7), (-7, 1), (1, 1), (0, 0)])
+def test_three_step_reaches_the_minimum_of_a_separable_basin(shift):
+    # steps 4, 2, 1 reach every displacement up to 7; on the separable single-basin surface each pass
+    # moves to the grid point nearest the true shift on both axes, so the result is the exhaustive one
+    cur, prev = smooth_pair(shift)
+    tss, sse_tss = orc.search(cur, prev, 16, 7, orc.SEARCH_TSS)
+    es, sse_es = orc.search(cur, prev, 16, 7, orc.SEARCH_ES)
+    inner = (slice(1, -1), slice(1, -1))
+    assert (es[inner][..., 0] == shift[0]).all() and (es[inner][..., 1] == shift[1]).all()
+    assert np.array_equal(tss[inner], es[inner]) and not sse_tss[inner].any()
+
+
+def test_three_step_first_step_rule():
+    # R = 8 still starts at S = 4 (2 * 8 - 1 > 8), so a shift of 8 is out of reach although inside the
+    # window; R = 15 starts at 8 and reaches it.  The pattern's period is 32 here so that 8 is unambiguous.
+    y, x = np.mgrid[0:128, 0:128].astype(np.float64)
+    v = 127.0 + 60.0 * np.sin(2 * np.pi * x / 32.0) + 60.0 * np.sin(2 * np.pi * y / 32.0)
+    prev = np.repeat(np.rint(v).astype(np.uint8)[:, :, None], 3, 2)
+    cur = np.roll(prev, (0, -8), axis=(0, 1))                # content shift (8, 0)
+    inner = (slice(1, -1), slice(1, -1))
+    es, _ = orc.search(cur, prev, 32, 8, orc.SEARCH_ES)
+    assert (es[inner][..., 0] == 8).all() and (es[inner][..., 1] == 0).all()
+    t8, s8 = orc.search(cur, prev, 32, 8, orc.SEARCH_TSS)
+    assert (t8[inner][..., 0] == 7).all() and (t8[inner][..., 1] == 0).all() and s8[inner].all()
+    t15, s15 = orc.search(cur, prev, 32, 15, orc.SEARCH_TSS)
+    assert (t15[inner][..., 0] == 8).all() and (t15[inner][..., 1] == 0).all() and not s15[inner].any()
+
+
+def tss_walk_reference(cur, prev, x0, y0, bw, bh, R):
+    """Independent restatement on a precomputed SSE surface: nine-point passes with halving step."""
+    surf = {}
+    for dy in range(-R, R + 1):
+        for dx in range(-R, R + 1):
+            s = brute_sse(cur, prev, x0, y0, bw, bh, dx, dy)
+            if s is not None:
+                surf[(dx, dy)] = (s, abs(dx) + abs(dy), dy, dx)
+    step = max(p for p in (1, 2, 4, 8, 16, 32, 64) if 2 * p - 1 <= R)
+    c, visited = (0, 0), {(0, 0)}
+    while step >= 1:
+        pts = [(c[0] + i * step, c[1] + j * step) for j in (-1, 0, 1) for i in (-1, 0, 1)]
+        visited.update(p for p in pts if p in surf)
+        c = min((p for p in pts if p in surf), key=lambda p: surf[p])
+        step //= 2
+    return c, surf[c][0], visited
+
+
+def test_three_step_invariants_on_video_frames():
+    w = configs.WORKLOADS[2]()
+    sb = w.streams(1, 6)
+    B = 16
+    for R, first in ((6, 2), (16, 8)):
+        for i in (1, 4):
+            cur, prev = sb.frame(i)[0][:80, :96], sb.frame(i - 1)[0][:80, :96]
+            mv, sse = orc.search(cur, prev, B, R, orc.SEARCH_TSS)
+            _, sse_es = orc.search(cur, prev, B, R, orc.SEARCH_ES)
+            assert (np.abs(mv) <= 2 * first - 1).all()           # reach of the step sequence
+            assert (sse >= sse_es).all()
+            for by in range(5):
+                for bx in range(6):
+                    dx, dy = (int(v) for v in mv[by, bx])
+                    assert orc.block_sse(cur, prev, bx * B, by * B, B, B, dx, dy) == int(sse[by, bx])
+                    best, s, visited = tss_walk_reference(cur, prev, bx * B, by * B, B, B, R)
+                    assert (dx, dy) == best and int(sse[by, bx]) == s
+                    assert len(visited) <= 1 + 8 * (first.bit_length())     # 9 points, then 8 new ones per pass
