@@ -43,6 +43,8 @@ def parse_args():
     ap.add_argument("--workload", type=int, default=5)
     ap.add_argument("--streams", type=int, default=0, help="override the number of streams per GPU")
     ap.add_argument("--skip-k", type=int, default=1, help="Step 2 on every k-th block row / column only (Section 4); default 1 = all blocks")
+    ap.add_argument("--search", default="", choices=["", "exhaustive", "diamond", "three_step"],
+                    help="Step 2 search unit; default: the workload's (diamond)")
     ap.add_argument("--no-lookahead", action="store_true", help="do not overlap the next frame's matching with this frame's inference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -61,7 +63,7 @@ def measured_peaks():
 
 def workload_config(w, n_streams, n_gpus):
     return {"workload": w.name, "streams_per_gpu": n_streams, "frame": f"{w.width}x{w.height}x3 uint8",
-            "block": w.block, "range": w.range, "search": "diamond" if w.search == 1 else "exhaustive",
+            "block": w.block, "range": w.range, "search": ("exhaustive", "diamond", "three_step")[w.search],
             "psnr_db": w.psnr_db, "expire_n": w.expire_n, "trunk_layers": len(w.layers),
             "parallelism": f"streams sharded over {n_gpus} GPU(s), no collective",
             "l2": "inputs larger than L2 (each step reads a fresh batch of frames)"}
@@ -380,6 +382,8 @@ def main():
     args = parse_args()
     from paper_1712_01670_b200.synth import configs
     w = configs.WORKLOADS[args.workload]()
+    if args.search:
+        w.search = {"exhaustive": configs.SEARCH_ES, "diamond": configs.SEARCH_DS, "three_step": configs.SEARCH_TSS}[args.search]
     if args.impl == "reference":
         reference_arm(args, w)
     else:

@@ -74,7 +74,10 @@ typedef struct {
     int32_t kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w;
 } dc_layer_desc;
 
-typedef enum { DC_SEARCH_EXHAUSTIVE = 0, DC_SEARCH_DIAMOND = 1 } dc_search_kind;
+/* The search unit of Step 2.  Exhaustive: every displacement within +-range.  Diamond: the paper's default
+ * (Section 4).  Three step: the alternative Section 7.5 compares; nine-point passes with step S0, S0/2, ..., 1
+ * where S0 is the largest power of two with 2 S0 - 1 <= range. */
+typedef enum { DC_SEARCH_EXHAUSTIVE = 0, DC_SEARCH_DIAMOND = 1, DC_SEARCH_THREE_STEP = 2 } dc_search_kind;
 typedef enum { DC_FP32 = 0, DC_BF16 = 1 } dc_dtype;
 
 /* The developer-facing knobs of Section 6 (threshold, block size, expiry) plus shapes. */

@@ -180,7 +180,7 @@ static void search_tss(const uint8_t* cur, const uint8_t* prev, int W, int H, in
 
 /* Step 2 for the blocks of the grid.  kind: 0 exhaustive, 1 diamond, 2 three step.
  * mv is [Gy][Gx][2] = (dx, dy); sse is [Gy][Gx].
- * skip_k (Section 4, "skipping some blocks"): only blocks whose row and column index are
+ * skip_k (Section 4, the k-skip acceleration): only blocks whose row and column index are
  * multiples of skip_k are searched; the others get mv = (0, 0), sse = ORC_NOT_SEARCHED and take
  * no part in Step 3.  skip_k = 1 searches every block. */
 void orc_search_k(const uint8_t* cur, const uint8_t* prev, int W, int H, int64_t pitch,

@@ -17,7 +17,7 @@ DC_OK = 0
 DC_ERR_ARG, DC_ERR_CONFIG, DC_ERR_ALLOC, DC_ERR_CUDA, DC_ERR_OVERFLOW, DC_ERR_TIMEOUT, DC_ERR_STATE, DC_ERR_LIMIT = range(-1, -9, -1)
 DC_NOALLOC_MAX_STREAMS = 64
 DC_CONV, DC_MAXPOOL, DC_RELU, DC_ADD, DC_CONCAT, DC_RESIZE_AREA, DC_LRN, DC_FC = range(8)
-DC_SEARCH_EXHAUSTIVE, DC_SEARCH_DIAMOND = 0, 1
+DC_SEARCH_EXHAUSTIVE, DC_SEARCH_DIAMOND, DC_SEARCH_THREE_STEP = 0, 1, 2
 DC_FP32, DC_BF16 = 0, 1
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdeepcache.so")

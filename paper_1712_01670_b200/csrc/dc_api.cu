@@ -58,7 +58,7 @@ int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
 {
     if (cfg->channels != 3 || cfg->width < 1 || cfg->height < 1 || cfg->n_streams < 1) return DC_ERR_CONFIG;
     if (cfg->block < 4 || cfg->block > 32 || cfg->range < 0 || cfg->range > 64) return DC_ERR_CONFIG;
-    if (cfg->search != DC_SEARCH_EXHAUSTIVE && cfg->search != DC_SEARCH_DIAMOND) return DC_ERR_CONFIG;
+    if (cfg->search < DC_SEARCH_EXHAUSTIVE || cfg->search > DC_SEARCH_THREE_STEP) return DC_ERR_CONFIG;
     if (cfg->skip_k < 1 || cfg->skip_k > 16 || cfg->expire_n < 1 || cfg->max_regions < 0) return DC_ERR_CONFIG;
     if (cfg->dtype != DC_FP32 && cfg->dtype != DC_BF16) return DC_ERR_CONFIG;
     if (!(cfg->psnr_db > 0.0) || !(cfg->psnr_db < 200.0)) return DC_ERR_CONFIG;

@@ -151,6 +151,22 @@ __global__ void __launch_bounds__(WARPS * 32) k_search(MatchArgs a)
                 unsigned long long k = cand_key(v, dx, dy);
                 if (k < bk) { bk = k; bs = v; bx_ = dx; by_ = dy; }
             }
+    } else if (a.search == DC_SEARCH_THREE_STEP) {
+        // nine-point passes with step S0, S0/2, ..., 1; S0 = largest power of two with 2 S0 - 1 <= R
+        int step = a.R < 1 ? 0 : 1;
+        while (4 * step - 1 <= a.R) step *= 2;
+        for (; step >= 1; step >>= 1) {
+            const int cx = bx_, cy = by_;
+#pragma unroll 1
+            for (int i = 0; i < 9; ++i) {
+                if (i == 4) continue;
+                const int dx = cx + (i % 3 - 1) * step, dy = cy + (i / 3 - 1) * step;
+                if (!c.valid(dx, dy)) continue;
+                uint32_t v = c.sse(dx, dy);
+                unsigned long long k = cand_key(v, dx, dy);
+                if (k < bk) { bk = k; bs = v; bx_ = dx; by_ = dy; }
+            }
+        }
     } else {
         // large diamond until its centre wins, then one small diamond
         const int lx[8] = {0, -1, 1, -2, 2, -1, 1, 0}, ly[8] = {-2, -1, -1, 0, 0, 1, 1, 2};
@@ -208,8 +224,8 @@ __global__ void __launch_bounds__(WARPS * 32) k_verify(MatchArgs a)
     int ok = 0;
     if (K > 0 && c.valid(Mx, My)) {
         const size_t g = (size_t)s * a.Gx * a.Gy + b;
-        // Section 4: "if the PSNR between (x_i, y_i) and (x_i + M_x, y_i + M_y) is already calculated
-        // in Step 2, we simply reuse the result" -- exact when the block's best vector is M itself
+        // Section 4's second acceleration: a score that Step 2 already computed for the pair (block, block + M)
+        // is taken over instead of being recomputed -- exact when the block's best vector is M itself
         uint32_t v = (a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My && a.sse[g] != 0xffffffffu) ? a.sse[g] : c.sse(Mx, My);
         ok = v <= a.limit[limit_index(a, c.bw, c.bh)];
     }

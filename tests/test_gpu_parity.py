@@ -56,7 +56,7 @@ def test_match_diamond_streams(widx, frames):
     check_pairs([(sb.frame(i - 1)[0], sb.frame(i)[0]) for i in frames], w.block, w.range, B.DC_SEARCH_DIAMOND)
 
 
-@pytest.mark.parametrize("search", [B.DC_SEARCH_EXHAUSTIVE, B.DC_SEARCH_DIAMOND])
+@pytest.mark.parametrize("search", [B.DC_SEARCH_EXHAUSTIVE, B.DC_SEARCH_DIAMOND, B.DC_SEARCH_THREE_STEP])
 @pytest.mark.parametrize("block,shape", [(8, (40, 56)), (10, (61, 47)), (16, (16, 16)), (16, (90, 131)), (32, (70, 100)), (5, (23, 29))])
 def test_match_edge_geometry(search, block, shape):
     g = rng(block * 7 + shape[0])
@@ -76,7 +76,7 @@ def test_match_ties_and_thresholds():
     row = ((x % 4) * 60).astype(np.uint8)
     prev = np.repeat(np.repeat(row[None, :, None], 48, 0), 3, 2)
     cur = np.roll(prev, -1, axis=1)
-    for search in (B.DC_SEARCH_EXHAUSTIVE, B.DC_SEARCH_DIAMOND):
+    for search in (B.DC_SEARCH_EXHAUSTIVE, B.DC_SEARCH_DIAMOND, B.DC_SEARCH_THREE_STEP):
         check_pairs([(prev, cur), (cur, prev)], 8, 6, search)
     # other thresholds move the integer SSE bound
     g = rng(3)
@@ -91,6 +91,27 @@ def test_match_full_hd_batch():
     w = configs.WORKLOADS[5]()
     sb = w.streams(2, 3)
     check_pairs([(sb.frame(1, s), sb.frame(2, s)) for s in range(2)], 16, 32, B.DC_SEARCH_DIAMOND)
+
+
+@pytest.mark.parametrize("widx,frames,R", [(2, (1, 2, 5), 16), (3, (1, 4), 7), (4, (2, 3), 24), (2, (3,), 1)])
+def test_match_three_step_streams(widx, frames, R):
+    """Three step search (Section 7.5) as the Step 2 unit: first steps 8, 4, 8 and 1 for these ranges."""
+    w = configs.WORKLOADS[widx]()
+    sb = w.streams(1, max(frames) + 1)
+    check_pairs([(sb.frame(i - 1)[0], sb.frame(i)[0]) for i in frames], w.block, R, B.DC_SEARCH_THREE_STEP)
+    check_pairs([(sb.frame(i - 1)[0], sb.frame(i)[0]) for i in frames], 10, R, B.DC_SEARCH_THREE_STEP, skip_k=2)
+
+
+def test_match_three_step_full_hd():
+    w = configs.WORKLOADS[5]()
+    sb = w.streams(2, 3)
+    check_pairs([(sb.frame(1, s), sb.frame(2, s)) for s in range(2)], 16, 32, B.DC_SEARCH_THREE_STEP)
+
+
+def test_infer_with_three_step():
+    w = configs.WORKLOADS[3]()
+    w.search = configs.SEARCH_TSS
+    U.run_stream_parity(w, 1, list(range(4)))
 
 
 @pytest.mark.parametrize("k", [2, 3])
