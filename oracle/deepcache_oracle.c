@@ -284,6 +284,58 @@ int orc_merge(const uint8_t* matched, int W, int H, int B, int Mx, int My, orc_r
     return n;
 }
 
+/* Per-block variant of Steps 4-5 (an extension: the paper moves every reused rectangle by the one global
+ * vector M; Section 4 notes that this loses blocks that move differently).  Here a searched block is
+ * accepted with its OWN best vector when that match passes the PSNR test of Step 2, and Step 5 merges
+ * only neighbours that carry the same vector: a horizontal run ends where the vector changes, and a run
+ * continues the rectangle above only when that run spans the same columns with the same vector.  Each
+ * rectangle's source is its position plus its blocks' vector.  Order and canonical form as orc_merge. */
+void orc_accept_own(const int16_t* mv, const uint32_t* sse, int W, int H, int B, double T, uint8_t* matched)
+{
+    int Gx = (W + B - 1) / B, Gy = (H + B - 1) / B;
+    for (int b = 0; b < Gx * Gy; ++b) {
+        int x0, y0, bw, bh;
+        block_geom(W, H, B, b % Gx, b / Gx, &x0, &y0, &bw, &bh);
+        matched[b] = (uint8_t)(sse[b] != ORC_NOT_SEARCHED && orc_psnr_pass(sse[b], (int64_t)bw * bh * 3, T));
+    }
+}
+
+int orc_merge_own(const uint8_t* matched, const int16_t* mv, int W, int H, int B, orc_region* out)
+{
+    int Gx = (W + B - 1) / B, Gy = (H + B - 1) / B, n = 0;
+    int* open_idx = (int*)malloc(sizeof(int) * Gx);      /* rectangle whose latest row has a run starting here */
+    int* open_end = (int*)malloc(sizeof(int) * Gx);
+    int* next_idx = (int*)malloc(sizeof(int) * Gx);
+    int* next_end = (int*)malloc(sizeof(int) * Gx);
+    for (int i = 0; i < Gx; ++i) open_idx[i] = -1;
+    for (int r = 0; r < Gy; ++r) {
+        for (int i = 0; i < Gx; ++i) next_idx[i] = -1;
+        int c = 0;
+        while (c < Gx) {
+            if (!matched[r * Gx + c]) { ++c; continue; }
+            int c0 = c, dx = mv[2 * (r * Gx + c)], dy = mv[2 * (r * Gx + c) + 1];
+            while (c < Gx && matched[r * Gx + c] && mv[2 * (r * Gx + c)] == dx && mv[2 * (r * Gx + c) + 1] == dy) ++c;
+            int c1 = c;
+            int y_px = r * B, y_end = (r + 1) * B < H ? (r + 1) * B : H;
+            int up = open_idx[c0];
+            if (up >= 0 && open_end[c0] == c1 && out[up].sx - out[up].x == dx && out[up].sy - out[up].y == dy) {
+                out[up].h += y_end - y_px;
+                next_idx[c0] = up;
+            } else {
+                int x_px = c0 * B, x_end = c1 * B < W ? c1 * B : W;
+                orc_region g = { x_px, y_px, x_end - x_px, y_end - y_px, x_px + dx, y_px + dy };
+                out[n] = g;
+                next_idx[c0] = n++;
+            }
+            next_end[c0] = c1;
+        }
+        memcpy(open_idx, next_idx, sizeof(int) * Gx);
+        memcpy(open_end, next_end, sizeof(int) * Gx);
+    }
+    free(open_idx); free(open_end); free(next_idx); free(next_end);
+    return n;
+}
+
 /* ------------------------------------------------------------------------
  * Section 5, "Propagation": the region transform D_t of Table 2
  * ---------------------------------------------------------------------- */

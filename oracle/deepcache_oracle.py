@@ -74,6 +74,10 @@ def lib():
         L.orc_verify.argtypes = [u8p, u8p, i, i, i64, i, i, i, i, d, u8p]
         L.orc_merge.restype = i
         L.orc_merge.argtypes = [u8p, i, i, i, i, i, rp]
+        L.orc_accept_own.restype = None
+        L.orc_accept_own.argtypes = [i16p, u32p, i, i, i, d, u8p]
+        L.orc_merge_own.restype = i
+        L.orc_merge_own.argtypes = [u8p, i16p, i, i, i, rp]
         L.orc_propagate_layer.restype = None
         L.orc_propagate_layer.argtypes = [lp, i, i, rp, rp, i, rp]
         L.orc_quant.restype = d
@@ -163,13 +167,38 @@ def merge(matched, W, H, B, Mx, My):
     return out[:n].copy()
 
 
-def match_blocks(cur, prev, B, R, kind, T, skip_k=1):
+REGIONS_GLOBAL, REGIONS_PER_BLOCK = 0, 1
+
+
+def accept_own(mv, sse, W, H, B, T):
+    """Per-block variant of Step 4: a block is matched when its own best vector passes the PSNR test."""
+    mv = np.ascontiguousarray(mv, np.int16)
+    sse = np.ascontiguousarray(sse, np.uint32)
+    matched = np.zeros(sse.shape, np.uint8)
+    lib().orc_accept_own(_p(mv, C.c_int16), _p(sse, C.c_uint32), W, H, B, float(T), _p(matched, C.c_uint8))
+    return matched
+
+
+def merge_own(matched, mv, W, H, B):
+    """Per-block variant of Step 5: only neighbours with the same vector merge; each rectangle carries its own."""
+    matched = _u8(matched)
+    mv = np.ascontiguousarray(mv, np.int16)
+    out = np.zeros(matched.size, REGION_DTYPE)
+    n = lib().orc_merge_own(_p(matched, C.c_uint8), _p(mv, C.c_int16), W, H, B, out.ctypes.data_as(C.POINTER(Region)))
+    return out[:n].copy()
+
+
+def match_blocks(cur, prev, B, R, kind, T, skip_k=1, region_mode=REGIONS_GLOBAL):
     """Steps 1-5 in order.  Returns dict(mv, sse, M, K, matched, regions)."""
     H, W = cur.shape[:2]
     mv, sse = search(cur, prev, B, R, kind, skip_k)
     Mx, My, K = mean_mv(mv, sse, W, H, B, T)
-    matched = verify(cur, prev, B, Mx, My, K, T)
-    regions = merge(matched, W, H, B, Mx, My)
+    if region_mode == REGIONS_PER_BLOCK:
+        matched = accept_own(mv, sse, W, H, B, T)
+        regions = merge_own(matched, mv, W, H, B)
+    else:
+        matched = verify(cur, prev, B, Mx, My, K, T)
+        regions = merge(matched, W, H, B, Mx, My)
     return dict(mv=mv, sse=sse, M=(Mx, My), K=K, matched=matched, regions=regions)
 
 
@@ -274,12 +303,13 @@ class OracleCache:
     """
 
     def __init__(self, width, height, layers, weights, biases, *, block=10, search_range=8,
-                 search_kind=SEARCH_DS, psnr_db=20.0, expire_n=10, quant=QUANT_NONE, use_cache=True, skip_k=1):
+                 search_kind=SEARCH_DS, psnr_db=20.0, expire_n=10, quant=QUANT_NONE, use_cache=True, skip_k=1,
+                 region_mode=0):
         self.W, self.H = width, height
         self.layers = layers
         self.block, self.R, self.kind = block, search_range, search_kind
         self.T, self.N, self.quant, self.use_cache = psnr_db, expire_n, quant, use_cache
-        self.skip_k = skip_k
+        self.skip_k, self.region_mode = skip_k, region_mode
         # weights are stored at the storage precision (bf16 workloads round them once)
         self.weights = [None if w is None else quant_array(w, quant) for w in weights]
         self.biases = [None if b is None else np.asarray(b, np.float64) for b in biases]
@@ -299,7 +329,8 @@ class OracleCache:
         info = dict(refreshed=bool(refresh), match=None, regions=None, reused=[None] * len(layers))
         per_layer_regions = None
         if not refresh:
-            m = match_blocks(frame, self.prev_frame, self.block, self.R, self.kind, self.T, self.skip_k)
+            m = match_blocks(frame, self.prev_frame, self.block, self.R, self.kind, self.T, self.skip_k,
+                             self.region_mode)
             per_layer_regions = propagate(layers, (self.H, self.W), m["regions"])
             info["match"], info["regions"] = m, per_layer_regions
         maps = []

@@ -182,3 +182,34 @@ def test_workload_1_end_to_end_reuse():
     # reused values are close to, but not the same as, fresh ones (sigma = 2 pixel noise)
     diff = np.abs(b["out"][mask] - fresh[mask])
     assert 0 < diff.max() < 0.2
+
+
+def test_per_block_mode_reuses_two_motions_end_to_end():
+    # left half static, right half moved by its own vector: the global mode can keep one of them only
+    g = rng(12)
+    w = configs.WORKLOADS[1]()                              # one 3x3 convolution on a 64x64 frame, block 8
+    f0 = g.integers(0, 256, size=(64, 64, 3), dtype=np.uint8)
+    f1 = f0.copy()
+    f1[:, 32:] = np.roll(f0, (-2, 3), axis=(0, 1))[:, 32:]  # f1[y][x] = f0[y + 2][x - 3] on the right half
+    own = make_cache(w, region_mode=orc.REGIONS_PER_BLOCK)
+    glob = make_cache(w)
+    a = own.infer_frame(f0)
+    b = own.infer_frame(f1)
+    glob.infer_frame(f0)
+    c = glob.infer_frame(f1)
+    vectors = {(int(r["sx"] - r["x"]), int(r["sy"] - r["y"])) for r in b["match"]["regions"]}
+    assert vectors == {(0, 0), (-3, 2)}
+    mask = b["reused"][0].astype(bool)
+    # the global vector is the mean of the two motions and fits neither half of this noise image
+    assert c["match"]["M"] == (-1, 1) and not c["reused"][0].any()
+    assert mask.mean() > 0.5
+    for r in b["regions"][0]:
+        if r["w"] == 0:
+            continue
+        d = b["out"][r["y"]:r["y"] + r["h"], r["x"]:r["x"] + r["w"]]
+        s = a["out"][r["sy"]:r["sy"] + r["h"], r["sx"]:r["sx"] + r["w"]]
+        assert np.array_equal(d, s)
+    fresh = make_cache(w, use_cache=False).infer_frame(f1)["out"]
+    assert np.array_equal(b["out"][~mask], fresh[~mask])
+    # exact copies of content: reused values equal fresh ones here (no noise was added)
+    assert np.abs(b["out"] - fresh).max() < 1e-12

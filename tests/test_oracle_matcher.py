@@ -418,3 +418,105 @@ def test_three_step_invariants_on_video_frames():
                     best, s, visited = tss_walk_reference(cur, prev, bx * B, by * B, B, B, R)
                     assert (dx, dy) == best and int(sse[by, bx]) == s
                     assert len(visited) <= 1 + 8 * (first.bit_length())     # 9 points, then 8 new ones per pass
+
+
+# ---------------------------------------------------------------------------
+# per-block region mode: every rectangle carries the vector of its own blocks
+# ---------------------------------------------------------------------------
+def merge_own_reference(matched, mv, W, H, B):
+    """Independent restatement: label runs per row, then chain runs with equal (columns, vector) downwards."""
+    Gy, Gx = matched.shape
+    runs = []                                               # per row: list of (c0, c1, dx, dy)
+    for r in range(Gy):
+        row, c = [], 0
+        while c < Gx:
+            if not matched[r, c]:
+                c += 1
+                continue
+            c0, v = c, tuple(mv[r, c])
+            while c < Gx and matched[r, c] and tuple(mv[r, c]) == v:
+                c += 1
+            row.append((c0, c, v[0], v[1]))
+        runs.append(row)
+    out = []
+    for r in range(Gy):
+        for run in runs[r]:
+            if r > 0 and run in runs[r - 1]:
+                continue                                    # continues the rectangle above
+            h = 1
+            while r + h < Gy and run in runs[r + h]:
+                h += 1
+            x, y = run[0] * B, r * B
+            x1, y1 = min(run[1] * B, W), min((r + h) * B, H)
+            out.append((x, y, x1 - x, y1 - y, x + run[2], y + run[3]))
+    return sorted(out, key=lambda t: (t[1], t[0]))
+
+
+def test_merge_own_equals_global_merge_when_all_vectors_agree():
+    g = rng(8)
+    W, H, B = 75, 52, 10
+    Gx, Gy = 8, 6
+    matched = (g.random((Gy, Gx)) < 0.7).astype(np.uint8)
+    mv = np.zeros((Gy, Gx, 2), np.int16)
+    mv[..., 0], mv[..., 1] = 3, -2
+    a = orc.merge_own(matched, mv, W, H, B)
+    b = orc.merge(matched, W, H, B, 3, -2)
+    assert [tuple(v) for v in a] == [tuple(v) for v in b]
+
+
+def test_merge_own_pins():
+    W, H, B = 40, 30, 10
+    mv = np.zeros((3, 4, 2), np.int16)
+    mv[:, :2] = (2, 0)                                      # left half moves by (2, 0), right half by (-3, 1)
+    mv[:, 2:] = (-3, 1)
+    r = orc.merge_own(np.ones((3, 4), np.uint8), mv, W, H, B)
+    assert [tuple(v) for v in r] == [(0, 0, 20, 30, 2, 0), (20, 0, 20, 30, 17, 1)]
+    # same columns, vector changes between rows 1 and 2: the rectangle is cut there
+    mv2 = np.zeros((3, 4, 2), np.int16)
+    mv2[2] = (1, 1)
+    r = orc.merge_own(np.ones((3, 4), np.uint8), mv2, W, H, B)
+    assert [tuple(v) for v in r] == [(0, 0, 40, 20, 0, 0), (0, 20, 40, 10, 1, 21)]
+    # a single odd block splits its row into three runs and breaks the column chains through it
+    mv3 = np.zeros((3, 4, 2), np.int16)
+    mv3[1, 1] = (0, -1)
+    r = orc.merge_own(np.ones((3, 4), np.uint8), mv3, W, H, B)
+    assert [tuple(v) for v in r] == [(0, 0, 40, 10, 0, 0), (0, 10, 10, 10, 0, 10), (10, 10, 10, 10, 10, 9),
+                                     (20, 10, 20, 10, 20, 10), (0, 20, 40, 10, 0, 20)]
+
+
+def test_merge_own_equals_reference_and_covers_matched_blocks():
+    g = rng(9)
+    for trial in range(40):
+        Gx, Gy, B = int(g.integers(1, 9)), int(g.integers(1, 8)), int(g.integers(4, 17))
+        W, H = Gx * B - int(g.integers(0, B)), Gy * B - int(g.integers(0, B))
+        matched = (g.random((Gy, Gx)) < 0.75).astype(np.uint8)
+        mv = g.integers(-1, 1, size=(Gy, Gx, 2)).astype(np.int16)      # few distinct vectors: long runs and chains
+        r = orc.merge_own(matched, mv, W, H, B)
+        assert [tuple(v) for v in r] == merge_own_reference(matched, mv, W, H, B)
+        m = cover(r, W, H)
+        expect = np.kron(matched, np.ones((B, B), np.int32))[:H, :W]
+        assert np.array_equal(m, expect)                                # disjoint, exactly the matched blocks
+        for v in r:                                                     # every block inside carries the rectangle's vector
+            blk = mv[v["y"] // B:-(-(v["y"] + v["h"]) // B), v["x"] // B:-(-(v["x"] + v["w"]) // B)]
+            assert (blk[..., 0] == v["sx"] - v["x"]).all() and (blk[..., 1] == v["sy"] - v["y"]).all()
+
+
+def test_accept_own_is_the_step_2_psnr_test():
+    g = rng(10)
+    prev = g.integers(0, 256, size=(48, 64, 3), dtype=np.uint8)
+    cur = prev.copy()
+    cur[:, 32:] = np.roll(prev, (-1, 3), axis=(0, 1))[:, 32:]           # right half: cur[y][x] = prev[y + 1][x - 3]
+    cur[16:32, 0:16] = g.integers(0, 256, size=(16, 16, 3))             # one block replaced by noise
+    m = orc.match_blocks(cur, prev, 16, 4, orc.SEARCH_ES, 20.0, region_mode=orc.REGIONS_PER_BLOCK)
+    lim = 16 * 16 * 3 * 65025 // 100                                    # 20 dB: SSE < n * 650.25
+    assert np.array_equal(m["matched"], (m["sse"] <= lim).astype(np.uint8))
+    assert m["matched"][1, 0] == 0 and m["matched"].sum() == 9          # bottom right row would leave the frame
+    regs = [tuple(v) for v in m["regions"]]
+    assert (0, 0, 32, 16, 0, 0) in regs                                 # left half above the noise block, unmoved
+    assert (32, 0, 32, 32, 29, 1) in regs                               # right half with its own vector
+    # the global mode keeps one vector only: with two motions it loses one half
+    g0 = orc.match_blocks(cur, prev, 16, 4, orc.SEARCH_ES, 20.0)
+    assert g0["matched"].sum() < m["matched"].sum()
+    # k-skip: blocks that were not searched have no vector of their own and stay unmatched
+    k = orc.match_blocks(cur, prev, 16, 4, orc.SEARCH_ES, 20.0, skip_k=2, region_mode=orc.REGIONS_PER_BLOCK)
+    assert not k["matched"][1::2].any() and not k["matched"][:, 1::2].any() and k["matched"][0, 0]
