@@ -79,6 +79,13 @@ typedef struct {
  * where S0 is the largest power of two with 2 S0 - 1 <= range. */
 typedef enum { DC_SEARCH_EXHAUSTIVE = 0, DC_SEARCH_DIAMOND = 1, DC_SEARCH_THREE_STEP = 2 } dc_search_kind;
 typedef enum { DC_FP32 = 0, DC_BF16 = 1 } dc_dtype;
+/* How matched blocks become rectangles.  DC_REGIONS_GLOBAL is the paper's Steps 3-5: one mean vector M per frame,
+ * blocks verified at M, every rectangle displaced by M.  DC_REGIONS_PER_BLOCK is an extension with no counterpart
+ * in the paper (Section 4 names the limit it lifts: content that moves against the global vector is lost):
+ * a searched block is accepted with its own Step 2 vector when that match passes the threshold, and only
+ * neighbours with the same vector merge, so each rectangle carries its own displacement.  The global vector
+ * is still computed and reported.  Blocks skipped by skip_k have no vector and stay unmatched in this mode. */
+typedef enum { DC_REGIONS_GLOBAL = 0, DC_REGIONS_PER_BLOCK = 1 } dc_region_mode;
 
 /* The developer-facing knobs of Section 6 (threshold, block size, expiry) plus shapes. */
 typedef struct {
@@ -93,6 +100,7 @@ typedef struct {
     double  psnr_db;                   /* similarity threshold T in dB (default 20) */
     int32_t dtype;                     /* dc_dtype of maps and arithmetic inputs */
     int32_t max_regions;               /* rectangles per stream; 0 = worst case of the grid */
+    int32_t region_mode;               /* dc_region_mode; 0 = the paper's global vector */
 } dc_config;
 
 /* Per-stream outcome of one dc_infer_frame. */

@@ -18,6 +18,7 @@ DC_ERR_ARG, DC_ERR_CONFIG, DC_ERR_ALLOC, DC_ERR_CUDA, DC_ERR_OVERFLOW, DC_ERR_TI
 DC_NOALLOC_MAX_STREAMS = 64
 DC_CONV, DC_MAXPOOL, DC_RELU, DC_ADD, DC_CONCAT, DC_RESIZE_AREA, DC_LRN, DC_FC = range(8)
 DC_SEARCH_EXHAUSTIVE, DC_SEARCH_DIAMOND, DC_SEARCH_THREE_STEP = 0, 1, 2
+DC_REGIONS_GLOBAL, DC_REGIONS_PER_BLOCK = 0, 1
 DC_FP32, DC_BF16 = 0, 1
 
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libdeepcache.so")
@@ -35,7 +36,8 @@ class dc_layer_desc(C.Structure):
 class dc_config(C.Structure):
     _fields_ = [("width", C.c_int32), ("height", C.c_int32), ("channels", C.c_int32), ("n_streams", C.c_int32),
                 ("block", C.c_int32), ("range", C.c_int32), ("search", C.c_int32), ("skip_k", C.c_int32),
-                ("expire_n", C.c_int32), ("psnr_db", C.c_double), ("dtype", C.c_int32), ("max_regions", C.c_int32)]
+                ("expire_n", C.c_int32), ("psnr_db", C.c_double), ("dtype", C.c_int32), ("max_regions", C.c_int32),
+                ("region_mode", C.c_int32)]
 
 
 class dc_frame_stats(C.Structure):

@@ -59,6 +59,7 @@ int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
     if (cfg->channels != 3 || cfg->width < 1 || cfg->height < 1 || cfg->n_streams < 1) return DC_ERR_CONFIG;
     if (cfg->block < 4 || cfg->block > 32 || cfg->range < 0 || cfg->range > 64) return DC_ERR_CONFIG;
     if (cfg->search < DC_SEARCH_EXHAUSTIVE || cfg->search > DC_SEARCH_THREE_STEP) return DC_ERR_CONFIG;
+    if (cfg->region_mode != DC_REGIONS_GLOBAL && cfg->region_mode != DC_REGIONS_PER_BLOCK) return DC_ERR_CONFIG;
     if (cfg->skip_k < 1 || cfg->skip_k > 16 || cfg->expire_n < 1 || cfg->max_regions < 0) return DC_ERR_CONFIG;
     if (cfg->dtype != DC_FP32 && cfg->dtype != DC_BF16) return DC_ERR_CONFIG;
     if (!(cfg->psnr_db > 0.0) || !(cfg->psnr_db < 200.0)) return DC_ERR_CONFIG;
@@ -317,7 +318,9 @@ int dc_cache_create(const dc_config* cfg, const dc_layer_desc* layers, int n_lay
     c->S = cfg->n_streams;
     c->Gx = dc_div_up(cfg->width, cfg->block); c->Gy = dc_div_up(cfg->height, cfg->block);
     // Step 5 never yields more than ceil(Gx / 2) * Gy rectangles (runs in a row are separated)
-    c->max_regions = cfg->max_regions > 0 ? cfg->max_regions : dc_div_up(c->Gx, 2) * c->Gy;
+    // worst case: alternating matched / unmatched blocks in every row; in per-block mode every block on its own
+    const int worst = cfg->region_mode == DC_REGIONS_PER_BLOCK ? c->Gx * c->Gy : dc_div_up(c->Gx, 2) * c->Gy;
+    c->max_regions = cfg->max_regions > 0 ? cfg->max_regions : worst;
     c->elt = cfg->dtype == DC_BF16 ? 2 : 4;
     c->executable = true;
     for (int i = 0; i < n_layers; ++i) if (!kind_executable(layers[i].kind)) c->executable = false;

@@ -23,7 +23,7 @@ constexpr int MAX_ROW_WORDS = 24;       // block <= 32 px -> 96 bytes per row
 struct MatchArgs {
     const uint8_t* cur;  size_t cur_pitch;  size_t cur_stream;
     const uint8_t* prev; size_t prev_pitch; size_t prev_stream;
-    int W, H, B, R, Gx, Gy, S, search, skip_k;
+    int W, H, B, R, Gx, Gy, S, search, skip_k, region_mode;
     uint32_t limit[4];
     int16_t* mv; uint32_t* sse; uint8_t* matched; int32_t* acc; int32_t* gmv;
 };
@@ -212,6 +212,27 @@ __device__ __forceinline__ int round_mean(int sum, int n)
     return sum < 0 ? -m : m;
 }
 
+// Per-block mode, in place of Step 4: a searched block is accepted with its own vector when that match passed
+// the PSNR test of Step 2.  One thread per block.  The global vector is still reported.
+__global__ void k_accept_own(MatchArgs a)
+{
+    const int per = a.Gx * a.Gy;
+    const int gi = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gi >= per * a.S) return;
+    const int s = gi / per, b = gi - s * per, by = b / a.Gx, bx = b - by * a.Gx;
+    const int bw = min(a.B, a.W - bx * a.B), bh = min(a.B, a.H - by * a.B);
+    const uint32_t v = a.sse[gi];
+    const int ok = v != 0xffffffffu && v <= a.limit[limit_index(a, bw, bh)];
+    a.matched[gi] = (uint8_t)ok;
+    if (ok) atomicAdd(&a.acc[4 * s + 3], 1);
+    if (b == 0) {
+        const int K = a.acc[4 * s + 2];
+        a.gmv[3 * s] = K > 0 ? round_mean(a.acc[4 * s + 0], K) : 0;
+        a.gmv[3 * s + 1] = K > 0 ? round_mean(a.acc[4 * s + 1], K) : 0;
+        a.gmv[3 * s + 2] = K;
+    }
+}
+
 template <int ITERS>
 __global__ void __launch_bounds__(WARPS * 32) k_verify(MatchArgs a)
 {
@@ -239,16 +260,27 @@ __global__ void __launch_bounds__(WARPS * 32) k_verify(MatchArgs a)
 // Step 5, part 1: for every block that starts a maximal horizontal run of matched blocks, the column
 // where the run ends; 0 for every other block (an end is never 0).  One thread per block; the forward
 // scan of a run start stays inside one row of bytes (cache hits after the first touch).
-__global__ void k_merge_runs(const uint8_t* matched, int Gx, int total, uint16_t* run_end)
+__global__ void k_merge_runs(const uint8_t* matched, const int16_t* mv, int Gx, int total, uint16_t* run_end)
 {
     const int b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b >= total) return;
     const int c = b % Gx;
     uint16_t e = 0;
-    if (matched[b] && (c == 0 || !matched[b - 1])) {
-        int j = c + 1;
-        while (j < Gx && matched[b - c + j]) ++j;
-        e = (uint16_t)j;
+    if (mv == nullptr) {
+        if (matched[b] && (c == 0 || !matched[b - 1])) {
+            int j = c + 1;
+            while (j < Gx && matched[b - c + j]) ++j;
+            e = (uint16_t)j;
+        }
+    } else if (matched[b]) {
+        // per-block mode: a run also ends where the vector changes
+        const uint32_t* v = (const uint32_t*)mv;                  // (dx, dy) as one word
+        const uint32_t mine = v[b];
+        if (c == 0 || !matched[b - 1] || v[b - 1] != mine) {
+            int j = c + 1;
+            while (j < Gx && matched[b - c + j] && v[b - c + j] == mine) ++j;
+            e = (uint16_t)j;
+        }
     }
     run_end[b] = e;
 }
@@ -256,7 +288,9 @@ __global__ void k_merge_runs(const uint8_t* matched, int Gx, int total, uint16_t
 // Step 5, part 2: a run continues the rectangle above it only when the run directly above starts and
 // ends at the same columns; every other run heads a rectangle that extends down while that holds.
 // One CTA per stream; heads are emitted in (y, x) order by a CTA-wide ordered compaction.
-__global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const int32_t* gmv, int W, int H, int B,
+// In per-block mode (mv != nullptr) the run above, and the runs below, must also carry the same vector,
+// and the rectangle's source is displaced by that vector instead of the global one.
+__global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const int16_t* mv, const int32_t* gmv, int W, int H, int B,
                                                 int Gx, int Gy, int max_regions, dc_region* regions,
                                                 int32_t* n_regions, int32_t* status)
 {
@@ -264,8 +298,9 @@ __global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const i
     __shared__ int base;
     const int s = blockIdx.x, tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
     const uint16_t* e = run_end + (size_t)s * Gx * Gy;
+    const uint32_t* v = mv ? (const uint32_t*)mv + (size_t)s * Gx * Gy : nullptr;
     dc_region* out = regions + (size_t)s * max_regions;
-    const int Mx = gmv[3 * s], My = gmv[3 * s + 1];
+    int Mx = gmv[3 * s], My = gmv[3 * s + 1];
     if (tid == 0) base = 0;
     __syncthreads();
     for (int start = 0; start < Gx * Gy; start += 1024) {
@@ -274,9 +309,9 @@ __global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const i
         if (b < Gx * Gy) {
             r = b / Gx; c0 = b - r * Gx;
             c1 = e[b];
-            if (c1 != 0 && !(r > 0 && e[b - Gx] == c1)) {
+            if (c1 != 0 && !(r > 0 && e[b - Gx] == c1 && (!v || v[b - Gx] == v[b]))) {
                 head = 1; h = 1;
-                while (r + h < Gy && e[b + h * Gx] == c1) ++h;
+                while (r + h < Gy && e[b + h * Gx] == c1 && (!v || v[b + h * Gx] == v[b])) ++h;
             }
         }
         // ordered compaction: exclusive scan of `head` over the 1024 threads
@@ -291,6 +326,7 @@ __global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const i
             if (idx < max_regions) {
                 const int x = c0 * B, y = r * B;
                 const int x1 = min(c1 * B, W), y1 = min((r + h) * B, H);
+                if (mv) { Mx = mv[2 * ((size_t)s * Gx * Gy + b)]; My = mv[2 * ((size_t)s * Gx * Gy + b) + 1]; }
                 dc_region g = { x, y, x1 - x, y1 - y, x + Mx, y + My };
                 out[idx] = g;
             } else {
@@ -690,7 +726,7 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
     a.cur = cur_key; a.cur_pitch = c->key_pitch; a.cur_stream = c->key_pitch * (size_t)c->cfg.height;
     a.prev = prev_key; a.prev_pitch = c->key_pitch; a.prev_stream = c->key_pitch * (size_t)c->cfg.height;
     a.W = c->cfg.width; a.H = c->cfg.height; a.B = c->cfg.block; a.R = c->cfg.range;
-    a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search; a.skip_k = c->cfg.skip_k;
+    a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search; a.skip_k = c->cfg.skip_k; a.region_mode = c->cfg.region_mode;
     for (int i = 0; i < 4; ++i) a.limit[i] = c->sse_limit[i];
     a.mv = c->blk_mv; a.sse = c->blk_sse; a.matched = c->matched; a.acc = c->mv_acc; a.gmv = c->gmv;
     // Step 3 sums and, behind them, the counter of walks handed to the second search phase
@@ -707,7 +743,10 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
     } else {
         launch_by_block(c, a, true);
     }
-    if (a.B == 16) {
+    if (a.region_mode == DC_REGIONS_PER_BLOCK) {
+        dc_prof_scope ps(c, DC_ST_VERIFY);
+        k_accept_own<<<dc_div_up(a.S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(a);
+    } else if (a.B == 16) {
         dc_prof_scope ps(c, DC_ST_VERIFY);
         k_verify16<<<dc_div_up(a.S * a.Gx * a.Gy, 16), 256, 0, c->stream>>>(a);
     } else {
@@ -715,8 +754,9 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
     }
     {
         dc_prof_scope ps(c, DC_ST_MERGE);
-        k_merge_runs<<<dc_div_up(c->S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(c->matched, a.Gx, c->S * a.Gx * a.Gy, c->run_end);
-        k_merge<<<c->S, 1024, 0, c->stream>>>(c->run_end, c->gmv, a.W, a.H, a.B, a.Gx, a.Gy, c->max_regions,
+        const int16_t* own = a.region_mode == DC_REGIONS_PER_BLOCK ? c->blk_mv : nullptr;
+        k_merge_runs<<<dc_div_up(c->S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(c->matched, own, a.Gx, c->S * a.Gx * a.Gy, c->run_end);
+        k_merge<<<c->S, 1024, 0, c->stream>>>(c->run_end, own, c->gmv, a.W, a.H, a.B, a.Gx, a.Gy, c->max_regions,
                                               c->regions0, c->n_regions, c->status);
     }
     c->launches += 4;

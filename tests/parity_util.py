@@ -64,7 +64,7 @@ def run_stream_parity(w, n_streams, frame_ids, check_layers=True, **kw):
     bit-exact matcher outputs, rectangles at every layer and reuse ratios, maps within tolerance."""
     bf16 = w.dtype == configs.DTYPE_BF16
     sb = w.streams(n_streams, max(frame_ids) + 1)
-    dc = DeepCache.from_workload(w, n_streams=n_streams, **{k: v for k, v in kw.items() if k in ("expire_n", "skip_k")})
+    dc = DeepCache.from_workload(w, n_streams=n_streams, **{k: v for k, v in kw.items() if k in ("expire_n", "skip_k", "region_mode")})
     oracles = make_oracles(w, n_streams, **kw)
     worst = 0.0
     try:

@@ -21,22 +21,23 @@ def rng(seed):
     return np.random.Generator(np.random.PCG64(seed))
 
 
-def matcher_only(width, height, n_streams, block, R, search, psnr_db=20.0, skip_k=1):
+def matcher_only(width, height, n_streams, block, R, search, psnr_db=20.0, skip_k=1, region_mode=0):
     layers = nets.single_conv(height, width)
     ws, bs = nets.random_weights(layers, 1)
     return DeepCache(width, height, layers, ws, bs, n_streams=n_streams, block=block, search_range=R,
-                     search=search, psnr_db=psnr_db, skip_k=skip_k)
+                     search=search, psnr_db=psnr_db, skip_k=skip_k, region_mode=region_mode)
 
 
-def check_pairs(pairs, block, R, search, psnr_db=20.0, skip_k=1):
+def check_pairs(pairs, block, R, search, psnr_db=20.0, skip_k=1, region_mode=0):
     """pairs: list of (prev, cur) frames of equal size, run as one batch of streams."""
     H, W = pairs[0][0].shape[:2]
-    dc = matcher_only(W, H, len(pairs), block, R, search, psnr_db, skip_k)
+    dc = matcher_only(W, H, len(pairs), block, R, search, psnr_db, skip_k, region_mode)
     try:
         dc.set_key(np.stack([p for p, _ in pairs]))
         got = dc.match_blocks(np.stack([c for _, c in pairs]))
         for s, (prev, cur) in enumerate(pairs):
-            U.assert_match_equal(got, s, orc.match_blocks(cur, prev, block, R, search, psnr_db, skip_k), f"stream {s}")
+            U.assert_match_equal(got, s, orc.match_blocks(cur, prev, block, R, search, psnr_db, skip_k, region_mode),
+                                 f"stream {s}")
         assert dc.status() == B.DC_OK
     finally:
         dc.close()
@@ -112,6 +113,43 @@ def test_infer_with_three_step():
     w = configs.WORKLOADS[3]()
     w.search = configs.SEARCH_TSS
     U.run_stream_parity(w, 1, list(range(4)))
+
+
+def two_motion_pair(g, H, W):
+    prev = g.integers(0, 256, size=(H, W, 3), dtype=np.uint8)
+    cur = prev.copy()
+    cur[:, W // 2:] = np.roll(prev, (-2, 3), axis=(0, 1))[:, W // 2:]
+    cur[H // 3:H // 3 + 7, 2:13] = g.integers(0, 256, size=(7, 11, 3))
+    return prev, cur
+
+
+@pytest.mark.parametrize("search", [B.DC_SEARCH_EXHAUSTIVE, B.DC_SEARCH_DIAMOND, B.DC_SEARCH_THREE_STEP])
+@pytest.mark.parametrize("block,shape", [(8, (40, 56)), (16, (90, 131)), (16, (64, 64)), (10, (61, 47))])
+def test_match_per_block_regions(search, block, shape):
+    """The per-block extension of Steps 4-5: own vectors, merge of equal vectors only (fast and generic kernels)."""
+    g = rng(block + shape[1])
+    H, W = shape
+    prev, cur = two_motion_pair(g, H, W)
+    smooth = np.clip(prev.astype(np.int32) + g.integers(-6, 7, size=prev.shape), 0, 255).astype(np.uint8)
+    check_pairs([(prev, cur), (prev, prev), (prev, smooth), (cur, prev)], block, 4, search,
+                region_mode=B.DC_REGIONS_PER_BLOCK)
+    check_pairs([(prev, cur)], block, 4, search, skip_k=2, region_mode=B.DC_REGIONS_PER_BLOCK)
+
+
+def test_match_per_block_streams_and_full_hd():
+    w = configs.WORKLOADS[4]()
+    sb = w.streams(1, 4)
+    check_pairs([(sb.frame(i - 1)[0], sb.frame(i)[0]) for i in (1, 2, 3)], 16, 24, B.DC_SEARCH_DIAMOND,
+                region_mode=B.DC_REGIONS_PER_BLOCK)
+    w = configs.WORKLOADS[5]()
+    sb = w.streams(2, 3)
+    check_pairs([(sb.frame(1, s), sb.frame(2, s)) for s in range(2)], 16, 32, B.DC_SEARCH_DIAMOND,
+                region_mode=B.DC_REGIONS_PER_BLOCK)
+
+
+@pytest.mark.parametrize("widx", [2, 3, 4])
+def test_infer_per_block_regions(widx):
+    U.run_stream_parity(configs.WORKLOADS[widx](), 1, list(range(4)), region_mode=B.DC_REGIONS_PER_BLOCK)
 
 
 @pytest.mark.parametrize("k", [2, 3])
