@@ -356,6 +356,24 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
                         "launches": prof["search"][1] + prof["verify"][1],
                         "bytes_per_frame_batch": 4.0 * frame_bytes * S}
 
+    if w.search == 0:
+        # Exhaustive search is plain integer arithmetic: every byte of every valid candidate takes one
+        # absolute difference and one multiply-accumulate.  Both run as 4-byte SIMD operations at 16 lanes
+        # per clock and SM sub-partition, on two pipes that work side by side, so the ceiling is
+        # SMs x 4 x 16 x 4 bytes per clock.
+        bw = np.minimum(w.block, w.width - np.arange(0, w.width, w.block))
+        bh = np.minimum(w.block, w.height - np.arange(0, w.height, w.block))
+        x0, y0 = np.arange(0, w.width, w.block), np.arange(0, w.height, w.block)
+        nx = np.minimum(w.range, w.width - bw - x0) + np.minimum(w.range, x0) + 1      # valid dx per block column
+        ny = np.minimum(w.range, w.height - bh - y0) + np.minimum(w.range, y0) + 1
+        byte_ops = 3.0 * float((nx * bw).sum()) * float((ny * bh).sum()) * S * n_cached
+        search_ms = prof["search"][0]
+        alu_peak = 148 * 4 * 16 * 4 * 1.965e9 / 1e12
+        ach = byte_ops / (search_ms * 1e-3) / 1e12 if search_ms > 0 else 0.0
+        roofline_matcher = {"kernel": "exhaustive block search", "bound": "alu", "achieved": ach, "peak": alu_peak,
+                            "unit": "T squared byte differences/s", "frac": ach / alu_peak,
+                            "peak_source": "148 SMs x 4 sub-partitions x 16 lanes x 4 bytes x 1965 MHz", "traffic": None,
+                            "launches": prof["search"][1], "ops_per_frame_batch": byte_ops / max(1, n_cached)}
     cpu_baseline = None
     if not args.no_cpu_baseline:
         fps, secs, what = run_oracle_sample(w, 3)

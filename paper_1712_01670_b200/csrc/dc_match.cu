@@ -24,6 +24,7 @@ struct MatchArgs {
     const uint8_t* cur;  size_t cur_pitch;  size_t cur_stream;
     const uint8_t* prev; size_t prev_pitch; size_t prev_stream;
     int W, H, B, R, Gx, Gy, S, search, skip_k, region_mode;
+    int edge_only;                       // generic search: only blocks clipped by the frame edge (the rest has a fast kernel)
     uint32_t limit[4];
     int16_t* mv; uint32_t* sse; uint8_t* matched; int32_t* acc; int32_t* gmv;
 };
@@ -98,6 +99,7 @@ __device__ __forceinline__ bool load_block(const MatchArgs& a, uint32_t* sm, Blo
     c.lane = threadIdx.x & 31;
     c.x0 = bx * a.B; c.y0 = by * a.B;
     c.bw = min(a.B, a.W - c.x0); c.bh = min(a.B, a.H - c.y0);
+    if (a.edge_only && c.bw == a.B && c.bh == a.B) return false;
     c.W = a.W; c.H = a.H; c.R = a.R;
     c.prev = a.prev + (size_t)s * a.prev_stream; c.prev_pitch = a.prev_pitch;
     c.cur_sm = sm;
@@ -660,6 +662,135 @@ __global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Fast Step 2: 16-pixel blocks, exhaustive search (plain integer ALU work: every displacement is scored)
+// ---------------------------------------------------------------------------------------------
+// One CTA per strip of 8 blocks, one warp per block.  The strip's search window (16 + 2R rows) is staged in
+// shared memory once.  A lane owns one horizontal displacement dx; for one 4-byte column of the block it
+// keeps the 16 rows of the current block in registers and walks down the window: every previous-frame word
+// it loads is scored against all block rows it can pair with, i.e. for E_DY vertical displacements at once,
+// so one (unaligned) load feeds up to 16 difference/accumulate pairs.  Displacements beyond the last full
+// group of 32 dx values are scored one candidate per lane.  Blocks clipped by the frame edge are left to
+// the generic kernel.
+constexpr int E_DY = 13;                        // vertical displacements scored together (65 = 5 * 13 for R = 32)
+constexpr int E_MAXR = 32;
+constexpr int E_PITCH = 152;                    // window row in words: (128 + 64) px * 3 B + 15 B alignment + one spare word, 16-byte multiple
+constexpr int E_MAXROWS = 16 + 2 * E_MAXR + E_DY - 1;   // plus rows only touched by displacements beyond R (scored, never compared)
+
+__global__ void __launch_bounds__(256, 3) k_search_es16(MatchArgs a)
+{
+    extern __shared__ uint32_t es_sm[];
+    const int R = a.R, n_d = 2 * R + 1;
+    const int chunks = (n_d + E_DY - 1) / E_DY;
+    const int rows = 16 + chunks * E_DY - 1;                     // <= E_MAXROWS
+    uint32_t* win = es_sm;
+    uint32_t* cur_all = es_sm + rows * E_PITCH;
+    const int strips = (a.Gx + 7) >> 3;
+    const int strip = blockIdx.x % strips, by = (blockIdx.x / strips) % a.Gy, s = blockIdx.x / (strips * a.Gy);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int xs = strip * 128, y0 = by * 16;
+    const int wx0 = ((xs - R) * 3) & ~15;                        // byte column of the window origin (may be < 0)
+    const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
+    const bool row_searched = (a.skip_k <= 1 || by % a.skip_k == 0) && a.H - y0 >= 16;
+    for (int i = threadIdx.x; row_searched && i < rows * (E_PITCH / 4); i += 256) {
+        const int row = i / (E_PITCH / 4), ci = i - row * (E_PITCH / 4);
+        const int gy = y0 - R + row, gb = wx0 + ci * 16;
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (gy >= 0 && gy < a.H && gb >= 0 && gb + 16 <= (int)a.prev_pitch)
+            v = __ldg((const uint4*)(prev + (size_t)gy * a.prev_pitch + gb));
+        *(uint4*)(win + row * E_PITCH + ci * 4) = v;
+    }
+    const int bx = strip * 8 + warp, x0 = bx * 16;
+    const bool full = bx < a.Gx && a.W - x0 >= 16 && a.H - y0 >= 16;
+    const bool skipped = a.skip_k > 1 && (bx % a.skip_k != 0 || by % a.skip_k != 0);
+    uint32_t* curw = cur_all + warp * 192;
+    if (full && !skipped) {                                       // the current block: 16 rows of 48 bytes
+        const uint8_t* cb = a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3;
+        for (int i = lane; i < 16 * 3; i += 32) {
+            const int r = i / 3, q = i - r * 3;
+            *(uint4*)(curw + r * 12 + q * 4) = __ldg((const uint4*)(cb + (size_t)r * a.cur_pitch) + q);
+        }
+    }
+    __syncthreads();
+    if (bx >= a.Gx) return;
+    const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
+    if (skipped) {
+        if (lane == 0) { a.mv[2 * g] = 0; a.mv[2 * g + 1] = 0; a.sse[g] = 0xffffffffu; }
+        return;
+    }
+    if (!full) return;                                            // clipped block: the generic kernel scores it
+
+    unsigned long long bk = ~0ull;
+    const int full_passes = n_d / 32;
+    for (int pass = 0; pass < full_passes; ++pass) {
+        const int dx = -R + pass * 32 + lane;
+        const int boff = (x0 + dx) * 3 - wx0;
+        const uint32_t sh = (boff & 3) * 8;
+        const bool x_ok = x0 + dx >= 0 && x0 + dx + 16 <= a.W;
+        for (int c = 0; c < chunks; ++c) {
+            const int dy0 = -R + c * E_DY;
+            uint32_t acc[E_DY];
+#pragma unroll
+            for (int d = 0; d < E_DY; ++d) acc[d] = 0;
+            const uint32_t* col = win + (c * E_DY) * E_PITCH + (boff >> 2);      // window row of displacement dy0, block row 0
+#pragma unroll 1
+            for (int j = 0; j < 12; ++j) {
+                uint32_t cw[16];
+#pragma unroll
+                for (int r = 0; r < 16; ++r) cw[r] = curw[r * 12 + j];
+#pragma unroll
+                for (int p = 0; p < 16 + E_DY - 1; ++p) {
+                    const uint32_t w = __funnelshift_r(col[p * E_PITCH + j], col[p * E_PITCH + j + 1], sh);
+#pragma unroll
+                    for (int r = 0; r < 16; ++r) {
+                        if (p - r >= 0 && p - r < E_DY) {
+                            const uint32_t t = __vabsdiffu4(cw[r], w);
+                            acc[p - r] = __dp4a(t, t, acc[p - r]);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int d = 0; d < E_DY; ++d) {
+                const int dy = dy0 + d;
+                if (x_ok && dy <= R && y0 + dy >= 0 && y0 + dy + 16 <= a.H) {
+                    const unsigned long long k = cand_key(acc[d], dx, dy);
+                    if (k < bk) bk = k;
+                }
+            }
+        }
+    }
+    // the remaining dx columns: one candidate per lane and round
+    const int dx_first = -R + full_passes * 32, n_left = (n_d - full_passes * 32) * n_d;
+    for (int i = lane; i < n_left; i += 32) {
+        const int dx = dx_first + i / n_d, dy = -R + i % n_d;
+        if (x0 + dx < 0 || x0 + dx + 16 > a.W || y0 + dy < 0 || y0 + dy + 16 > a.H) continue;
+        const int boff = (x0 + dx) * 3 - wx0;
+        const uint32_t sh = (boff & 3) * 8;
+        const uint32_t* col = win + (dy + R) * E_PITCH + (boff >> 2);
+        uint32_t acc = 0;
+#pragma unroll 2
+        for (int r = 0; r < 16; ++r) {
+            uint32_t lo = col[r * E_PITCH];
+#pragma unroll
+            for (int j = 0; j < 12; ++j) {
+                const uint32_t hi = col[r * E_PITCH + j + 1];
+                const uint32_t t = __vabsdiffu4(curw[r * 12 + j], __funnelshift_r(lo, hi, sh));
+                acc = __dp4a(t, t, acc);
+                lo = hi;
+            }
+        }
+        const unsigned long long k = cand_key(acc, dx, dy);
+        if (k < bk) bk = k;
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        const unsigned long long other = __shfl_xor_sync(0xffffffffu, bk, o);
+        if (other < bk) bk = other;
+    }
+    if (lane == 0) publish_block(a, s, g, 16, 16, bk);            // the zero vector is always valid, so bk is set
+}
+
 // Frame -> the library's aligned copy.  16-byte vectors when the source rows are aligned.
 __global__ void k_copy_frame(const uint8_t* src, size_t src_pitch, uint8_t* dst, size_t dst_pitch, int row_bytes,
                              int rows, int vec)
@@ -726,7 +857,7 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
     a.cur = cur_key; a.cur_pitch = c->key_pitch; a.cur_stream = c->key_pitch * (size_t)c->cfg.height;
     a.prev = prev_key; a.prev_pitch = c->key_pitch; a.prev_stream = c->key_pitch * (size_t)c->cfg.height;
     a.W = c->cfg.width; a.H = c->cfg.height; a.B = c->cfg.block; a.R = c->cfg.range;
-    a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search; a.skip_k = c->cfg.skip_k; a.region_mode = c->cfg.region_mode;
+    a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search; a.skip_k = c->cfg.skip_k; a.region_mode = c->cfg.region_mode; a.edge_only = 0;
     for (int i = 0; i < 4; ++i) a.limit[i] = c->sse_limit[i];
     a.mv = c->blk_mv; a.sse = c->blk_sse; a.matched = c->matched; a.acc = c->mv_acc; a.gmv = c->gmv;
     // Step 3 sums and, behind them, the counter of walks handed to the second search phase
@@ -740,6 +871,25 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
         if (grid > c->num_sms * 4) grid = c->num_sms * 4;
         k_search_ds16_long<<<grid, 256, 0, c->stream>>>(a, c->long_list, long_count);
         c->launches += 1;
+    } else if (a.B == 16 && a.search == DC_SEARCH_EXHAUSTIVE && a.R <= E_MAXR && a.W >= 16 && a.H >= 16) {
+        const int chunks = (2 * a.R + 1 + E_DY - 1) / E_DY;
+        const size_t smem = ((size_t)(16 + chunks * E_DY - 1) * E_PITCH + 8 * 192) * sizeof(uint32_t);
+        static bool attr_set = false;
+        if (!attr_set) {
+            DC_CUDA(cudaFuncSetAttribute(k_search_es16, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)(((size_t)E_MAXROWS * E_PITCH + 8 * 192) * sizeof(uint32_t))));
+            attr_set = true;
+        }
+        {
+            dc_prof_scope ps(c, DC_ST_SEARCH);
+            k_search_es16<<<((a.Gx + 7) / 8) * a.Gy * a.S, 256, smem, c->stream>>>(a);
+        }
+        if (a.W % 16 != 0 || a.H % 16 != 0) {                   // blocks clipped by the right / bottom edge
+            a.edge_only = 1;
+            launch_by_block(c, a, true);
+            a.edge_only = 0;
+            c->launches += 1;
+        }
     } else {
         launch_by_block(c, a, true);
     }

@@ -115,6 +115,31 @@ def test_infer_with_three_step():
     U.run_stream_parity(w, 1, list(range(4)))
 
 
+@pytest.mark.parametrize("R,shape", [(32, (97, 150)), (16, (64, 64)), (8, (50, 300)), (5, (33, 47)), (13, (80, 131)), (0, (32, 32))])
+def test_match_exhaustive_16_fast_path(R, shape):
+    """16-pixel blocks with exhaustive search run on the register-blocked kernel (full groups of 32 dx values,
+    the remaining columns one candidate per lane) and clipped edge blocks on the generic one."""
+    g = rng(R * 31 + shape[0])
+    H, W = shape
+    prev = g.integers(0, 256, size=(H, W, 3), dtype=np.uint8)
+    moved = np.roll(prev, (min(R, 3), -min(R, 7)), axis=(0, 1))
+    far = np.roll(prev, (-R, R), axis=(0, 1))                  # best vectors at the corner of the range
+    smooth = np.clip(prev.astype(np.int32) + g.integers(-6, 7, size=prev.shape), 0, 255).astype(np.uint8)
+    const = np.full_like(prev, 200)
+    check_pairs([(prev, moved), (prev, far), (prev, smooth), (const, const), (far, prev)], 16, R, B.DC_SEARCH_EXHAUSTIVE)
+    check_pairs([(prev, moved)], 16, R, B.DC_SEARCH_EXHAUSTIVE, skip_k=2)
+
+
+def test_match_exhaustive_video_streams():
+    w = configs.WORKLOADS[2]()
+    sb = w.streams(1, 4)
+    check_pairs([(sb.frame(i - 1)[0], sb.frame(i)[0]) for i in (1, 2, 3)], 16, 16, B.DC_SEARCH_EXHAUSTIVE)
+    w = configs.WORKLOADS[5]()                                 # 1920x1080: 120 full columns, last block row 8 px
+    sb = w.streams(1, 3)
+    f1, f2 = sb.frame(1, 0), sb.frame(2, 0)
+    check_pairs([(f1[:200, :1000], f2[:200, :1000])], 16, 32, B.DC_SEARCH_EXHAUSTIVE)
+
+
 def two_motion_pair(g, H, W):
     prev = g.integers(0, 256, size=(H, W, 3), dtype=np.uint8)
     cur = prev.copy()
