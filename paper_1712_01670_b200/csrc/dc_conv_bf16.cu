@@ -37,6 +37,7 @@ struct TcArgs {
     int BN, NB, BK, kchunks, stages, a_bytes, b_bytes;
     int MT, nbuf;                 // tiles per work item (1 or 2, sharing one B tile); TMEM accumulator sets (2, or 1 when MT * BN = 512)
     uint32_t idesc, sbo, layout_type;
+    uint32_t tmem_cols;           // TMEM columns this CTA allocates: a power of two >= nbuf * MT * BN (256 at most when two CTAs share an SM)
     int32_t* status;
 };
 
@@ -265,8 +266,8 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
     }
-    if (warp == 1) {       // 512 columns: two accumulators of up to 256 columns
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+    if (warp == 1) {       // up to 512 columns: two accumulators of up to 256 columns
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -358,7 +359,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(a.tmem_cols) : "memory");
     }
 }
 
@@ -410,7 +411,7 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
         ((uint4*)ring)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to TMA / MMA
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -477,7 +478,7 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(a.tmem_cols) : "memory");
     }
 }
 
@@ -531,7 +532,7 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     }
     if (warp == 1) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(512u) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     tc_fence_before();
@@ -638,7 +639,7 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(a.tmem_cols) : "memory");
     }
 }
 
@@ -698,9 +699,20 @@ EncodeTiledFn encode_fn()
     return fn;
 }
 
+// Two CTAs may share an SM when each needs at most 256 TMEM columns; each then gets half the operand-ring budget.
+// Layers with few output channels or a short K are bound by the epilogue (TMEM -> registers -> global), and a
+// second resident CTA doubles the epilogue warps per SM.
+static uint32_t tmem_cols_for(int nbuf, int mt, int bn)
+{
+    uint32_t need = (uint32_t)(nbuf * mt * bn), cols = 32;
+    while (cols < need) cols <<= 1;
+    return cols;
+}
+static int ring_budget(int ctas) { return 200 * 1024 / (ctas == 2 ? 2 : 1); }
+
 struct TcPlan { int BK, BN, NB, MT, nbuf, stages, a_bytes, b_bytes; CUtensorMapSwizzle swz; uint32_t layout_type, sbo; size_t smem; };
 
-bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn = 0)
+bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn = 0, int ctas = 1)
 {
     if (d.kind != DC_CONV) return false;
     if (d.sh < 1 || d.sw < 1 || DC_TILE_W * d.sw > 256 || DC_TILE_H * d.sh > 256) return false;   // TMA box limit
@@ -724,7 +736,8 @@ bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn =
     // MT * BN * nbuf accumulator columns
     p.MT = want_mt > 0 ? want_mt : 1;
     p.nbuf = p.MT * p.BN * 2 <= 512 ? 2 : 1;
-    int st = (200 * 1024) / (p.MT * p.a_bytes + p.b_bytes);
+    if (ctas == 2 && tmem_cols_for(p.nbuf, p.MT, p.BN) > 256) return false;
+    int st = ring_budget(ctas) / (p.MT * p.a_bytes + p.b_bytes);
     p.stages = st > kMaxStages ? kMaxStages : st;
     if (p.stages < 2) return false;
     p.smem = (size_t)p.stages * (p.MT * p.a_bytes + p.b_bytes) + sizeof(SmemCtl) + 1024;
@@ -823,7 +836,9 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     sa.PW = PW; sa.PH = PH;
     sa.stage_bytes = (PW * PH * 16 + 128 + 127) & ~127;          // patch + a readable pad behind its last pixel
     const int stage_bytes = sa.stage_bytes;
-    int st = (200 * 1024 - sa.w_bytes) / stage_bytes;
+    const int ctas = L.tc_ctas == 2 && tmem_cols_for(2, 1, d.cout) <= 256 ? 2 : 1;
+    a.tmem_cols = tmem_cols_for(2, 1, d.cout);
+    int st = (ring_budget(ctas) - sa.w_bytes) / stage_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
     const size_t smem = (size_t)a.stages * stage_bytes + ((sa.w_bytes + 127) & ~127) + sizeof(SmemCtl) + 256;
@@ -834,7 +849,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     }
     int grid_pad = (int)((pixels + 255) / 256); if (grid_pad > c->num_sms * 8) grid_pad = c->num_sms * 8;
     int items = max_tiles < 1 ? 1 : max_tiles;
-    int grid = items > c->num_sms ? c->num_sms : items;
+    int grid = items > c->num_sms * ctas ? c->num_sms * ctas : items;
     dc_prof_scope ps(c, DC_ST_CONV);
     k_pad_channels8<<<grid_pad, 256, 0, c->stream>>>((const __nv_bfloat16*)in, pixels, d.cin, (__nv_bfloat16*)L.in_padded);
     k_conv_tc_smallc<<<grid, kThreads, smem, c->stream>>>(tmA, sa);
@@ -871,12 +886,15 @@ static int launch_halo(dc_cache* c, int layer, int mt, const void* in, void* out
     ha.wpacked = (const __nv_bfloat16*)L.weight_halo;
     ha.PW = h.PW; ha.PH = h.PH; ha.plane_bytes = h.plane_bytes; ha.patch_bytes = h.patch_bytes;
     // patch ring: as deep as leaves at least 3 weight stages (a small-K item is one patch, so depth = items in flight)
+    a.tmem_cols = tmem_cols_for(a.nbuf, mt, h.BN);
+    const int ctas = L.tc_ctas == 2 && a.tmem_cols <= 256 ? 2 : 1;
+    const int budget = ring_budget(ctas);
     ha.a_stages = 2;
     for (int as = 4; as > 2; --as)
-        if (200 * 1024 - as * mt * h.patch_bytes >= 3 * h.b_bytes) { ha.a_stages = as; break; }
+        if (budget - as * mt * h.patch_bytes >= 3 * h.b_bytes) { ha.a_stages = as; break; }
     if (getenv("DC_HALO_ASTAGES")) ha.a_stages = atoi(getenv("DC_HALO_ASTAGES"));
     const int a_total = ha.a_stages * mt * h.patch_bytes;
-    int st = (200 * 1024 - a_total) / h.b_bytes;
+    int st = (budget - a_total) / h.b_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
     const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + sizeof(SmemCtl) + 256;
@@ -887,7 +905,7 @@ static int launch_halo(dc_cache* c, int layer, int mt, const void* in, void* out
         attr_set = true;
     }
     long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + mt - 1) / mt) * h.NB;
-    int grid = items > c->num_sms ? c->num_sms : (int)items;
+    int grid = items > c->num_sms * ctas ? c->num_sms * ctas : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
     if (mt == 2) k_conv_tc_halo<2><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
     else k_conv_tc_halo<1><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
@@ -903,7 +921,9 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     const dc_layer_desc& d = L.d;
     if (L.tc_mt >= 3) return launch_halo(c, layer, L.tc_mt - 2, in, out, tile_list, tile_count, masks, max_tiles);
     TcPlan p;
-    if (!make_plan(d, p, L.tc_mt, L.tc_bn)) {
+    int ctas = L.tc_ctas == 2 ? 2 : 1;
+    if (ctas == 2 && !make_plan(d, p, L.tc_mt, L.tc_bn, 2)) ctas = 1;
+    if (!make_plan(d, p, L.tc_mt, L.tc_bn, ctas)) {
         if (smallc_ok(d)) return launch_smallc(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
         return DC_ERR_CONFIG;
     }
@@ -937,6 +957,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
     a.BN = p.BN; a.NB = p.NB; a.BK = p.BK; a.kchunks = d.cin / p.BK; a.stages = p.stages; a.MT = p.MT; a.nbuf = p.nbuf;
     a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.sbo = p.sbo; a.layout_type = p.layout_type;
+    a.tmem_cols = tmem_cols_for(p.nbuf, p.MT, p.BN);
     // instruction descriptor: D = f32, A = B = bf16, both K-major, N = BN, M = 128
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
@@ -947,7 +968,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
         attr_set = true;
     }
     long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + p.MT - 1) / p.MT) * p.NB;
-    int grid = items > c->num_sms ? c->num_sms : (int)items;
+    int grid = items > c->num_sms * ctas ? c->num_sms * ctas : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
     if (p.MT == 2) k_conv_tc<2><<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
     else k_conv_tc<1><<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
@@ -964,53 +985,63 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
 {
     dc_layer_rt& L = c->L[layer];
     TcPlan p;
-    if (c->cfg.dtype != DC_BF16 || !encode_fn() || !make_plan(L.d, p) || getenv("DC_NO_TENSOR_CORES")) return DC_OK;
+    if (c->cfg.dtype != DC_BF16 || !encode_fn() || getenv("DC_NO_TENSOR_CORES")) return DC_OK;
+    const bool generic = make_plan(L.d, p);
+    if (!generic && !smallc_ok(L.d)) return DC_OK;
     if (getenv("DC_CONV_NO_TUNE")) return DC_OK;
     const int tiles = L.tiles_x * L.tiles_y * c->S;
     cudaEvent_t e0, e1;
     DC_CUDA(cudaEventCreate(&e0));
     DC_CUDA(cudaEventCreate(&e1));
-    float best = 1e30f; int best_mt = 1, best_bn = p.BN;
-    const int default_bn = p.BN;
-    for (int bn = default_bn; bn >= 64 && bn >= default_bn / 2; bn -= 32) {
-        if (L.d.cout % bn != 0) continue;
-        for (int mt = 1; mt <= 2; ++mt) {
-            TcPlan q;
-            if (!make_plan(L.d, q, mt, bn)) continue;
-            L.tc_mt = mt; L.tc_bn = bn;
-            int rc = DC_OK;
-            for (int rep = 0; rep < 3 && rc == DC_OK; ++rep) {
-                if (rep == 1) cudaEventRecord(e0, c->stream);
-                rc = dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles);
+    float best = 1e30f; int best_mt = L.tc_mt, best_bn = L.tc_bn, best_ctas = 1;
+    const bool verbose = getenv("DC_VERBOSE") != nullptr;
+    // times the launch the current L.tc_* fields select; keeps it when it is the fastest so far
+    auto trial = [&](const char* what) {
+        int rc = DC_OK;
+        for (int rep = 0; rep < 3 && rc == DC_OK; ++rep) {
+            if (rep == 1) cudaEventRecord(e0, c->stream);
+            rc = dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles);
+        }
+        cudaEventRecord(e1, c->stream);
+        if (rc != DC_OK || cudaEventSynchronize(e1) != cudaSuccess) { cudaGetLastError(); return; }
+        float ms = 0.f;
+        cudaEventElapsedTime(&ms, e0, e1);
+        if (verbose) fprintf(stderr, "libdeepcache: layer %d: %s, tiles/item code %d, %d channels per block, %d CTA(s) per SM: %.3f ms\n",
+                             layer, what, L.tc_mt, L.tc_bn, L.tc_ctas, ms / 2);
+        if (ms < best) { best = ms; best_mt = L.tc_mt; best_bn = L.tc_bn; best_ctas = L.tc_ctas; }
+    };
+    const int no_two = getenv("DC_CONV_ONE_CTA") != nullptr;
+    for (int ctas = 1; ctas <= (no_two ? 1 : 2); ++ctas) {
+        L.tc_ctas = ctas;
+        if (!generic) {                                               // few input channels: one kernel shape, 1 or 2 CTAs per SM
+            if (ctas == 2 && tmem_cols_for(2, 1, L.d.cout) > 256) continue;
+            trial("few-channel kernel");
+            continue;
+        }
+        const int default_bn = p.BN;
+        for (int bn = default_bn; bn >= 64 && bn >= default_bn / 2; bn -= 32) {
+            if (L.d.cout % bn != 0) continue;
+            for (int mt = 1; mt <= 2; ++mt) {
+                TcPlan q;
+                if (!make_plan(L.d, q, mt, bn, ctas)) continue;
+                L.tc_mt = mt; L.tc_bn = bn;
+                trial("tap-by-tap kernel");
             }
-            cudaEventRecord(e1, c->stream);
-            if (rc != DC_OK || cudaEventSynchronize(e1) != cudaSuccess) { cudaGetLastError(); continue; }
-            float ms = 0.f;
-            cudaEventElapsedTime(&ms, e0, e1);
-            if (ms < best) { best = ms; best_mt = mt; best_bn = bn; }
+        }
+        HaloPlan h;
+        if (L.weight_halo && halo_ok(L.d, h)) {
+            for (int mt = 1; mt <= 2; ++mt) {                          // tc_mt 3 / 4: patch-reuse kernel with 1 / 2 tiles per item
+                if (ctas == 2 && tmem_cols_for(mt * h.BN * 2 <= 512 ? 2 : 1, mt, h.BN) > 256) continue;
+                L.tc_mt = mt + 2; L.tc_bn = 0;
+                trial("patch-reuse kernel");
+            }
         }
     }
-    HaloPlan h;
-    if (L.weight_halo && halo_ok(L.d, h)) {
-        for (int mt = 1; mt <= 2; ++mt) {                          // tc_mt 3 / 4: patch-reuse kernel with 1 / 2 tiles per item
-            L.tc_mt = mt + 2; L.tc_bn = 0;
-            int rc = DC_OK;
-            for (int rep = 0; rep < 3 && rc == DC_OK; ++rep) {
-                if (rep == 1) cudaEventRecord(e0, c->stream);
-                rc = dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles);
-            }
-            cudaEventRecord(e1, c->stream);
-            if (rc != DC_OK || cudaEventSynchronize(e1) != cudaSuccess) { cudaGetLastError(); continue; }
-            float ms = 0.f;
-            cudaEventElapsedTime(&ms, e0, e1);
-            if (getenv("DC_VERBOSE")) fprintf(stderr, "libdeepcache: layer %d: patch-reuse kernel, %d tile(s) per item: %.3f ms\n", layer, mt, ms / 2);
-            if (ms < best) { best = ms; best_mt = mt + 2; best_bn = 0; }
-        }
-    }
-    if (getenv("DC_CONV_FORCE_HALO") && L.weight_halo) { best_mt = atoi(getenv("DC_CONV_FORCE_HALO")) + 2; best_bn = 0; }
-    L.tc_mt = best_mt; L.tc_bn = best_bn;
+    if (getenv("DC_CONV_FORCE_HALO") && L.weight_halo) { best_mt = atoi(getenv("DC_CONV_FORCE_HALO")) + 2; best_bn = 0; best_ctas = 1; }
+    L.tc_mt = best_mt; L.tc_bn = best_bn; L.tc_ctas = best_ctas;
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     c->launches = 0;
-    if (getenv("DC_VERBOSE")) fprintf(stderr, "libdeepcache: layer %d: %d tile(s) per item, %d channels per block (%.3f ms)\n", layer, best_mt, best_bn, best / 2);
+    if (verbose) fprintf(stderr, "libdeepcache: layer %d: chose code %d, %d channels per block, %d CTA(s) per SM (%.3f ms)\n",
+                         layer, best_mt, best_bn, best_ctas, best / 2);
     return DC_OK;
 }
