@@ -168,21 +168,20 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
     bool ok = true;
     // the tile index and this pixel's bitmap word of the NEXT item are fetched while the current one is
     // processed: two dependent global loads would otherwise sit on every item's critical path
-    int tile_n[2] = {-1, -1}; uint32_t mask_n[2] = {0, 0};
+    int tile_n0 = -1, tile_n1 = -1; uint32_t mask_n0 = 0, mask_n1 = 0;       // scalars: indexed arrays would live in local memory
     auto fetch = [&](int item) {
         if (item >= n_items) return;
-        const int group = item / a.NB;
-        for (int j = 0; j < a.MT; ++j) {
-            const int idx = group * a.MT + j;
-            tile_n[j] = idx < n_tiles ? a.tile_list[idx] : -1;   // odd tile count: the last item has one tile
-            mask_n[j] = tile_n[j] >= 0 ? a.masks[(size_t)tile_n[j] * 4 + mword_i] : 0u;
-        }
+        const int idx = (item / a.NB) * a.MT;
+        tile_n0 = a.tile_list[idx];
+        mask_n0 = a.masks[(size_t)tile_n0 * 4 + mword_i];
+        tile_n1 = (a.MT > 1 && idx + 1 < n_tiles) ? a.tile_list[idx + 1] : -1;     // odd tile count: the last item has one tile
+        mask_n1 = tile_n1 >= 0 ? a.masks[(size_t)tile_n1 * 4 + mword_i] : 0u;
     };
     fetch(blockIdx.x);
     for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
         const int nb = item % a.NB;
-        const int tile_c[2] = {tile_n[0], tile_n[1]};
-        const uint32_t mask_c[2] = {mask_n[0], mask_n[1]};
+        const int tile_c0 = tile_n0, tile_c1 = tile_n1;
+        const uint32_t mask_c0 = mask_n0, mask_c1 = mask_n1;
         fetch(item + gridDim.x);
         ok = mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, a.status);
         ok = __all_sync(0xffffffffu, ok);
@@ -190,11 +189,11 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
         tc_fence_after();
         const float* bias = a.bias + nb * a.BN;
         for (int j = 0; j < a.MT; ++j) {
-            const int tile = tile_c[j];
+            const int tile = j == 0 ? tile_c0 : tile_c1;
             if (tile < 0) break;
             const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
             const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
-            const bool reused = (mask_c[j] >> mbit) & 1u;
+            const bool reused = ((j == 0 ? mask_c0 : mask_c1) >> mbit) & 1u;
             const bool active = oy < a.Ho && ox < a.Wo && !reused;
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (acc * (uint32_t)a.MT + (uint32_t)j) * (uint32_t)a.BN;
             // Each lane owns one pixel (TMEM lane) and gets 32 channels = 64 bytes per step.  Storing them
@@ -203,6 +202,12 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
             // 4 lanes per pixel, so each pixel's 64 bytes leave as two whole sectors.
             const unsigned act_mask = __ballot_sync(0xffffffffu, active);
             uint8_t* stg = ctl->stage[q];
+            // write-back addressing, once per tile: piece k of this lane is the 16-byte part (lane & 3) of the pixel in
+            // tile row q * 4 + k, column lane >> 2 (the warp's 32 pixels are 4 tile rows of 8)
+            const size_t row_stride = (size_t)a.Wo * a.Co;
+            __nv_bfloat16* const wb = a.out + ((size_t)s * a.Ho + ty * DC_TILE_H + q * 4) * row_stride +
+                                      (size_t)(tx * DC_TILE_W + (lane >> 2)) * a.Co + nb * a.BN + (lane & 3) * 8;
+            const uint8_t* const rd = stg + (lane >> 2) * 80 + (lane & 3) * 16;
             for (int c = 0; c < a.BN / 32; ++c) {
                 uint32_t r[32];
                 tmem_ld32(taddr + c * 32, r);
@@ -225,12 +230,8 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
                 __syncwarp();
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
-                    const int piece = lane + 32 * k, pl = piece >> 2, part = piece & 3;    // pixel (lane) pl of this warp, 16-byte part
-                    if ((act_mask >> pl) & 1u) {
-                        const int mm = q * 32 + pl, pr = mm / DC_TILE_W, pc = mm % DC_TILE_W;
-                        __nv_bfloat16* o2 = a.out + (((size_t)s * a.Ho + ty * DC_TILE_H + pr) * a.Wo + tx * DC_TILE_W + pc) * a.Co + nb * a.BN + c * 32;
-                        ((uint4*)o2)[part] = *(const uint4*)(stg + pl * 80 + part * 16);
-                    }
+                    if ((act_mask >> ((lane >> 2) + 8 * k)) & 1u)
+                        *(uint4*)(wb + k * row_stride + c * 32) = *(const uint4*)(rd + k * (8 * 80));
                 }
                 __syncwarp();
             }
