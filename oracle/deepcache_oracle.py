@@ -283,6 +283,22 @@ def maxpool(x, layer):
     return out
 
 
+def pool_reuse(x, layer, prev_out=None, regions=None):
+    """Section 5 notes that the cache extends to other layer types; this is that extension for max pooling,
+    with the three steps of "Reuse": copy the layer's reusable rectangles from the cached pooled map, mark
+    them, pool the input only where nothing was copied.  Returns (out, reused byte map)."""
+    out = maxpool(x, layer)
+    reused = np.zeros(out.shape[:2], np.uint8)
+    if prev_out is not None and regions is not None:
+        for r in regions:
+            if r["w"] <= 0 or r["h"] <= 0:
+                continue
+            y, x0, h, w, sy, sx = (int(r[k]) for k in ("y", "x", "h", "w", "sy", "sx"))
+            out[y:y + h, x0:x0 + w] = prev_out[sy:sy + h, sx:sx + w]
+            reused[y:y + h, x0:x0 + w] = 1
+    return out, reused
+
+
 def add(a, b, relu, mode):
     a = np.ascontiguousarray(a, np.float64)
     b = np.ascontiguousarray(b, np.float64)
@@ -304,12 +320,12 @@ class OracleCache:
 
     def __init__(self, width, height, layers, weights, biases, *, block=10, search_range=8,
                  search_kind=SEARCH_DS, psnr_db=20.0, expire_n=10, quant=QUANT_NONE, use_cache=True, skip_k=1,
-                 region_mode=0):
+                 region_mode=0, cache_pool=False):
         self.W, self.H = width, height
         self.layers = layers
         self.block, self.R, self.kind = block, search_range, search_kind
         self.T, self.N, self.quant, self.use_cache = psnr_db, expire_n, quant, use_cache
-        self.skip_k, self.region_mode = skip_k, region_mode
+        self.skip_k, self.region_mode, self.cache_pool = skip_k, region_mode, cache_pool
         # weights are stored at the storage precision (bf16 workloads round them once)
         self.weights = [None if w is None else quant_array(w, quant) for w in weights]
         self.biases = [None if b is None else np.asarray(b, np.float64) for b in biases]
@@ -349,7 +365,11 @@ class OracleCache:
                 out, reused = conv_reuse(x, l, self.weights[i], self.biases[i], self.quant, prev, regs)
                 info["reused"][i] = reused
             elif k == KIND_MAXPOOL:
-                out = maxpool(x, l)
+                if self.cache_pool and not refresh:
+                    out, reused = pool_reuse(x, l, self.prev_maps[i], per_layer_regions[i])
+                    info["reused"][i] = reused
+                else:
+                    out = maxpool(x, l)
             elif k == KIND_ADD:
                 out = add(x, maps[l["in1"]], l["relu"], self.quant)
             elif k == KIND_RESIZE_AREA:
@@ -362,7 +382,8 @@ class OracleCache:
             maps.append(out)
         # the frame becomes the next key, the conv outputs the next values (Section 3)
         self.prev_frame = frame.copy()
-        self.prev_maps = [m if layers[i]["kind"] == KIND_CONV else None for i, m in enumerate(maps)]
+        kept = (KIND_CONV, KIND_MAXPOOL) if self.cache_pool else (KIND_CONV,)
+        self.prev_maps = [m if layers[i]["kind"] in kept else None for i, m in enumerate(maps)]
         self.frame_idx += 1
         info["maps"] = maps
         info["out"] = maps[-1]

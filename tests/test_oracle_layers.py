@@ -213,3 +213,59 @@ def test_per_block_mode_reuses_two_motions_end_to_end():
     assert np.array_equal(b["out"][~mask], fresh[~mask])
     # exact copies of content: reused values equal fresh ones here (no noise was added)
     assert np.abs(b["out"] - fresh).max() < 1e-12
+
+
+# ---------------------------------------------------------------------------
+# reuse in pooling layers (Section 5: the cache mechanism extends to other layer types)
+# ---------------------------------------------------------------------------
+def pool_layer(hi, wi, c, k=2, s=2, p=0):
+    return dict(kind=orc.KIND_MAXPOOL, kh=k, kw=k, sh=s, sw=s, ph=p, pw=p, cin=c, cout=c, relu=0, in0=-1, in1=-1,
+                out_h=(hi + 2 * p - k) // s + 1, out_w=(wi + 2 * p - k) // s + 1)
+
+
+def test_pool_reuse_copies_rectangles_and_pools_the_rest():
+    g = rng(21)
+    L = pool_layer(24, 20, 3)
+    x = g.normal(size=(24, 20, 3))
+    prev = g.normal(size=(12, 10, 3))
+    regions = np.zeros(3, orc.REGION_DTYPE)
+    regions[0] = (1, 2, 4, 3, 3, 0)
+    regions[2] = (6, 7, 4, 5, 5, 6)
+    out, reused = orc.pool_reuse(x, L, prev, regions)
+    full = orc.maxpool(x, L)
+    mask = np.zeros((12, 10), bool)
+    for r in regions:
+        mask[r["y"]:r["y"] + r["h"], r["x"]:r["x"] + r["w"]] = True
+    assert np.array_equal(reused.astype(bool), mask)
+    assert np.array_equal(out[~mask], full[~mask])
+    assert np.array_equal(out[2:5, 1:5], prev[0:3, 3:7]) and np.array_equal(out[7:12, 6:10], prev[6:11, 5:9])
+    a, b = orc.pool_reuse(x, L)                              # nothing cached: plain pooling
+    assert np.array_equal(a, full) and not b.any()
+
+
+def test_pool_reuse_is_exact_when_the_motion_is_a_multiple_of_the_stride():
+    # content moved by (4, -4): multiples of the cumulative stride at both 2x2 pooling layers, so a cached pooled pixel
+    # is the maximum over exactly the same conv outputs, and caching the pooling layers changes nothing in the result
+    g = rng(22)
+    w = configs.WORKLOADS[2]()
+    w.layers = nets.small_cnn(96, 96)
+    w.width = w.height = 96
+    f0 = g.integers(0, 256, size=(96, 96, 3), dtype=np.uint8)
+    f1 = np.roll(f0, (4, -4), axis=(0, 1))                   # f1[y][x] = f0[y - 4][x + 4]
+    es = dict(search_kind=orc.SEARCH_ES, search_range=5)     # noise frames: a walk would stall, score every vector
+    with_pool, without = make_cache(w, cache_pool=True, **es), make_cache(w, **es)
+    with_pool.infer_frame(f0); without.infer_frame(f0)
+    a, b = with_pool.infer_frame(f1), without.infer_frame(f1)
+    assert a["match"]["M"] == (4, -4)
+    pools = [i for i, l in enumerate(w.layers) if l["kind"] == orc.KIND_MAXPOOL]
+    assert pools and all(a["reused"][i] is not None and a["reused"][i].mean() > 0.3 for i in pools)
+    for ma, mb in zip(a["maps"], b["maps"]):
+        assert np.array_equal(ma, mb)
+    # an odd motion pairs a pooled pixel with a window shifted by one conv pixel: an approximation, like every
+    # reuse across a stride (the paper's reuse in strided convolutions has the same property)
+    f2 = np.roll(f0, (0, -3), axis=(0, 1))
+    c1, c2 = make_cache(w, cache_pool=True, **es), make_cache(w, **es)
+    c1.infer_frame(f0); c2.infer_frame(f0)
+    p, q = c1.infer_frame(f2), c2.infer_frame(f2)
+    assert p["match"]["M"] == (3, 0) and p["reused"][pools[0]].any()
+    assert not np.array_equal(p["maps"][pools[0]], q["maps"][pools[0]])
