@@ -45,6 +45,8 @@ def parse_args():
     ap.add_argument("--skip-k", type=int, default=1, help="Step 2 on every k-th block row / column only (Section 4); default 1 = all blocks")
     ap.add_argument("--search", default="", choices=["", "exhaustive", "diamond", "three_step"],
                     help="Step 2 search unit; default: the workload's (diamond)")
+    ap.add_argument("--cache-pool", action="store_true", help="also cache and reuse max-pooling outputs (Section 5's extension)")
+    ap.add_argument("--per-block-regions", action="store_true", help="rectangles carry their blocks' own vectors (extension)")
     ap.add_argument("--no-lookahead", action="store_true", help="do not overlap the next frame's matching with this frame's inference")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -214,7 +216,8 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
     dev_frames = host.to(dev, non_blocking=True)
     torch.cuda.synchronize()
 
-    dc = DeepCache.from_workload(w, n_streams=S, device=f"cuda:{local}", skip_k=args.skip_k)
+    dc = DeepCache.from_workload(w, n_streams=S, device=f"cuda:{local}", skip_k=args.skip_k,
+                                 cache_pool=args.cache_pool, region_mode=1 if args.per_block_regions else 0)
     pitch = w.width * 3
     last = w.layers[-1]
     out_bytes = S * last["out_h"] * last["out_w"] * last["cout"] * (2 if w.dtype == 1 else 4)

@@ -101,6 +101,10 @@ typedef struct {
     int32_t dtype;                     /* dc_dtype of maps and arithmetic inputs */
     int32_t max_regions;               /* rectangles per stream; 0 = worst case of the grid */
     int32_t region_mode;               /* dc_region_mode; 0 = the paper's global vector */
+    int32_t cache_pool;                /* 1: max-pooling layers keep their last output and reuse it like convolutions
+                                          (the extension Section 5 mentions; costs a second pooled map per layer).
+                                          Applies to pooling layers whose pixel is a multiple of 16 bytes.  0 = the
+                                          paper's choice: only convolutions are cached */
 } dc_config;
 
 /* Per-stream outcome of one dc_infer_frame. */

@@ -27,6 +27,13 @@ void dc_use_match_set(dc_cache* c, int k)
     c->long_list = m.long_list; c->gmv = m.gmv; c->regions0 = m.regions0; c->n_regions = m.n_regions;
 }
 
+bool dc_layer_cached(const dc_cache* c, int layer)
+{
+    const dc_layer_desc& d = c->L[layer].d;
+    if (d.kind == DC_CONV) return true;
+    return d.kind == DC_MAXPOOL && c->cfg.cache_pool && ((size_t)d.cout * c->elt) % 16 == 0;
+}
+
 namespace {
 
 // nearest bfloat16 (ties to even) of a double, as its 16 bit pattern
@@ -59,6 +66,7 @@ int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
     if (cfg->channels != 3 || cfg->width < 1 || cfg->height < 1 || cfg->n_streams < 1) return DC_ERR_CONFIG;
     if (cfg->block < 4 || cfg->block > 32 || cfg->range < 0 || cfg->range > 64) return DC_ERR_CONFIG;
     if (cfg->search < DC_SEARCH_EXHAUSTIVE || cfg->search > DC_SEARCH_THREE_STEP) return DC_ERR_CONFIG;
+    if (cfg->cache_pool != 0 && cfg->cache_pool != 1) return DC_ERR_CONFIG;
     if (cfg->region_mode != DC_REGIONS_GLOBAL && cfg->region_mode != DC_REGIONS_PER_BLOCK) return DC_ERR_CONFIG;
     if (cfg->skip_k < 1 || cfg->skip_k > 16 || cfg->expire_n < 1 || cfg->max_regions < 0) return DC_ERR_CONFIG;
     if (cfg->dtype != DC_FP32 && cfg->dtype != DC_BF16) return DC_ERR_CONFIG;
@@ -188,12 +196,13 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
         if (L.d.in0 < 0 && L.d.kind != DC_RESIZE_AREA) need_input_map = true;
         if (L.d.kind == DC_ADD && L.d.in1 < 0) need_input_map = true;
         L.map_bytes = (size_t)S * L.d.out_h * L.d.out_w * L.d.cout * c->elt;
-        const int copies = L.d.kind == DC_CONV ? 2 : 1;
+        const bool cached = dc_layer_cached(c, i);
+        const int copies = cached ? 2 : 1;
         for (int k = 0; k < copies; ++k) {
             DC_TRY(dev_alloc(c, (uint8_t**)&L.map[k], L.map_bytes));
             DC_CUDA(cudaMemsetAsync(L.map[k], 0, L.map_bytes, c->stream));
         }
-        if (L.d.kind == DC_CONV) {
+        if (cached) {
             L.tiles_x = dc_div_up(L.d.out_w, DC_TILE_W);
             L.tiles_y = dc_div_up(L.d.out_h, DC_TILE_H);
             size_t tiles = (size_t)L.tiles_x * L.tiles_y * S;
@@ -208,6 +217,8 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
             cudaError_t e = cudaMemcpy(L.all_list, iota, sizeof(int32_t) * tiles, cudaMemcpyHostToDevice);
             free(iota);
             DC_CUDA(e);
+        }
+        if (L.d.kind == DC_CONV) {
             if (!weights_dev || !bias_dev || !weights_dev[i] || !bias_dev[i]) return DC_ERR_ARG;
             DC_TRY(dc_pack_weights(c, i, (const float*)weights_dev[i], (const float*)bias_dev[i]));
         }
@@ -260,7 +271,7 @@ const void* layer_input(dc_cache* c, int idx)
 {
     if (idx < 0) return c->input_map;
     dc_layer_rt& P = c->L[idx];
-    return P.map[P.d.kind == DC_CONV ? P.cur : 0];
+    return P.map[dc_layer_cached(c, idx) ? P.cur : 0];
 }
 
 // Drops a pending lookahead: the main stream first waits for it, so nothing it wrote is still in flight.
@@ -294,7 +305,7 @@ int fill_stats(dc_cache* c, bool refreshed, dc_frame_stats* stats)
         st.mvx = h_gmv[3 * s]; st.mvy = h_gmv[3 * s + 1]; st.k_passed = h_gmv[3 * s + 2];
         st.n_matched = h_acc[4 * s + 3]; st.n_regions = h_nreg[s];
         for (int l = 0; l < n; ++l)
-            if (c->L[l].d.kind == DC_CONV)
+            if (dc_layer_cached(c, l))
                 st.reuse_ratio[l] = (float)h_reuse[(size_t)l * S + s] / (float)(c->L[l].d.out_h * c->L[l].d.out_w);
     }
     return DC_OK;
@@ -472,7 +483,18 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
             L.cur ^= 1;          // the newest output is next frame's cached value
             break;
         }
-        case DC_MAXPOOL: DC_TRY(dc_launch_maxpool(c, i, in)); break;
+        case DC_MAXPOOL: {
+            if (!dc_layer_cached(c, i)) { DC_TRY(dc_launch_maxpool(c, i, in, L.map[0], nullptr)); break; }
+            void* prev = L.map[L.cur]; void* out = L.map[L.cur ^ 1];
+            if (!refresh) {           // Section 5's three steps on a pooling layer: copy, mark, compute the rest
+                DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
+                DC_TRY(dc_launch_maxpool(c, i, in, out, L.masks));
+            } else {
+                DC_TRY(dc_launch_maxpool(c, i, in, out, nullptr));
+            }
+            L.cur ^= 1;
+            break;
+        }
         case DC_ADD: DC_TRY(dc_launch_add(c, i, in, layer_input(c, L.d.in1))); break;
         case DC_RELU: DC_TRY(dc_launch_relu(c, i, in)); break;
         case DC_RESIZE_AREA: DC_TRY(dc_launch_resize(c, i, frame_copy, c->key_pitch)); break;

@@ -103,8 +103,10 @@ template <> struct Vec16<__nv_bfloat16> {
     static __device__ __forceinline__ uint4 vmax(uint4 a, uint4 b) { return make_uint4(m2(a.x, b.x), m2(a.y, b.y), m2(a.z, b.z), m2(a.w, b.w)); }
 };
 
+// masks (optional): the layer's per-tile reuse bitmaps; a pixel whose bit is set was filled from the cache
 template <typename T>
-__global__ void k_maxpool_vec(const T* in, int Hi, int Wi, int C, int S, dc_layer_desc L, T* out)
+__global__ void k_maxpool_vec(const T* in, int Hi, int Wi, int C, int S, dc_layer_desc L, T* out, const uint32_t* masks,
+                              int tiles_x, int tiles_y)
 {
     constexpr int N = Vec16<T>::N;
     const int cv = C / N;
@@ -113,6 +115,11 @@ __global__ void k_maxpool_vec(const T* in, int Hi, int Wi, int C, int S, dc_laye
         int c = (int)(i % cv); size_t t = i / cv;
         int ox = (int)(t % L.out_w); t /= L.out_w;
         int oy = (int)(t % L.out_h); int s = (int)(t / L.out_h);
+        if (masks) {
+            const size_t tile = ((size_t)s * tiles_y + oy / DC_TILE_H) * tiles_x + ox / DC_TILE_W;
+            const int bit = DC_TILE_BIT(oy % DC_TILE_H, ox % DC_TILE_W);
+            if ((masks[tile * 4 + (bit >> 5)] >> (bit & 31)) & 1u) continue;
+        }
         uint4 m = make_uint4(0, 0, 0, 0);
         bool first = true;
         for (int ky = 0; ky < L.kh; ++ky) {
@@ -203,7 +210,7 @@ int dc_launch_resize(dc_cache* c, int layer, const uint8_t* frame, size_t pitch)
     return DC_OK;
 }
 
-int dc_launch_maxpool(dc_cache* c, int layer, const void* in)
+int dc_launch_maxpool(dc_cache* c, int layer, const void* in, void* out, const uint32_t* masks)
 {
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
@@ -211,15 +218,16 @@ int dc_launch_maxpool(dc_cache* c, int layer, const void* in)
     if ((L.d.cout * c->elt) % 16 == 0) {
         size_t nv = n * c->elt / 16;
         DISPATCH(c,
-            (k_maxpool_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)L.map[0])),
-            (k_maxpool_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)L.map[0])));
+            (k_maxpool_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)out, masks, L.tiles_x, L.tiles_y)),
+            (k_maxpool_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)out, masks, L.tiles_x, L.tiles_y)));
         c->launches += 1;
         DC_CUDA(cudaGetLastError());
         return DC_OK;
     }
+    if (masks) return DC_ERR_STATE;                             // cached pooling needs 16-byte pixels (checked at creation)
     DISPATCH(c,
-        (k_maxpool<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)L.map[0])),
-        (k_maxpool<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)L.map[0])));
+        (k_maxpool<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)out)),
+        (k_maxpool<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)out)));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;

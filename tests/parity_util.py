@@ -64,7 +64,7 @@ def run_stream_parity(w, n_streams, frame_ids, check_layers=True, **kw):
     bit-exact matcher outputs, rectangles at every layer and reuse ratios, maps within tolerance."""
     bf16 = w.dtype == configs.DTYPE_BF16
     sb = w.streams(n_streams, max(frame_ids) + 1)
-    dc = DeepCache.from_workload(w, n_streams=n_streams, **{k: v for k, v in kw.items() if k in ("expire_n", "skip_k", "region_mode")})
+    dc = DeepCache.from_workload(w, n_streams=n_streams, **{k: v for k, v in kw.items() if k in ("expire_n", "skip_k", "region_mode", "cache_pool")})
     oracles = make_oracles(w, n_streams, **kw)
     worst = 0.0
     try:
@@ -86,7 +86,7 @@ def run_stream_parity(w, n_streams, frame_ids, check_layers=True, **kw):
                     for li, l in enumerate(w.layers):
                         regs, _ = dc.layer_regions(li)
                         assert_regions_equal(regions_np(regs[s, :n]), o["regions"][li], what + f" layer {li}")
-                        if l["kind"] == orc.KIND_CONV:
+                        if l["kind"] == orc.KIND_CONV or (kw.get("cache_pool") and l["kind"] == orc.KIND_MAXPOOL):
                             want_ratio = float(o["reused"][li].mean())
                             assert abs(stats[s].reuse_ratio[li] - want_ratio) < 1e-6, what + f" layer {li} reuse"
                 if check_layers:

@@ -177,6 +177,27 @@ def test_infer_per_block_regions(widx):
     U.run_stream_parity(configs.WORKLOADS[widx](), 1, list(range(4)), region_mode=B.DC_REGIONS_PER_BLOCK)
 
 
+@pytest.mark.parametrize("widx,frames", [(2, 6), (3, 5), (5, 3)])
+def test_infer_with_cached_pooling(widx, frames):
+    """Reuse in max-pooling layers (the extension Section 5 mentions): maps, rectangles and per-layer reuse ratios
+    of the pooling layers against the oracle with the same switch."""
+    w = configs.WORKLOADS[widx]()
+    U.run_stream_parity(w, 2 if widx == 5 else 1, list(range(frames)), cache_pool=True)
+
+
+def test_cached_pooling_reuses_pixels():
+    w = configs.WORKLOADS[2]()
+    sb = w.streams(1, 3)
+    dc = DeepCache.from_workload(w, cache_pool=True)
+    try:
+        for i in range(3):
+            out, stats = dc.infer_frame(sb.frame(i), want_stats=True)
+        pools = [i for i, l in enumerate(w.layers) if l["kind"] == orc.KIND_MAXPOOL]
+        assert pools and all(stats[0].reuse_ratio[i] > 0.2 for i in pools)
+    finally:
+        dc.close()
+
+
 @pytest.mark.parametrize("k", [2, 3])
 def test_match_k_skip(k):
     """Section 4's k-skip: Step 2 on every k-th block row and column only (16-px fast path and generic path)."""
