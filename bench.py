@@ -386,7 +386,8 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
-            "config": dict(workload_config(w, S, world), skip_k=args.skip_k), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
+            "config": dict(workload_config(w, S, world), skip_k=args.skip_k, cache_pool=bool(args.cache_pool),
+                           regions="per_block" if args.per_block_regions else "global"), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "roofline_matcher": roofline_matcher, "cpu_baseline": cpu_baseline,
             "stage_ms": stage_ms, "stage_share": stage_share, "frames_cached": n_cached, "frames_full": n_full,
             "reuse_ratio_cached_frames": reuse, "cache_bytes": cache_bytes, "no_cache": no_cache,

@@ -230,6 +230,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     if (need_input_map)
         DC_TRY(dev_alloc(c, (uint8_t**)&c->input_map, (size_t)S * cfg.height * cfg.width * 3 * c->elt));
     size_t stat_ints = (size_t)S * (3 + 4 + 1) + (size_t)n * S;
+    if (c->executable) DC_TRY(dc_build_classify_table(c));
     if (cudaMallocHost(&c->stats_pinned, stat_ints * sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
     DC_CUDA(cudaStreamSynchronize(c->stream));      // layers / in_hw / all_count live on this stack frame
     for (int i = 0; i < n; ++i)
@@ -254,7 +255,7 @@ void release(dc_cache* c)
         cudaFree(m.blk_mv); cudaFree(m.blk_sse); cudaFree(m.matched); cudaFree(m.run_end); cudaFree(m.mv_acc);
         cudaFree(m.long_list); cudaFree(m.gmv); cudaFree(m.regions0); cudaFree(m.n_regions);
     }
-    cudaFree(c->table);
+    cudaFree(c->table); cudaFree(c->classify_table);
     cudaFree(c->layers_dev); cudaFree(c->in_hw_dev); cudaFree(c->dirty_count); cudaFree(c->all_count);
     cudaFree(c->reuse_px); cudaFree(c->zero_masks); cudaFree(c->status); cudaFree(c->input_map); cudaFree(c->pix_lut);
     if (c->stats_pinned) cudaFreeHost(c->stats_pinned);
@@ -467,6 +468,15 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
     }
     if (c->input_map) DC_TRY(dc_launch_input_map(c, frame_copy, c->key_pitch));
     const size_t per_layer = (size_t)S * c->max_regions;
+    // bitmaps, reuse copies and dirty lists of every cached layer in one launch (they need only the rectangles and
+    // each layer's own cached map); possible while all cached layers keep their newest map at the same index
+    bool classified = false;
+    if (!refresh && c->n_cached > 0) {
+        int cur = -1; bool same = true;
+        for (int i = 0; i < n; ++i)
+            if (dc_layer_cached(c, i)) { if (cur < 0) cur = c->L[i].cur; else if (c->L[i].cur != cur) same = false; }
+        if (same) { DC_TRY(dc_launch_classify_all(c, cur)); classified = true; }
+    }
     for (int i = 0; i < n; ++i) {
         dc_layer_rt& L = c->L[i];
         const void* in = layer_input(c, L.d.in0);
@@ -475,7 +485,7 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
             const int tiles = L.tiles_x * L.tiles_y * S;
             void* prev = L.map[L.cur]; void* out = L.map[L.cur ^ 1];
             if (!refresh) {
-                DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
+                if (!classified) DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
                 DC_TRY(dc_launch_conv(c, i, in, out, L.dirty_list, c->dirty_count + i, L.masks, tiles));
             } else {
                 DC_TRY(dc_launch_conv(c, i, in, out, L.all_list, c->all_count + i, c->zero_masks, tiles));
@@ -487,7 +497,7 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
             if (!dc_layer_cached(c, i)) { DC_TRY(dc_launch_maxpool(c, i, in, L.map[0], nullptr)); break; }
             void* prev = L.map[L.cur]; void* out = L.map[L.cur ^ 1];
             if (!refresh) {           // Section 5's three steps on a pooling layer: copy, mark, compute the rest
-                DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
+                if (!classified) DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
                 DC_TRY(dc_launch_maxpool(c, i, in, out, L.masks));
             } else {
                 DC_TRY(dc_launch_maxpool(c, i, in, out, nullptr));

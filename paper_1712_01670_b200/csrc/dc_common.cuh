@@ -76,6 +76,7 @@ struct dc_cache {
     cudaEvent_t ev_key, ev_match;   // main stream: frame copied in; side stream: lookahead finished
     const uint8_t* la_frame; size_t la_pitch; bool la_matched;
     bool last_refreshed;
+    void* classify_table; int n_cached, classify_warps;   // all cached layers' classification in one launch (dc_regions.cu)
     size_t key_pitch;
     int num_sms;
     uint8_t* staging[2];            // device copies of host frames for dc_infer_frame_host (one in use, one prefetching)
@@ -136,4 +137,6 @@ int dc_launch_relu(dc_cache* c, int layer, const void* a);
 int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_dev);
 // true for layers that keep their last output as cached values: convolutions, and max pooling when cfg.cache_pool
 bool dc_layer_cached(const dc_cache* c, int layer);
+int dc_build_classify_table(dc_cache* c);
+int dc_launch_classify_all(dc_cache* c, int cur);
 int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in);

@@ -108,12 +108,9 @@ struct ClassifyArgs {
     unsigned long long* reused_total;
 };
 
-__global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
+__device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int tile, const int lane)
 {
-    const int lane = threadIdx.x & 31;
-    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
     const int per = a.tiles_x * a.tiles_y;
-    if (tile >= per * a.S) return;
     const int s = tile / per, t = tile - s * per, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
     const int X0 = tx * DC_TILE_W, Y0 = ty * DC_TILE_H;
     const int X1 = min(X0 + DC_TILE_W, a.Wo), Y1 = min(Y0 + DC_TILE_H, a.Ho);
@@ -172,7 +169,90 @@ __global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
     }
 }
 
+__global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
+{
+    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (tile >= a.tiles_x * a.tiles_y * a.S) return;
+    classify_tile(a, tile, threadIdx.x & 31);
+}
+
+// Every cached layer of a frame in one launch: the bitmaps, reuse copies and dirty lists of a layer depend only
+// on the rectangles (known once propagation has run) and on the layer's own cached map, not on the layers before it.
+// Warps are numbered through all layers' tiles; first_warp is the running sum.
+struct ClassifyLayer {
+    const dc_region* regions; uint8_t* map[2];
+    int Ho, Wo, px_bytes, tiles_x, tiles_y, first_warp;
+    uint32_t* masks; int32_t* dirty_list; int32_t* dirty_count; int32_t* reuse_px;
+    const int32_t* alive; unsigned long long* reused_total;
+};
+
+__global__ void __launch_bounds__(256) k_classify_copy_all(const ClassifyLayer* layers, int n_cached, int total_warps,
+                                                           const int32_t* n_regions, int max_regions, int S, int cur)
+{
+    const int w = blockIdx.x * 8 + (threadIdx.x >> 5);
+    if (w >= total_warps) return;
+    int lo = 0, hi = n_cached - 1;
+    while (lo < hi) {
+        const int mid = (lo + hi + 1) >> 1;
+        if (layers[mid].first_warp <= w) lo = mid; else hi = mid - 1;
+    }
+    const ClassifyLayer& L = layers[lo];
+    ClassifyArgs a;
+    a.regions = L.regions; a.n_regions = n_regions; a.max_regions = max_regions;
+    a.prev = L.map[cur]; a.out = L.map[cur ^ 1];
+    a.Ho = L.Ho; a.Wo = L.Wo; a.px_bytes = L.px_bytes; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y; a.S = S;
+    a.masks = L.masks; a.dirty_list = L.dirty_list; a.dirty_count = L.dirty_count; a.reuse_px = L.reuse_px;
+    a.alive = L.alive; a.reused_total = L.reused_total;
+    classify_tile(a, w - L.first_warp, threadIdx.x & 31);
+}
+
 }  // namespace
+
+// Builds the device table for k_classify_copy_all (once, after every map is allocated).
+int dc_build_classify_table(dc_cache* c)
+{
+    const int n = c->n_layers;
+    ClassifyLayer* h = (ClassifyLayer*)malloc(sizeof(ClassifyLayer) * (n > 0 ? n : 1));
+    if (!h) return DC_ERR_ALLOC;
+    int k = 0, warps = 0;
+    for (int i = 0; i < n; ++i) {
+        if (!dc_layer_cached(c, i)) continue;
+        dc_layer_rt& L = c->L[i];
+        ClassifyLayer& e = h[k++];
+        e.regions = c->table + (size_t)i * c->S * c->max_regions;
+        e.map[0] = (uint8_t*)L.map[0]; e.map[1] = (uint8_t*)L.map[1];
+        e.Ho = L.d.out_h; e.Wo = L.d.out_w; e.px_bytes = L.d.cout * c->elt;
+        e.tiles_x = L.tiles_x; e.tiles_y = L.tiles_y; e.first_warp = warps;
+        e.masks = L.masks; e.dirty_list = L.dirty_list; e.dirty_count = c->dirty_count + i;
+        e.reuse_px = c->reuse_px + (size_t)i * c->S; e.alive = c->alive + (size_t)i * c->S;
+        e.reused_total = c->reused_total + i;
+        warps += L.tiles_x * L.tiles_y * c->S;
+    }
+    c->n_cached = k; c->classify_warps = warps;
+    int rc = DC_OK;
+    if (k > 0) {
+        if (cudaMalloc(&c->classify_table, sizeof(ClassifyLayer) * k) != cudaSuccess) { cudaGetLastError(); rc = DC_ERR_ALLOC; }
+        else if (cudaMemcpy(c->classify_table, h, sizeof(ClassifyLayer) * k, cudaMemcpyHostToDevice) != cudaSuccess) rc = DC_ERR_CUDA;
+        else c->bytes += sizeof(ClassifyLayer) * k;
+    }
+    free(h);
+    return rc;
+}
+
+// All cached layers at once; `cur` is the index of the map that holds the cached values (the same for every layer:
+// they all flip once per frame).  The caller has zeroed the dirty counts and the reuse counters on the stream.
+int dc_launch_classify_all(dc_cache* c, int cur)
+{
+    if (c->n_cached <= 0) return DC_OK;
+    {
+        dc_prof_scope ps(c, DC_ST_CLASSIFY_COPY);
+        k_classify_copy_all<<<dc_div_up(c->classify_warps, 8), 256, 0, c->stream>>>(
+            (const ClassifyLayer*)c->classify_table, c->n_cached, c->classify_warps, c->n_regions, c->max_regions, c->S, cur);
+    }
+    c->launches += 1;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
 
 int dc_launch_propagate(dc_cache* c, const dc_region* in, const int32_t* n_in, int layer_end)
 {

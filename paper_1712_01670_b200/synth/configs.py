@@ -60,8 +60,9 @@ def small_cnn_stream() -> Workload:
     sd = _seed(2)
     return Workload("small_cnn_stream", 2, 227, 227, 1, 30, 16, 16, SEARCH_DS, DTYPE_FP32,
                     nets.small_cnn(227, 227),
-                    lambda s, f: streams.StreamBatch(
-                        [streams.PannedStream(227, 227, f, sd, max_pan=3, disturbance="rects")]),
+                    lambda s, f, first=0: streams.StreamBatch(
+                        [streams.PannedStream(227, 227, f, sd + 1000 * k, max_pan=3, disturbance="rects")
+                         for k in range(first, first + s)]),
                     seed=sd)
 
 
@@ -70,9 +71,9 @@ def alexnet_stream() -> Workload:
     n_patches = int(np.ceil(0.10 * 227 * 227 / (24 * 24)))
     return Workload("alexnet_stream", 3, 227, 227, 1, 100, 16, 16, SEARCH_DS, DTYPE_BF16,
                     nets.alexnet_trunk(227, 227),
-                    lambda s, f: streams.StreamBatch(
-                        [streams.PannedStream(227, 227, f, sd, max_pan=4, disturbance="patches",
-                                              patch=24, n_patches=n_patches)]),
+                    lambda s, f, first=0: streams.StreamBatch(
+                        [streams.PannedStream(227, 227, f, sd + 1000 * k, max_pan=4, disturbance="patches",
+                                              patch=24, n_patches=n_patches) for k in range(first, first + s)]),
                     seed=sd)
 
 
@@ -80,9 +81,9 @@ def resnet50_stream() -> Workload:
     sd = _seed(4)
     return Workload("resnet50_stream", 4, 224, 224, 1, 300, 16, 24, SEARCH_DS, DTYPE_BF16,
                     nets.resnet50_trunk(224, 224),
-                    lambda s, f: streams.StreamBatch(
-                        [streams.PannedStream(224, 224, f, sd, max_pan=6, disturbance="window",
-                                              window_frac=0.15, zoom=0.02)]),
+                    lambda s, f, first=0: streams.StreamBatch(
+                        [streams.PannedStream(224, 224, f, sd + 1000 * k, max_pan=6, disturbance="window",
+                                              window_frac=0.15, zoom=0.02) for k in range(first, first + s)]),
                     seed=sd)
 
 
