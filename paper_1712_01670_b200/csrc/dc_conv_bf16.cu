@@ -672,6 +672,32 @@ __global__ void k_pad_channels8(const __nv_bfloat16* in, size_t pixels, int C, _
     }
 }
 
+// [S][H][W][C] -> [S][H][W][16] with zero padding, C < 16
+__global__ void k_pad_channels16(const __nv_bfloat16* in, size_t pixels, int C, __nv_bfloat16* out)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < pixels; i += (size_t)gridDim.x * blockDim.x) {
+        unsigned short v[16];
+#pragma unroll
+        for (int c = 0; c < 16; ++c) v[c] = 0;
+        const unsigned short* p = (const unsigned short*)in + i * C;
+        for (int c = 0; c < C; ++c) v[c] = p[c];
+        ((uint4*)out)[2 * i] = make_uint4(v[0] | ((uint32_t)v[1] << 16), v[2] | ((uint32_t)v[3] << 16),
+                                          v[4] | ((uint32_t)v[5] << 16), v[6] | ((uint32_t)v[7] << 16));
+        ((uint4*)out)[2 * i + 1] = make_uint4(v[8] | ((uint32_t)v[9] << 16), v[10] | ((uint32_t)v[11] << 16),
+                                              v[12] | ((uint32_t)v[13] << 16), v[14] | ((uint32_t)v[15] << 16));
+    }
+}
+
+// weights [cout][taps][cin] -> [cout][taps][16], channels beyond cin zero
+__global__ void k_pack_pad16(const __nv_bfloat16* w, size_t cout_taps, int cin, __nv_bfloat16* out)
+{
+    const size_t total = cout_taps * 16;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const size_t ct = i >> 4; const int ch = (int)(i & 15);
+        out[i] = ch < cin ? w[ct * cin + ch] : __float2bfloat16(0.f);
+    }
+}
+
 // weights [cout][taps][cin] -> [kblocks][cout][8]: block j holds tap j (cin real channels, rest zero)
 __global__ void k_pack_smallc(const __nv_bfloat16* w, int cout, int taps, int cin, int kblocks, __nv_bfloat16* out)
 {
@@ -767,6 +793,16 @@ bool smallc_ok(const dc_layer_desc& d)
            d.kh * d.kw <= 64;
 }
 
+// Few input channels with a stride or a large kernel (e.g. 11 x 11 stride 4 on RGB): the channels are padded
+// to 16 and the layer runs on the tap-by-tap kernel as a 16-channel convolution (K = taps x 16; the padded
+// products are zeros).  Far more tensor work than needed, still many times faster than the CUDA-core kernel.
+dc_layer_desc padded16(const dc_layer_desc& d) { dc_layer_desc e = d; e.cin = 16; return e; }
+bool pad16_ok(const dc_layer_desc& d)
+{
+    TcPlan p;
+    return d.kind == DC_CONV && d.cin < 16 && !make_plan(d, p) && !smallc_ok(d) && make_plan(padded16(d), p);
+}
+
 }  // namespace
 
 int dc_conv_bf16_supported(const dc_cache* c, int layer)
@@ -774,7 +810,7 @@ int dc_conv_bf16_supported(const dc_cache* c, int layer)
     TcPlan p;
     if (getenv("DC_NO_TENSOR_CORES")) return 0;
     if (c->cfg.dtype != DC_BF16 || encode_fn() == nullptr) return 0;
-    return make_plan(c->L[layer].d, p) || smallc_ok(c->L[layer].d);
+    return make_plan(c->L[layer].d, p) || smallc_ok(c->L[layer].d) || pad16_ok(c->L[layer].d);
 }
 
 // Normal layers need no repacking ([cout][kh][kw][cin] is already K-major); few-channel layers
@@ -784,7 +820,7 @@ int dc_pack_weights_bf16(dc_cache* c, int layer)
     dc_layer_rt& L = c->L[layer];
     TcPlan p;
     HaloPlan h;
-    if (halo_ok(L.d, h) && !getenv("DC_CONV_NO_HALO")) {
+    if (halo_ok(L.d, h)) {
         const size_t n = (size_t)L.d.cout * L.d.kh * L.d.kw * L.d.cin;
         DC_CUDA(cudaMalloc(&L.weight_halo, n * 2));
         c->bytes += n * 2;
@@ -792,6 +828,18 @@ int dc_pack_weights_bf16(dc_cache* c, int layer)
         k_pack_halo<<<grid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, L.d.cout, L.d.kh * L.d.kw, L.d.cin, h.BN,
                                                  (__nv_bfloat16*)L.weight_halo);
         DC_CUDA(cudaGetLastError());
+    }
+    if (pad16_ok(L.d)) {
+        const size_t cout_taps = (size_t)L.d.cout * L.d.kh * L.d.kw;
+        const size_t wbytes = cout_taps * 16 * 2, pbytes = (size_t)c->S * L.in_h * L.in_w * 32;
+        DC_CUDA(cudaMalloc(&L.weight_packed, wbytes));
+        DC_CUDA(cudaMalloc(&L.in_padded, pbytes));
+        c->bytes += wbytes + pbytes;
+        L.k_packed = L.d.kh * L.d.kw * 16;
+        k_pack_pad16<<<dc_div_up((int)(cout_taps * 16), 256), 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, cout_taps, L.d.cin,
+                                                                                   (__nv_bfloat16*)L.weight_packed);
+        DC_CUDA(cudaGetLastError());
+        return DC_OK;
     }
     if (make_plan(L.d, p) || !smallc_ok(L.d)) return DC_OK;
     const int taps = L.d.kh * L.d.kw, kblocks = (taps + 1) / 2 * 2;
@@ -893,7 +941,6 @@ static int launch_halo(dc_cache* c, int layer, int mt, const void* in, void* out
     ha.a_stages = 2;
     for (int as = 4; as > 2; --as)
         if (budget - as * mt * h.patch_bytes >= 3 * h.b_bytes) { ha.a_stages = as; break; }
-    if (getenv("DC_HALO_ASTAGES")) ha.a_stages = atoi(getenv("DC_HALO_ASTAGES"));
     const int a_total = ha.a_stages * mt * h.patch_bytes;
     int st = (budget - a_total) / h.b_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
@@ -919,8 +966,18 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
-    const dc_layer_desc& d = L.d;
     if (L.tc_mt >= 3) return launch_halo(c, layer, L.tc_mt - 2, in, out, tile_list, tile_count, masks, max_tiles);
+    const bool pad16 = pad16_ok(L.d) && L.weight_packed && L.in_padded;
+    const dc_layer_desc d = pad16 ? padded16(L.d) : L.d;
+    const void* weights = pad16 ? L.weight_packed : L.weight;
+    if (pad16) {
+        const size_t pixels = (size_t)c->S * L.in_h * L.in_w;
+        int grid_pad = (int)((pixels + 255) / 256); if (grid_pad > c->num_sms * 8) grid_pad = c->num_sms * 8;
+        dc_prof_scope ps(c, DC_ST_CONV);
+        k_pad_channels16<<<grid_pad, 256, 0, c->stream>>>((const __nv_bfloat16*)in, pixels, L.d.cin, (__nv_bfloat16*)L.in_padded);
+        c->launches += 1;
+        in = L.in_padded;
+    }
     TcPlan p;
     int ctas = L.tc_ctas == 2 ? 2 : 1;
     if (ctas == 2 && !make_plan(d, p, L.tc_mt, L.tc_bn, 2)) ctas = 1;
@@ -948,7 +1005,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
         cuuint64_t strides[1] = {K * 2};
         cuuint32_t box[2] = {(cuuint32_t)p.BK, (cuuint32_t)p.BN};
         cuuint32_t estr[2] = {1, 1};
-        if (enc(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L.weight, dims, strides, box, estr,
+        if (enc(&tmB, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(weights), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, p.swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return DC_ERR_CUDA;
     }
@@ -987,7 +1044,8 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
     dc_layer_rt& L = c->L[layer];
     TcPlan p;
     if (c->cfg.dtype != DC_BF16 || !encode_fn() || getenv("DC_NO_TENSOR_CORES")) return DC_OK;
-    const bool generic = make_plan(L.d, p);
+    const dc_layer_desc de = pad16_ok(L.d) ? padded16(L.d) : L.d;
+    const bool generic = make_plan(de, p);
     if (!generic && !smallc_ok(L.d)) return DC_OK;
     if (getenv("DC_CONV_NO_TUNE")) return DC_OK;
     const int tiles = L.tiles_x * L.tiles_y * c->S;
@@ -1011,8 +1069,7 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
                              layer, what, L.tc_mt, L.tc_bn, L.tc_ctas, ms / 2);
         if (ms < best) { best = ms; best_mt = L.tc_mt; best_bn = L.tc_bn; best_ctas = L.tc_ctas; }
     };
-    const int no_two = getenv("DC_CONV_ONE_CTA") != nullptr;
-    for (int ctas = 1; ctas <= (no_two ? 1 : 2); ++ctas) {
+    for (int ctas = 1; ctas <= 2; ++ctas) {
         L.tc_ctas = ctas;
         if (!generic) {                                               // few input channels: one kernel shape, 1 or 2 CTAs per SM
             if (ctas == 2 && tmem_cols_for(2, 1, L.d.cout) > 256) continue;
@@ -1024,7 +1081,7 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
             if (L.d.cout % bn != 0) continue;
             for (int mt = 1; mt <= 2; ++mt) {
                 TcPlan q;
-                if (!make_plan(L.d, q, mt, bn, ctas)) continue;
+                if (!make_plan(de, q, mt, bn, ctas)) continue;
                 L.tc_mt = mt; L.tc_bn = bn;
                 trial("tap-by-tap kernel");
             }
@@ -1038,7 +1095,6 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
             }
         }
     }
-    if (getenv("DC_CONV_FORCE_HALO") && L.weight_halo) { best_mt = atoi(getenv("DC_CONV_FORCE_HALO")) + 2; best_bn = 0; best_ctas = 1; }
     L.tc_mt = best_mt; L.tc_bn = best_bn; L.tc_ctas = best_ctas;
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     c->launches = 0;
