@@ -176,6 +176,43 @@ __global__ void k_relu(const T* a, size_t n, T* out)
         out[i] = from_f<T>(fmaxf(to_f(a[i]), 0.f));
 }
 
+// 16-byte vectors: element-wise add (+ ReLU) and ReLU are pure HBM traffic, one vector per thread and pass
+template <typename T> struct VecOps;
+template <> struct VecOps<float> {
+    static __device__ __forceinline__ uint4 add(uint4 a, uint4 b, int relu)
+    {
+        float r[4] = {__uint_as_float(a.x) + __uint_as_float(b.x), __uint_as_float(a.y) + __uint_as_float(b.y),
+                      __uint_as_float(a.z) + __uint_as_float(b.z), __uint_as_float(a.w) + __uint_as_float(b.w)};
+        if (relu) { for (int i = 0; i < 4; ++i) r[i] = fmaxf(r[i], 0.f); }
+        return make_uint4(__float_as_uint(r[0]), __float_as_uint(r[1]), __float_as_uint(r[2]), __float_as_uint(r[3]));
+    }
+};
+template <> struct VecOps<__nv_bfloat16> {
+    static __device__ __forceinline__ uint32_t add2(uint32_t a, uint32_t b, int relu)
+    {
+        const float2 fa = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&a));
+        const float2 fb = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&b));
+        float x = fa.x + fb.x, y = fa.y + fb.y;                   // fp32 sum, one rounding to bf16 (as the scalar kernel)
+        if (relu) { x = fmaxf(x, 0.f); y = fmaxf(y, 0.f); }
+        __nv_bfloat162 r = __floats2bfloat162_rn(x, y);
+        return *reinterpret_cast<uint32_t*>(&r);
+    }
+    static __device__ __forceinline__ uint4 add(uint4 a, uint4 b, int relu)
+    {
+        return make_uint4(add2(a.x, b.x, relu), add2(a.y, b.y, relu), add2(a.z, b.z, relu), add2(a.w, b.w, relu));
+    }
+};
+
+// out = a + b (+ ReLU); with b == nullptr: out = ReLU(a) (a + 0 is exact)
+template <typename T>
+__global__ void k_add_vec(const uint4* a, const uint4* b, size_t nvec, int relu, uint4* out)
+{
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < nvec; i += (size_t)gridDim.x * blockDim.x) {
+        const uint4 va = __ldg(a + i), vb = b ? __ldg(b + i) : make_uint4(0, 0, 0, 0);
+        out[i] = VecOps<T>::add(va, vb, relu);
+    }
+}
+
 inline int grid_for(size_t n, int block) { size_t g = (n + block - 1) / block; return (int)(g > 148 * 16 ? 148 * 16 : (g ? g : 1)); }
 
 }  // namespace
@@ -238,9 +275,16 @@ int dc_launch_add(dc_cache* c, int layer, const void* a, const void* b)
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
     dc_prof_scope ps(c, DC_ST_POINTWISE);
-    DISPATCH(c,
-        (k_add<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, (const float*)b, n, L.d.relu, (float*)L.map[0])),
-        (k_add<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, n, L.d.relu, (__nv_bfloat16*)L.map[0])));
+    if ((n * c->elt) % 16 == 0) {                                 // maps come from cudaMalloc: 256-byte aligned
+        const size_t nv = n * c->elt / 16;
+        DISPATCH(c,
+            (k_add_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, (const uint4*)b, nv, L.d.relu, (uint4*)L.map[0])),
+            (k_add_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, (const uint4*)b, nv, L.d.relu, (uint4*)L.map[0])));
+    } else {
+        DISPATCH(c,
+            (k_add<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, (const float*)b, n, L.d.relu, (float*)L.map[0])),
+            (k_add<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, n, L.d.relu, (__nv_bfloat16*)L.map[0])));
+    }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -251,9 +295,16 @@ int dc_launch_relu(dc_cache* c, int layer, const void* a)
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
     dc_prof_scope ps(c, DC_ST_POINTWISE);
-    DISPATCH(c,
-        (k_relu<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, n, (float*)L.map[0])),
-        (k_relu<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, n, (__nv_bfloat16*)L.map[0])));
+    if ((n * c->elt) % 16 == 0) {
+        const size_t nv = n * c->elt / 16;
+        DISPATCH(c,
+            (k_add_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, nullptr, nv, 1, (uint4*)L.map[0])),
+            (k_add_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, nullptr, nv, 1, (uint4*)L.map[0])));
+    } else {
+        DISPATCH(c,
+            (k_relu<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, n, (float*)L.map[0])),
+            (k_relu<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, n, (__nv_bfloat16*)L.map[0])));
+    }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
