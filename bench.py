@@ -344,10 +344,14 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
     bf16 = w.dtype == 1
     conv_tflops = useful_flops / (conv_ms * 1e-3) / 1e12 if conv_ms > 0 else 0.0
     conv_peak = peaks["bf16_tflops_sustained"] if bf16 else None
+    # DRAM bytes per convolution launch from the ncu capture summarised in profiles/dram_traffic_batched_stress.md
+    # (32 streams of workload 5, kernels as committed with that file); other shapes were not captured
+    conv_traffic = 78.0e6 if (w.index == 5 and S == 32 and bf16 and not args.cache_pool) else None
     roofline = {"kernel": "partial convolution (all conv launches of the timed region)",
                 "bound": "tensor" if bf16 else "alu", "achieved": conv_tflops,
                 "peak": conv_peak, "unit": "TFLOP/s", "frac": (conv_tflops / conv_peak) if conv_peak else None,
-                "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": None,
+                "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": conv_traffic,
+                "traffic_unit": "bytes per launch (dram read + write, ncu, one-pass capture of this workload)",
                 "launches": conv_n, "avg_launch_ms": conv_ms / max(1, conv_n),
                 "flops_per_launch": useful_flops / max(1, conv_n)}
     match_ms = prof["search"][0] + prof["verify"][0]
@@ -355,7 +359,9 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
     match_gbs = match_bytes / (match_ms * 1e-3) / 1e9 if match_ms > 0 else 0.0
     roofline_matcher = {"kernel": "block search + verify", "bound": "hbm", "achieved": match_gbs,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": match_gbs / peaks["hbm_gbs"],
-                        "peak_source": f"hbm_gbs, {peaks['source']}", "traffic": None,
+                        "peak_source": f"hbm_gbs, {peaks['source']}",
+                        "traffic": 942.0e6 if (w.index == 5 and S == 32 and w.search == 1 and args.skip_k == 1) else None,
+                        "traffic_unit": "bytes per batch-frame (search + long walks + verify; dram read + write, ncu)",
                         "launches": prof["search"][1] + prof["verify"][1],
                         "bytes_per_frame_batch": 4.0 * frame_bytes * S}
 
