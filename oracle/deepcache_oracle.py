@@ -299,6 +299,38 @@ def pool_reuse(x, layer, prev_out=None, regions=None):
     return out, reused
 
 
+def lrn(x, layer, alpha, beta, k, mode):
+    """Local response normalisation over a spatial window inside each channel: the form Table 2's LRN row
+    describes (a radius r erodes the rectangle by r on every side).  With n = 2 r + 1:
+        b[y, x, c] = a[y, x, c] / (k + alpha / n^2 * sum_{|dy|,|dx| <= r} a[y + dy, x + dx, c]^2) ^ beta
+    pixels outside the map count as zero; the divisor n^2 is the same at the borders.  r = layer's ph."""
+    x = np.ascontiguousarray(x, np.float64)
+    r = int(layer["ph"])
+    n = 2 * r + 1
+    H, W, _ = x.shape
+    sq = np.zeros((H + 2 * r, W + 2 * r, x.shape[2]), np.float64)
+    sq[r:r + H, r:r + W] = x * x
+    total = np.zeros_like(x)
+    for dy in range(n):
+        for dx in range(n):
+            total += sq[dy:dy + H, dx:dx + W]
+    out = x / (k + alpha / (n * n) * total) ** beta
+    return quant_array(out, mode)
+
+
+def concat(a, b):
+    """Channel concatenation (Table 2's Concat row, two inputs): the channels of a, then those of b."""
+    return np.concatenate([np.asarray(a, np.float64), np.asarray(b, np.float64)], axis=2)
+
+
+def fully_connected(x, layer, weight, bias, mode):
+    """A fully-connected layer on an H x W x C map is the convolution whose kernel covers the whole map without
+    padding (one output pixel); weight is [cout][H][W][cin].  Table 2: nothing of its output is reusable."""
+    L = dict(layer, kind=KIND_CONV, kh=x.shape[0], kw=x.shape[1], sh=1, sw=1, ph=0, pw=0, out_h=1, out_w=1)
+    out, _ = conv_reuse(x, L, weight, bias, mode)
+    return out
+
+
 def add(a, b, relu, mode):
     a = np.ascontiguousarray(a, np.float64)
     b = np.ascontiguousarray(b, np.float64)
@@ -320,12 +352,13 @@ class OracleCache:
 
     def __init__(self, width, height, layers, weights, biases, *, block=10, search_range=8,
                  search_kind=SEARCH_DS, psnr_db=20.0, expire_n=10, quant=QUANT_NONE, use_cache=True, skip_k=1,
-                 region_mode=0, cache_pool=False):
+                 region_mode=0, cache_pool=False, lrn=(1e-4, 0.75, 1.0)):
         self.W, self.H = width, height
         self.layers = layers
         self.block, self.R, self.kind = block, search_range, search_kind
         self.T, self.N, self.quant, self.use_cache = psnr_db, expire_n, quant, use_cache
         self.skip_k, self.region_mode, self.cache_pool = skip_k, region_mode, cache_pool
+        self.lrn = lrn                 # (alpha, beta, k) of every LRN layer
         # weights are stored at the storage precision (bf16 workloads round them once)
         self.weights = [None if w is None else quant_array(w, quant) for w in weights]
         self.biases = [None if b is None else np.asarray(b, np.float64) for b in biases]
@@ -377,6 +410,12 @@ class OracleCache:
                 out = resize_area(frame, l["out_h"], l["out_w"], self.quant)
             elif k == KIND_RELU:
                 out = np.maximum(x, 0.0)
+            elif k == KIND_LRN:
+                out = lrn(x, l, *self.lrn, self.quant)
+            elif k == KIND_CONCAT:
+                out = concat(x, maps[l["in1"]])
+            elif k == KIND_FC:
+                out = fully_connected(x, l, self.weights[i], self.biases[i], self.quant)
             else:
                 raise ValueError(f"layer kind {k} has no execution rule in the oracle")
             maps.append(out)

@@ -52,6 +52,27 @@ class NetBuilder:
         self.layers.append(_layer(KIND_ADD, a, h, w, c, c, relu=relu, in1=b))
         return len(self.layers) - 1
 
+    def lrn(self, src: int, radius: int) -> int:
+        """Within-channel local response normalisation over a (2 radius + 1)^2 window (Table 2's LRN row)."""
+        h, w, c = self.shape(src)
+        self.layers.append(_layer(KIND_LRN, src, h, w, c, c, 2 * radius + 1, 1, radius))
+        return len(self.layers) - 1
+
+    def concat(self, a: int, b: int) -> int:
+        h, w, ca = self.shape(a)
+        hb, wb, cb = self.shape(b)
+        assert (h, w) == (hb, wb)
+        self.layers.append(_layer(KIND_CONCAT, a, h, w, ca, ca + cb, in1=b))
+        return len(self.layers) - 1
+
+    def fc(self, src: int, cout: int, relu: int = 0) -> int:
+        """Fully connected = a convolution whose kernel covers the whole input map (weights [cout][h][w][cin])."""
+        h, w, c = self.shape(src)
+        l = _layer(KIND_FC, src, 1, 1, c, cout, 1, 1, 0, relu)
+        l["kh"], l["kw"] = h, w
+        self.layers.append(l)
+        return len(self.layers) - 1
+
     def resize_area(self, src: int, oh: int, ow: int) -> int:
         h, w, c = self.shape(src)
         self.layers.append(_layer(KIND_RESIZE_AREA, src, oh, ow, c, c))
@@ -73,6 +94,25 @@ def small_cnn(h=227, w=227):
     x = b.conv(x, 64, 3, 1, 1)
     x = b.maxpool(x, 2, 2)
     b.conv(x, 128, 3, 1, 1)
+    return b.layers
+
+
+def inception_lrn_net(h=64, w=64):
+    """A small GoogLeNet-flavoured graph that uses every layer kind of Table 2: convolution, LRN, pooling, two
+    branches joined by a channel concatenation, and a fully connected head."""
+    b = NetBuilder(h, w)
+    x = b.conv(-1, 32, 3, 1, 1)
+    x = b.lrn(x, 1)
+    x = b.maxpool(x, 2, 2)
+    p1 = b.conv(x, 32, 1, 1, 0)
+    p2 = b.conv(x, 16, 3, 1, 1)
+    p2 = b.conv(p2, 32, 3, 1, 1)
+    x = b.concat(p1, p2)
+    x = b.conv(x, 64, 3, 1, 1)
+    x = b.maxpool(x, 2, 2)
+    x = b.lrn(x, 2)
+    x = b.maxpool(x, 4, 4)
+    b.fc(x, 48)
     return b.layers
 
 
@@ -120,7 +160,7 @@ def vgg16_trunk(h=224, w=224, src_h=None, src_w=None):
 
 
 def random_weights(layers, seed: int, *, std: float | None = None, bias_std: float = 0.05):
-    """He-normal (or fixed-``std``) weights for every conv layer; ``None`` elsewhere.
+    """He-normal (or fixed-``std``) weights for every conv and fully-connected layer; ``None`` elsewhere.
 
     The last conv of a residual branch (a conv feeding an add with relu=0) is
     scaled by 0.5 so activations stay tame through deep residual stacks.
@@ -132,7 +172,7 @@ def random_weights(layers, seed: int, *, std: float | None = None, bias_std: flo
             feeds_add.add(l["in0"])
     weights, biases = [], []
     for i, l in enumerate(layers):
-        if l["kind"] != KIND_CONV:
+        if l["kind"] not in (KIND_CONV, KIND_FC):
             weights.append(None)
             biases.append(None)
             continue

@@ -269,3 +269,65 @@ def test_pool_reuse_is_exact_when_the_motion_is_a_multiple_of_the_stride():
     p, q = c1.infer_frame(f2), c2.infer_frame(f2)
     assert p["match"]["M"] == (3, 0) and p["reused"][pools[0]].any()
     assert not np.array_equal(p["maps"][pools[0]], q["maps"][pools[0]])
+
+
+# ---------------------------------------------------------------------------
+# the remaining layer kinds of Table 2 as executable layers: LRN, concat, fully connected
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("r,alpha,beta,k", [(1, 1e-4, 0.75, 1.0), (2, 0.05, 0.75, 2.0), (0, 0.3, 0.5, 1.0)])
+def test_lrn_equals_average_pooling_form(r, alpha, beta, k):
+    g = rng(30 + r)
+    x = g.normal(size=(11, 9, 5)) * 3.0
+    L = dict(kind=orc.KIND_LRN, kh=2 * r + 1, kw=2 * r + 1, sh=1, sw=1, ph=r, pw=r, cin=5, cout=5, relu=0, in0=-1, in1=-1,
+             out_h=11, out_w=9)
+    got = orc.lrn(x, L, alpha, beta, k, orc.QUANT_NONE)
+    t = torch.from_numpy(x).permute(2, 0, 1)[None]
+    avg = F.avg_pool2d(t * t, 2 * r + 1, 1, r, count_include_pad=True)          # zero padding, divisor n^2 everywhere
+    ref = (t / (k + alpha * avg) ** beta)[0].permute(1, 2, 0).numpy()
+    assert np.abs(got - ref).max() < 1e-13
+
+
+def test_lrn_closed_forms():
+    L = dict(kind=orc.KIND_LRN, kh=3, kw=3, sh=1, sw=1, ph=1, pw=1, cin=1, cout=1, relu=0, in0=-1, in1=-1, out_h=5, out_w=5)
+    x = np.full((5, 5, 1), 2.0)
+    b = orc.lrn(x, L, 0.9, 0.5, 1.0, orc.QUANT_NONE)
+    assert abs(b[2, 2, 0] - 2.0 / np.sqrt(1.0 + 0.9 * 4.0)) < 1e-15             # interior: mean of squares = 4
+    assert abs(b[0, 0, 0] - 2.0 / np.sqrt(1.0 + 0.9 * 16.0 / 9.0)) < 1e-15      # corner: 4 of the 9 taps are inside
+    assert abs(b[0, 2, 0] - 2.0 / np.sqrt(1.0 + 0.9 * 24.0 / 9.0)) < 1e-15      # edge: 6 of 9
+    # the region rule and the arithmetic agree: an output pixel depends exactly on the (2r+1)^2 window
+    y = x.copy(); y[4, 4, 0] = 7.0
+    c = orc.lrn(y, L, 0.9, 0.5, 1.0, orc.QUANT_NONE)
+    changed = np.argwhere(c[..., 0] != b[..., 0])
+    assert set(map(tuple, changed)) == {(3, 3), (3, 4), (4, 3), (4, 4)}
+
+
+def test_concat_and_fully_connected():
+    g = rng(33)
+    a, b = g.normal(size=(4, 5, 3)), g.normal(size=(4, 5, 2))
+    c = orc.concat(a, b)
+    assert c.shape == (4, 5, 5) and np.array_equal(c[..., :3], a) and np.array_equal(c[..., 3:], b)
+    x = g.normal(size=(3, 4, 6))
+    w = g.normal(size=(7, 3, 4, 6))
+    bias = g.normal(size=7)
+    L = dict(kind=orc.KIND_FC, kh=3, kw=4, sh=1, sw=1, ph=0, pw=0, cin=6, cout=7, relu=1, in0=-1, in1=-1, out_h=1, out_w=1)
+    got = orc.fully_connected(x, L, w, bias, orc.QUANT_NONE)
+    ref = F.linear(torch.from_numpy(x).reshape(1, -1), torch.from_numpy(w).reshape(7, -1), torch.from_numpy(bias)).clamp_min(0)
+    assert got.shape == (1, 1, 7) and np.abs(got[0, 0] - ref[0].numpy()).max() < 1e-12
+
+
+def test_graph_with_every_layer_kind_runs_and_reuses():
+    w = configs.WORKLOADS[2]()
+    w.layers = nets.inception_lrn_net(64, 64)
+    w.width = w.height = 64
+    sb = w.streams(1, 3)
+    frames = [sb.frame(i)[0][:64, :64] for i in range(3)]
+    cached, plain = make_cache(w), make_cache(w, use_cache=False)
+    for i, f in enumerate(frames):
+        a, b = cached.infer_frame(f), plain.infer_frame(f)
+        assert a["out"].shape == (1, 1, 48)
+        if i == 0:
+            assert np.array_equal(a["out"], b["out"])
+        else:
+            assert a["reused"][0].any()                                          # first convolution reuses
+            assert len(a["regions"][-1]) == 0 or not a["regions"][-1]["w"].any()  # Table 2: nothing reusable after FC
+            assert np.abs(a["out"] - b["out"]).max() < 0.5
