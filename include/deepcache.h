@@ -71,8 +71,15 @@ typedef enum {
  * DC_CONV: kh x kw kernel, stride, padding, cin -> cout, optional fused ReLU.
  * DC_MAXPOOL: floor mode, padded taps ignored.  DC_ADD: element-wise, optional ReLU.
  * DC_RESIZE_AREA: box average of the input frame (in0 must be -1) to out_h x out_w.
- * DC_LRN (radius = ph), DC_CONCAT, DC_FC are known to region propagation only;
- * a cache containing them cannot run dc_infer_frame. */
+ * DC_LRN: local response normalisation inside each channel over a (2 ph + 1)^2 spatial window (the form Table 2's
+ *   radius describes): b = a / (k + alpha / n^2 * sum of a^2 over the window)^beta, outside pixels count as zero;
+ *   alpha, beta, k come from dc_config.  Executable when kh = kw = 2 ph + 1 and pw = ph.
+ * DC_CONCAT: channels of in0 followed by those of in1.
+ * DC_FC: fully connected; executable when kh, kw equal the input map's height and width (then it is the convolution
+ *   whose kernel covers the whole map: weights [cout][kh][kw][cin], out 1 x 1, optional ReLU).  Table 2: nothing of
+ *   its output is reusable.
+ * A layer table with an LRN or FC layer of another shape is accepted for region propagation, but such a cache
+ * cannot run dc_infer_frame. */
 typedef struct {
     int32_t kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w;
 } dc_layer_desc;
@@ -108,6 +115,7 @@ typedef struct {
                                           (the extension Section 5 mentions; costs a second pooled map per layer).
                                           Applies to pooling layers whose pixel is a multiple of 16 bytes.  0 = the
                                           paper's choice: only convolutions are cached */
+    double  lrn_alpha, lrn_beta, lrn_k;/* parameters of every DC_LRN layer; all three 0 selects 1e-4, 0.75, 1 */
 } dc_config;
 
 /* Per-stream outcome of one dc_infer_frame. */

@@ -37,7 +37,8 @@ class dc_config(C.Structure):
     _fields_ = [("width", C.c_int32), ("height", C.c_int32), ("channels", C.c_int32), ("n_streams", C.c_int32),
                 ("block", C.c_int32), ("range", C.c_int32), ("search", C.c_int32), ("skip_k", C.c_int32),
                 ("expire_n", C.c_int32), ("psnr_db", C.c_double), ("dtype", C.c_int32), ("max_regions", C.c_int32),
-                ("region_mode", C.c_int32), ("cache_pool", C.c_int32)]
+                ("region_mode", C.c_int32), ("cache_pool", C.c_int32),
+                ("lrn_alpha", C.c_double), ("lrn_beta", C.c_double), ("lrn_k", C.c_double)]
 
 
 class dc_frame_stats(C.Structure):

@@ -59,7 +59,17 @@ int dev_alloc(dc_cache* c, T** p, size_t count)
 }
 #define DC_TRY(expr) do { int rc__ = (expr); if (rc__ != DC_OK) return rc__; } while (0)
 
-bool kind_executable(int k) { return k == DC_CONV || k == DC_MAXPOOL || k == DC_RELU || k == DC_ADD || k == DC_RESIZE_AREA; }
+// Can dc_infer_frame run this layer?  LRN needs its window stated consistently, a fully-connected layer must cover
+// its whole input map (it then runs as that convolution).
+bool layer_executable(const dc_layer_desc& L, int in_h, int in_w)
+{
+    switch (L.kind) {
+    case DC_CONV: case DC_MAXPOOL: case DC_RELU: case DC_ADD: case DC_RESIZE_AREA: case DC_CONCAT: return true;
+    case DC_LRN: return L.kh == 2 * L.ph + 1 && L.kw == L.kh && L.pw == L.ph;
+    case DC_FC: return L.kh == in_h && L.kw == in_w && L.out_h == 1 && L.out_w == 1;
+    default: return false;
+    }
+}
 
 int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
 {
@@ -105,6 +115,10 @@ int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
             break;
         case DC_LRN:
             if (L.ph < 0 || L.out_h != ih || L.out_w != iw || L.cout != ic) return DC_ERR_CONFIG;
+            break;
+        case DC_FC:
+            if (L.cin != ic) return DC_ERR_CONFIG;
+            if (layer_executable(L, ih, iw) && (L.cout * elt) % 16 != 0) return DC_ERR_CONFIG;
             break;
         case DC_RELU:
             if (L.out_h != ih || L.out_w != iw || L.cout != ic) return DC_ERR_CONFIG;
@@ -188,13 +202,16 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     for (int i = 0; i < n; ++i) {
         dc_layer_rt& L = c->L[i];
         L.d = layers[i];
+        // an executable fully-connected layer runs as the convolution that covers its input map; the device copy of the
+        // layer table keeps DC_FC, so Table 2 still marks nothing of its output reusable and every tile is computed
+        if (L.d.kind == DC_FC && c->executable) { L.d.kind = DC_CONV; L.d.sh = L.d.sw = 1; L.d.ph = L.d.pw = 0; }
         L.in_h = L.d.in0 < 0 ? cfg.height : layers[L.d.in0].out_h;
         L.in_w = L.d.in0 < 0 ? cfg.width : layers[L.d.in0].out_w;
         in_hw[2 * i] = L.in_h; in_hw[2 * i + 1] = L.in_w;
         all_count[i] = 0;
         if (!c->executable) continue;
         if (L.d.in0 < 0 && L.d.kind != DC_RESIZE_AREA) need_input_map = true;
-        if (L.d.kind == DC_ADD && L.d.in1 < 0) need_input_map = true;
+        if ((L.d.kind == DC_ADD || L.d.kind == DC_CONCAT) && L.d.in1 < 0) need_input_map = true;
         L.map_bytes = (size_t)S * L.d.out_h * L.d.out_w * L.d.cout * c->elt;
         const bool cached = dc_layer_cached(c, i);
         const int copies = cached ? 2 : 1;
@@ -335,7 +352,11 @@ int dc_cache_create(const dc_config* cfg, const dc_layer_desc* layers, int n_lay
     c->max_regions = cfg->max_regions > 0 ? cfg->max_regions : worst;
     c->elt = cfg->dtype == DC_BF16 ? 2 : 4;
     c->executable = true;
-    for (int i = 0; i < n_layers; ++i) if (!kind_executable(layers[i].kind)) c->executable = false;
+    for (int i = 0; i < n_layers; ++i) {
+        const int ih = layers[i].in0 < 0 ? cfg->height : layers[layers[i].in0].out_h;
+        const int iw = layers[i].in0 < 0 ? cfg->width : layers[layers[i].in0].out_w;
+        if (!layer_executable(layers[i], ih, iw)) c->executable = false;
+    }
     rc = build(c, layers, weights_dev, bias_dev);
     if (rc != DC_OK) { release(c); return rc; }
     *out = c;
@@ -507,6 +528,12 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
         }
         case DC_ADD: DC_TRY(dc_launch_add(c, i, in, layer_input(c, L.d.in1))); break;
         case DC_RELU: DC_TRY(dc_launch_relu(c, i, in)); break;
+        case DC_LRN: DC_TRY(dc_launch_lrn(c, i, in)); break;
+        case DC_CONCAT: {
+            const int ca = L.d.in0 < 0 ? 3 : c->L[L.d.in0].d.cout, cb = L.d.in1 < 0 ? 3 : c->L[L.d.in1].d.cout;
+            DC_TRY(dc_launch_concat(c, i, in, ca, layer_input(c, L.d.in1), cb));
+            break;
+        }
         case DC_RESIZE_AREA: DC_TRY(dc_launch_resize(c, i, frame_copy, c->key_pitch)); break;
         default: return DC_ERR_STATE;
         }

@@ -213,6 +213,43 @@ __global__ void k_add_vec(const uint4* a, const uint4* b, size_t nvec, int relu,
     }
 }
 
+// Local response normalisation inside each channel over a (2 r + 1)^2 window; pixels outside the map count as zero
+// and the divisor stays n^2 at the borders.  One thread per output element; sums in float.
+template <typename T>
+__global__ void k_lrn(const T* in, int H, int W, int C, int S, int r, float alpha_n2, float beta, float kappa, T* out)
+{
+    const size_t total = (size_t)S * H * W * C;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C); size_t t = i / C;
+        const int x = (int)(t % W); t /= W;
+        const int y = (int)(t % H); const int s = (int)(t / H);
+        float sum = 0.f;
+        for (int dy = -r; dy <= r; ++dy) {
+            const int yy = y + dy;
+            if (yy < 0 || yy >= H) continue;
+            for (int dx = -r; dx <= r; ++dx) {
+                const int xx = x + dx;
+                if (xx < 0 || xx >= W) continue;
+                const float v = to_f(in[(((size_t)s * H + yy) * W + xx) * C + c]);
+                sum += v * v;
+            }
+        }
+        out[i] = from_f<T>(to_f(in[i]) * powf(kappa + alpha_n2 * sum, -beta));
+    }
+}
+
+// Channel concatenation of two NHWC maps
+template <typename T>
+__global__ void k_concat(const T* a, int Ca, const T* b, int Cb, size_t pixels, T* out)
+{
+    const int C = Ca + Cb;
+    const size_t total = pixels * C;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
+        const int c = (int)(i % C); const size_t px = i / C;
+        out[i] = c < Ca ? a[px * Ca + c] : b[px * Cb + (c - Ca)];
+    }
+}
+
 inline int grid_for(size_t n, int block) { size_t g = (n + block - 1) / block; return (int)(g > 148 * 16 ? 148 * 16 : (g ? g : 1)); }
 
 }  // namespace
@@ -305,6 +342,36 @@ int dc_launch_relu(dc_cache* c, int layer, const void* a)
             (k_relu<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, n, (float*)L.map[0])),
             (k_relu<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, n, (__nv_bfloat16*)L.map[0])));
     }
+    c->launches += 1;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
+
+int dc_launch_lrn(dc_cache* c, int layer, const void* in)
+{
+    dc_layer_rt& L = c->L[layer];
+    const size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
+    const int r = L.d.ph, win = 2 * r + 1;
+    const bool defaults = c->cfg.lrn_alpha == 0.0 && c->cfg.lrn_beta == 0.0 && c->cfg.lrn_k == 0.0;
+    const float alpha = (float)(defaults ? 1e-4 : c->cfg.lrn_alpha), beta = (float)(defaults ? 0.75 : c->cfg.lrn_beta);
+    const float kappa = (float)(defaults ? 1.0 : c->cfg.lrn_k);
+    dc_prof_scope ps(c, DC_ST_POINTWISE);
+    DISPATCH(c,
+        (k_lrn<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (float*)L.map[0])),
+        (k_lrn<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (__nv_bfloat16*)L.map[0])));
+    c->launches += 1;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
+
+int dc_launch_concat(dc_cache* c, int layer, const void* a, int ca, const void* b, int cb)
+{
+    dc_layer_rt& L = c->L[layer];
+    const size_t pixels = (size_t)c->S * L.d.out_h * L.d.out_w;
+    dc_prof_scope ps(c, DC_ST_POINTWISE);
+    DISPATCH(c,
+        (k_concat<float><<<grid_for(pixels * L.d.cout, 256), 256, 0, c->stream>>>((const float*)a, ca, (const float*)b, cb, pixels, (float*)L.map[0])),
+        (k_concat<__nv_bfloat16><<<grid_for(pixels * L.d.cout, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, ca, (const __nv_bfloat16*)b, cb, pixels, (__nv_bfloat16*)L.map[0])));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;

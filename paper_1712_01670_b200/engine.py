@@ -30,7 +30,7 @@ def device_view(ptr: int, shape, dtype: torch.dtype, device) -> torch.Tensor:
 class DeepCache:
     def __init__(self, width, height, layers, weights, biases, *, n_streams=1, block=10, search_range=8,
                  search=B.DC_SEARCH_DIAMOND, psnr_db=20.0, expire_n=10, dtype=B.DC_FP32, max_regions=0, skip_k=1,
-                 region_mode=B.DC_REGIONS_GLOBAL, cache_pool=False, device="cuda:0"):
+                 region_mode=B.DC_REGIONS_GLOBAL, cache_pool=False, lrn=(1e-4, 0.75, 1.0), device="cuda:0"):
         if not torch.cuda.is_available():
             raise RuntimeError("DeepCache needs a CUDA device; there is no CPU fallback")
         self.device = torch.device(device)
@@ -39,7 +39,7 @@ class DeepCache:
         self.cfg = B.dc_config(width=width, height=height, channels=3, n_streams=n_streams, block=block,
                                range=search_range, search=search, skip_k=skip_k, expire_n=expire_n, psnr_db=psnr_db,
                                dtype=dtype, max_regions=max_regions, region_mode=region_mode,
-                               cache_pool=int(bool(cache_pool)))
+                               cache_pool=int(bool(cache_pool)), lrn_alpha=lrn[0], lrn_beta=lrn[1], lrn_k=lrn[2])
         self.S, self.W, self.H = n_streams, width, height
         self.Gx, self.Gy = -(-width // block), -(-height // block)
         worst = self.Gx * self.Gy if region_mode == B.DC_REGIONS_PER_BLOCK else -(-self.Gx // 2) * self.Gy

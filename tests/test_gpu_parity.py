@@ -198,6 +198,30 @@ def test_cached_pooling_reuses_pixels():
         dc.close()
 
 
+@pytest.mark.parametrize("dtype", [configs.DTYPE_FP32, configs.DTYPE_BF16])
+def test_infer_graph_with_every_layer_kind(dtype):
+    """Convolution, LRN, pooling, two branches joined by a concat and a fully-connected head (all rows of Table 2),
+    every layer's map and rectangles against the oracle over a refresh, cached frames and the next refresh."""
+    w = configs.WORKLOADS[2]()
+    w.layers = nets.inception_lrn_net(80, 96)
+    w.width, w.height, w.dtype, w.expire_n = 96, 80, dtype, 3
+    crop = w.make_streams
+    w.make_streams = lambda s, f, first=0: _cropped(crop(s, f, first), 80, 96)
+    U.run_stream_parity(w, 2, list(range(5)))
+    U.run_stream_parity(w, 1, list(range(3)), cache_pool=True, region_mode=B.DC_REGIONS_PER_BLOCK)
+
+
+class _cropped:
+    """A stream batch cut to the top-left h x w pixels of every frame."""
+
+    def __init__(self, batch, h, w):
+        self.batch, self.h, self.w = batch, h, w
+
+    def frame(self, i, s=None):
+        f = self.batch.frame(i) if s is None else self.batch.frame(i, s)
+        return np.ascontiguousarray(f[..., :self.h, :self.w, :])
+
+
 @pytest.mark.parametrize("k", [2, 3])
 def test_match_k_skip(k):
     """Section 4's k-skip: Step 2 on every k-th block row and column only (16-px fast path and generic path)."""
