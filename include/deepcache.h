@@ -111,9 +111,9 @@ typedef struct {
     int32_t dtype;                     /* dc_dtype of maps and arithmetic inputs */
     int32_t max_regions;               /* rectangles per stream; 0 = worst case of the grid */
     int32_t region_mode;               /* dc_region_mode; 0 = the paper's global vector */
-    int32_t cache_pool;                /* 1: max-pooling layers keep their last output and reuse it like convolutions
+    int32_t cache_pool;                /* 1: max-pooling and LRN layers keep their last output and reuse it like convolutions
                                           (the extension Section 5 mentions; costs a second pooled map per layer).
-                                          Applies to pooling layers whose pixel is a multiple of 16 bytes.  0 = the
+                                          Applies to such layers whose pixel is a multiple of 16 bytes.  0 = the
                                           paper's choice: only convolutions are cached */
     double  lrn_alpha, lrn_beta, lrn_k;/* parameters of every DC_LRN layer; all three 0 selects 1e-4, 0.75, 1 */
 } dc_config;

@@ -287,7 +287,15 @@ def pool_reuse(x, layer, prev_out=None, regions=None):
     """Section 5 notes that the cache extends to other layer types; this is that extension for max pooling,
     with the three steps of "Reuse": copy the layer's reusable rectangles from the cached pooled map, mark
     them, pool the input only where nothing was copied.  Returns (out, reused byte map)."""
-    out = maxpool(x, layer)
+    return _copy_rectangles(maxpool(x, layer), prev_out, regions)
+
+
+def lrn_reuse(x, layer, alpha, beta, k, mode, prev_out=None, regions=None):
+    """The same extension for an LRN layer: cached rectangles copied, the rest normalised from the input."""
+    return _copy_rectangles(lrn(x, layer, alpha, beta, k, mode), prev_out, regions)
+
+
+def _copy_rectangles(out, prev_out, regions):
     reused = np.zeros(out.shape[:2], np.uint8)
     if prev_out is not None and regions is not None:
         for r in regions:
@@ -411,7 +419,11 @@ class OracleCache:
             elif k == KIND_RELU:
                 out = np.maximum(x, 0.0)
             elif k == KIND_LRN:
-                out = lrn(x, l, *self.lrn, self.quant)
+                if self.cache_pool and not refresh:
+                    out, reused = lrn_reuse(x, l, *self.lrn, self.quant, self.prev_maps[i], per_layer_regions[i])
+                    info["reused"][i] = reused
+                else:
+                    out = lrn(x, l, *self.lrn, self.quant)
             elif k == KIND_CONCAT:
                 out = concat(x, maps[l["in1"]])
             elif k == KIND_FC:
@@ -421,7 +433,7 @@ class OracleCache:
             maps.append(out)
         # the frame becomes the next key, the conv outputs the next values (Section 3)
         self.prev_frame = frame.copy()
-        kept = (KIND_CONV, KIND_MAXPOOL) if self.cache_pool else (KIND_CONV,)
+        kept = (KIND_CONV, KIND_MAXPOOL, KIND_LRN) if self.cache_pool else (KIND_CONV,)
         self.prev_maps = [m if layers[i]["kind"] in kept else None for i, m in enumerate(maps)]
         self.frame_idx += 1
         info["maps"] = maps

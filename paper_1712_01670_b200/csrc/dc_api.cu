@@ -31,7 +31,7 @@ bool dc_layer_cached(const dc_cache* c, int layer)
 {
     const dc_layer_desc& d = c->L[layer].d;
     if (d.kind == DC_CONV) return true;
-    return d.kind == DC_MAXPOOL && c->cfg.cache_pool && ((size_t)d.cout * c->elt) % 16 == 0;
+    return (d.kind == DC_MAXPOOL || d.kind == DC_LRN) && c->cfg.cache_pool && ((size_t)d.cout * c->elt) % 16 == 0;
 }
 
 namespace {
@@ -528,7 +528,18 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
         }
         case DC_ADD: DC_TRY(dc_launch_add(c, i, in, layer_input(c, L.d.in1))); break;
         case DC_RELU: DC_TRY(dc_launch_relu(c, i, in)); break;
-        case DC_LRN: DC_TRY(dc_launch_lrn(c, i, in)); break;
+        case DC_LRN: {
+            if (!dc_layer_cached(c, i)) { DC_TRY(dc_launch_lrn(c, i, in, L.map[0], nullptr)); break; }
+            void* prev = L.map[L.cur]; void* out = L.map[L.cur ^ 1];
+            if (!refresh) {
+                if (!classified) DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
+                DC_TRY(dc_launch_lrn(c, i, in, out, L.masks));
+            } else {
+                DC_TRY(dc_launch_lrn(c, i, in, out, nullptr));
+            }
+            L.cur ^= 1;
+            break;
+        }
         case DC_CONCAT: {
             const int ca = L.d.in0 < 0 ? 3 : c->L[L.d.in0].d.cout, cb = L.d.in1 < 0 ? 3 : c->L[L.d.in1].d.cout;
             DC_TRY(dc_launch_concat(c, i, in, ca, layer_input(c, L.d.in1), cb));

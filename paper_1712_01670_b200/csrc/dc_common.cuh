@@ -132,12 +132,12 @@ int dc_launch_conv(dc_cache* c, int layer, const void* in, void* out, const int3
 int dc_launch_input_map(dc_cache* c, const uint8_t* frame, size_t pitch);
 int dc_launch_resize(dc_cache* c, int layer, const uint8_t* frame, size_t pitch);   // frame: 16-byte aligned rows
 int dc_launch_maxpool(dc_cache* c, int layer, const void* in, void* out, const uint32_t* masks);
-int dc_launch_lrn(dc_cache* c, int layer, const void* in);
+int dc_launch_lrn(dc_cache* c, int layer, const void* in, void* out, const uint32_t* masks);
 int dc_launch_concat(dc_cache* c, int layer, const void* a, int ca, const void* b, int cb);
 int dc_launch_add(dc_cache* c, int layer, const void* a, const void* b);
 int dc_launch_relu(dc_cache* c, int layer, const void* a);
 int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_dev);
-// true for layers that keep their last output as cached values: convolutions, and max pooling when cfg.cache_pool
+// true for layers that keep their last output as cached values: convolutions, and max pooling / LRN when cfg.cache_pool
 bool dc_layer_cached(const dc_cache* c, int layer);
 int dc_build_classify_table(dc_cache* c);
 int dc_launch_classify_all(dc_cache* c, int cur);

@@ -216,13 +216,19 @@ __global__ void k_add_vec(const uint4* a, const uint4* b, size_t nvec, int relu,
 // Local response normalisation inside each channel over a (2 r + 1)^2 window; pixels outside the map count as zero
 // and the divisor stays n^2 at the borders.  One thread per output element; sums in float.
 template <typename T>
-__global__ void k_lrn(const T* in, int H, int W, int C, int S, int r, float alpha_n2, float beta, float kappa, T* out)
+__global__ void k_lrn(const T* in, int H, int W, int C, int S, int r, float alpha_n2, float beta, float kappa, T* out,
+                      const uint32_t* masks, int tiles_x, int tiles_y)
 {
     const size_t total = (size_t)S * H * W * C;
     for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (size_t)gridDim.x * blockDim.x) {
         const int c = (int)(i % C); size_t t = i / C;
         const int x = (int)(t % W); t /= W;
         const int y = (int)(t % H); const int s = (int)(t / H);
+        if (masks) {                                             // pixel filled from the cache
+            const size_t tile = ((size_t)s * tiles_y + y / DC_TILE_H) * tiles_x + x / DC_TILE_W;
+            const int bit = DC_TILE_BIT(y % DC_TILE_H, x % DC_TILE_W);
+            if ((masks[tile * 4 + (bit >> 5)] >> (bit & 31)) & 1u) continue;
+        }
         float sum = 0.f;
         for (int dy = -r; dy <= r; ++dy) {
             const int yy = y + dy;
@@ -347,7 +353,7 @@ int dc_launch_relu(dc_cache* c, int layer, const void* a)
     return DC_OK;
 }
 
-int dc_launch_lrn(dc_cache* c, int layer, const void* in)
+int dc_launch_lrn(dc_cache* c, int layer, const void* in, void* out, const uint32_t* masks)
 {
     dc_layer_rt& L = c->L[layer];
     const size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
@@ -357,8 +363,8 @@ int dc_launch_lrn(dc_cache* c, int layer, const void* in)
     const float kappa = (float)(defaults ? 1.0 : c->cfg.lrn_k);
     dc_prof_scope ps(c, DC_ST_POINTWISE);
     DISPATCH(c,
-        (k_lrn<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (float*)L.map[0])),
-        (k_lrn<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (__nv_bfloat16*)L.map[0])));
+        (k_lrn<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (float*)out, masks, L.tiles_x, L.tiles_y)),
+        (k_lrn<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (__nv_bfloat16*)out, masks, L.tiles_x, L.tiles_y)));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;

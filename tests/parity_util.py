@@ -86,7 +86,7 @@ def run_stream_parity(w, n_streams, frame_ids, check_layers=True, **kw):
                     for li, l in enumerate(w.layers):
                         regs, _ = dc.layer_regions(li)
                         assert_regions_equal(regions_np(regs[s, :n]), o["regions"][li], what + f" layer {li}")
-                        if l["kind"] == orc.KIND_CONV or (kw.get("cache_pool") and l["kind"] == orc.KIND_MAXPOOL):
+                        if l["kind"] == orc.KIND_CONV or (kw.get("cache_pool") and l["kind"] in (orc.KIND_MAXPOOL, orc.KIND_LRN)):
                             want_ratio = float(o["reused"][li].mean())
                             assert abs(stats[s].reuse_ratio[li] - want_ratio) < 1e-6, what + f" layer {li} reuse"
                 if check_layers:

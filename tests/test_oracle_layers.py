@@ -331,3 +331,17 @@ def test_graph_with_every_layer_kind_runs_and_reuses():
             assert a["reused"][0].any()                                          # first convolution reuses
             assert len(a["regions"][-1]) == 0 or not a["regions"][-1]["w"].any()  # Table 2: nothing reusable after FC
             assert np.abs(a["out"] - b["out"]).max() < 0.5
+
+
+def test_lrn_reuse_copies_rectangles_and_normalises_the_rest():
+    g = rng(35)
+    L = dict(kind=orc.KIND_LRN, kh=3, kw=3, sh=1, sw=1, ph=1, pw=1, cin=2, cout=2, relu=0, in0=-1, in1=-1, out_h=9, out_w=8)
+    x = g.normal(size=(9, 8, 2))
+    prev = g.normal(size=(9, 8, 2))
+    regions = np.zeros(2, orc.REGION_DTYPE)
+    regions[1] = (2, 3, 4, 5, 1, 2)
+    out, reused = orc.lrn_reuse(x, L, 0.1, 0.75, 1.0, orc.QUANT_NONE, prev, regions)
+    full = orc.lrn(x, L, 0.1, 0.75, 1.0, orc.QUANT_NONE)
+    mask = np.zeros((9, 8), bool); mask[3:8, 2:6] = True
+    assert np.array_equal(reused.astype(bool), mask)
+    assert np.array_equal(out[3:8, 2:6], prev[2:7, 1:5]) and np.array_equal(out[~mask], full[~mask])
