@@ -5,10 +5,11 @@
 //              (two aligned loads + funnel shift), |a-b| per byte by vabsdiff4, squares summed
 //              by dp4a, warp-reduced.  Candidates are ordered by (SSE, |dx|+|dy|, dy, dx).
 //              Blocks that pass the PSNR bound add their vector to the Step 3 sums.
-//   k_search_ds16  Step 2 for 16-pixel blocks with diamond search (the common case): one CTA per strip
-//              of 8 blocks, the previous frame's window (+-10 px) staged once in shared memory,
-//              each lane owns one block row, the two half-warps score two candidates at a time,
-//              and points already scored by the previous diamond are skipped (they cannot win).
+//   k_search_ds16q  Step 2 for 16-pixel blocks with diamond search (the common case): one CTA per 8 x 4
+//              blocks, the previous frame's window (+-10 px) staged once in shared memory; a warp walks
+//              8 blocks in lockstep, 4 lanes per block with 4 block rows each in registers, one candidate
+//              per block and pass; points already scored by the previous diamond are skipped (they cannot
+//              win).  Walks that leave the window continue in k_search_ds16q_long with private windows.
 //   k_verify   Steps 3-4: rounds the mean vector M, scores every block at M (reusing the Step 2
 //              score when the block's own best vector is M).
 //   k_merge_runs, k_merge   Step 5: maximal horizontal runs per block row, merged vertically when the
@@ -24,7 +25,7 @@ struct MatchArgs {
     const uint8_t* cur;  size_t cur_pitch;  size_t cur_stream;
     const uint8_t* prev; size_t prev_pitch; size_t prev_stream;
     int W, H, B, R, Gx, Gy, S, search, skip_k, region_mode;
-    int edge_only;                       // generic search: only blocks clipped by the frame edge (the rest has a fast kernel)
+    int edge_only;                       // generic search: 1 = only blocks clipped by the frame edge, 2 = only blocks clipped in width (the rest has a fast kernel)
     uint32_t limit[4];
     int16_t* mv; uint32_t* sse; uint8_t* matched; int32_t* acc; int32_t* gmv;
 };
@@ -99,7 +100,7 @@ __device__ __forceinline__ bool load_block(const MatchArgs& a, uint32_t* sm, Blo
     c.lane = threadIdx.x & 31;
     c.x0 = bx * a.B; c.y0 = by * a.B;
     c.bw = min(a.B, a.W - c.x0); c.bh = min(a.B, a.H - c.y0);
-    if (a.edge_only && c.bw == a.B && c.bh == a.B) return false;
+    if ((a.edge_only == 1 && c.bw == a.B && c.bh == a.B) || (a.edge_only == 2 && c.bw == a.B)) return false;
     c.W = a.W; c.H = a.H; c.R = a.R;
     c.prev = a.prev + (size_t)s * a.prev_stream; c.prev_pitch = a.prev_pitch;
     c.cur_sm = sm;
@@ -351,9 +352,6 @@ constexpr int F_WORDS = 120;                   // strip window row: (128 + 2 * 1
 constexpr int F_PITCH = 121;                   // odd word pitch: the 16 rows of a half-warp hit 16 banks
 constexpr int L_WORDS = 32;                    // private window row: (16 + 2 * 10) px * 3 B = 108 B + slack
 constexpr int L_PITCH = 33;
-constexpr int F_CANDS = 2;                     // candidates scored per pass (2: half-warp each, 4: quarter-warp each)
-constexpr int F_LPC = 32 / F_CANDS;            // lanes per candidate
-constexpr int F_NR = 16 / F_LPC;               // block rows per lane
 
 // NR rows (48 bytes each) of the current block per lane, masked for clipped edge blocks.
 template <int NR>
@@ -395,13 +393,13 @@ struct RowCtx {
         load(rows, bw, on);
     }
     // partial SSE of row k against 13 consecutive words at q, the row starting sh bits into q[0]
-    template <typename P>
+    template <bool CLIP = true, typename P>
     __device__ __forceinline__ uint32_t sse(int k, P q, uint32_t sh) const
     {
         uint32_t w[13], acc[3] = {0, 0, 0};                     // three chains hide the dp4a latency
 #pragma unroll
         for (int j = 0; j < 13; ++j) w[j] = q[j];
-        if (!clipped) {
+        if (!CLIP || !clipped) {
 #pragma unroll
             for (int j = 0; j < 12; ++j) {
                 uint32_t d = __vabsdiffu4(cw[k][j], __funnelshift_r(w[j], w[j + 1], sh));
@@ -418,93 +416,6 @@ struct RowCtx {
     }
 };
 
-// Search points relative to a centre: 0-7 the large diamond, 8 the centre itself, 9-12 the small diamond.
-__constant__ signed char kPointX[13] = {0, -1, 1, -2, 2, -1, 1, 0, 0, 0, -1, 1, 0};
-__constant__ signed char kPointY[13] = {-2, -1, -1, 0, 0, 1, 1, 2, 0, -1, 0, 0, 1};
-// After a move by (mx, my) (one of the 8 large-diamond offsets) the new large diamond overlaps the old
-// one; entry (my + 2) * 5 + (mx + 2) has bit j set for every point j of the new diamond that the old
-// diamond (its 8 points and its centre) did not contain.
-__constant__ unsigned char kNewPoints[25] = {0, 0, 31, 0, 0, 0, 11, 0, 21, 0, 171, 0, 0, 0, 213, 0, 168, 0, 208, 0, 0, 0, 248, 0, 0};
-
-// The diamond walk of one block by one warp.  `Win` supplies the staged previous-frame pixels:
-//   reach(cx, cy)      true when every point a step around centre (cx, cy) may touch is staged
-//   row(r, dx, dy, sh) pointer to the words holding row r of the candidate displaced by (dx, dy)
-// Returns false when the walk must continue elsewhere (bk then holds the state to resume from).
-template <typename Win>
-__device__ __forceinline__ bool diamond_walk(const MatchArgs& a, const RowCtx<F_NR>& rc, Win& win, int x0, int y0, int bw,
-                                             int bh, int lane, bool resume, unsigned long long& bk)
-{
-    const int r = lane & (F_LPC - 1), group = lane / F_LPC;       // lane owns block rows r, r + F_LPC, ...
-    // displacements that keep the block inside the previous frame and within the search range
-    const int dx_lo = max(-a.R, -x0), dy_lo = max(-a.R, -y0);
-    const unsigned dx_span = (unsigned)(min(a.R, a.W - bw - x0) - dx_lo), dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
-    uint32_t bs = (uint32_t)(bk >> 32), bt = (uint32_t)bk;        // best so far: SSE and tie-break word
-    // Scores the points of `mask` (bit i = point i around centre (cx, cy)), F_CANDS per pass: each
-    // group of F_LPC lanes takes one candidate, each lane F_NR block rows.  One call site keeps
-    // the code small.
-    auto score_points = [&](int cx, int cy, unsigned mask) {
-#pragma unroll 1
-        while (mask) {
-            int i = -1;
-#pragma unroll
-            for (int k = 0; k < F_CANDS; ++k) {
-                if (mask) {
-                    const int b = __ffs(mask) - 1; mask &= mask - 1;
-                    if (group == k) i = b;
-                }
-            }
-            const int ii = i < 0 ? 8 : i;
-            const int dx = cx + kPointX[ii], dy = cy + kPointY[ii];
-            // inside the frame and the range: one unsigned compare per axis against the block's valid span
-            const bool ok = i >= 0 && (unsigned)(dx - dx_lo) <= dx_span && (unsigned)(dy - dy_lo) <= dy_span;
-            uint32_t acc = 0;
-            if (ok) {
-                uint32_t sh;
-#pragma unroll
-                for (int k = 0; k < F_NR; ++k)
-                    if (rc.row_on[k]) { const uint32_t* q = win.row(r + k * F_LPC, dx, dy, sh); acc += rc.sse(k, q, sh); }
-            }
-            uint32_t ks = acc;                                     // sum over the candidate's lanes
-#pragma unroll
-            for (int off = F_LPC / 2; off > 0; off >>= 1) ks += __shfl_xor_sync(0xffffffffu, ks, off);
-            // candidate order (SSE, |dx| + |dy|, dy, dx) as two 32-bit words; all-ones = no candidate
-            uint32_t kt = ((uint32_t)(abs(dx) + abs(dy)) << 16) | ((uint32_t)(dy + 128) << 8) | (uint32_t)(dx + 128);
-            if (!ok) { ks = 0xffffffffu; kt = 0xffffffffu; }
-#pragma unroll
-            for (int off = F_LPC; off < 32; off <<= 1) {
-                const uint32_t os = __shfl_xor_sync(0xffffffffu, ks, off), ot = __shfl_xor_sync(0xffffffffu, kt, off);
-                if (os < ks || (os == ks && ot < kt)) { ks = os; kt = ot; }
-            }
-            if (ks < bs || (ks == bs && kt < bt)) { bs = ks; bt = kt; }
-        }
-    };
-    int cx, cy;
-    if (!resume) {
-        bs = 0xffffffffu; bt = 0xffffffffu;
-        cx = 0; cy = 0;
-        score_points(0, 0, 0x1ffu);                               // the centre (0, 0) and its large diamond
-    } else {
-        // resumed walk: the best point so far is the centre; score its whole large diamond
-        cx = (int)(bt & 0xff) - 128; cy = (int)((bt >> 8) & 0xff) - 128;
-        if (!win.reach(cx, cy)) return false;
-        score_points(cx, cy, 0xffu);
-    }
-    const int max_steps = (2 * a.R + 1) * (2 * a.R + 1);          // every move strictly lowers the key
-#pragma unroll 1
-    for (int step = 0; step < max_steps; ++step) {
-        const int nx = (int)(bt & 0xff) - 128, ny = (int)((bt >> 8) & 0xff) - 128;
-        if (nx == cx && ny == cy) break;                           // the centre won: large diamond done
-        if (!win.reach(nx, ny)) { bk = ((unsigned long long)bs << 32) | bt; return false; }
-        const int mx = nx - cx, my = ny - cy;
-        cx = nx; cy = ny;
-        // points of the new diamond that the old one already scored lost to the new centre: skip them
-        score_points(cx, cy, kNewPoints[(my + 2) * 5 + (mx + 2)]);
-    }
-    score_points(cx, cy, 0x1e00u);                                // small diamond around the final centre
-    bk = ((unsigned long long)bs << 32) | bt;
-    return true;
-}
-
 __device__ __forceinline__ void publish_block(const MatchArgs& a, int s, size_t g, int bw, int bh, unsigned long long bk)
 {
     const int fx = (int)(bk & 0xff) - 128, fy = (int)((bk >> 8) & 0xff) - 128;
@@ -517,64 +428,201 @@ __device__ __forceinline__ void publish_block(const MatchArgs& a, int s, size_t 
     }
 }
 
-// Window shared by the 8 blocks of a strip, centred on zero motion.
-struct StripWin {
-    const uint32_t* win; int x0, wx0;
+// ---------------------------------------------------------------------------------------------
+// Step 2 for 16-pixel blocks, diamond search, several blocks per warp
+// ---------------------------------------------------------------------------------------------
+// A warp walks 32 / LPB blocks in lockstep: LPB lanes share a block, each owning 16 / LPB of its rows
+// (kept in registers), and every pass scores ONE candidate per block.  The per-pass bookkeeping
+// (next point, bounds, addresses, best-so-far) is then paid once for 32 / LPB candidates instead of
+// once for two, and the sum over a candidate's rows needs log2(LPB) shuffles.  The search points and
+// the new-point masks are packed into immediates, so lanes that look up different entries do not
+// serialise on the constant cache.
+constexpr int kPX[13] = {0, -1, 1, -2, 2, -1, 1, 0, 0, 0, -1, 1, 0};
+constexpr int kPY[13] = {-2, -1, -1, 0, 0, 1, 1, 2, 0, -1, 0, 0, 1};
+constexpr int kNP[25] = {0, 0, 31, 0, 0, 0, 11, 0, 21, 0, 171, 0, 0, 0, 213, 0, 168, 0, 208, 0, 0, 0, 248, 0, 0};
+constexpr unsigned long long pack_nibbles(const int (&v)[13])
+{
+    unsigned long long r = 0;
+    for (int i = 0; i < 13; ++i) r |= (unsigned long long)(v[i] + 2) << (4 * i);
+    return r;
+}
+// new-point masks of the 8 possible moves; a move's table index (my + 2) * 5 + (mx + 2) is always even
+constexpr unsigned long long pack_moves(int first)
+{
+    unsigned long long r = 0;
+    for (int h = first; h < first + 8 && 2 * h < 25; ++h) r |= (unsigned long long)kNP[2 * h] << (8 * (h - first));
+    return r;
+}
+constexpr unsigned long long kPackX = pack_nibbles(kPX), kPackY = pack_nibbles(kPY);
+constexpr unsigned long long kMovesLo = pack_moves(0), kMovesHi = pack_moves(8);
+
+// st: 0 walking, 1 finished, 2 the walk left the staged window (resume elsewhere), 3 no block
+struct WalkState { int cx, cy, phase, st; uint32_t mask, bs, bt; };
+
+__device__ __forceinline__ void walk_begin(WalkState& w, bool on)
+{
+    w.cx = 0; w.cy = 0; w.phase = 0; w.st = on ? 0 : 3;
+    w.mask = on ? 0x1ffu : 0u;                                    // the centre (0, 0) and its large diamond
+    w.bs = 0xffffffffu; w.bt = 0xffffffffu;
+}
+// continue from the best point found so far, which becomes the centre of a whole large diamond
+__device__ __forceinline__ void walk_resume(WalkState& w)
+{
+    w.cx = (int)(w.bt & 0xff) - 128; w.cy = (int)((w.bt >> 8) & 0xff) - 128;
+    w.phase = 0; w.st = 0; w.mask = 0xffu;
+}
+
+// The walks of all blocks of a warp, until every one has finished or left its window.
+//   win.reach(cx, cy)      true when every point around centre (cx, cy) is staged
+//   win.row(r, dx, dy, sh) words holding row r of the candidate displaced by (dx, dy)
+// (dx_lo, dx_span), (dy_lo, dy_span): displacements that keep the block inside the previous frame and the range.
+template <int LPB, typename Win>
+__device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<16 / LPB>& rc, const Win& win, int q,
+                                              int dx_lo, unsigned dx_span, int dy_lo, unsigned dy_span, WalkState& w)
+{
+    constexpr int NR = 16 / LPB;
+    const int max_passes = 16 + 5 * (2 * a.R + 1) * (2 * a.R + 1);   // every move strictly lowers the key
+#pragma unroll 1
+    for (int pass = 0; pass < max_passes; ++pass) {
+        if (w.st == 0 && w.mask == 0) {
+            if (w.phase == 0) {
+                const int nx = (int)(w.bt & 0xff) - 128, ny = (int)((w.bt >> 8) & 0xff) - 128;
+                if (nx == w.cx && ny == w.cy) { w.phase = 1; w.mask = 0x1e00u; }    // centre won: small diamond
+                else if (!win.reach(nx, ny)) w.st = 2;
+                else {
+                    // points of the new diamond that the old one already scored lost to the new centre: skip them
+                    const int h = ((ny - w.cy + 2) * 5 + (nx - w.cx + 2)) >> 1;
+                    w.mask = (uint32_t)((h < 8 ? kMovesLo >> (8 * h) : kMovesHi >> (8 * (h - 8))) & 0xffu);
+                    w.cx = nx; w.cy = ny;
+                }
+            } else w.st = 1;
+        }
+        if (!__any_sync(0xffffffffu, w.st == 0)) break;
+        const bool run = w.st == 0;
+        const int i = run ? __ffs(w.mask) - 1 : 8;
+        w.mask &= w.mask - 1;
+        const int dx = w.cx + (int)((kPackX >> (4 * i)) & 7) - 2, dy = w.cy + (int)((kPackY >> (4 * i)) & 7) - 2;
+        const bool ok = run && (unsigned)(dx - dx_lo) <= dx_span && (unsigned)(dy - dy_lo) <= dy_span;
+        uint32_t ks = 0;
+        if (ok) {
+            // rows below a clipped block's last row hold zeros and are scored against staged words, then dropped:
+            // no branch between the rows, so their load / difference / accumulate chains interleave
+            uint32_t sh;
+#pragma unroll
+            for (int k = 0; k < NR; ++k) {
+                const uint32_t* p = win.row(q + k * LPB, dx, dy, sh);
+                const uint32_t v = rc.template sse<false>(k, p, sh);
+                ks += rc.row_on[k] ? v : 0u;
+            }
+        }
+#pragma unroll
+        for (int off = LPB / 2; off > 0; off >>= 1) ks += __shfl_xor_sync(0xffffffffu, ks, off);
+        const uint32_t kt = ((uint32_t)(abs(dx) + abs(dy)) << 16) | ((uint32_t)(dy + 128) << 8) | (uint32_t)(dx + 128);
+        if (ok && (ks < w.bs || (ks == w.bs && kt < w.bt))) { w.bs = ks; w.bt = kt; }
+    }
+}
+
+// Window shared by the VS x 8 blocks of a CTA; every block's reach is centred on zero motion.
+struct StackWin {
+    const uint32_t* win; int x0, wx0, row0;
     __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx) + 2 <= F_WR && abs(cy) + 2 <= F_WR; }
     __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
     {
         const int off = (x0 + dx) * 3 - wx0;
         sh = (off & 3) * 8;
-        return win + (r + dy + F_WR) * F_PITCH + (off >> 2);
+        return win + (row0 + r + dy + F_WR) * F_PITCH + (off >> 2);
     }
 };
 
-// Phase 1: one CTA per strip of 8 blocks.  A walk that leaves the strip window is handed to phase 2.
-__global__ void __launch_bounds__(256, 5) k_search_ds16(MatchArgs a, uint4* long_list, int32_t* long_count)
+// Phase 1: one CTA per 8 x VS blocks (VS strips stacked vertically share window rows), 32 / LPB blocks per
+// warp.  A walk that leaves the window is handed to phase 2.  Blocks clipped in width are left to the
+// generic kernel.  Launched without k-skip only (every block is searched).
+template <int LPB, int VS, int MINB>
+__global__ void __launch_bounds__(LPB * 8 * VS, MINB) k_search_ds16q(MatchArgs a, uint4* long_list, int32_t* long_count)
 {
-    __shared__ uint32_t win[F_ROWS * F_PITCH];
-    const int strips = (a.Gx + 7) >> 3;
-    const int strip = blockIdx.x % strips, by = (blockIdx.x / strips) % a.Gy, s = blockIdx.x / (strips * a.Gy);
-    const int xs = strip * 128, y0 = by * 16;
+    constexpr int THREADS = LPB * 8 * VS, ROWS = 16 * VS + 2 * F_WR, CHUNKS = ROWS * (F_WORDS / 4);
+    __shared__ uint32_t win[ROWS * F_PITCH];
+    const int strips = (a.Gx + 7) >> 3, vgroups = (a.Gy + VS - 1) / VS;
+    const int strip = blockIdx.x % strips, vg = (blockIdx.x / strips) % vgroups, s = blockIdx.x / (strips * vgroups);
+    const int xs = strip * 128, yb = vg * 16 * VS;
     const int wx0 = ((xs - F_WR) * 3) & ~15;                  // byte column of the window origin (may be < 0)
+    // this lane's block: LPB lanes per block, 8 blocks per strip, VS strips
+    const int lane = threadIdx.x & 31, q = lane % LPB;
+    const int blk = threadIdx.x / LPB, by = vg * VS + (blk >> 3), bx = strip * 8 + (blk & 7);
+    const bool in_grid = bx < a.Gx && by < a.Gy;
+    const int x0 = bx * 16, y0 = by * 16;
+    const bool searched = in_grid && a.W - x0 >= 16;
+    const int bw = searched ? 16 : 0, bh = searched ? min(16, a.H - y0) : 0;
+    RowCtx<16 / LPB> rc;                                      // issued first: in flight while the window is staged
+    rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)(searched ? y0 : 0) * a.cur_pitch + (size_t)(searched ? x0 : 0) * 3,
+                  a.cur_pitch, q, LPB, bw, bh);
     const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
-    const bool row_searched = a.skip_k <= 1 || by % a.skip_k == 0;
-    for (int i = threadIdx.x; row_searched && i < F_ROWS * (F_WORDS / 4); i += 256) {   // 16-byte chunks; wx0 and the pitch are 16-byte multiples
-        const int row = i / (F_WORDS / 4), ci = i - row * (F_WORDS / 4);
-        const int gy = y0 - F_WR + row, gb = wx0 + ci * 16;
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (gy >= 0 && gy < a.H && gb >= 0 && gb + 16 <= (int)a.prev_pitch)
-            v = __ldg((const uint4*)(prev + (size_t)gy * a.prev_pitch + gb));
-        uint32_t* d = win + row * F_PITCH + ci * 4;
-        d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    constexpr int UNR = 4;                                    // 16-byte chunks; wx0 and the pitch are 16-byte multiples
+    for (int i0 = threadIdx.x; i0 < CHUNKS; i0 += THREADS * UNR) {
+        uint4 v[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int i = i0 + u * THREADS, row = i / (F_WORDS / 4), ci = i - row * (F_WORDS / 4);
+            const int gy = yb - F_WR + row, gb = wx0 + ci * 16;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (i < CHUNKS && gy >= 0 && gy < a.H && gb >= 0 && gb + 16 <= (int)a.prev_pitch)
+                v[u] = __ldg((const uint4*)(prev + (size_t)gy * a.prev_pitch + gb));
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int i = i0 + u * THREADS, row = i / (F_WORDS / 4), ci = i - row * (F_WORDS / 4);
+            if (i < CHUNKS) {
+                uint32_t* d = win + row * F_PITCH + ci * 4;
+                d[0] = v[u].x; d[1] = v[u].y; d[2] = v[u].z; d[3] = v[u].w;
+            }
+        }
     }
     __syncthreads();
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int bx = strip * 8 + warp;
-    if (bx >= a.Gx) return;
-    if (a.skip_k > 1 && (bx % a.skip_k != 0 || by % a.skip_k != 0)) {      // Section 4, k-skip: not searched
-        if (lane == 0) {
-            const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
-            a.mv[2 * g] = 0; a.mv[2 * g + 1] = 0; a.sse[g] = 0xffffffffu;
-        }
-        return;
+    const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
+    const int dx_lo = max(-a.R, -x0), dy_lo = max(-a.R, -y0);
+    const unsigned dx_span = (unsigned)(min(a.R, a.W - bw - x0) - dx_lo), dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
+    StackWin sw = {win, x0, wx0, (blk >> 3) * 16};
+    WalkState w;
+    walk_begin(w, searched);
+    lockstep_walk<LPB>(a, rc, sw, q, dx_lo, dx_span, dy_lo, dy_span, w);
+    // finished blocks: results, and Step 3's sums once per warp (all blocks of a CTA belong to one stream)
+    const int fx = (int)(w.bt & 0xff) - 128, fy = (int)((w.bt >> 8) & 0xff) - 128;
+    const bool fin = searched && q == 0 && w.st != 2;
+    if (fin) { a.mv[2 * g] = (int16_t)fx; a.mv[2 * g + 1] = (int16_t)fy; a.sse[g] = w.bs; }
+    const bool pass = fin && w.bs <= a.limit[limit_index(a, bw, bh)];     // PSNR > T: member of Step 3's set S
+    const int n_pass = __popc(__ballot_sync(0xffffffffu, pass));
+    const int sum_x = __reduce_add_sync(0xffffffffu, pass ? fx : 0), sum_y = __reduce_add_sync(0xffffffffu, pass ? fy : 0);
+    if (lane == 0 && n_pass) {
+        atomicAdd(&a.acc[4 * s + 0], sum_x);
+        atomicAdd(&a.acc[4 * s + 1], sum_y);
+        atomicAdd(&a.acc[4 * s + 2], n_pass);
     }
-    const int x0 = bx * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
-    RowCtx<F_NR> rc;
-    rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, lane & (F_LPC - 1), F_LPC, bw, bh);
-    StripWin sw = {win, x0, wx0};
-    unsigned long long bk = 0;
-    const bool done = diamond_walk(a, rc, sw, x0, y0, bw, bh, lane, false, bk);
-    if (lane == 0) {
-        const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
-        if (done) publish_block(a, s, g, bw, bh, bk);
-        else long_list[atomicAdd(long_count, 1)] = make_uint4((uint32_t)g, (uint32_t)bk, (uint32_t)(bk >> 32), 0u);
+    const bool far = searched && q == 0 && w.st == 2;
+    const unsigned fm = __ballot_sync(0xffffffffu, far);
+    if (fm) {
+        int base = 0;
+        if (lane == 0) base = atomicAdd(long_count, __popc(fm));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (far) long_list[base + __popc(fm & ((1u << lane) - 1u))] = make_uint4((uint32_t)g, w.bt, w.bs, 0u);
     }
 }
 
-// Private window of one warp, centred on (wcx, wcy) relative to the block.
-struct WarpWin {
-    uint32_t* win; const uint8_t* prev; size_t pitch; int H, x0, y0, wcx, wcy, wx0, lane;
+// Section 4, k-skip: blocks that are not searched report vector (0, 0) and SSE 2^32 - 1.  One thread per block.
+__global__ void k_mark_unsearched(MatchArgs a)
+{
+    const int gi = blockIdx.x * blockDim.x + threadIdx.x;
+    if (gi >= a.S * a.Gx * a.Gy) return;
+    const int b = gi % (a.Gx * a.Gy), by = b / a.Gx, bx = b - by * a.Gx;
+    if (bx % a.skip_k != 0 || by % a.skip_k != 0) { a.mv[2 * gi] = 0; a.mv[2 * gi + 1] = 0; a.sse[gi] = 0xffffffffu; }
+}
+
+constexpr int P1_LPB = 4, P1_VS = 4;           // phase 1: 4 lanes per block (8 blocks per warp), 4 strips per CTA
+constexpr int P2_LPB = 16;                     // phase 2: 16 lanes per block; its 8 windows per CTA limit the resident warps,
+                                               // so fewer lanes per block would leave the SM short of warps
+
+// Private window of one block, centred on (wcx, wcy) relative to the block.
+struct BlockWin {
+    uint32_t* win; const uint8_t* prev; size_t pitch; int H, x0, y0, wcx, wcy, wx0;
     __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx - wcx) + 2 <= F_WR && abs(cy - wcy) + 2 <= F_WR; }
     __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
     {
@@ -582,48 +630,103 @@ struct WarpWin {
         sh = (off & 3) * 8;
         return win + (r + dy - wcy + F_WR) * L_PITCH + (off >> 2);
     }
-    __device__ __forceinline__ void stage(int cx, int cy)
+    // the block's LPB lanes fill the window around (cx, cy)
+    template <int LPB>
+    __device__ __forceinline__ void stage(int cx, int cy, int q)
     {
         wcx = cx; wcy = cy;
         wx0 = ((x0 + cx - F_WR) * 3) & ~15;
-        __syncwarp();
         static_assert(L_WORDS == 32, "8 chunks of 16 bytes per window row");
-        for (int i = lane; i < F_ROWS * 8; i += 32) {                 // wx0 and the pitch are 16-byte multiples
-            const int row = i >> 3, ci = i & 7;
-            const int gy = y0 + cy - F_WR + row, gb = wx0 + ci * 16;
-            uint4 v = make_uint4(0, 0, 0, 0);
-            if (gy >= 0 && gy < H && gb >= 0 && gb + 16 <= (int)pitch) v = __ldg((const uint4*)(prev + (size_t)gy * pitch + gb));
-            uint32_t* d = win + row * L_PITCH + ci * 4;
-            d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+        for (int i0 = q; i0 < F_ROWS * 8; i0 += LPB * 4) {            // wx0 and the pitch are 16-byte multiples
+            uint4 v[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * LPB, row = i >> 3, ci = i & 7;
+                const int gy = y0 + cy - F_WR + row, gb = wx0 + ci * 16;
+                v[u] = make_uint4(0, 0, 0, 0);
+                if (i < F_ROWS * 8 && gy >= 0 && gy < H && gb >= 0 && gb + 16 <= (int)pitch)
+                    v[u] = __ldg((const uint4*)(prev + (size_t)gy * pitch + gb));
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int i = i0 + u * LPB, row = i >> 3, ci = i & 7;
+                uint32_t* d = win + row * L_PITCH + ci * 4;
+                if (i < F_ROWS * 8) { d[0] = v[u].x; d[1] = v[u].y; d[2] = v[u].z; d[3] = v[u].w; }
+            }
         }
-        __syncwarp();
     }
 };
 
-// Phase 2: the walks that left their strip window, one warp each, re-staging a private window
-// around the walk's centre whenever it nears the window's edge.
-__global__ void __launch_bounds__(256, 4) k_search_ds16_long(MatchArgs a, const uint4* long_list, const int32_t* long_count)
+// Phase 2: the walks that left their window.  Each group of LPB lanes takes walks off the list one after the
+// other; a walk's private window is re-staged around its centre whenever it nears the window's edge.
+// 8 walks per CTA (LPB / 4 warps).
+// With k-skip (Section 4) the searched blocks lie k blocks apart and share no window: there is no phase 1 then,
+// and this kernel walks every searched full-width block from its start (long_list == nullptr; item i is the
+// i-th searched block in stream / row / column order).
+template <int LPB, int MINB>
+__global__ void __launch_bounds__(LPB * 8, MINB) k_search_ds16q_long(MatchArgs a, const uint4* long_list, const int32_t* long_count, int32_t* cursor)
 {
     __shared__ uint32_t win_all[8][F_ROWS * L_PITCH];
-    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int n = *long_count, per = a.Gx * a.Gy;
-    for (int i = blockIdx.x * 8 + warp; i < n; i += gridDim.x * 8) {
-        const uint4 e = long_list[i];
-        const size_t g = e.x;
-        unsigned long long bk = ((unsigned long long)e.z << 32) | e.y;
-        const int s = (int)(g / per), b = (int)(g - (size_t)s * per), by = b / a.Gx, bx = b - by * a.Gx;
-        const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
-        RowCtx<F_NR> rc;
-        rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, lane & (F_LPC - 1), F_LPC, bw, bh);
-        WarpWin ww = {win_all[warp], a.prev + (size_t)s * a.prev_stream, a.prev_pitch, a.H, x0, y0, 0, 0, 0, lane};
-        const int limit = 4 * a.R + 8;                           // each re-staging moves the centre >= 8 px
-        bool done = false;
-        for (int round = 0; round < limit && !done; ++round) {
-            ww.stage((int)(bk & 0xff) - 128, (int)((bk >> 8) & 0xff) - 128);
-            done = diamond_walk(a, rc, ww, x0, y0, bw, bh, lane, true, bk);
+    const int lane = threadIdx.x & 31, q = lane % LPB, qb = lane / LPB;
+    const int per = a.Gx * a.Gy;
+    const bool direct = long_list == nullptr;
+    const int sgx = (a.W / 16 + a.skip_k - 1) / a.skip_k, sgy = (a.Gy + a.skip_k - 1) / a.skip_k;   // searched columns (full width only), rows
+    const int n = direct ? a.S * sgx * sgy : *long_count;
+    bool fresh = false;
+    const int limit = 4 * a.R + 8;                                    // each re-staging moves the centre >= 8 px
+    WalkState w; walk_begin(w, false); w.st = 1;
+    RowCtx<16 / LPB> rc; rc.clipped = false; rc.row_bytes = 48;
+#pragma unroll
+    for (int k = 0; k < 16 / LPB; ++k) {
+        rc.row_on[k] = false;
+#pragma unroll
+        for (int j = 0; j < 12; ++j) rc.cw[k][j] = 0;
+    }
+    BlockWin bw_ = {win_all[threadIdx.x / LPB], nullptr, a.prev_pitch, a.H, 0, 0, 0, 0, 0};
+    int s = 0, bh = 16, rounds = 0, dx_lo = 0, dy_lo = 0; unsigned dx_span = 0, dy_span = 0; size_t g = 0;
+#pragma unroll 1
+    for (;;) {
+        const bool need = w.st == 1;
+        const unsigned m = __ballot_sync(0xffffffffu, need && q == 0);
+        if (m) {
+            const int leader = __ffs(m) - 1;
+            int base = 0;
+            if (lane == leader) base = atomicAdd(cursor, __popc(m));
+            base = __shfl_sync(0xffffffffu, base, leader);
+            const int idx = base + __popc(m & ((1u << (qb * LPB)) - 1u));
+            if (need) {
+                if (idx < n) {
+                    if (direct) {
+                        const int ss = idx / (sgx * sgy), r = idx - ss * sgx * sgy, sby = r / sgx, sbx = r - sby * sgx;
+                        g = (size_t)ss * per + (size_t)(sby * a.skip_k) * a.Gx + sbx * a.skip_k;
+                        fresh = true;
+                    } else {
+                        const uint4 e = long_list[idx];
+                        g = e.x; w.bt = e.y; w.bs = e.z;
+                    }
+                    s = (int)(g / per);
+                    const int b = (int)(g - (size_t)s * per), by = b / a.Gx, bx = b - by * a.Gx;
+                    const int x0 = bx * 16, y0 = by * 16;
+                    bh = min(16, a.H - y0);
+                    rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, q, LPB, 16, bh);
+                    bw_.prev = a.prev + (size_t)s * a.prev_stream; bw_.x0 = x0; bw_.y0 = y0;
+                    dx_lo = max(-a.R, -x0); dy_lo = max(-a.R, -y0);
+                    dx_span = (unsigned)(min(a.R, a.W - 16 - x0) - dx_lo); dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
+                    rounds = 0; w.st = 2;
+                } else w.st = 3;
+            }
+        }
+        if (!__any_sync(0xffffffffu, w.st == 2)) break;
+        __syncwarp();
+        if (w.st == 2) {
+            if (fresh) { bw_.stage<LPB>(0, 0, q); walk_begin(w, true); fresh = false; }
+            else { bw_.stage<LPB>((int)(w.bt & 0xff) - 128, (int)((w.bt >> 8) & 0xff) - 128, q); walk_resume(w); }
+            ++rounds;
         }
         __syncwarp();
-        if (lane == 0) publish_block(a, s, g, bw, bh, bk);
+        lockstep_walk<LPB>(a, rc, bw_, q, dx_lo, dx_span, dy_lo, dy_span, w);
+        if (w.st == 2 && rounds >= limit) w.st = 1;
+        if (w.st == 1 && q == 0) publish_block(a, s, g, 16, bh, ((unsigned long long)w.bs << 32) | w.bt);
     }
 }
 
@@ -864,13 +967,24 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
     DC_CUDA(cudaMemsetAsync(c->mv_acc, 0, sizeof(int32_t) * (4 * c->S + 4), c->stream));
     int32_t* long_count = c->mv_acc + 4 * c->S;
     if (a.B == 16 && a.search == DC_SEARCH_DIAMOND) {
-        dc_prof_scope ps(c, DC_ST_SEARCH);
-        k_search_ds16<<<((a.Gx + 7) / 8) * a.Gy * a.S, 256, 0, c->stream>>>(a, c->long_list, long_count);
-        int blocks = a.S * a.Gx * a.Gy;
-        int grid = dc_div_up(blocks, 8);
-        if (grid > c->num_sms * 4) grid = c->num_sms * 4;
-        k_search_ds16_long<<<grid, 256, 0, c->stream>>>(a, c->long_list, long_count);
-        c->launches += 1;
+        {
+            dc_prof_scope ps(c, DC_ST_SEARCH);
+            if (a.skip_k <= 1) {
+                const int ctas = ((a.Gx + 7) / 8) * ((a.Gy + P1_VS - 1) / P1_VS) * a.S;
+                k_search_ds16q<P1_LPB, P1_VS, 4><<<ctas, P1_LPB * 8 * P1_VS, 0, c->stream>>>(a, c->long_list, long_count);
+                k_search_ds16q_long<P2_LPB, 5><<<c->num_sms * 5, P2_LPB * 8, 0, c->stream>>>(a, c->long_list, long_count, long_count + 1);
+            } else {
+                k_mark_unsearched<<<dc_div_up(a.S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(a);
+                k_search_ds16q_long<P2_LPB, 5><<<c->num_sms * 5, P2_LPB * 8, 0, c->stream>>>(a, nullptr, long_count, long_count + 1);
+            }
+            c->launches += 1;
+        }
+        if (a.W % 16 != 0) {                                        // blocks clipped by the right edge
+            a.edge_only = 2;
+            launch_by_block(c, a, true);
+            a.edge_only = 0;
+            c->launches += 1;
+        }
     } else if (a.B == 16 && a.search == DC_SEARCH_EXHAUSTIVE && a.R <= E_MAXR && a.W >= 16 && a.H >= 16) {
         const int chunks = (2 * a.R + 1 + E_DY - 1) / E_DY;
         const size_t smem = ((size_t)(16 + chunks * E_DY - 1) * E_PITCH + 8 * 192) * sizeof(uint32_t);

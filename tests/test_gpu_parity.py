@@ -91,7 +91,10 @@ def test_match_full_hd_batch():
     """Workload 5's matcher geometry (1920x1080, block 16, range 32, last block row 8 px) on 2 streams."""
     w = configs.WORKLOADS[5]()
     sb = w.streams(2, 3)
-    check_pairs([(sb.frame(1, s), sb.frame(2, s)) for s in range(2)], 16, 32, B.DC_SEARCH_DIAMOND)
+    pairs = [(sb.frame(1, s), sb.frame(2, s)) for s in range(2)]
+    check_pairs(pairs, 16, 32, B.DC_SEARCH_DIAMOND)
+    # k-skip at this size: every searched block is walked with a private window from its start
+    check_pairs(pairs, 16, 32, B.DC_SEARCH_DIAMOND, skip_k=2)
 
 
 @pytest.mark.parametrize("widx,frames,R", [(2, (1, 2, 5), 16), (3, (1, 4), 7), (4, (2, 3), 24), (2, (3,), 1)])
