@@ -346,10 +346,8 @@ __global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const i
 // ---------------------------------------------------------------------------------------------
 // Fast Steps 2 and 4: 16-pixel blocks, diamond search
 // ---------------------------------------------------------------------------------------------
-constexpr int F_WR = 10;                       // reach of a staged window around a block, pixels
+constexpr int F_WR = 10;                       // reach of a block's private window, pixels
 constexpr int F_ROWS = 16 + 2 * F_WR;          // window rows
-constexpr int F_WORDS = 120;                   // strip window row: (128 + 2 * 10) px * 3 B = 444 B + alignment slack
-constexpr int F_PITCH = 121;                   // odd word pitch: the 16 rows of a half-warp hit 16 banks
 constexpr int L_WORDS = 32;                    // private window row: (16 + 2 * 10) px * 3 B = 108 B + slack
 constexpr int L_PITCH = 33;
 
@@ -476,7 +474,9 @@ __device__ __forceinline__ void walk_resume(WalkState& w)
 //   win.reach(cx, cy)      true when every point around centre (cx, cy) is staged
 //   win.row(r, dx, dy, sh) words holding row r of the candidate displaced by (dx, dy)
 // (dx_lo, dx_span), (dy_lo, dy_span): displacements that keep the block inside the previous frame and the range.
-template <int LPB, typename Win>
+// QUIT: a walk that is about to move while at most QUIT blocks of the warp are still walking gives up its
+//       place (st = 2, as if it had left the window), so that a few long walks do not hold the whole warp; 0 = never.
+template <int LPB, int QUIT, typename Win>
 __device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<16 / LPB>& rc, const Win& win, int q,
                                               int dx_lo, unsigned dx_span, int dy_lo, unsigned dy_span, WalkState& w)
 {
@@ -484,11 +484,13 @@ __device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<1
     const int max_passes = 16 + 5 * (2 * a.R + 1) * (2 * a.R + 1);   // every move strictly lowers the key
 #pragma unroll 1
     for (int pass = 0; pass < max_passes; ++pass) {
+        const unsigned walking = __ballot_sync(0xffffffffu, w.st == 0);
+        if (!walking) break;
         if (w.st == 0 && w.mask == 0) {
             if (w.phase == 0) {
                 const int nx = (int)(w.bt & 0xff) - 128, ny = (int)((w.bt >> 8) & 0xff) - 128;
                 if (nx == w.cx && ny == w.cy) { w.phase = 1; w.mask = 0x1e00u; }    // centre won: small diamond
-                else if (!win.reach(nx, ny)) w.st = 2;
+                else if (!win.reach(nx, ny) || (QUIT > 0 && __popc(walking) <= QUIT * LPB)) w.st = 2;
                 else {
                     // points of the new diamond that the old one already scored lost to the new centre: skip them
                     const int h = ((ny - w.cy + 2) * 5 + (nx - w.cx + 2)) >> 1;
@@ -497,7 +499,6 @@ __device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<1
                 }
             } else w.st = 1;
         }
-        if (!__any_sync(0xffffffffu, w.st == 0)) break;
         const bool run = w.st == 0;
         const int i = run ? __ffs(w.mask) - 1 : 8;
         w.mask &= w.mask - 1;
@@ -522,30 +523,36 @@ __device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<1
     }
 }
 
-// Window shared by the VS x 8 blocks of a CTA; every block's reach is centred on zero motion.
+// Window shared by the VS x 8 blocks of a CTA; every block may move WR pixels from zero motion inside it.
+// Row length: a candidate starts at most (112 + 2 WR) * 3 + 15 bytes into the row (15 = alignment of the
+// window's origin) and reads 13 words from the word that holds its first byte.
+template <int WR>
 struct StackWin {
+    static constexpr int WORDS = ((((112 + 2 * WR) * 3 + 15) >> 2) + 13 + 3) & ~3;   // staged in 16-byte chunks
+    static constexpr int PITCH = WORDS | 1;                    // odd: the rows of a block's lanes fall in different banks
     const uint32_t* win; int x0, wx0, row0;
-    __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx) + 2 <= F_WR && abs(cy) + 2 <= F_WR; }
+    __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx) + 2 <= WR && abs(cy) + 2 <= WR; }
     __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
     {
         const int off = (x0 + dx) * 3 - wx0;
         sh = (off & 3) * 8;
-        return win + (row0 + r + dy + F_WR) * F_PITCH + (off >> 2);
+        return win + (row0 + r + dy + WR) * PITCH + (off >> 2);
     }
 };
 
 // Phase 1: one CTA per 8 x VS blocks (VS strips stacked vertically share window rows), 32 / LPB blocks per
 // warp.  A walk that leaves the window is handed to phase 2.  Blocks clipped in width are left to the
 // generic kernel.  Launched without k-skip only (every block is searched).
-template <int LPB, int VS, int MINB>
+template <int LPB, int VS, int WR, int QUIT, int MINB>
 __global__ void __launch_bounds__(LPB * 8 * VS, MINB) k_search_ds16q(MatchArgs a, uint4* long_list, int32_t* long_count)
 {
-    constexpr int THREADS = LPB * 8 * VS, ROWS = 16 * VS + 2 * F_WR, CHUNKS = ROWS * (F_WORDS / 4);
-    __shared__ uint32_t win[ROWS * F_PITCH];
+    using Win = StackWin<WR>;
+    constexpr int THREADS = LPB * 8 * VS, ROWS = 16 * VS + 2 * WR, CPR = Win::WORDS / 4, CHUNKS = ROWS * CPR;
+    __shared__ uint32_t win[ROWS * Win::PITCH];
     const int strips = (a.Gx + 7) >> 3, vgroups = (a.Gy + VS - 1) / VS;
     const int strip = blockIdx.x % strips, vg = (blockIdx.x / strips) % vgroups, s = blockIdx.x / (strips * vgroups);
     const int xs = strip * 128, yb = vg * 16 * VS;
-    const int wx0 = ((xs - F_WR) * 3) & ~15;                  // byte column of the window origin (may be < 0)
+    const int wx0 = ((xs - WR) * 3) & ~15;                  // byte column of the window origin (may be < 0)
     // this lane's block: LPB lanes per block, 8 blocks per strip, VS strips
     const int lane = threadIdx.x & 31, q = lane % LPB;
     const int blk = threadIdx.x / LPB, by = vg * VS + (blk >> 3), bx = strip * 8 + (blk & 7);
@@ -562,17 +569,17 @@ __global__ void __launch_bounds__(LPB * 8 * VS, MINB) k_search_ds16q(MatchArgs a
         uint4 v[UNR];
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            const int i = i0 + u * THREADS, row = i / (F_WORDS / 4), ci = i - row * (F_WORDS / 4);
-            const int gy = yb - F_WR + row, gb = wx0 + ci * 16;
+            const int i = i0 + u * THREADS, row = i / CPR, ci = i - row * CPR;
+            const int gy = yb - WR + row, gb = wx0 + ci * 16;
             v[u] = make_uint4(0, 0, 0, 0);
             if (i < CHUNKS && gy >= 0 && gy < a.H && gb >= 0 && gb + 16 <= (int)a.prev_pitch)
                 v[u] = __ldg((const uint4*)(prev + (size_t)gy * a.prev_pitch + gb));
         }
 #pragma unroll
         for (int u = 0; u < UNR; ++u) {
-            const int i = i0 + u * THREADS, row = i / (F_WORDS / 4), ci = i - row * (F_WORDS / 4);
+            const int i = i0 + u * THREADS, row = i / CPR, ci = i - row * CPR;
             if (i < CHUNKS) {
-                uint32_t* d = win + row * F_PITCH + ci * 4;
+                uint32_t* d = win + row * Win::PITCH + ci * 4;
                 d[0] = v[u].x; d[1] = v[u].y; d[2] = v[u].z; d[3] = v[u].w;
             }
         }
@@ -581,10 +588,10 @@ __global__ void __launch_bounds__(LPB * 8 * VS, MINB) k_search_ds16q(MatchArgs a
     const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
     const int dx_lo = max(-a.R, -x0), dy_lo = max(-a.R, -y0);
     const unsigned dx_span = (unsigned)(min(a.R, a.W - bw - x0) - dx_lo), dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
-    StackWin sw = {win, x0, wx0, (blk >> 3) * 16};
+    const Win sw = {win, x0, wx0, (blk >> 3) * 16};
     WalkState w;
     walk_begin(w, searched);
-    lockstep_walk<LPB>(a, rc, sw, q, dx_lo, dx_span, dy_lo, dy_span, w);
+    lockstep_walk<LPB, QUIT>(a, rc, sw, q, dx_lo, dx_span, dy_lo, dy_span, w);
     // finished blocks: results, and Step 3's sums once per warp (all blocks of a CTA belong to one stream)
     const int fx = (int)(w.bt & 0xff) - 128, fy = (int)((w.bt >> 8) & 0xff) - 128;
     const bool fin = searched && q == 0 && w.st != 2;
@@ -617,6 +624,8 @@ __global__ void k_mark_unsearched(MatchArgs a)
 }
 
 constexpr int P1_LPB = 4, P1_VS = 4;           // phase 1: 4 lanes per block (8 blocks per warp), 4 strips per CTA
+constexpr int P1_WR = 10;                      // phase 1 follows a walk up to 8 px from zero motion
+constexpr int P1_QUIT = 2;                     // ... and hands over the last two walks of a warp at their next move
 constexpr int P2_LPB = 16;                     // phase 2: 16 lanes per block; its 8 windows per CTA limit the resident warps,
                                                // so fewer lanes per block would leave the SM short of warps
 
@@ -724,7 +733,7 @@ __global__ void __launch_bounds__(LPB * 8, MINB) k_search_ds16q_long(MatchArgs a
             ++rounds;
         }
         __syncwarp();
-        lockstep_walk<LPB>(a, rc, bw_, q, dx_lo, dx_span, dy_lo, dy_span, w);
+        lockstep_walk<LPB, 0>(a, rc, bw_, q, dx_lo, dx_span, dy_lo, dy_span, w);
         if (w.st == 2 && rounds >= limit) w.st = 1;
         if (w.st == 1 && q == 0) publish_block(a, s, g, 16, bh, ((unsigned long long)w.bs << 32) | w.bt);
     }
@@ -971,7 +980,7 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
             dc_prof_scope ps(c, DC_ST_SEARCH);
             if (a.skip_k <= 1) {
                 const int ctas = ((a.Gx + 7) / 8) * ((a.Gy + P1_VS - 1) / P1_VS) * a.S;
-                k_search_ds16q<P1_LPB, P1_VS, 4><<<ctas, P1_LPB * 8 * P1_VS, 0, c->stream>>>(a, c->long_list, long_count);
+                k_search_ds16q<P1_LPB, P1_VS, P1_WR, P1_QUIT, 4><<<ctas, P1_LPB * 8 * P1_VS, 0, c->stream>>>(a, c->long_list, long_count);
                 k_search_ds16q_long<P2_LPB, 5><<<c->num_sms * 5, P2_LPB * 8, 0, c->stream>>>(a, c->long_list, long_count, long_count + 1);
             } else {
                 k_mark_unsearched<<<dc_div_up(a.S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(a);
