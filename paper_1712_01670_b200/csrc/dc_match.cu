@@ -463,11 +463,21 @@ __device__ __forceinline__ void walk_begin(WalkState& w, bool on)
     w.mask = on ? 0x1ffu : 0u;                                    // the centre (0, 0) and its large diamond
     w.bs = 0xffffffffu; w.bt = 0xffffffffu;
 }
-// continue from the best point found so far, which becomes the centre of a whole large diamond
+// points of the large diamond around a new centre that the diamond around the old one did not contain:
+// the others lost to the new centre already and cannot win (mx, my: the move, one of the 8 diamond offsets)
+__device__ __forceinline__ uint32_t new_points(int mx, int my)
+{
+    const int h = ((my + 2) * 5 + (mx + 2)) >> 1;
+    return (uint32_t)((h < 8 ? kMovesLo >> (8 * h) : kMovesHi >> (8 * (h - 8))) & 0xffu);
+}
+// A walk that stopped with st = 2 had chosen its next centre (the best point so far) but not moved yet:
+// make that move now, exactly as the uninterrupted walk would have.
 __device__ __forceinline__ void walk_resume(WalkState& w)
 {
-    w.cx = (int)(w.bt & 0xff) - 128; w.cy = (int)((w.bt >> 8) & 0xff) - 128;
-    w.phase = 0; w.st = 0; w.mask = 0xffu;
+    const int nx = (int)(w.bt & 0xff) - 128, ny = (int)((w.bt >> 8) & 0xff) - 128;
+    w.mask = new_points(nx - w.cx, ny - w.cy);
+    w.cx = nx; w.cy = ny;
+    w.phase = 0; w.st = 0;
 }
 
 // The walks of all blocks of a warp, until every one has finished or left its window.
@@ -492,9 +502,7 @@ __device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<1
                 if (nx == w.cx && ny == w.cy) { w.phase = 1; w.mask = 0x1e00u; }    // centre won: small diamond
                 else if (!win.reach(nx, ny) || (QUIT > 0 && __popc(walking) <= QUIT * LPB)) w.st = 2;
                 else {
-                    // points of the new diamond that the old one already scored lost to the new centre: skip them
-                    const int h = ((ny - w.cy + 2) * 5 + (nx - w.cx + 2)) >> 1;
-                    w.mask = (uint32_t)((h < 8 ? kMovesLo >> (8 * h) : kMovesHi >> (8 * (h - 8))) & 0xffu);
+                    w.mask = new_points(nx - w.cx, ny - w.cy);
                     w.cx = nx; w.cy = ny;
                 }
             } else w.st = 1;
@@ -610,7 +618,7 @@ __global__ void __launch_bounds__(LPB * 8 * VS, MINB) k_search_ds16q(MatchArgs a
         int base = 0;
         if (lane == 0) base = atomicAdd(long_count, __popc(fm));
         base = __shfl_sync(0xffffffffu, base, 0);
-        if (far) long_list[base + __popc(fm & ((1u << lane) - 1u))] = make_uint4((uint32_t)g, w.bt, w.bs, 0u);
+        if (far) long_list[base + __popc(fm & ((1u << lane) - 1u))] = make_uint4((uint32_t)g, w.bt, w.bs, (uint32_t)(w.cx + 128) | ((uint32_t)(w.cy + 128) << 8));   // block, best point, centre it was found from
     }
 }
 
@@ -712,6 +720,7 @@ __global__ void __launch_bounds__(LPB * 8, MINB) k_search_ds16q_long(MatchArgs a
                     } else {
                         const uint4 e = long_list[idx];
                         g = e.x; w.bt = e.y; w.bs = e.z;
+                        w.cx = (int)(e.w & 0xff) - 128; w.cy = (int)((e.w >> 8) & 0xff) - 128;
                     }
                     s = (int)(g / per);
                     const int b = (int)(g - (size_t)s * per), by = b / a.Gx, bx = b - by * a.Gx;
