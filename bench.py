@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--cache-pool", action="store_true", help="also cache and reuse max-pooling outputs (Section 5's extension)")
     ap.add_argument("--per-block-regions", action="store_true", help="rectangles carry their blocks' own vectors (extension)")
     ap.add_argument("--no-lookahead", action="store_true", help="do not overlap the next frame's matching with this frame's inference")
+    ap.add_argument("--matcher-only", action="store_true",
+                    help="time Steps 1-5 alone (dc_cache_set_key + dc_match_blocks per step) and print a short JSON line; "
+                         "a small, single-purpose run for profiling the matcher kernels")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -227,6 +230,28 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
             dist.barrier()
         torch.cuda.synchronize()
 
+    if args.matcher_only:
+        for i in range(1, args.warmup + 1):
+            B.dc_cache_set_key(dc.handle, dev_frames[max(i - 1, 0)], pitch)
+            B.dc_match_blocks(dc.handle, dev_frames[i], pitch)
+        barrier()
+        m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        m0.record()
+        for i in range(args.warmup, total):
+            B.dc_cache_set_key(dc.handle, dev_frames[max(i - 1, 0)], pitch)
+            B.dc_match_blocks(dc.handle, dev_frames[i], pitch)
+        m1.record()
+        barrier()
+        ms = m0.elapsed_time(m1) / args.steps
+        if rank == 0:
+            print(json.dumps({"stage": "matcher (key copy, frame copy, Steps 2-5)", "ms_per_step": ms, "streams": S,
+                              "steps": args.steps, "warmup": args.warmup, "config": workload_config(w, S, world),
+                              "algorithmic_gbs": 4.0 * frame_bytes * S / (ms * 1e-3) / 1e9}))
+        dc.close()
+        if world > 1:
+            dist.destroy_process_group()
+        return
+
     # ---- device-resident timing: value ----
     # The loop a user runs: infer frame t, then announce frame t+1 so that its matching runs on a side stream
     # beside the convolutions of frame t (dc_lookahead_frame; results are identical without it).
@@ -346,7 +371,7 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
     conv_peak = peaks["bf16_tflops_sustained"] if bf16 else None
     # DRAM bytes per convolution launch from the ncu capture summarised in profiles/dram_traffic_batched_stress.md
     # (32 streams of workload 5, kernels as committed with that file); other shapes were not captured
-    conv_traffic = 78.0e6 if (w.index == 5 and S == 32 and bf16 and not args.cache_pool) else None
+    conv_traffic = 77.8e6 if (w.index == 5 and S == 32 and bf16 and not args.cache_pool) else None
     roofline = {"kernel": "partial convolution (all conv launches of the timed region)",
                 "bound": "tensor" if bf16 else "alu", "achieved": conv_tflops,
                 "peak": conv_peak, "unit": "TFLOP/s", "frac": (conv_tflops / conv_peak) if conv_peak else None,
@@ -360,7 +385,7 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
     roofline_matcher = {"kernel": "block search + verify", "bound": "hbm", "achieved": match_gbs,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": match_gbs / peaks["hbm_gbs"],
                         "peak_source": f"hbm_gbs, {peaks['source']}",
-                        "traffic": 942.0e6 if (w.index == 5 and S == 32 and w.search == 1 and args.skip_k == 1) else None,
+                        "traffic": 936.0e6 if (w.index == 5 and S == 32 and w.search == 1 and args.skip_k == 1) else None,
                         "traffic_unit": "bytes per batch-frame (search + long walks + verify; dram read + write, ncu)",
                         "launches": prof["search"][1] + prof["verify"][1],
                         "bytes_per_frame_batch": 4.0 * frame_bytes * S}
