@@ -137,6 +137,20 @@ __global__ void k_maxpool_vec(const T* in, int Hi, int Wi, int C, int S, dc_laye
     }
 }
 
+// 2 x 2 windows at stride 2 without padding (every window inside the map), no reuse bitmap: the four 16-byte
+// loads of an output vector are independent and issued together; 32-bit index arithmetic.
+template <typename T>
+__global__ void k_maxpool2x2_vec(const uint4* in, int Hi, int Wi, int cv, int out_h, int out_w, unsigned total, uint4* out)
+{
+    for (unsigned i = blockIdx.x * blockDim.x + threadIdx.x; i < total; i += gridDim.x * blockDim.x) {
+        const unsigned c = i % cv, t = i / cv, ox = t % out_w, u = t / out_w, oy = u % out_h, s = u / out_h;
+        const uint4* p = in + (((size_t)s * Hi + 2 * oy) * Wi + 2 * ox) * cv + c;
+        const size_t row = (size_t)Wi * cv;
+        const uint4 v00 = __ldg(p), v01 = __ldg(p + cv), v10 = __ldg(p + row), v11 = __ldg(p + row + cv);
+        out[i] = Vec16<T>::vmax(Vec16<T>::vmax(v00, v01), Vec16<T>::vmax(v10, v11));
+    }
+}
+
 template <typename T>
 __global__ void k_maxpool(const T* in, int Hi, int Wi, int C, int S, dc_layer_desc L, T* out)
 {
@@ -295,6 +309,17 @@ int dc_launch_maxpool(dc_cache* c, int layer, const void* in, void* out, const u
     dc_layer_rt& L = c->L[layer];
     size_t n = (size_t)c->S * L.d.out_h * L.d.out_w * L.d.cout;
     dc_prof_scope ps(c, DC_ST_POINTWISE);
+    if ((L.d.cout * c->elt) % 16 == 0 && !masks && L.d.kh == 2 && L.d.kw == 2 && L.d.sh == 2 && L.d.sw == 2 && L.d.ph == 0 &&
+        L.d.pw == 0 && 2 * L.d.out_h <= L.in_h && 2 * L.d.out_w <= L.in_w && n * c->elt / 16 < 0x7fffffffull) {
+        const unsigned nv = (unsigned)(n * c->elt / 16);
+        const int cv = L.d.cout * c->elt / 16;
+        DISPATCH(c,
+            (k_maxpool2x2_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)in, L.in_h, L.in_w, cv, L.d.out_h, L.d.out_w, nv, (uint4*)out)),
+            (k_maxpool2x2_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)in, L.in_h, L.in_w, cv, L.d.out_h, L.d.out_w, nv, (uint4*)out)));
+        c->launches += 1;
+        DC_CUDA(cudaGetLastError());
+        return DC_OK;
+    }
     if ((L.d.cout * c->elt) % 16 == 0) {
         size_t nv = n * c->elt / 16;
         DISPATCH(c,
