@@ -394,9 +394,16 @@ struct RowCtx {
     template <bool CLIP = true, typename P>
     __device__ __forceinline__ uint32_t sse(int k, P q, uint32_t sh) const
     {
-        uint32_t w[13], acc[3] = {0, 0, 0};                     // three chains hide the dp4a latency
+        uint32_t w[13];
 #pragma unroll
         for (int j = 0; j < 13; ++j) w[j] = q[j];
+        return sse_words<CLIP>(k, w, sh);
+    }
+    // the same on 13 words already in registers
+    template <bool CLIP = true>
+    __device__ __forceinline__ uint32_t sse_words(int k, const uint32_t (&w)[13], uint32_t sh) const
+    {
+        uint32_t acc[3] = {0, 0, 0};                            // three chains hide the dp4a latency
         if (!CLIP || !clipped) {
 #pragma unroll
             for (int j = 0; j < 12; ++j) {
@@ -758,9 +765,10 @@ __global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
     const int s = in_grid ? (int)(gi / (unsigned)per) : 0, b = in_grid ? (int)(gi - (unsigned)s * per) : 0;
     const int by = b / a.Gx, bx = b - by * a.Gx;
     const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
-    const int K = a.acc[4 * s + 2];
+    const int4 sums = __ldcg((const int4*)a.acc + s);                            // Step 3: sum dx, sum dy, K (one 16-byte load)
+    const int K = sums.z;
     int Mx = 0, My = 0;
-    if (K > 0) { Mx = round_mean(a.acc[4 * s + 0], K); My = round_mean(a.acc[4 * s + 1], K); }
+    if (K > 0) { Mx = round_mean(sums.x, K); My = round_mean(sums.y, K); }
     const bool cand_ok = in_grid && K > 0 && abs(Mx) <= a.R && abs(My) <= a.R && x0 + Mx >= 0 && y0 + My >= 0 &&
                          x0 + Mx + bw <= a.W && y0 + My + bh <= a.H;
     const size_t g = (size_t)s * per + b;
@@ -770,16 +778,55 @@ __global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
     if (cand_ok && !known && r < bh) {
         RowCtx<1> rc;
         rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, r, 16, bw, bh);
+        // the 48 bytes of the displaced row lie in four aligned 16-byte chunks (rows of the frame copy are padded):
+        // four wide loads instead of thirteen narrow ones, then a word offset that is the same for a whole stream
         const uint8_t* p = a.prev + (size_t)s * a.prev_stream + (size_t)(y0 + My + r) * a.prev_pitch + (size_t)(x0 + Mx) * 3;
-        acc = rc.sse(0, (const uint32_t*)((uintptr_t)p & ~(uintptr_t)3), ((uint32_t)(uintptr_t)p & 3u) * 8u);
+        const uint4* p16 = (const uint4*)((uintptr_t)p & ~(uintptr_t)15);
+        const uint4 c0 = __ldg(p16), c1 = __ldg(p16 + 1), c2 = __ldg(p16 + 2), c3 = __ldg(p16 + 3);
+        const uint32_t ww[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
+        const uint32_t boff = (uint32_t)(uintptr_t)p & 15u, sh = (boff & 3u) * 8u;
+        uint32_t w[13];
+        switch (boff >> 2) {
+        case 0:
+#pragma unroll
+            for (int j = 0; j < 13; ++j) w[j] = ww[j];
+            break;
+        case 1:
+#pragma unroll
+            for (int j = 0; j < 13; ++j) w[j] = ww[j + 1];
+            break;
+        case 2:
+#pragma unroll
+            for (int j = 0; j < 13; ++j) w[j] = ww[j + 2];
+            break;
+        default:
+#pragma unroll
+            for (int j = 0; j < 13; ++j) w[j] = ww[j + 3];
+            break;
+        }
+        acc = rc.sse_words(0, w, sh);
     }
     const uint32_t sse = __reduce_add_sync(half ? 0xffff0000u : 0x0000ffffu, acc);
+    int ok = 0;
     if (r == 0 && in_grid) {
         const uint32_t v = known ? a.sse[g] : sse;
-        const int ok = cand_ok && v <= a.limit[limit_index(a, bw, bh)];
+        ok = cand_ok && v <= a.limit[limit_index(a, bw, bh)];
         a.matched[g] = (uint8_t)ok;
-        if (ok) atomicAdd(&a.acc[4 * s + 3], 1);
         if (b == 0) { a.gmv[3 * s] = Mx; a.gmv[3 * s + 1] = My; a.gmv[3 * s + 2] = K; }
+    }
+    // count of matched blocks: one atomic per CTA and stream (the sums above share its 16 bytes, so every
+    // atomic saved also shortens the other CTAs' loads of them)
+    if (per < 16) {                                                               // tiny frames: a CTA may span many streams
+        if (ok) atomicAdd(&a.acc[4 * s + 3], 1);
+        return;
+    }
+    const unsigned first = blockIdx.x * 16u, last = min(first + 15u, (unsigned)(per * a.S) - 1u);
+    const int s_first = (int)(first / (unsigned)per), s_last = (int)(last / (unsigned)per);
+    const int n_first = __syncthreads_count(ok && s == s_first);
+    if (threadIdx.x == 0 && n_first) atomicAdd(&a.acc[4 * s_first + 3], n_first);
+    if (s_last != s_first) {                                                      // the CTA's 16 blocks span two streams
+        const int n_last = __syncthreads_count(ok && s != s_first);
+        if (threadIdx.x == 0 && n_last) atomicAdd(&a.acc[4 * s_last + 3], n_last);
     }
 }
 
