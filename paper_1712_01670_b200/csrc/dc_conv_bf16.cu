@@ -507,7 +507,14 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
                  ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
 }
 
-template <int MT>
+// SLAB = false: the A side of a 64-channel chunk is one (16 + kh - 1) x (8 + kw - 1) patch in eight 16-byte planes
+//               (unswizzled core matrices), read in place by every tap.
+// SLAB = true:  the A side of a (chunk, kx) pair is one column slab: the (16 + kh - 1) x 8 pixels of the tile's
+//               columns displaced by kx, 128 bytes (64 channels) per pixel, 128-byte swizzled.  The eight pixels of
+//               a tile row are one 1024-byte swizzle atom, so tap (ky, kx) is the slab from atom ky on: a plain
+//               K-major tile.  kw loads of whole 128-byte rows per chunk instead of kh * kw (tap by tap) or eight
+//               loads of 16-byte rows (patch).  ha.patch_bytes then holds the bytes of one slab.
+template <int MT, bool SLAB>
 __global__ void __launch_bounds__(kThreads, 1)
 k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
 {
@@ -516,7 +523,8 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
     const int n_tiles = *a.tile_count;
     const int n_items = (n_tiles + MT - 1) / MT * a.NB;
     if ((int)blockIdx.x >= n_items) return;
-    uint8_t* aring = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    constexpr uintptr_t kAlign = SLAB ? 1023 : 127;           // swizzle atoms start on 1024-byte boundaries
+    uint8_t* aring = (uint8_t*)(((uintptr_t)smem_raw + kAlign) & ~kAlign);
     const int a_slot = MT * ha.patch_bytes;
     uint8_t* bring = aring + (size_t)ha.a_stages * a_slot;
     SmemCtl* ctl = (SmemCtl*)(bring + (size_t)a.stages * a.b_bytes);
@@ -556,30 +564,42 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
                 sN[j] = s; xb[j] = tx * DC_TILE_W - a.pw; yb[j] = ty * DC_TILE_H - a.ph;
             }
             for (int cc = 0; cc < a.kchunks && ok; ++cc) {
-                if (lane == 0) {
-                    ok = mbar_wait(&ctl->a_empty[sa], pa ^ 1u, ctl, a.status);
-                    if (ok) {
-                        mbar_expect_tx(&ctl->a_full[sa], (uint32_t)(MT * 8 * ha.PW * ha.PH * 16));
-#pragma unroll
-                        for (int j = 0; j < MT; ++j)
-                            for (int g = 0; g < 8; ++g)
-                                tma_load_4d(aring + (size_t)sa * a_slot + j * ha.patch_bytes + g * ha.plane_bytes, &tmA,
-                                            cc * 64 + g * 8, xb[j], yb[j], sN[j], &ctl->a_full[sa]);
-                    }
-                }
-                ok = __shfl_sync(0xffffffffu, ok, 0);
-                if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
-                for (int tap = 0; tap < taps && ok; ++tap) {
+                for (int kx = 0; kx < (SLAB ? a.kw : 1) && ok; ++kx) {
                     if (lane == 0) {
-                        ok = mbar_wait(&ctl->empty[sb], pb ^ 1u, ctl, a.status);
+                        ok = mbar_wait(&ctl->a_empty[sa], pa ^ 1u, ctl, a.status);
                         if (ok) {
-                            mbar_expect_tx(&ctl->full[sb], (uint32_t)a.b_bytes);
-                            const uint8_t* src = (const uint8_t*)ha.wpacked + ((size_t)(nb * taps + tap) * a.kchunks + cc) * a.b_bytes;
-                            bulk_copy_g2s(bring + (size_t)sb * a.b_bytes, src, (uint32_t)a.b_bytes, &ctl->full[sb]);
+                            if (SLAB) {
+                                mbar_expect_tx(&ctl->a_full[sa], (uint32_t)(MT * ha.patch_bytes));
+#pragma unroll
+                                for (int j = 0; j < MT; ++j)
+                                    tma_load_4d(aring + (size_t)sa * a_slot + j * ha.patch_bytes, &tmA, cc * 64, xb[j] + kx, yb[j], sN[j],
+                                                &ctl->a_full[sa]);
+                            } else {
+                                mbar_expect_tx(&ctl->a_full[sa], (uint32_t)(MT * 8 * ha.PW * ha.PH * 16));
+#pragma unroll
+                                for (int j = 0; j < MT; ++j)
+                                    for (int g = 0; g < 8; ++g)
+                                        tma_load_4d(aring + (size_t)sa * a_slot + j * ha.patch_bytes + g * ha.plane_bytes, &tmA,
+                                                    cc * 64 + g * 8, xb[j], yb[j], sN[j], &ctl->a_full[sa]);
+                            }
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (++sb == a.stages) { sb = 0; pb ^= 1u; }
+                    if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
+                    // the weight tiles that go with this A stage: all taps (patch), or the taps of column kx (slab)
+                    for (int t = 0; t < (SLAB ? a.kh : taps) && ok; ++t) {
+                        const int tap = SLAB ? t * a.kw + kx : t;
+                        if (lane == 0) {
+                            ok = mbar_wait(&ctl->empty[sb], pb ^ 1u, ctl, a.status);
+                            if (ok) {
+                                mbar_expect_tx(&ctl->full[sb], (uint32_t)a.b_bytes);
+                                const uint8_t* src = (const uint8_t*)ha.wpacked + ((size_t)(nb * taps + tap) * a.kchunks + cc) * a.b_bytes;
+                                bulk_copy_g2s(bring + (size_t)sb * a.b_bytes, src, (uint32_t)a.b_bytes, &ctl->full[sb]);
+                            }
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (++sb == a.stages) { sb = 0; pb ^= 1u; }
+                    }
                 }
             }
         }
@@ -588,11 +608,13 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
         // ---------------- MMA issuer (lane 0 only) ----------------
         if (lane == 0) {
             const uint32_t b_lbo = (uint32_t)a.BN * 16u;
-            const uint64_t aconst = umma_desc(0, (uint32_t)ha.PW * 16u, 0, (uint32_t)ha.plane_bytes);
+            // A: patch planes (rows PW * 16 bytes apart, planes along K), or a 128-byte swizzled K-major slab
+            const uint64_t aconst = SLAB ? umma_desc(0, 1024, 2) : umma_desc(0, (uint32_t)ha.PW * 16u, 0, (uint32_t)ha.plane_bytes);
             const uint64_t bconst = umma_desc(0, 128, 0, b_lbo);
             const uint32_t aring_lo = smem_u32(aring) >> 4, bring_lo = smem_u32(bring) >> 4;
             const uint32_t a_slot_lo = (uint32_t)a_slot >> 4, patch_lo = (uint32_t)ha.patch_bytes >> 4;
-            const uint32_t a_kstep = (uint32_t)(2 * ha.plane_bytes) >> 4, b_kstep = (2 * b_lbo) >> 4, b_lo = (uint32_t)a.b_bytes >> 4;
+            const uint32_t a_kstep = SLAB ? 2u : (uint32_t)(2 * ha.plane_bytes) >> 4;    // 16 channels further along K
+            const uint32_t b_kstep = (2 * b_lbo) >> 4, b_lo = (uint32_t)a.b_bytes >> 4;
             int sa = 0, sb = 0; uint32_t pa = 0, pb = 0, acc = 0, acc_ph = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
@@ -601,11 +623,13 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
                 tc_fence_after();
                 uint32_t accumulate = 0;
                 for (int cc = 0; cc < a.kchunks && ok; ++cc) {
-                    ok = mbar_wait(&ctl->a_full[sa], pa, ctl, a.status);
-                    const uint64_t apatch = aconst + (aring_lo + (uint32_t)sa * a_slot_lo);
-                    uint32_t tap_lo = 0;                                // (ky * PW + kx) * 16 bytes, in 16-byte units
-                    for (int ky = 0; ky < a.kh && ok; ++ky, tap_lo += (uint32_t)(ha.PW - a.kw)) {
-                        for (int kx = 0; kx < a.kw && ok; ++kx, ++tap_lo) {
+                    for (int ax = 0; ax < (SLAB ? a.kw : 1) && ok; ++ax) {     // A stages of this chunk: one patch, or kw slabs
+                        ok = mbar_wait(&ctl->a_full[sa], pa, ctl, a.status);
+                        const uint64_t apatch = aconst + (aring_lo + (uint32_t)sa * a_slot_lo);
+                        // patch: taps in (ky, kx) order at (ky * PW + kx) * 16 bytes; slab ax: taps (ky, ax) at ky atoms of 1024 bytes
+                        const int n_t = SLAB ? a.kh : taps;
+                        for (int t = 0; t < n_t && ok; ++t) {
+                            const uint32_t tap_lo = SLAB ? (uint32_t)t * 64u : (uint32_t)((t / a.kw) * ha.PW + t % a.kw);
                             ok = mbar_wait(&ctl->full[sb], pb, ctl, a.status);
                             if (!ok) break;
                             tc_fence_after();
@@ -615,7 +639,7 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
                                 const uint64_t adesc = apatch + j * patch_lo + tap_lo;
                                 uint32_t acc_j = accumulate;
 #pragma unroll
-                                for (int kk = 0; kk < 4; ++kk) {        // K = 16: two 8-channel planes
+                                for (int kk = 0; kk < 4; ++kk) {        // K = 16 per instruction, 64 channels per chunk
                                     umma_f16(d_tmem + j * a.BN, adesc + kk * a_kstep, bdesc + kk * b_kstep, a.idesc, acc_j);
                                     acc_j = 1;
                                 }
@@ -624,9 +648,9 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
                             umma_commit(&ctl->empty[sb]);
                             if (++sb == a.stages) { sb = 0; pb ^= 1u; }
                         }
+                        if (ok) umma_commit(&ctl->a_empty[sa]);         // the A stage is free once its taps retire
+                        if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
                     }
-                    if (ok) umma_commit(&ctl->a_empty[sa]);             // the patch is free once its taps retire
-                    if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
                 }
                 if (ok) umma_commit(&ctl->tmem_full[acc]);
                 if (++acc == (uint32_t)a.nbuf) { acc = 0; acc_ph ^= 1u; }
@@ -907,7 +931,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     return DC_OK;
 }
 
-static int launch_halo(dc_cache* c, int layer, int mt, const void* in, void* out, const int32_t* tile_list,
+static int launch_halo(dc_cache* c, int layer, int mt, bool slab, const void* in, void* out, const int32_t* tile_list,
                        const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
@@ -919,10 +943,11 @@ static int launch_halo(dc_cache* c, int layer, int mt, const void* in, void* out
     cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
     cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
     cuuint32_t box[4] = {8, (cuuint32_t)h.PW, (cuuint32_t)h.PH, 1};
+    if (slab) { box[0] = 64; box[1] = DC_TILE_W; }                // a column slab: 64 channels x 8 pixels x PH rows
     cuuint32_t estr[4] = {1, 1, 1, 1};
     if (enc(&tmA, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return DC_ERR_CUDA;
+            CU_TENSOR_MAP_INTERLEAVE_NONE, slab ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) return DC_ERR_CUDA;
     TcHaloArgs ha;
     TcArgs& a = ha.t;
     a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
@@ -933,30 +958,39 @@ static int launch_halo(dc_cache* c, int layer, int mt, const void* in, void* out
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(h.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
     ha.wpacked = (const __nv_bfloat16*)L.weight_halo;
-    ha.PW = h.PW; ha.PH = h.PH; ha.plane_bytes = h.plane_bytes; ha.patch_bytes = h.patch_bytes;
+    ha.PW = h.PW; ha.PH = h.PH; ha.plane_bytes = h.plane_bytes;
+    ha.patch_bytes = slab ? h.PH * DC_TILE_W * 128 : h.patch_bytes;
     // patch ring: as deep as leaves at least 3 weight stages (a small-K item is one patch, so depth = items in flight)
     a.tmem_cols = tmem_cols_for(a.nbuf, mt, h.BN);
     const int ctas = L.tc_ctas == 2 && a.tmem_cols <= 256 ? 2 : 1;
     const int budget = ring_budget(ctas);
     ha.a_stages = 2;
     for (int as = 4; as > 2; --as)
-        if (budget - as * mt * h.patch_bytes >= 3 * h.b_bytes) { ha.a_stages = as; break; }
-    const int a_total = ha.a_stages * mt * h.patch_bytes;
+        if (budget - as * mt * ha.patch_bytes >= 3 * h.b_bytes) { ha.a_stages = as; break; }
+    const int a_total = ha.a_stages * mt * ha.patch_bytes;
     int st = (budget - a_total) / h.b_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
-    const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + sizeof(SmemCtl) + 256;
+    const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + sizeof(SmemCtl) + (slab ? 1280 : 256);
+    if (smem > 227 * 1024) return DC_ERR_CONFIG;
     static bool attr_set = false;
     if (!attr_set) {
-        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
-        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_halo<2, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
         attr_set = true;
     }
     long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + mt - 1) / mt) * h.NB;
     int grid = items > c->num_sms * ctas ? c->num_sms * ctas : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
-    if (mt == 2) k_conv_tc_halo<2><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
-    else k_conv_tc_halo<1><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+    if (slab) {
+        if (mt == 2) k_conv_tc_halo<2, true><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+        else k_conv_tc_halo<1, true><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+    } else {
+        if (mt == 2) k_conv_tc_halo<2, false><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+        else k_conv_tc_halo<1, false><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+    }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -966,7 +1000,8 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
-    if (L.tc_mt >= 3) return launch_halo(c, layer, L.tc_mt - 2, in, out, tile_list, tile_count, masks, max_tiles);
+    if (L.tc_mt >= 5) return launch_halo(c, layer, L.tc_mt - 4, true, in, out, tile_list, tile_count, masks, max_tiles);
+    if (L.tc_mt >= 3) return launch_halo(c, layer, L.tc_mt - 2, false, in, out, tile_list, tile_count, masks, max_tiles);
     const bool pad16 = pad16_ok(L.d) && L.weight_packed && L.in_padded;
     const dc_layer_desc d = pad16 ? padded16(L.d) : L.d;
     const void* weights = pad16 ? L.weight_packed : L.weight;
@@ -1096,6 +1131,8 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
                 if (ctas == 2 && tmem_cols_for(mt * h.BN * 2 <= 512 ? 2 : 1, mt, h.BN) > 256) continue;
                 L.tc_mt = mt + 2; L.tc_bn = 0;
                 trial("patch-reuse kernel");
+                L.tc_mt = mt + 4;                                       // tc_mt 5 / 6: column slabs with 1 / 2 tiles per item
+                trial("column-slab kernel");
             }
         }
     }
