@@ -41,7 +41,8 @@ struct dc_layer_rt {
     int tc_ctas;                    // conv, bf16: CTAs per SM the tuned launch uses (1 or 2)
     int tc_mt, tc_bn;               // conv, bf16: tuned tiles per work item (3, 4: patch-reuse kernel with 1, 2; 5, 6: column-slab kernel) and
                                     // channels per block (0 = default)
-    void* weight_halo;              // conv, bf16: weights packed for the patch-reuse kernel
+    void* weight_halo;              // conv, bf16: weights packed for the patch-reuse and column-slab kernels
+    int halo_bn;                    // channels per block that packing is grouped by
     void* in_padded;                // conv, bf16, cin <= 8: input with channels padded to 8
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation

@@ -797,12 +797,16 @@ bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn =
 
 struct HaloPlan { int BN, NB, PW, PH, plane_bytes, patch_bytes, b_bytes; };
 
-bool halo_ok(const dc_layer_desc& d, HaloPlan& h)
+bool halo_ok(const dc_layer_desc& d, HaloPlan& h, int want_bn = 0)
 {
     if (d.kind != DC_CONV || d.sh != 1 || d.sw != 1 || d.cin % 64 != 0 || d.kh * d.kw < 2 || d.kh > 5 || d.kw > 5) return false;
     h.BN = 0;
     for (int bn = 256; bn >= 32; bn -= 32) if (d.cout % bn == 0) { h.BN = bn; break; }
     if (!h.BN) return false;
+    if (want_bn > 0) {                                           // a tuned choice: must divide cout like the default
+        if (want_bn % 32 != 0 || want_bn > 256 || d.cout % want_bn != 0) return false;
+        h.BN = want_bn;
+    }
     h.NB = d.cout / h.BN;
     h.PW = DC_TILE_W + d.kw - 1; h.PH = DC_TILE_H + d.kh - 1;
     h.plane_bytes = (h.PW * h.PH * 16 + 127) & ~127;       // TMA destinations are 128-byte aligned
@@ -851,6 +855,7 @@ int dc_pack_weights_bf16(dc_cache* c, int layer)
         int grid = (int)((n + 255) / 256); if (grid > c->num_sms * 8) grid = c->num_sms * 8;
         k_pack_halo<<<grid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, L.d.cout, L.d.kh * L.d.kw, L.d.cin, h.BN,
                                                  (__nv_bfloat16*)L.weight_halo);
+        L.halo_bn = h.BN;
         DC_CUDA(cudaGetLastError());
     }
     if (pad16_ok(L.d)) {
@@ -938,7 +943,16 @@ static int launch_halo(dc_cache* c, int layer, int mt, bool slab, const void* in
     const dc_layer_desc& d = L.d;
     HaloPlan h;
     EncodeTiledFn enc = encode_fn();
-    if (!enc || !L.weight_halo || !halo_ok(d, h)) return DC_ERR_CONFIG;
+    if (!enc || !L.weight_halo || !halo_ok(d, h, L.tc_bn)) return DC_ERR_CONFIG;
+    if (L.halo_bn != h.BN) {
+        // the packed weights are grouped by channel block: another block width needs another packing (same size).
+        // Happens while the tuner tries widths and once more for its final choice, never in steady state.
+        const size_t n = (size_t)d.cout * d.kh * d.kw * d.cin;
+        int pgrid = (int)((n + 255) / 256); if (pgrid > c->num_sms * 8) pgrid = c->num_sms * 8;
+        k_pack_halo<<<pgrid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, d.cout, d.kh * d.kw, d.cin, h.BN,
+                                                  (__nv_bfloat16*)L.weight_halo);
+        L.halo_bn = h.BN;
+    }
     CUtensorMap tmA;
     cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
     cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
@@ -1125,14 +1139,18 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
                 trial("tap-by-tap kernel");
             }
         }
-        HaloPlan h;
-        if (L.weight_halo && halo_ok(L.d, h)) {
-            for (int mt = 1; mt <= 2; ++mt) {                          // tc_mt 3 / 4: patch-reuse kernel with 1 / 2 tiles per item
-                if (ctas == 2 && tmem_cols_for(mt * h.BN * 2 <= 512 ? 2 : 1, mt, h.BN) > 256) continue;
-                L.tc_mt = mt + 2; L.tc_bn = 0;
-                trial("patch-reuse kernel");
-                L.tc_mt = mt + 4;                                       // tc_mt 5 / 6: column slabs with 1 / 2 tiles per item
-                trial("column-slab kernel");
+        HaloPlan h0;
+        if (L.weight_halo && halo_ok(L.d, h0)) {
+            for (int bn = h0.BN; bn >= 64 && bn >= h0.BN / 2; bn -= 32) {
+                HaloPlan h;
+                if (!halo_ok(L.d, h, bn)) continue;
+                for (int mt = 1; mt <= 2; ++mt) {                      // tc_mt 3 / 4: patch-reuse kernel with 1 / 2 tiles per item
+                    if (ctas == 2 && tmem_cols_for(mt * h.BN * 2 <= 512 ? 2 : 1, mt, h.BN) > 256) continue;
+                    L.tc_bn = bn;
+                    if (bn == h0.BN) { L.tc_mt = mt + 2; trial("patch-reuse kernel"); }
+                    L.tc_mt = mt + 4;                                   // tc_mt 5 / 6: column slabs with 1 / 2 tiles per item
+                    trial("column-slab kernel");
+                }
             }
         }
     }
