@@ -11,7 +11,7 @@
 //              per block and pass; points already scored by the previous diamond are skipped (they cannot
 //              win).  Walks that leave the window continue in k_search_ds16q_long with private windows.
 //   k_verify   Steps 3-4: rounds the mean vector M, scores every block at M (reusing the Step 2
-//              score when the block's own best vector is M).
+//              score when the block's own best vector is M); k_verify16_prep / k_verify16_list for 16-pixel blocks.
 //   k_merge_runs, k_merge   Step 5: maximal horizontal runs per block row, merged vertically when the
 //              spans are identical, emitted in (y, x) order by a CTA-wide ordered compaction.
 #include "dc_common.cuh"
@@ -755,14 +755,18 @@ __global__ void __launch_bounds__(LPB * 8, MINB) k_search_ds16q_long(MatchArgs a
     }
 }
 
-// Step 4 for 16-pixel blocks: one half-warp per block, one lane per block row.
-__global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
+// Step 4 for 16-pixel blocks, in two launches.
+// k_verify16_prep (one thread per block) rounds M, settles every block that needs no pixels -- M leaves the frame
+// or the range for it, or its own best vector is M, so that Step 2 already holds the score (Section 4's second
+// acceleration, exact in that case) -- and lists the others.  k_verify16_list scores the listed blocks, one
+// half-warp per block and one lane per block row, so that no warp idles on blocks that were settled.
+__global__ void __launch_bounds__(256) k_verify16_prep(MatchArgs a, uint32_t* list, int32_t* list_count)
 {
-    const int lane = threadIdx.x & 31, r = lane & 15, half = lane >> 4;
+    const int lane = threadIdx.x & 31;
     const int per = a.Gx * a.Gy;
-    const unsigned gi = (blockIdx.x * 8u + (threadIdx.x >> 5)) * 2u + half;     // S * Gx * Gy < 2^31
+    const unsigned gi = blockIdx.x * 256u + threadIdx.x;                          // S * Gx * Gy < 2^31
     const bool in_grid = gi < (unsigned)(per * a.S);
-    const int s = in_grid ? (int)(gi / (unsigned)per) : 0, b = in_grid ? (int)(gi - (unsigned)s * per) : 0;
+    const int s = in_grid ? (int)(gi / (unsigned)per) : a.S - 1, b = in_grid ? (int)(gi - (unsigned)s * per) : 0;
     const int by = b / a.Gx, bx = b - by * a.Gx;
     const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
     const int4 sums = __ldcg((const int4*)a.acc + s);                            // Step 3: sum dx, sum dy, K (one 16-byte load)
@@ -771,62 +775,82 @@ __global__ void __launch_bounds__(256) k_verify16(MatchArgs a)
     if (K > 0) { Mx = round_mean(sums.x, K); My = round_mean(sums.y, K); }
     const bool cand_ok = in_grid && K > 0 && abs(Mx) <= a.R && abs(My) <= a.R && x0 + Mx >= 0 && y0 + My >= 0 &&
                          x0 + Mx + bw <= a.W && y0 + My + bh <= a.H;
-    const size_t g = (size_t)s * per + b;
-    // Section 4: reuse the Step 2 score when that step already scored this pair (best vector == M)
-    const bool known = cand_ok && a.mv[2 * g] == Mx && a.mv[2 * g + 1] == My && a.sse[g] != 0xffffffffu;
-    uint32_t acc = 0;
-    if (cand_ok && !known && r < bh) {
-        RowCtx<1> rc;
-        rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, r, 16, bw, bh);
-        // the 48 bytes of the displaced row lie in four aligned 16-byte chunks (rows of the frame copy are padded):
-        // four wide loads instead of thirteen narrow ones, then a word offset that is the same for a whole stream
-        const uint8_t* p = a.prev + (size_t)s * a.prev_stream + (size_t)(y0 + My + r) * a.prev_pitch + (size_t)(x0 + Mx) * 3;
-        const uint4* p16 = (const uint4*)((uintptr_t)p & ~(uintptr_t)15);
-        const uint4 c0 = __ldg(p16), c1 = __ldg(p16 + 1), c2 = __ldg(p16 + 2), c3 = __ldg(p16 + 3);
-        const uint32_t ww[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
-        const uint32_t boff = (uint32_t)(uintptr_t)p & 15u, sh = (boff & 3u) * 8u;
-        uint32_t w[13];
-        switch (boff >> 2) {
-        case 0:
+    bool known = false; uint32_t v = 0;
+    if (cand_ok) {
+        const uint32_t own = ((const uint32_t*)a.mv)[gi];                         // (dx, dy) as one word
+        v = a.sse[gi];
+        known = (int16_t)(own & 0xffffu) == Mx && (int16_t)(own >> 16) == My && v != 0xffffffffu;
+    }
+    const bool settled = in_grid && (!cand_ok || known);
+    const int ok = known && v <= a.limit[limit_index(a, bw, bh)];
+    if (settled) a.matched[gi] = (uint8_t)ok;
+    if (in_grid && b == 0) { a.gmv[3 * s] = Mx; a.gmv[3 * s + 1] = My; a.gmv[3 * s + 2] = K; }
+    // matched count: one atomic per warp and stream
+    const unsigned same = __match_any_sync(0xffffffffu, s);
+    const unsigned oks = __ballot_sync(0xffffffffu, ok);
+    if (lane == __ffs(same) - 1 && (oks & same)) atomicAdd(&a.acc[4 * s + 3], __popc(oks & same));
+    // the blocks whose pixels must be read
+    const bool todo = in_grid && !settled;
+    const unsigned tm = __ballot_sync(0xffffffffu, todo);
+    if (tm) {
+        int base = 0;
+        if (lane == 0) base = atomicAdd(list_count, __popc(tm));
+        base = __shfl_sync(0xffffffffu, base, 0);
+        if (todo) list[base + __popc(tm & ((1u << lane) - 1u))] = gi;
+    }
+}
+
+__global__ void __launch_bounds__(256) k_verify16_list(MatchArgs a, const uint32_t* list, const int32_t* list_count)
+{
+    const int lane = threadIdx.x & 31, r = lane & 15, half = lane >> 4;
+    const int per = a.Gx * a.Gy, n = *list_count;
+    const int stride = gridDim.x * 16;
+    for (int i0 = (blockIdx.x * 8 + (threadIdx.x >> 5)) * 2; i0 < n; i0 += stride) {      // both halves of a warp stay in the loop together
+        const int i = i0 + half;
+        const bool on = i < n;
+        const unsigned gi = on ? list[i] : 0u;
+        const int s = (int)(gi / (unsigned)per), b = (int)(gi - (unsigned)s * per);
+        const int by = b / a.Gx, bx = b - by * a.Gx;
+        const int x0 = bx * 16, y0 = by * 16, bw = min(16, a.W - x0), bh = min(16, a.H - y0);
+        const int Mx = a.gmv[3 * s], My = a.gmv[3 * s + 1];
+        uint32_t acc = 0;
+        if (on && r < bh) {
+            RowCtx<1> rc;
+            rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, r, 16, bw, bh);
+            // the 48 bytes of the displaced row lie in four aligned 16-byte chunks (rows of the frame copy are padded):
+            // four wide loads instead of thirteen narrow ones, then a word offset that is the same for a whole stream
+            const uint8_t* p = a.prev + (size_t)s * a.prev_stream + (size_t)(y0 + My + r) * a.prev_pitch + (size_t)(x0 + Mx) * 3;
+            const uint4* p16 = (const uint4*)((uintptr_t)p & ~(uintptr_t)15);
+            const uint4 c0 = __ldg(p16), c1 = __ldg(p16 + 1), c2 = __ldg(p16 + 2), c3 = __ldg(p16 + 3);
+            const uint32_t ww[16] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w, c2.x, c2.y, c2.z, c2.w, c3.x, c3.y, c3.z, c3.w};
+            const uint32_t boff = (uint32_t)(uintptr_t)p & 15u, sh = (boff & 3u) * 8u;
+            uint32_t w[13];
+            switch (boff >> 2) {
+            case 0:
 #pragma unroll
-            for (int j = 0; j < 13; ++j) w[j] = ww[j];
-            break;
-        case 1:
+                for (int j = 0; j < 13; ++j) w[j] = ww[j];
+                break;
+            case 1:
 #pragma unroll
-            for (int j = 0; j < 13; ++j) w[j] = ww[j + 1];
-            break;
-        case 2:
+                for (int j = 0; j < 13; ++j) w[j] = ww[j + 1];
+                break;
+            case 2:
 #pragma unroll
-            for (int j = 0; j < 13; ++j) w[j] = ww[j + 2];
-            break;
-        default:
+                for (int j = 0; j < 13; ++j) w[j] = ww[j + 2];
+                break;
+            default:
 #pragma unroll
-            for (int j = 0; j < 13; ++j) w[j] = ww[j + 3];
-            break;
+                for (int j = 0; j < 13; ++j) w[j] = ww[j + 3];
+                break;
+            }
+            acc = rc.sse_words(0, w, sh);
         }
-        acc = rc.sse_words(0, w, sh);
-    }
-    const uint32_t sse = __reduce_add_sync(half ? 0xffff0000u : 0x0000ffffu, acc);
-    int ok = 0;
-    if (r == 0 && in_grid) {
-        const uint32_t v = known ? a.sse[g] : sse;
-        ok = cand_ok && v <= a.limit[limit_index(a, bw, bh)];
-        a.matched[g] = (uint8_t)ok;
-        if (b == 0) { a.gmv[3 * s] = Mx; a.gmv[3 * s + 1] = My; a.gmv[3 * s + 2] = K; }
-    }
-    // count of matched blocks: one atomic per CTA and stream (the sums above share its 16 bytes, so every
-    // atomic saved also shortens the other CTAs' loads of them)
-    if (per < 16) {                                                               // tiny frames: a CTA may span many streams
-        if (ok) atomicAdd(&a.acc[4 * s + 3], 1);
-        return;
-    }
-    const unsigned first = blockIdx.x * 16u, last = min(first + 15u, (unsigned)(per * a.S) - 1u);
-    const int s_first = (int)(first / (unsigned)per), s_last = (int)(last / (unsigned)per);
-    const int n_first = __syncthreads_count(ok && s == s_first);
-    if (threadIdx.x == 0 && n_first) atomicAdd(&a.acc[4 * s_first + 3], n_first);
-    if (s_last != s_first) {                                                      // the CTA's 16 blocks span two streams
-        const int n_last = __syncthreads_count(ok && s != s_first);
-        if (threadIdx.x == 0 && n_last) atomicAdd(&a.acc[4 * s_last + 3], n_last);
+        const uint32_t sse = __reduce_add_sync(half ? 0xffff0000u : 0x0000ffffu, acc);
+        if (r == 0 && on) {
+            const int ok = sse <= a.limit[limit_index(a, bw, bh)];
+            a.matched[gi] = (uint8_t)ok;
+            if (ok) atomicAdd(&a.acc[4 * s + 3], 1);
+        }
     }
 }
 
@@ -1077,7 +1101,10 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
         k_accept_own<<<dc_div_up(a.S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(a);
     } else if (a.B == 16) {
         dc_prof_scope ps(c, DC_ST_VERIFY);
-        k_verify16<<<dc_div_up(a.S * a.Gx * a.Gy, 16), 256, 0, c->stream>>>(a);
+        int32_t* todo_count = long_count + 2;                       // zeroed with the Step 3 sums; the walk list is free again
+        k_verify16_prep<<<dc_div_up(a.S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(a, (uint32_t*)c->long_list, todo_count);
+        k_verify16_list<<<c->num_sms * 8, 256, 0, c->stream>>>(a, (const uint32_t*)c->long_list, todo_count);
+        c->launches += 1;
     } else {
         launch_by_block(c, a, false);
     }
