@@ -388,7 +388,12 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
                         "traffic": 936.0e6 if (w.index == 5 and S == 32 and w.search == 1 and args.skip_k == 1) else None,
                         "traffic_unit": "bytes per batch-frame (search + long walks + verify; dram read + write, ncu)",
                         "launches": prof["search"][1] + prof["verify"][1],
-                        "bytes_per_frame_batch": 4.0 * frame_bytes * S}
+                        "bytes_per_frame_batch": 4.0 * frame_bytes * S,
+                        "note": "Step 4 is credited with both frames for every block although blocks whose own best vector is M "
+                                "are settled without reading pixels; step2_only credits and times Step 2 alone",
+                        "step2_only": {"bytes_per_frame_batch": 2.0 * frame_bytes * S,
+                                       "achieved": (2.0 * frame_bytes * S * n_cached / (prof["search"][0] * 1e-3) / 1e9) if prof["search"][0] > 0 else 0.0,
+                                       "frac": (2.0 * frame_bytes * S * n_cached / (prof["search"][0] * 1e-3) / 1e9 / peaks["hbm_gbs"]) if prof["search"][0] > 0 else 0.0}}
 
     if w.search == 0:
         # Exhaustive search is plain integer arithmetic: every byte of every valid candidate takes one

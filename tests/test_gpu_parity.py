@@ -407,6 +407,41 @@ def test_infer_workload_5_two_streams():
     U.run_stream_parity(configs.WORKLOADS[5](), 2, [0, 1, 2])
 
 
+def test_infer_workload_5_full_batch_sampled_streams():
+    """The benchmark's own configuration: all 32 full-HD streams in one cache, the loop bench.py times
+    (dc_infer_frame(t), then dc_lookahead_frame(t + 1)), frames 0-3.  The oracle follows three of the streams
+    (first, one in the middle, last): motion vector, counts, frame rectangles and the final map of every frame."""
+    w = configs.WORKLOADS[5]()
+    S, n_frames, sample = w.n_streams, 4, (0, 13, w.n_streams - 1)
+    bf16 = w.dtype == configs.DTYPE_BF16
+    sb = w.streams(S, n_frames)
+    frames = [torch.from_numpy(np.ascontiguousarray(sb.frame(i))).cuda() for i in range(n_frames)]
+    oracles = dict(zip(sample, U.make_oracles(w, len(sample))))
+    dc = DeepCache.from_workload(w, n_streams=S)
+    try:
+        pitch = w.width * 3
+        for i in range(n_frames):
+            out, st = dc.infer_frame(frames[i], want_stats=True)
+            out = out.clone()
+            regs0, _ = dc.layer_regions(-1)
+            regs0 = regs0.clone()
+            if i + 1 < n_frames:
+                B.dc_lookahead_frame(dc.handle, frames[i + 1], pitch)
+            for s in sample:
+                o = oracles[s].infer_frame(sb.frame(i, s))
+                what = f"frame {i} stream {s} of {S}"
+                assert bool(st[s].refreshed) == o["refreshed"], what
+                if not o["refreshed"]:
+                    m = o["match"]
+                    assert (st[s].mvx, st[s].mvy, st[s].k_passed) == (m["M"][0], m["M"][1], m["K"]), what
+                    assert st[s].n_matched == int(m["matched"].sum()) and st[s].n_regions == len(m["regions"]), what
+                    U.assert_regions_equal(U.regions_np(regs0[s, :len(m["regions"])]), m["regions"], what + " frame rectangles")
+                U.assert_map_close(out[s], o["out"], bf16, what + " output")
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
+
+
 def test_infer_identical_frames_and_reset():
     w = configs.WORKLOADS[2]()
     f = w.streams(1, 1).frame(0)
