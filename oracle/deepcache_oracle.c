@@ -9,7 +9,7 @@
  * Conventions
  *   frames   uint8, HWC (3 channels), row pitch in bytes
  *   maps     double, NHWC (one stream at a time: HWC)
- *   weights  double, [cout][kh][kw][cin]
+ *   weights  double, [cout][kh][kw][cin] ([cout][kh][kw][cin / groups] for a grouped convolution)
  *   motion   MV = (dx, dy) points from a block of the current frame to its
  *            match in the previous frame: previous = current + MV
  *            (Section 4, Step 2: (x'_i - x_i, y'_i - y_i))
@@ -36,6 +36,7 @@ typedef struct { int32_t x, y, w, h, sx, sy; } orc_region;
 
 typedef struct {
     int32_t kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w;
+    int32_t groups;   /* convolution only: the channels are cut into this many independent groups (0 or 1: one) */
 } orc_layer;
 
 enum { ORC_CONV = 0, ORC_MAXPOOL = 1, ORC_RELU = 2, ORC_ADD = 3, ORC_CONCAT = 4,
@@ -497,6 +498,9 @@ void orc_conv_reuse(const double* in, int Hi, int Wi, const orc_layer* L,
                     double* out, uint8_t* reused)
 {
     const int Ho = L->out_h, Wo = L->out_w, Ci = L->cin, Co = L->cout;
+    /* grouped convolution (the form the cited AlexNet uses): output channel co of group g = co / (Co / G) sees
+     * only the input channels g * Ci / G ... (g + 1) * Ci / G - 1; weights [cout][kh][kw][cin / G] */
+    const int G = L->groups > 1 ? L->groups : 1, Cig = Ci / G, Cog = Co / G;
     #pragma omp parallel for schedule(dynamic, 1)
     for (int oy = 0; oy < Ho; ++oy)
         for (int ox = 0; ox < Wo; ++ox) {
@@ -520,9 +524,9 @@ void orc_conv_reuse(const double* in, int Hi, int Wi, const orc_layer* L,
                     for (int kx = 0; kx < L->kw; ++kx) {
                         int ix = ox * L->sw - L->pw + kx;
                         if (ix < 0 || ix >= Wi) continue;
-                        const double* a = in + ((int64_t)iy * Wi + ix) * Ci;
-                        const double* w = weight + (((int64_t)co * L->kh + ky) * L->kw + kx) * Ci;
-                        for (int ci = 0; ci < Ci; ++ci) acc += a[ci] * w[ci];
+                        const double* a = in + ((int64_t)iy * Wi + ix) * Ci + (co / Cog) * Cig;
+                        const double* w = weight + (((int64_t)co * L->kh + ky) * L->kw + kx) * Cig;
+                        for (int ci = 0; ci < Cig; ++ci) acc += a[ci] * w[ci];
                     }
                 }
                 acc += bias[co];

@@ -35,7 +35,7 @@ class Region(C.Structure):
 
 class Layer(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("kind", "kh", "kw", "sh", "sw", "ph", "pw", "cin", "cout",
-                                         "relu", "in0", "in1", "out_h", "out_w")]
+                                         "relu", "in0", "in1", "out_h", "out_w", "groups")]
 
 
 REGION_DTYPE = np.dtype([(n, "<i4") for n in ("x", "y", "w", "h", "sx", "sy")])
@@ -110,7 +110,7 @@ def _u8(a):
 
 
 def make_layer(d: dict) -> Layer:
-    return Layer(**{k: int(d[k]) for k, _ in Layer._fields_})
+    return Layer(**{k: int(d.get(k, 0)) for k, _ in Layer._fields_})       # groups is optional (0 = ungrouped)
 
 
 # ---------------------------------------------------------------------------

@@ -4,9 +4,9 @@ Input description only: shapes, strides, graph wiring and random numbers.  No
 convolution, erosion or matching arithmetic lives here.
 
 A layer is a plain dict with the keys of the C struct ``dc_layer_desc``:
-``kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w``.
+``kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w, groups``.
 ``in0`` / ``in1`` index the producing layer; ``-1`` is the input frame.
-Weights are float32, laid out ``[cout][kh][kw][cin]``; biases float32 ``[cout]``.
+Weights are float32, laid out ``[cout][kh][kw][cin / groups]``; biases float32 ``[cout]``.
 """
 from __future__ import annotations
 
@@ -16,9 +16,9 @@ import numpy as np
 KIND_CONV, KIND_MAXPOOL, KIND_RELU, KIND_ADD, KIND_CONCAT, KIND_RESIZE_AREA, KIND_LRN, KIND_FC = range(8)
 
 
-def _layer(kind, in0, out_h, out_w, cin, cout, k=1, s=1, p=0, relu=0, in1=-1):
+def _layer(kind, in0, out_h, out_w, cin, cout, k=1, s=1, p=0, relu=0, in1=-1, groups=1):
     return dict(kind=kind, kh=k, kw=k, sh=s, sw=s, ph=p, pw=p, cin=cin, cout=cout,
-                relu=relu, in0=in0, in1=in1, out_h=out_h, out_w=out_w)
+                relu=relu, in0=in0, in1=in1, out_h=out_h, out_w=out_w, groups=groups)
 
 
 class NetBuilder:
@@ -34,10 +34,11 @@ class NetBuilder:
         l = self.layers[idx]
         return (l["out_h"], l["out_w"], l["cout"])
 
-    def conv(self, src: int, cout: int, k: int, s: int = 1, p: int = 0, relu: int = 1) -> int:
+    def conv(self, src: int, cout: int, k: int, s: int = 1, p: int = 0, relu: int = 1, groups: int = 1) -> int:
         h, w, c = self.shape(src)
+        assert c % groups == 0 and cout % groups == 0
         oh, ow = (h + 2 * p - k) // s + 1, (w + 2 * p - k) // s + 1
-        self.layers.append(_layer(KIND_CONV, src, oh, ow, c, cout, k, s, p, relu))
+        self.layers.append(_layer(KIND_CONV, src, oh, ow, c, cout, k, s, p, relu, groups=groups))
         return len(self.layers) - 1
 
     def maxpool(self, src: int, k: int, s: int, p: int = 0) -> int:
@@ -116,15 +117,18 @@ def inception_lrn_net(h=64, w=64):
     return b.layers
 
 
-def alexnet_trunk(h=227, w=227):
+def alexnet_trunk(h=227, w=227, grouped=False):
+    """AlexNet-shaped trunk.  ``grouped``: the second, fourth and fifth convolutions in two channel groups,
+    as in the two-GPU original; the stated workload uses the ungrouped form."""
+    g = 2 if grouped else 1
     b = NetBuilder(h, w)
     x = b.conv(-1, 96, 11, 4, 0)
     x = b.maxpool(x, 3, 2)
-    x = b.conv(x, 256, 5, 1, 2)
+    x = b.conv(x, 256, 5, 1, 2, groups=g)
     x = b.maxpool(x, 3, 2)
     x = b.conv(x, 384, 3, 1, 1)
-    x = b.conv(x, 384, 3, 1, 1)
-    x = b.conv(x, 256, 3, 1, 1)
+    x = b.conv(x, 384, 3, 1, 1, groups=g)
+    x = b.conv(x, 256, 3, 1, 1, groups=g)
     b.maxpool(x, 3, 2)
     return b.layers
 
@@ -176,11 +180,12 @@ def random_weights(layers, seed: int, *, std: float | None = None, bias_std: flo
             weights.append(None)
             biases.append(None)
             continue
-        fan_in = l["kh"] * l["kw"] * l["cin"]
+        cin_g = l["cin"] // max(1, l.get("groups", 1))            # a grouped convolution sees cin / groups channels
+        fan_in = l["kh"] * l["kw"] * cin_g
         sd = std if std is not None else float(np.sqrt(2.0 / fan_in))
         if i in feeds_add:
             sd *= 0.5
-        w = rng.normal(0.0, sd, size=(l["cout"], l["kh"], l["kw"], l["cin"])).astype(np.float32)
+        w = rng.normal(0.0, sd, size=(l["cout"], l["kh"], l["kw"], cin_g)).astype(np.float32)
         bvec = (rng.normal(0.0, bias_std, size=l["cout"]) if bias_std > 0 else np.zeros(l["cout"]))
         weights.append(w)
         biases.append(bvec.astype(np.float32))

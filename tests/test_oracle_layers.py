@@ -37,6 +37,34 @@ def test_conv_equals_torch_float64(hi, wi, cin, cout, k, s, p, relu):
     assert not reused.any()
 
 
+@pytest.mark.parametrize("groups,cin,cout,k,s,p", [(2, 8, 12, 3, 1, 1), (4, 8, 8, 5, 2, 2), (3, 9, 6, 1, 1, 0), (2, 96, 64, 5, 1, 2)])
+def test_grouped_conv_equals_torch_float64(groups, cin, cout, k, s, p):
+    """Grouped convolution (the cited AlexNet's layers 2, 4, 5): library routine in float64, and the structural
+    fact that an output channel does not depend on the input channels of another group."""
+    g = rng(groups * 1000 + cin)
+    hi, wi = 13, 17
+    x = g.normal(size=(hi, wi, cin))
+    w = g.normal(size=(cout, k, k, cin // groups))
+    b = g.normal(size=cout)
+    L = dict(conv_layer(hi, wi, cin, cout, k, s, p, 1), groups=groups)
+    out, _ = orc.conv_reuse(x, L, w, b, orc.QUANT_NONE)
+    ref = F.conv2d(torch.from_numpy(x).permute(2, 0, 1)[None], torch.from_numpy(w).permute(0, 3, 1, 2),
+                   torch.from_numpy(b), stride=s, padding=p, groups=groups).clamp_min(0)[0].permute(1, 2, 0).numpy()
+    assert np.abs(out - ref).max() < 1e-12
+    x2 = x.copy()
+    x2[..., :cin // groups] += 1.0                               # disturb group 0's inputs only
+    out2, _ = orc.conv_reuse(x2, L, w, b, orc.QUANT_NONE)
+    assert np.array_equal(out2[..., cout // groups:], out[..., cout // groups:])
+    assert not np.array_equal(out2[..., :cout // groups], out[..., :cout // groups])
+    # groups = 1 and a missing key are the ordinary convolution
+    w1 = g.normal(size=(cout, k, k, cin))
+    L1 = conv_layer(hi, wi, cin, cout, k, s, p, 0)
+    a1, _ = orc.conv_reuse(x, dict(L1, groups=1), w1, b, orc.QUANT_NONE)
+    L1.pop("groups", None)
+    a0, _ = orc.conv_reuse(x, L1, w1, b, orc.QUANT_NONE)
+    assert np.array_equal(a0, a1)
+
+
 @pytest.mark.parametrize("k,s,p", [(2, 2, 0), (3, 2, 0), (3, 2, 1)])
 def test_maxpool_equals_torch(k, s, p):
     g = rng(k + s)
