@@ -68,7 +68,7 @@ typedef enum {
 
 /* One layer.  in0 / in1: index of the producing layer, -1 = the input frame
  * (in1 is used by DC_ADD / DC_CONCAT only).  out_h, out_w: output size.
- * DC_CONV: kh x kw kernel, stride, padding, cin -> cout, optional fused ReLU.
+ * DC_CONV: kh x kw kernel, stride, padding, cin -> cout, optional fused ReLU, optionally in channel groups.
  * DC_MAXPOOL: floor mode, padded taps ignored.  DC_ADD: element-wise, optional ReLU.
  * DC_RESIZE_AREA: box average of the input frame (in0 must be -1) to out_h x out_w.
  * DC_LRN: local response normalisation inside each channel over a (2 ph + 1)^2 spatial window (the form Table 2's
@@ -82,6 +82,10 @@ typedef enum {
  * cannot run dc_infer_frame. */
 typedef struct {
     int32_t kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w;
+    int32_t groups;   /* DC_CONV only: grouped convolution (the cited AlexNet's form); 0 or 1 = ordinary.  Output channel
+                         co belongs to group co / (cout / groups) and sees input channels group * cin / groups ...; both
+                         cin and cout must be multiples of groups; weights [cout][kh][kw][cin / groups].  Must be 0 or 1
+                         for every other kind. */
 } dc_layer_desc;
 
 /* The search unit of Step 2.  Exhaustive: every displacement within +-range.  Diamond: the paper's default

@@ -30,7 +30,7 @@ class dc_region(C.Structure):
 
 class dc_layer_desc(C.Structure):
     _fields_ = [(n, C.c_int32) for n in ("kind", "kh", "kw", "sh", "sw", "ph", "pw", "cin", "cout",
-                                         "relu", "in0", "in1", "out_h", "out_w")]
+                                         "relu", "in0", "in1", "out_h", "out_w", "groups")]
 
 
 class dc_config(C.Structure):
@@ -125,7 +125,7 @@ def make_layers(layers) -> C.Array:
     arr = (dc_layer_desc * len(layers))()
     for k, l in enumerate(layers):
         for name, _ in dc_layer_desc._fields_:
-            setattr(arr[k], name, int(l[name]))
+            setattr(arr[k], name, int(l.get(name, 0)) if name == "groups" else int(l[name]))
     return arr
 
 

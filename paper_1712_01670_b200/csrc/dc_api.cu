@@ -91,6 +91,7 @@ int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
         int iw = L.in0 < 0 ? cfg->width : layers[L.in0].out_w;
         int ic = L.in0 < 0 ? 3 : layers[L.in0].cout;
         if (L.out_h < 1 || L.out_w < 1 || L.cout < 1) return DC_ERR_CONFIG;
+        if (L.groups < 0 || (L.groups > 1 && L.kind != DC_CONV)) return DC_ERR_CONFIG;
         switch (L.kind) {
         case DC_CONV: case DC_MAXPOOL:
             if (L.kh < 1 || L.kw < 1 || L.sh < 1 || L.sw < 1 || L.ph < 0 || L.pw < 0) return DC_ERR_CONFIG;
@@ -98,6 +99,7 @@ int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
             if ((ih + 2 * L.ph - L.kh) / L.sh + 1 != L.out_h || (iw + 2 * L.pw - L.kw) / L.sw + 1 != L.out_w) return DC_ERR_CONFIG;
             if (ih + 2 * L.ph < L.kh || iw + 2 * L.pw < L.kw) return DC_ERR_CONFIG;
             if (L.cin != ic) return DC_ERR_CONFIG;
+            if (L.kind == DC_CONV && L.groups > 1 && (L.cin % L.groups != 0 || L.cout % L.groups != 0)) return DC_ERR_CONFIG;
             if (L.kind == DC_MAXPOOL && L.cout != ic) return DC_ERR_CONFIG;
             if (L.kind == DC_CONV && (L.cout * elt) % 16 != 0) return DC_ERR_CONFIG;   // 16-byte pixel vectors
             break;

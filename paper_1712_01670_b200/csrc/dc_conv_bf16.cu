@@ -838,6 +838,7 @@ int dc_conv_bf16_supported(const dc_cache* c, int layer)
     TcPlan p;
     if (getenv("DC_NO_TENSOR_CORES")) return 0;
     if (c->cfg.dtype != DC_BF16 || encode_fn() == nullptr) return 0;
+    if (c->L[layer].d.groups > 1) return 0;                       // grouped layers run on the CUDA-core kernel
     return make_plan(c->L[layer].d, p) || smallc_ok(c->L[layer].d) || pad16_ok(c->L[layer].d);
 }
 
@@ -1092,7 +1093,7 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
 {
     dc_layer_rt& L = c->L[layer];
     TcPlan p;
-    if (c->cfg.dtype != DC_BF16 || !encode_fn() || getenv("DC_NO_TENSOR_CORES")) return DC_OK;
+    if (c->cfg.dtype != DC_BF16 || !encode_fn() || getenv("DC_NO_TENSOR_CORES") || L.d.groups > 1) return DC_OK;
     const dc_layer_desc de = pad16_ok(L.d) ? padded16(L.d) : L.d;
     const bool generic = make_plan(de, p);
     if (!generic && !smallc_ok(L.d)) return DC_OK;

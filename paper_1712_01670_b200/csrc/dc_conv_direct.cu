@@ -2,7 +2,7 @@
 // pixels that were not filled from the cache).
 //
 // Used for float32 networks, whose 1e-4 accuracy bound rules out tensor-core input formats,
-// and for layer shapes the tensor-core kernel does not take.  One CTA of 128 threads owns one
+// for layer shapes the tensor-core kernel does not take, and for grouped convolutions.  One CTA of 128 threads owns one
 // dirty 16x8 output tile and a group of 32 output channels; thread t owns pixel t and keeps 32
 // float accumulators.  Weights for one kernel row and 8 input channels are staged in shared
 // memory as floats [kx][ci][co] and read as broadcast float4; inputs come straight from the
@@ -27,6 +27,7 @@ struct ConvArgs {
     const void* in; const void* w; const float* bias; void* out;
     const int32_t* tile_list; const int32_t* tile_count; const uint32_t* masks;
     int Hi, Wi, Ci, Ho, Wo, Co, kh, kw, sh, sw, ph, pw, relu, tiles_x, tiles_y;
+    int Cig, Cog, co_blocks;     // grouped convolution: input / output channels per group, CTAs (of CO_T channels) per group
 };
 
 template <typename T>
@@ -35,7 +36,10 @@ __global__ void __launch_bounds__(DC_TILE_PX) k_conv_direct(ConvArgs a)
     __shared__ __align__(16) float wsm[MAX_KW * CI_T * CO_T];
     const T* in = (const T*)a.in; const T* wt = (const T*)a.w; T* out = (T*)a.out;
     const int tid = threadIdx.x, prow = tid / DC_TILE_W, pcol = tid % DC_TILE_W;
-    const int co0 = blockIdx.y * CO_T, con = min(CO_T, a.Co - co0);
+    // blockIdx.y = (group, block of CO_T output channels inside the group): a CTA never straddles two groups
+    const int grp = blockIdx.y / a.co_blocks, co0 = grp * a.Cog + (blockIdx.y % a.co_blocks) * CO_T;
+    const int con = min(CO_T, (grp + 1) * a.Cog - co0);
+    const int ci_base = grp * a.Cig;                              // the group's first input channel
     const int per = a.tiles_x * a.tiles_y;
     const int n_tiles = *a.tile_count;
     for (int ti = blockIdx.x; ti < n_tiles; ti += gridDim.x) {
@@ -52,14 +56,14 @@ __global__ void __launch_bounds__(DC_TILE_PX) k_conv_direct(ConvArgs a)
         const T* in_s = in + (size_t)s * a.Hi * a.Wi * a.Ci;
         for (int ky = 0; ky < a.kh; ++ky) {
             const int iy = oy * a.sh - a.ph + ky;
-            for (int ci0 = 0; ci0 < a.Ci; ci0 += CI_T) {
-                const int cn = min(CI_T, a.Ci - ci0);
+            for (int ci0 = 0; ci0 < a.Cig; ci0 += CI_T) {
+                const int cn = min(CI_T, a.Cig - ci0);
                 __syncthreads();
                 for (int e = tid; e < a.kw * CI_T * CO_T; e += DC_TILE_PX) {
                     int co = e % CO_T, ci = (e / CO_T) % CI_T, kx = e / (CO_T * CI_T);
                     float v = 0.f;
                     if (co < con && ci < cn)
-                        v = ld_f(wt + (((size_t)(co0 + co) * a.kh + ky) * a.kw + kx) * a.Ci + ci0 + ci);
+                        v = ld_f(wt + (((size_t)(co0 + co) * a.kh + ky) * a.kw + kx) * a.Cig + ci0 + ci);
                     wsm[e] = v;
                 }
                 __syncthreads();
@@ -67,7 +71,7 @@ __global__ void __launch_bounds__(DC_TILE_PX) k_conv_direct(ConvArgs a)
                 for (int kx = 0; kx < a.kw; ++kx) {
                     const int ix = ox * a.sw - a.pw + kx;
                     if (ix < 0 || ix >= a.Wi) continue;
-                    const T* ap = in_s + ((size_t)iy * a.Wi + ix) * a.Ci + ci0;
+                    const T* ap = in_s + ((size_t)iy * a.Wi + ix) * a.Ci + ci_base + ci0;
                     float av[CI_T];
 #pragma unroll
                     for (int ci = 0; ci < CI_T; ++ci) av[ci] = ci < cn ? ld_f(ap + ci) : 0.f;
@@ -125,7 +129,9 @@ int dc_launch_conv(dc_cache* c, int layer, const void* in, void* out, const int3
     a.Hi = L.in_h; a.Wi = L.in_w; a.Ci = L.d.cin; a.Ho = L.d.out_h; a.Wo = L.d.out_w; a.Co = L.d.cout;
     a.kh = L.d.kh; a.kw = L.d.kw; a.sh = L.d.sh; a.sw = L.d.sw; a.ph = L.d.ph; a.pw = L.d.pw; a.relu = L.d.relu;
     a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
-    int co_groups = dc_div_up(L.d.cout, CO_T);
+    const int G = L.d.groups > 1 ? L.d.groups : 1;
+    a.Cig = L.d.cin / G; a.Cog = L.d.cout / G; a.co_blocks = dc_div_up(a.Cog, CO_T);
+    int co_groups = G * a.co_blocks;
     int gx = max_tiles < 1 ? 1 : max_tiles;
     int cap = dc_div_up(148 * 8, co_groups);
     if (gx > cap) gx = cap;
@@ -143,7 +149,7 @@ int dc_pack_weights_bf16(dc_cache* c, int layer);
 int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_dev)
 {
     dc_layer_rt& L = c->L[layer];
-    size_t n = (size_t)L.d.cout * L.d.kh * L.d.kw * L.d.cin;
+    size_t n = (size_t)L.d.cout * L.d.kh * L.d.kw * (L.d.cin / (L.d.groups > 1 ? L.d.groups : 1));
     if (L.d.kw > MAX_KW) return DC_ERR_CONFIG;
     DC_CUDA(cudaMalloc(&L.weight, n * c->elt));
     DC_CUDA(cudaMalloc((void**)&L.bias, sizeof(float) * L.d.cout));
@@ -153,6 +159,6 @@ int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_d
     else k_convert_weights<float><<<grid, 256, 0, c->stream>>>(w_dev, n, (float*)L.weight);
     DC_CUDA(cudaGetLastError());
     DC_CUDA(cudaMemcpyAsync(L.bias, b_dev, sizeof(float) * L.d.cout, cudaMemcpyDeviceToDevice, c->stream));
-    if (c->cfg.dtype == DC_BF16) return dc_pack_weights_bf16(c, layer);
+    if (c->cfg.dtype == DC_BF16 && L.d.groups <= 1) return dc_pack_weights_bf16(c, layer);   // grouped: no tensor-core packing
     return DC_OK;
 }

@@ -66,11 +66,13 @@ def small_cnn_stream() -> Workload:
                     seed=sd)
 
 
-def alexnet_stream() -> Workload:
+def alexnet_stream(grouped: bool = False, dtype: int = DTYPE_BF16) -> Workload:
+    """Workload 3.  ``grouped``: the trunk with the cited network's two channel groups in layers 2, 4, 5
+    (an extra; the stated workload is ungrouped)."""
     sd = _seed(3)
     n_patches = int(np.ceil(0.10 * 227 * 227 / (24 * 24)))
-    return Workload("alexnet_stream", 3, 227, 227, 1, 100, 16, 16, SEARCH_DS, DTYPE_BF16,
-                    nets.alexnet_trunk(227, 227),
+    return Workload("alexnet_stream" + ("_grouped" if grouped else ""), 3, 227, 227, 1, 100, 16, 16, SEARCH_DS, dtype,
+                    nets.alexnet_trunk(227, 227, grouped=grouped),
                     lambda s, f, first=0: streams.StreamBatch(
                         [streams.PannedStream(227, 227, f, sd + 1000 * k, max_pan=4, disturbance="patches",
                                               patch=24, n_patches=n_patches) for k in range(first, first + s)]),

@@ -27,7 +27,7 @@ def test_library_builds_and_exports_header_symbols():
 
 def test_struct_layouts_match_the_header():
     assert ctypes.sizeof(binding.dc_region) == 24
-    assert ctypes.sizeof(binding.dc_layer_desc) == 56
+    assert ctypes.sizeof(binding.dc_layer_desc) == 60
     assert ctypes.sizeof(binding.dc_config) == 88 and binding.dc_config.psnr_db.offset == 40
     assert binding.dc_config.region_mode.offset == 56
     assert ctypes.sizeof(binding.dc_frame_stats) == 7 * 4 + 4 * binding.DC_MAX_LAYERS

@@ -398,6 +398,13 @@ def test_infer_workload_3_alexnet_bf16():
     U.run_stream_parity(configs.WORKLOADS[3](), 1, list(range(12)))
 
 
+@pytest.mark.parametrize("dtype", [configs.DTYPE_FP32, configs.DTYPE_BF16])
+def test_infer_alexnet_with_grouped_convolutions(dtype):
+    """The AlexNet trunk with two channel groups in its second, fourth and fifth convolutions: every layer's
+    rectangles, reuse ratios and maps against the oracle, cached frames included."""
+    U.run_stream_parity(configs.alexnet_stream(grouped=True, dtype=dtype), 1, list(range(4)))
+
+
 def test_infer_workload_4_resnet50_bf16():
     U.run_stream_parity(configs.WORKLOADS[4](), 1, list(range(4)))
 
