@@ -10,6 +10,8 @@
 //              8 blocks in lockstep, 4 lanes per block with 4 block rows each in registers, one candidate
 //              per block and pass; points already scored by the previous diamond are skipped (they cannot
 //              win).  Walks that leave the window continue in k_search_ds16q_long with private windows.
+//   k_search_tss16q  Step 2 for 16-pixel blocks with three step search: the same lane layout, one window that
+//              covers the whole reach of the search.
 //   k_verify   Steps 3-4: rounds the mean vector M, scores every block at M (reusing the Step 2
 //              score when the block's own best vector is M); k_verify16_prep / k_verify16_list for 16-pixel blocks.
 //   k_merge_runs, k_merge   Step 5: maximal horizontal runs per block row, merged vertically when the
@@ -629,6 +631,134 @@ __global__ void __launch_bounds__(LPB * 8 * VS, MINB) k_search_ds16q(MatchArgs a
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Step 2 for 16-pixel blocks, three step search (Section 7.5), several blocks per warp
+// ---------------------------------------------------------------------------------------------
+// Same lane layout as the diamond kernel.  Every block scores the same number of points (the centre, then
+// eight per step), so the blocks of a warp stay in step without loss.  WalkState: phase = current step size,
+// mask = points of the 3 x 3 grid still to score (bit 4 = its centre).
+template <int LPB, typename Win>
+__device__ __forceinline__ void lockstep_tss(const MatchArgs& a, const RowCtx<16 / LPB>& rc, const Win& win, int q,
+                                             int dx_lo, unsigned dx_span, int dy_lo, unsigned dy_span, WalkState& w)
+{
+    constexpr int NR = 16 / LPB;
+#pragma unroll 1
+    for (int pass = 0; pass < 9 * 8; ++pass) {                   // at most 1 + 8 * log2(2 S0) points, S0 <= 64
+        if (w.st == 0 && w.mask == 0) {
+            w.phase >>= 1;                                        // next, halved step around the best point so far
+            if (w.phase == 0) w.st = 1;
+            else { w.cx = (int)(w.bt & 0xff) - 128; w.cy = (int)((w.bt >> 8) & 0xff) - 128; w.mask = 0x1efu; }
+        }
+        if (!__any_sync(0xffffffffu, w.st == 0)) break;
+        const bool run = w.st == 0;
+        const int i = run ? __ffs(w.mask) - 1 : 4;
+        w.mask &= w.mask - 1;
+        const int dx = w.cx + (i % 3 - 1) * w.phase, dy = w.cy + (i / 3 - 1) * w.phase;
+        const bool ok = run && (unsigned)(dx - dx_lo) <= dx_span && (unsigned)(dy - dy_lo) <= dy_span;
+        uint32_t ks = 0;
+        if (ok) {
+            uint32_t sh;
+#pragma unroll
+            for (int k = 0; k < NR; ++k) {
+                const uint32_t* p = win.row(q + k * LPB, dx, dy, sh);
+                const uint32_t v = rc.template sse<false>(k, p, sh);
+                ks += rc.row_on[k] ? v : 0u;
+            }
+        }
+#pragma unroll
+        for (int off = LPB / 2; off > 0; off >>= 1) ks += __shfl_xor_sync(0xffffffffu, ks, off);
+        const uint32_t kt = ((uint32_t)(abs(dx) + abs(dy)) << 16) | ((uint32_t)(dy + 128) << 8) | (uint32_t)(dx + 128);
+        if (ok && (ks < w.bs || (ks == w.bs && kt < w.bt))) { w.bs = ks; w.bt = kt; }
+    }
+}
+
+// Window of a CTA's 8 x VS blocks whose reach is known at launch only (three step search: 2 S0 - 1 pixels).
+struct StackWinR {
+    const uint32_t* win; int x0, wx0, row0, wr, pitch;
+    __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
+    {
+        const int off = (x0 + dx) * 3 - wx0;
+        sh = (off & 3) * 8;
+        return win + (row0 + r + dy + wr) * pitch + (off >> 2);
+    }
+};
+
+// One CTA per 8 x VS blocks; the window (dynamic shared memory) reaches wr = 2 S0 - 1 pixels around the tile, which
+// covers every point the search can visit.  Blocks clipped in width are left to the generic kernel.
+template <int LPB, int VS>
+__global__ void __launch_bounds__(LPB * 8 * VS) k_search_tss16q(MatchArgs a, int s0, int wr, int words, int pitch)
+{
+    extern __shared__ uint32_t tss_win[];
+    constexpr int THREADS = LPB * 8 * VS;
+    const int rows = 16 * VS + 2 * wr, cpr = words / 4, chunks = rows * cpr;
+    const int strips = (a.Gx + 7) >> 3, vgroups = (a.Gy + VS - 1) / VS;
+    const int strip = blockIdx.x % strips, vg = (blockIdx.x / strips) % vgroups, s = blockIdx.x / (strips * vgroups);
+    const int xs = strip * 128, yb = vg * 16 * VS;
+    const int wx0 = ((xs - wr) * 3) & ~15;                    // byte column of the window origin (may be < 0)
+    const int lane = threadIdx.x & 31, q = lane % LPB;
+    const int blk = threadIdx.x / LPB, by = vg * VS + (blk >> 3), bx = strip * 8 + (blk & 7);
+    const bool in_grid = bx < a.Gx && by < a.Gy;
+    const int x0 = bx * 16, y0 = by * 16;
+    const bool searched = in_grid && a.W - x0 >= 16;
+    const int bw = searched ? 16 : 0, bh = searched ? min(16, a.H - y0) : 0;
+    RowCtx<16 / LPB> rc;                                      // issued first: in flight while the window is staged
+    rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)(searched ? y0 : 0) * a.cur_pitch + (size_t)(searched ? x0 : 0) * 3,
+                  a.cur_pitch, q, LPB, bw, bh);
+    const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
+    constexpr int UNR = 4;                                    // 16-byte chunks; wx0 and the pitch are 16-byte multiples
+    for (int i0 = threadIdx.x; i0 < chunks; i0 += THREADS * UNR) {
+        uint4 v[UNR];
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int i = i0 + u * THREADS, row = i / cpr, ci = i - row * cpr;
+            const int gy = yb - wr + row, gb = wx0 + ci * 16;
+            v[u] = make_uint4(0, 0, 0, 0);
+            if (i < chunks && gy >= 0 && gy < a.H && gb >= 0 && gb + 16 <= (int)a.prev_pitch)
+                v[u] = __ldg((const uint4*)(prev + (size_t)gy * a.prev_pitch + gb));
+        }
+#pragma unroll
+        for (int u = 0; u < UNR; ++u) {
+            const int i = i0 + u * THREADS, row = i / cpr, ci = i - row * cpr;
+            if (i < chunks) {
+                uint32_t* d = tss_win + row * pitch + ci * 4;
+                d[0] = v[u].x; d[1] = v[u].y; d[2] = v[u].z; d[3] = v[u].w;
+            }
+        }
+    }
+    __syncthreads();
+    const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
+    const int dx_lo = max(-a.R, -x0), dy_lo = max(-a.R, -y0);
+    const unsigned dx_span = (unsigned)(min(a.R, a.W - bw - x0) - dx_lo), dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
+    const StackWinR sw = {tss_win, x0, wx0, (blk >> 3) * 16, wr, pitch};
+    WalkState w;
+    walk_begin(w, searched);
+    w.phase = s0;                                             // first pass: the centre and its eight neighbours at step S0
+    if (searched && s0 == 0) w.mask = 0x010u;                 // range 0: the zero vector alone
+    lockstep_tss<LPB>(a, rc, sw, q, dx_lo, dx_span, dy_lo, dy_span, w);
+    const int fx = (int)(w.bt & 0xff) - 128, fy = (int)((w.bt >> 8) & 0xff) - 128;
+    const bool fin = searched && q == 0;
+    if (fin) { a.mv[2 * g] = (int16_t)fx; a.mv[2 * g + 1] = (int16_t)fy; a.sse[g] = w.bs; }
+    const bool pass = fin && w.bs <= a.limit[limit_index(a, bw, bh)];     // PSNR > T: member of Step 3's set S
+    const int n_pass = __popc(__ballot_sync(0xffffffffu, pass));
+    const int sum_x = __reduce_add_sync(0xffffffffu, pass ? fx : 0), sum_y = __reduce_add_sync(0xffffffffu, pass ? fy : 0);
+    if (lane == 0 && n_pass) {
+        atomicAdd(&a.acc[4 * s + 0], sum_x);
+        atomicAdd(&a.acc[4 * s + 1], sum_y);
+        atomicAdd(&a.acc[4 * s + 2], n_pass);
+    }
+}
+
+constexpr int TSS_LPB = 4, TSS_VS = 4;
+// shared memory of one k_search_tss16q CTA for search range R
+static size_t tss_window_bytes(int R)
+{
+    int s0 = R < 1 ? 0 : 1;
+    while (s0 > 0 && 4 * s0 - 1 <= R) s0 *= 2;
+    const int wr = s0 > 0 ? 2 * s0 - 1 : 1;
+    const int words = ((((112 + 2 * wr) * 3 + 15) >> 2) + 13 + 3) & ~3;
+    return (size_t)(16 * TSS_VS + 2 * wr) * (words | 1) * sizeof(uint32_t);
+}
+
 // Section 4, k-skip: blocks that are not searched report vector (0, 0) and SSE 2^32 - 1.  One thread per block.
 __global__ void k_mark_unsearched(MatchArgs a)
 {
@@ -1067,6 +1197,28 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
                 k_search_ds16q_long<P2_LPB, 5><<<c->num_sms * 5, P2_LPB * 8, 0, c->stream>>>(a, nullptr, long_count, long_count + 1);
             }
             c->launches += 1;
+        }
+        if (a.W % 16 != 0) {                                        // blocks clipped by the right edge
+            a.edge_only = 2;
+            launch_by_block(c, a, true);
+            a.edge_only = 0;
+            c->launches += 1;
+        }
+    } else if (a.B == 16 && a.search == DC_SEARCH_THREE_STEP && a.skip_k <= 1 && tss_window_bytes(a.R) <= 160 * 1024) {
+        int s0 = a.R < 1 ? 0 : 1;                                   // first step: the largest power of two with 2 S0 - 1 <= R
+        while (s0 > 0 && 4 * s0 - 1 <= a.R) s0 *= 2;
+        const int wr = s0 > 0 ? 2 * s0 - 1 : 1;
+        const int words = ((((112 + 2 * wr) * 3 + 15) >> 2) + 13 + 3) & ~3, pitch = words | 1;
+        const size_t smem = tss_window_bytes(a.R);
+        static bool attr_set = false;
+        if (!attr_set) {
+            DC_CUDA(cudaFuncSetAttribute(k_search_tss16q<TSS_LPB, TSS_VS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
+            attr_set = true;
+        }
+        {
+            dc_prof_scope ps(c, DC_ST_SEARCH);
+            const int ctas = ((a.Gx + 7) / 8) * ((a.Gy + TSS_VS - 1) / TSS_VS) * a.S;
+            k_search_tss16q<TSS_LPB, TSS_VS><<<ctas, TSS_LPB * 8 * TSS_VS, smem, c->stream>>>(a, s0, wr, words, pitch);
         }
         if (a.W % 16 != 0) {                                        // blocks clipped by the right edge
             a.edge_only = 2;
