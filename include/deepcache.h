@@ -20,7 +20,8 @@
  *     asynchronous unless stated otherwise.
  *   - Environment switches read by the library (diagnostics only): DC_VERBOSE prints CUDA error strings and the
  *     per-layer kernel choices made by dc_cache_create; DC_CONV_NO_TUNE skips the per-layer timing and keeps the
- *     default work split; DC_NO_TENSOR_CORES runs every convolution on the CUDA-core kernel.
+ *     default work split; DC_NO_TENSOR_CORES runs every convolution on the CUDA-core kernel; DC_CONV_SCHEME=<1..6>
+ *     restricts that timing to one operand scheme of the tensor-core convolution (used by the tests to reach each one).
  *   - Frames are uint8, interleaved HWC with 3 channels; n_streams frames are
  *     stacked, stream s starting at frame + s * height * pitch_bytes.
  *   - Feature maps are NHWC, N = n_streams, element type float (DC_FP32) or

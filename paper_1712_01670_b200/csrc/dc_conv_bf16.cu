@@ -1109,7 +1109,11 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
         if (dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles) != DC_OK) break;
     const bool verbose = getenv("DC_VERBOSE") != nullptr;
     // times the launch the current L.tc_* fields select; keeps it when it is the fastest so far
+    // DC_CONV_SCHEME=<code> (diagnostics, tests): only candidates of that operand scheme are timed, so the scheme runs
+    // wherever it can (1, 2 tap by tap; 3, 4 patch; 5, 6 column slabs; the second of each pair with two tiles per item)
+    const int only = getenv("DC_CONV_SCHEME") ? atoi(getenv("DC_CONV_SCHEME")) : 0;
     auto trial = [&](const char* what) {
+        if (only > 0 && generic && L.tc_mt != only) return;
         int rc = DC_OK;
         for (int rep = 0; rep < kTuneReps + 1 && rc == DC_OK; ++rep) {
             if (rep == 1) cudaEventRecord(e0, c->stream);

@@ -385,6 +385,25 @@ def test_conv_partial(dtype, hi, wi, cin, cout, k, s, p, relu):
         dc.close()
 
 
+@pytest.mark.parametrize("scheme", [1, 2, 3, 4, 5, 6])
+def test_conv_schemes_forced(scheme, monkeypatch):
+    """Every operand scheme of the tensor-core convolution (tap by tap, patch, column slabs; one or two tiles per
+    item) on layers it can take: VGG-shaped 3x3 layers, a 5x5 layer and odd map sizes, through cached frames."""
+    monkeypatch.setenv("DC_CONV_SCHEME", str(scheme))
+    b = nets.NetBuilder(45, 53)
+    x = b.conv(-1, 64, 3, 1, 1)
+    x = b.conv(x, 64, 3, 1, 1)
+    x = b.conv(x, 128, 5, 1, 2)
+    x = b.maxpool(x, 2, 2)
+    x = b.conv(x, 256, 3, 1, 1)
+    b.conv(x, 256, 3, 1, 1, relu=0)
+    w = configs.small_cnn_stream()
+    w.layers, w.dtype, w.width, w.height = b.layers, configs.DTYPE_BF16, 53, 45
+    inner = w.make_streams
+    w.make_streams = lambda s, f, first=0: _cropped(inner(s, f), 45, 53)
+    U.run_stream_parity(w, 2, [0, 1, 2])
+
+
 # ------------------------------------------------------------------ dc_infer_frame
 def test_infer_workload_1():
     U.run_stream_parity(configs.WORKLOADS[1](), 1, [0, 1])
