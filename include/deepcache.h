@@ -268,6 +268,7 @@ int dc_cache_counters(dc_cache* cache, int64_t* reused_px_host, int64_t* frames_
  * Runs Steps 2 and 3 of the matcher on caller-owned frames: for each block of frame_dev the best
  * motion vector into prev_dev and its SSE, and per stream the rounded mean vector of the blocks
  * that pass the PSNR test.  Same definitions, candidate order and outputs as dc_match_blocks.
+ * search must be DC_SEARCH_EXHAUSTIVE or DC_SEARCH_DIAMOND (three step search: DC_ERR_CONFIG).
  *   frame_dev, prev_dev   uint8 HWC frames, n_streams stacked, any alignment, row pitch pitch_bytes
  *   block_mv_dev   int16  [S][Gy][Gx][2],  block_sse_dev uint32 [S][Gy][Gx],  global_mv_dev int32 [S][3]
  *   cuda_stream    cudaStream_t the work is enqueued on (asynchronous)

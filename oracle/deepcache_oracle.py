@@ -340,10 +340,20 @@ def fully_connected(x, layer, weight, bias, mode):
 
 
 def add(a, b, relu, mode):
+    """Residual add (a multi-input layer of Table 2): element-wise sum, optional ReLU, storage rounding."""
     a = np.ascontiguousarray(a, np.float64)
     b = np.ascontiguousarray(b, np.float64)
     out = np.empty_like(a)
     lib().orc_add(_p(a, C.c_double), _p(b, C.c_double), a.size, relu, mode, _p(out, C.c_double))
+    return out
+
+
+def relu(a):
+    """A stand-alone ReLU layer (Table 2, "others": the rectangle passes unchanged).  max(a, 0) of a stored value
+    is a stored value, so there is no rounding step."""
+    a = np.ascontiguousarray(a, np.float64)
+    out = np.empty_like(a)
+    lib().orc_relu(_p(a, C.c_double), a.size, _p(out, C.c_double))
     return out
 
 
@@ -417,7 +427,7 @@ class OracleCache:
                 assert l["in0"] < 0, "area resize reads the input frame"
                 out = resize_area(frame, l["out_h"], l["out_w"], self.quant)
             elif k == KIND_RELU:
-                out = np.maximum(x, 0.0)
+                out = relu(x)
             elif k == KIND_LRN:
                 if self.cache_pool and not refresh:
                     out, reused = lrn_reuse(x, l, *self.lrn, self.quant, self.prev_maps[i], per_layer_regions[i])

@@ -4,8 +4,8 @@
 // The regular matcher keeps its Step 3 accumulators (sum of motion vectors and count of blocks
 // that pass the PSNR test, per stream) in memory that dc_cache_create allocates.  Some callers
 // have no chance to create a cache: code that runs where cudaMalloc is off limits (for instance
-// inside a host callback or a latency-critical loop whose memory was fixed at start-up), or a
-// plug-in whose host forbids allocation after initialisation.  This entry point does the same
+// a latency-critical loop whose memory was fixed at start-up), or a plug-in whose host forbids
+// allocation after initialisation.  This entry point does the same
 // search with the accumulators in a fixed array that lives in the library image itself.
 //
 // The array holds DC_NOALLOC_MAX_STREAMS x 4 32-bit words (1 KiB).  Every GPU that loads the

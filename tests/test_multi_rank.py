@@ -25,13 +25,14 @@ def _worker(rank, world, port, out):
         mine = sharding.shard_streams(rank, world, S)
         gathered = [None] * world
         dist.all_gather_object(gathered, mine)
-        # each rank renders only its own streams, from the global stream index: same pixels whoever renders them
-        w = configs.WORKLOADS[2]()
-        frames = w.make_streams(1, 2).frame(1)
+        # each rank renders only its own streams, from the global stream index (as bench.py does with first=):
+        # the pixels of a stream depend on that index alone, not on who renders it
+        w = configs.batched_stress(96, 64, 128)
+        frames = w.streams(S, 2, first=mine[0]).frame(1)
         local_time = 1.0 + rank                      # rank 1 is slower
         t = sharding.max_over_ranks(local_time)
         out[rank] = dict(mine=mine, gathered=gathered, t=t, rate=sharding.aggregate_rate(S * 10, world, t),
-                         checksum=int(frames.sum()))
+                         frames=frames.tobytes(), shape=frames.shape)
     finally:
         dist.destroy_process_group()
 
@@ -47,7 +48,13 @@ def test_two_ranks_shard_streams_and_reduce_time():
     assert flat == list(range(6))                                    # disjoint and complete
     assert res[0]["t"] == res[1]["t"] == 2.0                         # the slowest rank sets the time
     assert res[0]["rate"] == 3 * 10 * 2 / 2.0
-    assert res[0]["checksum"] == res[1]["checksum"]                  # seeded inputs do not depend on the rank
+    # one process renders all six streams: rank r's frames are streams r * S ... r * S + S - 1 of that batch
+    whole = configs.batched_stress(96, 64, 128).streams(6, 2).frame(1)
+    assert whole.shape == (6, 64, 96, 3)
+    for r in range(world):
+        assert tuple(res[r]["shape"]) == (3, 64, 96, 3)
+        assert res[r]["frames"] == whole[3 * r:3 * r + 3].tobytes()
+    assert res[0]["frames"] != res[1]["frames"]                      # different streams, different pixels
 
 
 def test_single_process_is_identity():

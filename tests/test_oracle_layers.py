@@ -373,3 +373,96 @@ def test_lrn_reuse_copies_rectangles_and_normalises_the_rest():
     mask = np.zeros((9, 8), bool); mask[3:8, 2:6] = True
     assert np.array_equal(reused.astype(bool), mask)
     assert np.array_equal(out[3:8, 2:6], prev[2:7, 1:5]) and np.array_equal(out[~mask], full[~mask])
+
+
+# ---------------------------------------------------------------------------
+# residual add and stand-alone ReLU (the multi-input and "others" rows of Table 2 as executable layers)
+# ---------------------------------------------------------------------------
+@pytest.mark.parametrize("relu", [0, 1])
+def test_add_equals_torch_float64(relu):
+    g = rng(40 + relu)
+    a, b = g.normal(size=(7, 5, 6)), g.normal(size=(7, 5, 6))
+    ref = torch.from_numpy(a) + torch.from_numpy(b)
+    if relu:
+        ref = ref.clamp_min(0)
+    got = orc.add(a, b, relu, orc.QUANT_NONE)
+    assert np.array_equal(got, ref.numpy())                             # one float64 addition: no rounding freedom
+    assert (got < 0).any() != bool(relu)
+    # a swapped or dropped operand, or a ReLU applied before the sum, would show here
+    a2, b2 = np.array([[[-3.0, 2.0]]]), np.array([[[1.0, -5.0]]])
+    assert np.array_equal(orc.add(a2, b2, 0, orc.QUANT_NONE), [[[-2.0, -3.0]]])
+    assert np.array_equal(orc.add(a2, b2, 1, orc.QUANT_NONE), [[[0.0, 0.0]]])
+    assert np.array_equal(orc.add(-a2, -b2, 1, orc.QUANT_NONE), [[[2.0, 3.0]]])
+
+
+def test_add_rounds_the_sum_to_bf16_once():
+    # operands as a bf16 workload stores them (8 significant bits), close in magnitude: their sum is exact in
+    # float32, so torch's double -> float -> bfloat16 conversion rounds only once, like the oracle
+    g = rng(42)
+    a = g.integers(-255, 256, size=4000) / 64.0
+    b = g.integers(-255, 256, size=4000) / 32.0
+    for relu in (0, 1):
+        ref = torch.from_numpy(a + b)
+        if relu:
+            ref = ref.clamp_min(0)
+        ref = ref.to(torch.bfloat16).to(torch.float64).numpy()
+        assert np.array_equal(orc.add(a, b, relu, orc.QUANT_BF16), ref)
+    # exact ties go to the even neighbour: 1 + 2^-8 -> 1; (1 + 2^-7) + 2^-8 -> 1 + 2^-6
+    tie = orc.add(np.array([1.0, 1.0078125]), np.array([0.00390625, 0.00390625]), 0, orc.QUANT_BF16)
+    assert np.array_equal(tie, [1.0, 1.015625])
+    # the ReLU acts on the sum before rounding; a negative sum never rounds to a positive value
+    assert np.array_equal(orc.add(np.array([-1.0]), np.array([0.99609375]), 1, orc.QUANT_BF16), [0.0])
+
+
+def test_relu_layer_equals_torch():
+    g = rng(43)
+    x = g.normal(size=(5, 4, 3))
+    assert np.array_equal(orc.relu(x), torch.from_numpy(x).clamp_min(0).numpy())
+    assert np.array_equal(orc.relu(np.array([-0.5, 0.0, 2.5])), [0.0, 0.0, 2.5])
+    q = orc.quant_array(x, orc.QUANT_BF16)
+    assert np.array_equal(orc.quant_array(orc.relu(q), orc.QUANT_BF16), orc.relu(q))    # stored values stay stored values
+
+
+def _residual_net(h, w):
+    """conv 3x3 -> [branch: conv 3x3 + ReLU, conv 1x1] + skip -> add (+ReLU) -> stand-alone ReLU of a signed 1x1 conv."""
+    nb = nets.NetBuilder(h, w)
+    stem = nb.conv(-1, 4, 3, 1, 1, relu=1)
+    b1 = nb.conv(stem, 4, 3, 1, 1, relu=1)
+    b2 = nb.conv(b1, 4, 1, 1, 0, relu=0)
+    s = nb.add(b2, stem, relu=1)
+    lin = nb.conv(s, 5, 1, 1, 0, relu=0)
+    nb.layers.append(dict(kind=orc.KIND_RELU, kh=1, kw=1, sh=1, sw=1, ph=0, pw=0, cin=5, cout=5, relu=0, in0=lin, in1=-1,
+                          out_h=h, out_w=w, groups=1))
+    return nb.layers
+
+
+def _torch_conv(x, w, b, p, relu):
+    y = F.conv2d(x, torch.from_numpy(w).permute(0, 3, 1, 2), torch.from_numpy(b), padding=p)
+    return y.clamp_min(0) if relu else y
+
+
+def test_residual_block_through_the_cache_equals_torch_float64():
+    h, w_ = 24, 20
+    layers = _residual_net(h, w_)
+    ws, bs = nets.random_weights(layers, 7)
+    oc = orc.OracleCache(w_, h, layers, ws, bs, block=8, search_range=4, search_kind=orc.SEARCH_DS)
+    f = rng(44).integers(0, 256, size=(h, w_, 3), dtype=np.uint8)
+    a = oc.infer_frame(f)
+    x = torch.from_numpy(f.astype(np.float64) / 255.0).permute(2, 0, 1)[None]
+    W = [None if v is None else np.asarray(v, np.float64) for v in ws]
+    Bv = [None if v is None else np.asarray(v, np.float64) for v in bs]
+    stem = _torch_conv(x, W[0], Bv[0], 1, True)
+    b1 = _torch_conv(stem, W[1], Bv[1], 1, True)
+    b2 = _torch_conv(b1, W[2], Bv[2], 0, False)
+    s = (b2 + stem).clamp_min(0)                      # in0 = branch, in1 = skip
+    lin = _torch_conv(s, W[4], Bv[4], 0, False)
+    out = lin.clamp_min(0)
+    for got, ref in ((a["maps"][3], s), (a["maps"][4], lin), (a["maps"][5], out)):
+        assert np.abs(got - ref[0].permute(1, 2, 0).numpy()).max() < 1e-12
+    assert (a["maps"][4] < 0).any() and not (a["maps"][5] < 0).any()
+    # the same frame again: both inputs of the add carry the same rectangles, so its output is reusable and the
+    # whole network output is the cached one
+    b = oc.infer_frame(f)
+    assert not b["refreshed"] and b["regions"][3]["w"].any()
+    for ma, mb in zip(a["maps"], b["maps"]):
+        assert np.array_equal(ma, mb)
