@@ -51,6 +51,9 @@ def parse_args():
     ap.add_argument("--matcher-only", action="store_true",
                     help="time Steps 1-5 alone (dc_cache_set_key + dc_match_blocks per step) and print a short JSON line; "
                          "a small, single-purpose run for profiling the matcher kernels")
+    ap.add_argument("--reuse-copy", action="store_true",
+                    help="time the reuse copy alone (Section 5 'Reuse', step 1) on one 64-channel 224x224 bf16 layer with "
+                         "rectangles covering most of the map, through dc_conv_partial; prints a short JSON line")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -64,6 +67,30 @@ def measured_peaks():
         return dict(hbm_gbs=p["hbm_gbs"], bf16_tflops=p["bf16_tflops"],
                     bf16_tflops_sustained=p.get("bf16_tflops_sustained", p["bf16_tflops"]), source="measured")
     return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, bf16_tflops_sustained=1400.0, source="fallback")
+
+
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) from committed ncu captures.  Each entry names
+# its capture and carries the SHA-256 of the kernel source it was taken with; when that source has changed since, the
+# number no longer describes the kernels that run and null is printed instead.
+CAPTURED_TRAFFIC = {
+    "conv": {"bytes": None, "source": "paper_1712_01670_b200/csrc/dc_conv_bf16.cu", "sha256": None, "capture": None},
+    "matcher": {"bytes": None, "source": "paper_1712_01670_b200/csrc/dc_match.cu", "sha256": None, "capture": None},
+}
+
+
+def captured_traffic(key, applies):
+    import hashlib
+    e = CAPTURED_TRAFFIC[key]
+    if not applies or e["bytes"] is None:
+        return None, None
+    try:
+        with open(os.path.join(ROOT, e["source"]), "rb") as f:
+            sha = hashlib.sha256(f.read()).hexdigest()
+    except OSError:
+        return None, None
+    if sha != e["sha256"]:
+        return None, f"{e['capture']} predates the current {os.path.basename(e['source'])}"
+    return e["bytes"], e["capture"]
 
 
 def workload_config(w, n_streams, n_gpus):
@@ -201,8 +228,65 @@ def gpu_arm(args, w):
         gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local, dev)
 
 
+def reuse_copy_bench(args, B, DeepCache, rank, dev):
+    """Reuse copy alone: one 3 -> 64 channel 3x3 layer at 224 x 224, bf16, S streams; six rectangles per stream cover
+    about 79 % of the map, each displaced by its own vector.  dc_conv_partial runs the three steps of "Reuse"; the
+    event profile separates the copy + bitmap kernel from the convolution of the rest."""
+    import torch
+    from paper_1712_01670_b200.synth import nets
+    S = args.streams or 32
+    H = W = 224
+    nb = nets.NetBuilder(H, W)
+    nb.conv(-1, 64, 3, 1, 1, 1)
+    ws, bs = nets.random_weights(nb.layers, 5)
+    dc = DeepCache(W, H, nb.layers, ws, bs, n_streams=S, block=16, search_range=8, dtype=B.DC_BF16, max_regions=8)
+    g = np.random.Generator(np.random.PCG64(1712))
+    regs = np.zeros((S, dc.max_regions, 6), np.int32)
+    reused_px = 0
+    cw, ch = W // 3, H // 2
+    for s in range(S):
+        for i in range(6):
+            w_, h_ = cw - 8, ch - 12
+            x0, y0 = (i % 3) * cw + int(g.integers(0, 9)), (i // 3) * ch + int(g.integers(0, 13))
+            sx = min(max(x0 + int(g.integers(-8, 9)), 0), W - w_)
+            sy = min(max(y0 + int(g.integers(-8, 9)), 0), H - h_)
+            regs[s, i] = (x0, y0, w_, h_, sx, sy)
+            reused_px += w_ * h_
+    regs_d = torch.from_numpy(regs).to(dev)
+    n_d = torch.full((S,), 6, dtype=torch.int32, device=dev)
+    x = torch.rand((S, H, W, 3), device=dev).to(torch.bfloat16)
+    maps = [torch.randn((S, H, W, 64), device=dev).to(torch.bfloat16) for _ in range(2)]
+    for i in range(args.warmup):
+        B.dc_conv_partial(dc.handle, 0, x, maps[i & 1], regs_d, n_d, maps[(i & 1) ^ 1])
+    torch.cuda.synchronize()
+    B.dc_cache_set_profiling(dc.handle, True)
+    B.dc_cache_profile(dc.handle)
+    for i in range(args.steps):
+        B.dc_conv_partial(dc.handle, 0, x, maps[i & 1], regs_d, n_d, maps[(i & 1) ^ 1])
+    torch.cuda.synchronize()
+    prof = B.dc_cache_profile(dc.handle)
+    status = dc.status()
+    dc.close()
+    ms = prof["classify_copy"][0] / max(1, prof["classify_copy"][1])
+    bytes_per_launch = 2.0 * reused_px * 64 * 2
+    peaks = measured_peaks()
+    gbs = bytes_per_launch / (ms * 1e-3) / 1e9
+    if rank == 0:
+        print(json.dumps({"stage": "reuse copy + bitmaps (k_classify_copy), one 64-channel 224x224 bf16 layer",
+                          "streams": S, "reuse_ratio": reused_px / (S * H * W), "ms_per_launch": ms,
+                          "launches": prof["classify_copy"][1], "bytes_per_launch": bytes_per_launch,
+                          "roofline_copy": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                                            "frac": gbs / peaks["hbm_gbs"], "peak_source": f"hbm_gbs, {peaks['source']}"},
+                          "conv_ms_per_launch": prof["conv"][0] / max(1, prof["conv"][1]), "status": status}))
+
+
 def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local, dev):
     import torch
+    if args.reuse_copy:
+        reuse_copy_bench(args, B, DeepCache, rank, dev)
+        if world > 1:
+            dist.destroy_process_group()
+        return
     S = args.streams or w.n_streams
     total = args.warmup + args.steps
     # every rank renders its own streams: global stream index = rank * S + s
@@ -369,25 +453,45 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
     stage_share = {k: round(v[0] / max(1e-9, sum(x[0] for x in prof.values())), 4) for k, v in prof.items()}
     bf16 = w.dtype == 1
     conv_tflops = useful_flops / (conv_ms * 1e-3) / 1e12 if conv_ms > 0 else 0.0
-    conv_peak = peaks["bf16_tflops_sustained"] if bf16 else None
-    # DRAM bytes per convolution launch from the ncu capture summarised in profiles/dram_traffic_batched_stress.md
-    # (32 streams of workload 5, kernels as committed with that file); other shapes were not captured
-    conv_traffic = 77.8e6 if (w.index == 5 and S == 32 and bf16 and not args.cache_pool) else None
+    # Which measured peak applies: the burst figure for a region that ran at full clock without a power cap, the
+    # sustained one when the sampled clocks show the cap (long dense steps).  Both fractions are printed.
+    capped = "sw_power_cap" in (clocks.get("reasons") or []) or \
+             (clocks.get("sm_mhz") and clocks.get("sm_max_mhz") and clocks["sm_mhz"] < 0.9 * clocks["sm_max_mhz"])
+    conv_peak = (peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]) if bf16 else None
+    conv_traffic, conv_traffic_from = captured_traffic("conv", w.index == 5 and S == 32 and bf16 and not args.cache_pool)
     roofline = {"kernel": "partial convolution (all conv launches of the timed region)",
                 "bound": "tensor" if bf16 else "alu", "achieved": conv_tflops,
                 "peak": conv_peak, "unit": "TFLOP/s", "frac": (conv_tflops / conv_peak) if conv_peak else None,
-                "peak_source": f"bf16_tflops_sustained, {peaks['source']}", "traffic": conv_traffic,
-                "traffic_unit": "bytes per launch (dram read + write, ncu, one-pass capture of this workload)",
+                "peak_source": f"{'bf16_tflops_sustained' if capped else 'bf16_tflops (burst)'}, {peaks['source']}; "
+                               f"chosen by the clocks sampled in the timed region ({clocks.get('sm_mhz')} MHz, reasons {clocks.get('reasons')})",
+                "frac_burst": (conv_tflops / peaks["bf16_tflops"]) if bf16 else None,
+                "frac_sustained": (conv_tflops / peaks["bf16_tflops_sustained"]) if bf16 else None,
+                "traffic": conv_traffic, "traffic_from": conv_traffic_from,
+                "traffic_unit": "bytes per launch (dram read + write, ncu)",
                 "launches": conv_n, "avg_launch_ms": conv_ms / max(1, conv_n),
                 "flops_per_launch": useful_flops / max(1, conv_n)}
+    # Reuse copy (Section 5 "Reuse", step 1): 2 x reused pixels x channels x element size over the time of the kernel
+    # that also builds the bitmaps and dirty lists.  Meaningful where reuse is high (see bench.py --reuse-copy).
+    elt = 2 if bf16 else 4
+    copy_bytes = sum(2.0 * (px1[li] - px0[li]) * l["cout"] * elt for li, l in enumerate(w.layers)
+                     if l["kind"] == 0 or (args.cache_pool and l["kind"] in (1, 6)))
+    copy_ms, copy_n = prof["classify_copy"]
+    copy_gbs = copy_bytes / (copy_ms * 1e-3) / 1e9 if copy_ms > 0 else 0.0
+    roofline_copy = {"kernel": "reuse copy + bitmaps + dirty lists (k_classify_copy_all)", "bound": "hbm", "achieved": copy_gbs,
+                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": copy_gbs / peaks["hbm_gbs"],
+                     "peak_source": f"hbm_gbs, {peaks['source']}", "traffic": None, "launches": copy_n,
+                     "bytes_per_launch": copy_bytes / max(1, copy_n),
+                     "note": "little is reusable on this workload, so the kernel mostly classifies tiles; "
+                             "bench.py --reuse-copy times the copy at 79 % reuse"}
     match_ms = prof["search"][0] + prof["verify"][0]
     match_bytes = 4.0 * frame_bytes * S * n_cached            # Step 2: cur + prev once; Step 4: both again
     match_gbs = match_bytes / (match_ms * 1e-3) / 1e9 if match_ms > 0 else 0.0
+    match_traffic, match_traffic_from = captured_traffic("matcher", w.index == 5 and S == 32 and w.search == 1 and args.skip_k == 1)
     roofline_matcher = {"kernel": "block search + verify", "bound": "hbm", "achieved": match_gbs,
                         "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": match_gbs / peaks["hbm_gbs"],
                         "peak_source": f"hbm_gbs, {peaks['source']}",
-                        "traffic": 936.0e6 if (w.index == 5 and S == 32 and w.search == 1 and args.skip_k == 1) else None,
-                        "traffic_unit": "bytes per batch-frame (search + long walks + verify; dram read + write, ncu)",
+                        "traffic": match_traffic, "traffic_from": match_traffic_from,
+                        "traffic_unit": "bytes per batch-frame (search + verify kernels; dram read + write, ncu)",
                         "launches": prof["search"][1] + prof["verify"][1],
                         "bytes_per_frame_batch": 4.0 * frame_bytes * S,
                         "note": "Step 4 is credited with both frames for every block although blocks whose own best vector is M "
@@ -425,7 +529,7 @@ def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local,
             "vs_baseline": None, "dtype": "bf16" if bf16 else "f32", "data": "synthetic",
             "config": dict(workload_config(w, S, world), skip_k=args.skip_k, cache_pool=bool(args.cache_pool),
                            regions="per_block" if args.per_block_regions else "global"), "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
-            "roofline": roofline, "roofline_matcher": roofline_matcher, "cpu_baseline": cpu_baseline,
+            "roofline": roofline, "roofline_matcher": roofline_matcher, "roofline_copy": roofline_copy, "cpu_baseline": cpu_baseline,
             "stage_ms": stage_ms, "stage_share": stage_share, "frames_cached": n_cached, "frames_full": n_full,
             "reuse_ratio_cached_frames": reuse, "cache_bytes": cache_bytes, "no_cache": no_cache,
             "serial": {"value": sharding.aggregate_rate(S * args.steps, world, serial_ms * 1e-3), "unit": UNIT,

@@ -176,6 +176,7 @@ int dc_match_blocks(dc_cache* cache, const uint8_t* frame_dev, size_t pitch_byte
  *   in_dev   dc_region [S][max_regions], n_in_dev int32 [S]: rectangles on the input frame
  *   out_dev  dc_region [layer_end-layer_begin][S][max_regions]
  *   n_out_dev int32 [layer_end-layer_begin][S] (slot count, equal to n_in; may be NULL)
+ * Slots at or beyond max_regions are never written, whatever n_in_dev says.
  * Errors: DC_ERR_ARG, DC_ERR_CUDA. */
 int dc_propagate_regions(dc_cache* cache, const dc_region* in_dev, const int32_t* n_in_dev,
                          int layer_begin, int layer_end, dc_region* out_dev, int32_t* n_out_dev);
@@ -188,6 +189,9 @@ int dc_propagate_regions(dc_cache* cache, const dc_region* in_dev, const int32_t
  *   regions_dev   dc_region [S][max_regions], n_regions_dev int32 [S]: rectangles in output
  *                 coordinates (c_regions); both NULL = plain full convolution
  *   out_map_dev   [S][Ho][Wo][cout]  (top blob); must not alias prev_out_dev
+ * A count above max_regions is cut to max_regions.  A rectangle that does not lie inside the Ho x Wo map on
+ * both sides (current and cached) is not reused -- its pixels are convolved like any other -- and the device
+ * status word is set to DC_ERR_ARG (dc_get_status); no map is ever addressed outside its bounds.
  * Errors: DC_ERR_ARG, DC_ERR_CONFIG (not a convolution), DC_ERR_CUDA. */
 int dc_conv_partial(dc_cache* cache, int layer, const void* in_map_dev, const void* prev_out_dev,
                     const dc_region* regions_dev, const int32_t* n_regions_dev, void* out_map_dev);
@@ -235,8 +239,10 @@ int dc_cache_layer_map(dc_cache* cache, int layer, void** map_dev, size_t* bytes
  * `layer` ([S][max_regions]) and of their per-stream count ([S]). */
 int dc_cache_layer_regions(dc_cache* cache, int layer, dc_region** regions_dev, int32_t** n_dev);
 
-/* Waits for the stream and returns the device status word: DC_OK, DC_ERR_OVERFLOW or
- * DC_ERR_TIMEOUT as recorded by a kernel since the last reset.  Synchronous. */
+/* Waits for the stream and returns the device status word: DC_OK, or what a kernel recorded since the
+ * last reset: DC_ERR_OVERFLOW (Step 5 found more rectangles than max_regions), DC_ERR_TIMEOUT (a bounded
+ * device-side wait or walk ran out; the affected results are not valid), DC_ERR_ARG (a caller's rectangle
+ * outside its map was ignored).  Synchronous. */
 int dc_get_status(dc_cache* cache, int32_t* status_host);
 
 /* Kernels of this library launched on this cache since creation (for reporting). */

@@ -147,6 +147,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
         DC_CUDA(cudaGetDevice(&dev));
         DC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         c->num_sms = sms;
+        c->device = dev;
     }
     const size_t nblk = (size_t)S * c->Gx * c->Gy;
     for (int k = 0; k < 2; ++k) {

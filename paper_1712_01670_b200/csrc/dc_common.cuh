@@ -27,6 +27,13 @@ enum dc_stage { DC_ST_SEARCH = 0, DC_ST_VERIFY, DC_ST_MERGE, DC_ST_PROPAGATE, DC
 
 struct dc_prof;      // event pool, allocated when profiling is switched on
 
+// A tensor map (CUtensorMap, 128 bytes) encoded for one base address and one operand scheme, kept so that a launch
+// need not encode it again.  A layer's input alternates between at most two buffers (its producer's ping-pong maps).
+struct dc_tm_slot {
+    const void* base; int code, bn; bool valid;
+    alignas(64) unsigned char map[128];
+};
+
 struct dc_layer_rt {
     dc_layer_desc d;
     int in_h, in_w;                 // size of the input map (or of the frame)
@@ -47,6 +54,8 @@ struct dc_layer_rt {
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation
     int32_t* all_list;              // conv: every tile (used by full frames)
+    dc_tm_slot tm_a[2], tm_b;       // conv, bf16: tensor maps of the input (two bases) and of the weights
+    int tm_next;                    // which of tm_a[] a new input base replaces
 };
 
 // Everything one run of the matcher writes.  Two sets exist so that the matcher may already work on the
@@ -80,6 +89,8 @@ struct dc_cache {
     void* classify_table; int n_cached, classify_warps;   // all cached layers' classification in one launch (dc_regions.cu)
     size_t key_pitch;
     int num_sms;
+    int device;                     // ordinal of the device the cache lives on
+    int debug_stall_ms;             // > 0: the next tensor-core convolution launch is made to time out (tests)
     uint8_t* staging[2];            // device copies of host frames for dc_infer_frame_host (one in use, one prefetching)
     cudaStream_t copy_stream;       // dc_prefetch_frame_host copies on its own stream
     cudaEvent_t copied[2];
@@ -120,6 +131,20 @@ struct dc_prof_scope {
 };
 
 static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }
+
+// A kernel's opt-in to more than 48 KB of dynamic shared memory (cudaFuncSetAttribute) holds for one device only.
+// One of these per call site remembers on which devices it has been made.  Two threads may both find it unset and
+// both set it: same value, harmless.
+struct dc_once_per_device {
+    bool done[64];
+    bool first(int dev)
+    {
+        if (dev < 0 || dev >= 64) return true;        // beyond the table: set it every time
+        if (done[dev]) return false;
+        done[dev] = true;
+        return true;
+    }
+};
 
 // ---- kernels' host-side launchers (each returns DC_OK or DC_ERR_CUDA) ----
 int dc_launch_copy_frame(dc_cache* c, const uint8_t* frame, size_t pitch, uint8_t* dst);

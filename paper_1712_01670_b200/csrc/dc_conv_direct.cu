@@ -133,7 +133,7 @@ int dc_launch_conv(dc_cache* c, int layer, const void* in, void* out, const int3
     a.Cig = L.d.cin / G; a.Cog = L.d.cout / G; a.co_blocks = dc_div_up(a.Cog, CO_T);
     int co_groups = G * a.co_blocks;
     int gx = max_tiles < 1 ? 1 : max_tiles;
-    int cap = dc_div_up(148 * 8, co_groups);
+    int cap = dc_div_up(c->num_sms * 8, co_groups);
     if (gx > cap) gx = cap;
     dim3 grid(gx, co_groups);
     dc_prof_scope ps(c, DC_ST_CONV);
@@ -154,7 +154,7 @@ int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_d
     DC_CUDA(cudaMalloc(&L.weight, n * c->elt));
     DC_CUDA(cudaMalloc((void**)&L.bias, sizeof(float) * L.d.cout));
     c->bytes += n * c->elt + sizeof(float) * L.d.cout;
-    int grid = (int)((n + 255) / 256); if (grid > 148 * 8) grid = 148 * 8;
+    int grid = (int)((n + 255) / 256); if (grid > c->num_sms * 8) grid = c->num_sms * 8;
     if (c->cfg.dtype == DC_BF16) k_convert_weights<__nv_bfloat16><<<grid, 256, 0, c->stream>>>(w_dev, n, (__nv_bfloat16*)L.weight);
     else k_convert_weights<float><<<grid, 256, 0, c->stream>>>(w_dev, n, (float*)L.weight);
     DC_CUDA(cudaGetLastError());

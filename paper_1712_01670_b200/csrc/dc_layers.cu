@@ -270,7 +270,11 @@ __global__ void k_concat(const T* a, int Ca, const T* b, int Cb, size_t pixels, 
     }
 }
 
-inline int grid_for(size_t n, int block) { size_t g = (n + block - 1) / block; return (int)(g > 148 * 16 ? 148 * 16 : (g ? g : 1)); }
+inline int grid_for(const dc_cache* c, size_t n, int block)
+{
+    const size_t g = (n + block - 1) / block, cap = (size_t)c->num_sms * 16;
+    return (int)(g > cap ? cap : (g ? g : 1));
+}
 
 }  // namespace
 
@@ -282,8 +286,8 @@ int dc_launch_input_map(dc_cache* c, const uint8_t* frame, size_t pitch)
     int W = c->cfg.width, H = c->cfg.height;
     dc_prof_scope ps(c, DC_ST_INPUT);
     DISPATCH(c,
-        (k_input_map<float><<<grid_for(n, 256), 256, 0, c->stream>>>(frame, pitch, W, H, c->S, (const float*)c->pix_lut, (float*)c->input_map)),
-        (k_input_map<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>(frame, pitch, W, H, c->S, (const __nv_bfloat16*)c->pix_lut, (__nv_bfloat16*)c->input_map)));
+        (k_input_map<float><<<grid_for(c, n, 256), 256, 0, c->stream>>>(frame, pitch, W, H, c->S, (const float*)c->pix_lut, (float*)c->input_map)),
+        (k_input_map<__nv_bfloat16><<<grid_for(c, n, 256), 256, 0, c->stream>>>(frame, pitch, W, H, c->S, (const __nv_bfloat16*)c->pix_lut, (__nv_bfloat16*)c->input_map)));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -314,8 +318,8 @@ int dc_launch_maxpool(dc_cache* c, int layer, const void* in, void* out, const u
         const unsigned nv = (unsigned)(n * c->elt / 16);
         const int cv = L.d.cout * c->elt / 16;
         DISPATCH(c,
-            (k_maxpool2x2_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)in, L.in_h, L.in_w, cv, L.d.out_h, L.d.out_w, nv, (uint4*)out)),
-            (k_maxpool2x2_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)in, L.in_h, L.in_w, cv, L.d.out_h, L.d.out_w, nv, (uint4*)out)));
+            (k_maxpool2x2_vec<float><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const uint4*)in, L.in_h, L.in_w, cv, L.d.out_h, L.d.out_w, nv, (uint4*)out)),
+            (k_maxpool2x2_vec<__nv_bfloat16><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const uint4*)in, L.in_h, L.in_w, cv, L.d.out_h, L.d.out_w, nv, (uint4*)out)));
         c->launches += 1;
         DC_CUDA(cudaGetLastError());
         return DC_OK;
@@ -323,16 +327,16 @@ int dc_launch_maxpool(dc_cache* c, int layer, const void* in, void* out, const u
     if ((L.d.cout * c->elt) % 16 == 0) {
         size_t nv = n * c->elt / 16;
         DISPATCH(c,
-            (k_maxpool_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)out, masks, L.tiles_x, L.tiles_y)),
-            (k_maxpool_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)out, masks, L.tiles_x, L.tiles_y)));
+            (k_maxpool_vec<float><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)out, masks, L.tiles_x, L.tiles_y)),
+            (k_maxpool_vec<__nv_bfloat16><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)out, masks, L.tiles_x, L.tiles_y)));
         c->launches += 1;
         DC_CUDA(cudaGetLastError());
         return DC_OK;
     }
     if (masks) return DC_ERR_STATE;                             // cached pooling needs 16-byte pixels (checked at creation)
     DISPATCH(c,
-        (k_maxpool<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)out)),
-        (k_maxpool<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)out)));
+        (k_maxpool<float><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const float*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (float*)out)),
+        (k_maxpool<__nv_bfloat16><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.in_h, L.in_w, L.d.cout, c->S, L.d, (__nv_bfloat16*)out)));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -346,12 +350,12 @@ int dc_launch_add(dc_cache* c, int layer, const void* a, const void* b)
     if ((n * c->elt) % 16 == 0) {                                 // maps come from cudaMalloc: 256-byte aligned
         const size_t nv = n * c->elt / 16;
         DISPATCH(c,
-            (k_add_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, (const uint4*)b, nv, L.d.relu, (uint4*)L.map[0])),
-            (k_add_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, (const uint4*)b, nv, L.d.relu, (uint4*)L.map[0])));
+            (k_add_vec<float><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const uint4*)a, (const uint4*)b, nv, L.d.relu, (uint4*)L.map[0])),
+            (k_add_vec<__nv_bfloat16><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const uint4*)a, (const uint4*)b, nv, L.d.relu, (uint4*)L.map[0])));
     } else {
         DISPATCH(c,
-            (k_add<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, (const float*)b, n, L.d.relu, (float*)L.map[0])),
-            (k_add<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, n, L.d.relu, (__nv_bfloat16*)L.map[0])));
+            (k_add<float><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const float*)a, (const float*)b, n, L.d.relu, (float*)L.map[0])),
+            (k_add<__nv_bfloat16><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, (const __nv_bfloat16*)b, n, L.d.relu, (__nv_bfloat16*)L.map[0])));
     }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
@@ -366,12 +370,12 @@ int dc_launch_relu(dc_cache* c, int layer, const void* a)
     if ((n * c->elt) % 16 == 0) {
         const size_t nv = n * c->elt / 16;
         DISPATCH(c,
-            (k_add_vec<float><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, nullptr, nv, 1, (uint4*)L.map[0])),
-            (k_add_vec<__nv_bfloat16><<<grid_for(nv, 256), 256, 0, c->stream>>>((const uint4*)a, nullptr, nv, 1, (uint4*)L.map[0])));
+            (k_add_vec<float><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const uint4*)a, nullptr, nv, 1, (uint4*)L.map[0])),
+            (k_add_vec<__nv_bfloat16><<<grid_for(c, nv, 256), 256, 0, c->stream>>>((const uint4*)a, nullptr, nv, 1, (uint4*)L.map[0])));
     } else {
         DISPATCH(c,
-            (k_relu<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)a, n, (float*)L.map[0])),
-            (k_relu<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, n, (__nv_bfloat16*)L.map[0])));
+            (k_relu<float><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const float*)a, n, (float*)L.map[0])),
+            (k_relu<__nv_bfloat16><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, n, (__nv_bfloat16*)L.map[0])));
     }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
@@ -388,8 +392,8 @@ int dc_launch_lrn(dc_cache* c, int layer, const void* in, void* out, const uint3
     const float kappa = (float)(defaults ? 1.0 : c->cfg.lrn_k);
     dc_prof_scope ps(c, DC_ST_POINTWISE);
     DISPATCH(c,
-        (k_lrn<float><<<grid_for(n, 256), 256, 0, c->stream>>>((const float*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (float*)out, masks, L.tiles_x, L.tiles_y)),
-        (k_lrn<__nv_bfloat16><<<grid_for(n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (__nv_bfloat16*)out, masks, L.tiles_x, L.tiles_y)));
+        (k_lrn<float><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const float*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (float*)out, masks, L.tiles_x, L.tiles_y)),
+        (k_lrn<__nv_bfloat16><<<grid_for(c, n, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)in, L.d.out_h, L.d.out_w, L.d.cout, c->S, r, alpha / (win * win), beta, kappa, (__nv_bfloat16*)out, masks, L.tiles_x, L.tiles_y)));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -401,8 +405,8 @@ int dc_launch_concat(dc_cache* c, int layer, const void* a, int ca, const void* 
     const size_t pixels = (size_t)c->S * L.d.out_h * L.d.out_w;
     dc_prof_scope ps(c, DC_ST_POINTWISE);
     DISPATCH(c,
-        (k_concat<float><<<grid_for(pixels * L.d.cout, 256), 256, 0, c->stream>>>((const float*)a, ca, (const float*)b, cb, pixels, (float*)L.map[0])),
-        (k_concat<__nv_bfloat16><<<grid_for(pixels * L.d.cout, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, ca, (const __nv_bfloat16*)b, cb, pixels, (__nv_bfloat16*)L.map[0])));
+        (k_concat<float><<<grid_for(c, pixels * L.d.cout, 256), 256, 0, c->stream>>>((const float*)a, ca, (const float*)b, cb, pixels, (float*)L.map[0])),
+        (k_concat<__nv_bfloat16><<<grid_for(c, pixels * L.d.cout, 256), 256, 0, c->stream>>>((const __nv_bfloat16*)a, ca, (const __nv_bfloat16*)b, cb, pixels, (__nv_bfloat16*)L.map[0])));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;

@@ -30,6 +30,7 @@ struct MatchArgs {
     int edge_only;                       // generic search: 1 = only blocks clipped by the frame edge, 2 = only blocks clipped in width (the rest has a fast kernel)
     uint32_t limit[4];
     int16_t* mv; uint32_t* sse; uint8_t* matched; int32_t* acc; int32_t* gmv;
+    int32_t* status;                     // device status word: a walk ended by its step limit records DC_ERR_TIMEOUT
 };
 
 __device__ __forceinline__ unsigned long long cand_key(uint32_t sse, int dx, int dy)
@@ -176,8 +177,9 @@ __global__ void __launch_bounds__(WARPS * 32) k_search(MatchArgs a)
         // large diamond until its centre wins, then one small diamond
         const int lx[8] = {0, -1, 1, -2, 2, -1, 1, 0}, ly[8] = {-2, -1, -1, 0, 0, 1, 1, 2};
         const int sx[4] = {0, -1, 1, 0}, sy[4] = {-1, 0, 0, 1};
-        const int max_steps = (2 * a.R + 1) * (2 * a.R + 1);   // every move strictly lowers the key
-        for (int step = 0; step < max_steps; ++step) {
+        const int max_steps = (2 * a.R + 1) * (2 * a.R + 1);   // every move strictly lowers the key: never reached
+        bool settled = false;
+        for (int step = 0; step < max_steps && !settled; ++step) {
             int cx = bx_, cy = by_;
 #pragma unroll 1
             for (int i = 0; i < 8; ++i) {
@@ -187,8 +189,9 @@ __global__ void __launch_bounds__(WARPS * 32) k_search(MatchArgs a)
                 unsigned long long k = cand_key(v, dx, dy);
                 if (k < bk) { bk = k; bs = v; bx_ = dx; by_ = dy; }
             }
-            if (bx_ == cx && by_ == cy) break;
+            settled = bx_ == cx && by_ == cy;
         }
+        if (!settled && c.lane == 0) atomicExch(a.status, (int)DC_ERR_TIMEOUT);   // the limit ended the walk: result not valid
         int cx = bx_, cy = by_;
 #pragma unroll 1
         for (int i = 0; i < 4; ++i) {
@@ -538,6 +541,9 @@ __device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<1
         const uint32_t kt = ((uint32_t)(abs(dx) + abs(dy)) << 16) | ((uint32_t)(dy + 128) << 8) | (uint32_t)(dx + 128);
         if (ok && (ks < w.bs || (ks == w.bs && kt < w.bt))) { w.bs = ks; w.bt = kt; }
     }
+    // Every move strictly lowers the key, so a walk ends long before max_passes.  Should the limit ever end one, its
+    // result is not the walk's: the status word says so.
+    if (w.st == 0) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
 }
 
 // Window shared by the VS x 8 blocks of a CTA; every block may move WR pixels from zero motion inside it.
@@ -880,7 +886,10 @@ __global__ void __launch_bounds__(LPB * 8, MINB) k_search_ds16q_long(MatchArgs a
         }
         __syncwarp();
         lockstep_walk<LPB, 0>(a, rc, bw_, q, dx_lo, dx_span, dy_lo, dy_span, w);
-        if (w.st == 2 && rounds >= limit) w.st = 1;
+        if (w.st == 2 && rounds >= limit) {                          // never reached; a walk cut here is not valid
+            w.st = 1;
+            if (q == 0) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
+        }
         if (w.st == 1 && q == 0) publish_block(a, s, g, 16, bh, ((unsigned long long)w.bs << 32) | w.bt);
     }
 }
@@ -1182,6 +1191,7 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
     a.Gx = c->Gx; a.Gy = c->Gy; a.S = c->S; a.search = c->cfg.search; a.skip_k = c->cfg.skip_k; a.region_mode = c->cfg.region_mode; a.edge_only = 0;
     for (int i = 0; i < 4; ++i) a.limit[i] = c->sse_limit[i];
     a.mv = c->blk_mv; a.sse = c->blk_sse; a.matched = c->matched; a.acc = c->mv_acc; a.gmv = c->gmv;
+    a.status = c->status;
     // Step 3 sums and, behind them, the counter of walks handed to the second search phase
     DC_CUDA(cudaMemsetAsync(c->mv_acc, 0, sizeof(int32_t) * (4 * c->S + 4), c->stream));
     int32_t* long_count = c->mv_acc + 4 * c->S;
@@ -1210,10 +1220,9 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
         const int wr = s0 > 0 ? 2 * s0 - 1 : 1;
         const int words = ((((112 + 2 * wr) * 3 + 15) >> 2) + 13 + 3) & ~3, pitch = words | 1;
         const size_t smem = tss_window_bytes(a.R);
-        static bool attr_set = false;
-        if (!attr_set) {
+        static dc_once_per_device attr_set;
+        if (attr_set.first(c->device)) {
             DC_CUDA(cudaFuncSetAttribute(k_search_tss16q<TSS_LPB, TSS_VS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 160 * 1024));
-            attr_set = true;
         }
         {
             dc_prof_scope ps(c, DC_ST_SEARCH);
@@ -1229,11 +1238,10 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
     } else if (a.B == 16 && a.search == DC_SEARCH_EXHAUSTIVE && a.R <= E_MAXR && a.W >= 16 && a.H >= 16) {
         const int chunks = (2 * a.R + 1 + E_DY - 1) / E_DY;
         const size_t smem = ((size_t)(16 + chunks * E_DY - 1) * E_PITCH + 8 * 192) * sizeof(uint32_t);
-        static bool attr_set = false;
-        if (!attr_set) {
+        static dc_once_per_device attr_set;
+        if (attr_set.first(c->device)) {
             DC_CUDA(cudaFuncSetAttribute(k_search_es16, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)(((size_t)E_MAXROWS * E_PITCH + 8 * 192) * sizeof(uint32_t))));
-            attr_set = true;
         }
         {
             dc_prof_scope ps(c, DC_ST_SEARCH);

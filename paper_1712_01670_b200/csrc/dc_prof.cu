@@ -1,4 +1,5 @@
 // Optional event profiler: one cudaEvent pair around every launch site, summed per stage.
+#include <new>
 #include <vector>
 
 #include "dc_common.cuh"
@@ -26,14 +27,22 @@ dc_prof_scope::dc_prof_scope(dc_cache* cache, int st) : c(cache), stage(st)
     if (p->open_start) cudaEventRecord(p->open_start, c->stream);
 }
 
+// The event lists grow with push_back; a failed allocation must not leave through the C ABI: the pair is
+// dropped (its events destroyed) and that launch goes untimed.
+static bool keep_event(std::vector<cudaEvent_t>& v, cudaEvent_t e)
+{
+    try { v.push_back(e); return true; } catch (...) { cudaEventDestroy(e); return false; }
+}
+
 dc_prof_scope::~dc_prof_scope()
 {
     dc_prof* p = c->prof;
     if (!p || !p->on || !p->open_start) return;
     cudaEvent_t b = p->get();
-    if (!b) { p->pool.push_back(p->open_start); p->open_start = nullptr; return; }
+    if (!b) { keep_event(p->pool, p->open_start); p->open_start = nullptr; return; }
     cudaEventRecord(b, c->stream);
-    p->pairs.push_back({p->open_start, b, stage});
+    try { p->pairs.push_back({p->open_start, b, stage}); }
+    catch (...) { cudaEventDestroy(p->open_start); cudaEventDestroy(b); }
     p->open_start = nullptr;
 }
 
@@ -49,7 +58,8 @@ void dc_prof_release(dc_cache* c)
 extern "C" int dc_cache_set_profiling(dc_cache* c, int enable)
 {
     if (!c) return DC_ERR_ARG;
-    if (!c->prof) c->prof = new dc_prof();
+    if (!c->prof) c->prof = new (std::nothrow) dc_prof();
+    if (!c->prof) return DC_ERR_ALLOC;
     c->prof->on = enable != 0;
     return DC_OK;
 }
@@ -66,7 +76,7 @@ extern "C" int dc_cache_profile(dc_cache* c, float* ms_host, int64_t* launches_h
             ms_host[pr.stage] += ms;
             if (launches_host) launches_host[pr.stage] += 1;
         }
-        c->prof->pool.push_back(pr.a); c->prof->pool.push_back(pr.b);
+        keep_event(c->prof->pool, pr.a); keep_event(c->prof->pool, pr.b);
     }
     cudaGetLastError();
     c->prof->pairs.clear();

@@ -6,8 +6,9 @@
 //                    so no synchronisation is needed; a vanished rectangle is all zeros.
 //   k_classify_copy  one warp per 16x8 output tile: lanes test the stream's rectangles against
 //                    the tile, OR their coverage into a 128-bit bitmap, the warp copies each
-//                    covered span from the cached map with 16-byte vectors, and tiles that
-//                    still hold uncovered pixels are appended to the layer's dirty list.
+//                    covered row span from the cached map with bulk copies (global -> shared ->
+//                    global through the copy engine, no registers), and tiles that still hold
+//                    uncovered pixels are appended to the layer's dirty list.
 #include "dc_common.cuh"
 
 namespace {
@@ -83,7 +84,7 @@ __global__ void k_propagate(const dc_layer_desc* layers, const int32_t* in_hw, i
 {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     int s = blockIdx.y;
-    if (i >= n_in[s]) return;
+    if (i >= max_regions || i >= n_in[s]) return;          // a caller's count beyond the table is cut, never written
     const size_t slot = (size_t)s * max_regions + i;
     const size_t layer_stride = (size_t)S * max_regions;
     const dc_region r0 = in[slot];
@@ -98,6 +99,62 @@ __global__ void k_propagate(const dc_layer_desc* layers, const int32_t* in_hw, i
     }
 }
 
+// ---- bulk copies (cp.async.bulk) for the reuse copy ----
+constexpr int kCopyWarps = 4;                    // warps per CTA
+constexpr int kSeg = 512;                        // bytes one lane moves per round; a row span is cut into such segments
+constexpr int kStageBytes = 32 * kSeg;           // staging of one warp: one segment per lane
+constexpr size_t kCopySmem = (size_t)kCopyWarps * kStageBytes + 128 + kCopyWarps * sizeof(unsigned long long);
+constexpr unsigned long long kCopyWaitNs = 2000000000ull;   // a warp gives up on its staging barrier after 2 s (far beyond any copy)
+
+__device__ __forceinline__ uint32_t rs_smem(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void rs_bar_init(void* bar)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(rs_smem(bar)) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ __forceinline__ void rs_expect(void* bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(rs_smem(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool rs_try(void* bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(rs_smem(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void rs_load(void* dst_smem, const void* src, uint32_t bytes, void* bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(rs_smem(dst_smem)), "l"(src), "r"(bytes), "r"(rs_smem(bar)) : "memory");
+}
+__device__ __forceinline__ void rs_store(void* dst, const void* src_smem, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(dst), "r"(rs_smem(src_smem)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ unsigned long long rs_now()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait for a phase of the staging barrier; false when the limit passed.
+__device__ __forceinline__ bool rs_wait(void* bar, uint32_t parity)
+{
+    if (rs_try(bar, parity)) return true;
+    const unsigned long long t0 = rs_now();
+    for (unsigned spin = 1;; ++spin) {
+        if (rs_try(bar, parity)) return true;
+        if ((spin & 255u) == 0 && rs_now() - t0 > kCopyWaitNs) return false;
+    }
+}
+__device__ __forceinline__ void rs_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void rs_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
+__device__ __forceinline__ void rs_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+// What a warp needs for its bulk copies: 16 KB of staging, one mbarrier and its phase.
+struct CopyLane { uint8_t* stage; unsigned long long* bar; uint32_t phase; bool dead; };
+
 struct ClassifyArgs {
     const dc_region* regions; const int32_t* n_regions; int max_regions;
     const uint8_t* prev; uint8_t* out;           // maps as bytes
@@ -106,9 +163,10 @@ struct ClassifyArgs {
     uint32_t* masks; int32_t* dirty_list; int32_t* dirty_count; int32_t* reuse_px;
     const int32_t* alive;                        // per stream: rectangles alive at this layer, or NULL (unknown)
     unsigned long long* reused_total;
+    int32_t* status;                             // device status word
 };
 
-__device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int tile, const int lane)
+__device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int tile, const int lane, CopyLane& cl)
 {
     const int per = a.tiles_x * a.tiles_y;
     const int s = tile / per, t = tile - s * per, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
@@ -116,7 +174,7 @@ __device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int t
     const int X1 = min(X0 + DC_TILE_W, a.Wo), Y1 = min(Y0 + DC_TILE_H, a.Ho);
     const dc_region* regs = a.regions + (size_t)s * a.max_regions;
     // every rectangle of this stream has eroded away before this layer: nothing to test or copy
-    const int n = (a.alive && a.alive[s] == 0) ? 0 : a.n_regions[s];
+    const int n = (a.alive && a.alive[s] == 0) ? 0 : min(a.n_regions[s], a.max_regions);
     const size_t map_base = (size_t)s * a.Ho * a.Wo * a.px_bytes;
     uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;      // bit (row * DC_TILE_W + col) of the tile, row-major
     for (int base = 0; base < n; base += 32) {
@@ -125,6 +183,15 @@ __device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int t
         int ix0 = 0, ix1 = 0, iy0 = 0, iy1 = 0;
         if (i < n) {
             r = regs[i];
+            // Rectangles made by Step 5 and Table 2 lie inside the map on both sides.  One that does not (a caller's
+            // own list) is not reused: neither side is ever addressed outside its map; the status word records it.
+            const bool inside = r.x >= 0 && r.y >= 0 && r.sx >= 0 && r.sy >= 0 && r.w <= a.Wo && r.h <= a.Ho &&
+                                r.x <= a.Wo - r.w && r.y <= a.Ho - r.h && r.sx <= a.Wo - r.w && r.sy <= a.Ho - r.h;
+            if (r.w <= 0 || r.h <= 0) r = empty_region();
+            else if (!inside) {
+                if (t == 0 && a.status) atomicExch(a.status, (int)DC_ERR_ARG);
+                r = empty_region();
+            }
             ix0 = max(r.x, X0); ix1 = min(r.x + r.w, X1);
             iy0 = max(r.y, Y0); iy1 = min(r.y + r.h, Y1);
         }
@@ -145,12 +212,36 @@ __device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int t
             int rsx = __shfl_sync(0xffffffffu, r.sx, src_lane), rsy = __shfl_sync(0xffffffffu, r.sy, src_lane);
             int cx0 = __shfl_sync(0xffffffffu, ix0, src_lane), cx1 = __shfl_sync(0xffffffffu, ix1, src_lane);
             int cy0 = __shfl_sync(0xffffffffu, iy0, src_lane), cy1 = __shfl_sync(0xffffffffu, iy1, src_lane);
-            int span_vec = (cx1 - cx0) * (a.px_bytes >> 4);          // 16-byte vectors per row
-            for (int y = cy0; y < cy1; ++y) {
-                const uint4* src = (const uint4*)(a.prev + map_base +
-                    ((size_t)(y - ry + rsy) * a.Wo + (cx0 - rx + rsx)) * a.px_bytes);
-                uint4* dst = (uint4*)(a.out + map_base + ((size_t)y * a.Wo + cx0) * a.px_bytes);
-                for (int v = lane; v < span_vec; v += 32) dst[v] = __ldg(src + v);
+            // Section 5 "Reuse", step 1.  Inside the tile the rectangle is (cy1 - cy0) row spans, each contiguous in both
+            // maps (all channels of cx1 - cx0 pixels).  Spans are cut into segments of kSeg bytes; per round every lane
+            // moves one segment: a bulk copy into the warp's staging, then a bulk copy out to the new map.  Addresses
+            // and sizes are multiples of 16 bytes (px_bytes is).
+            const int span_bytes = (cx1 - cx0) * a.px_bytes;
+            const int segs = (span_bytes + kSeg - 1) / kSeg, items = (cy1 - cy0) * segs;
+            const uint8_t* src0 = a.prev + map_base + ((size_t)(cy0 - ry + rsy) * a.Wo + (cx0 - rx + rsx)) * a.px_bytes;
+            uint8_t* dst0 = a.out + map_base + ((size_t)cy0 * a.Wo + cx0) * a.px_bytes;
+            const size_t row_pitch = (size_t)a.Wo * a.px_bytes;
+            for (int i0 = 0; i0 < items && !cl.dead; i0 += 32) {
+                const int it = i0 + lane;
+                const bool on = it < items;
+                const int row = on ? it / segs : 0, sg = it - row * segs;
+                const uint32_t bytes = on ? (uint32_t)min(kSeg, span_bytes - sg * kSeg) : 0u;
+                const size_t off = (size_t)row * row_pitch + (size_t)sg * kSeg;
+                const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+                if (lane == 0) rs_expect(cl.bar, total);
+                __syncwarp();
+                if (on) rs_load(cl.stage + lane * kSeg, src0 + off, bytes, cl.bar);
+                const bool landed = rs_wait(cl.bar, cl.phase);
+                if (!__all_sync(0xffffffffu, landed)) {                     // never seen; leave rather than spin for ever
+                    if (lane == 0 && a.status) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
+                    cl.dead = true;
+                    break;
+                }
+                cl.phase ^= 1u;
+                if (on) rs_store(dst0 + off, cl.stage + lane * kSeg, bytes);
+                rs_commit();
+                rs_wait_read();                                             // staging may be overwritten by the next round
+                __syncwarp();
             }
         }
     }
@@ -169,11 +260,27 @@ __device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int t
     }
 }
 
-__global__ void __launch_bounds__(256) k_classify_copy(ClassifyArgs a)
+// Staging and barrier of this warp, carved from the CTA's dynamic shared memory.
+__device__ __forceinline__ CopyLane copy_lane_setup(uint8_t* smem_raw)
 {
-    const int tile = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (tile >= a.tiles_x * a.tiles_y * a.S) return;
-    classify_tile(a, tile, threadIdx.x & 31);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
+    CopyLane cl;
+    cl.stage = base + (size_t)warp * kStageBytes;
+    cl.bar = (unsigned long long*)(base + (size_t)kCopyWarps * kStageBytes) + warp;
+    cl.phase = 0; cl.dead = false;
+    if (lane == 0) rs_bar_init(cl.bar);
+    __syncwarp();
+    return cl;
+}
+
+__global__ void __launch_bounds__(kCopyWarps * 32) k_classify_copy(ClassifyArgs a)
+{
+    extern __shared__ uint8_t copy_smem[];
+    CopyLane cl = copy_lane_setup(copy_smem);
+    const int tile = blockIdx.x * kCopyWarps + (threadIdx.x >> 5);
+    if (tile < a.tiles_x * a.tiles_y * a.S) classify_tile(a, tile, threadIdx.x & 31, cl);
+    rs_wait_all();
 }
 
 // Every cached layer of a frame in one launch: the bitmaps, reuse copies and dirty lists of a layer depend only
@@ -183,14 +290,16 @@ struct ClassifyLayer {
     const dc_region* regions; uint8_t* map[2];
     int Ho, Wo, px_bytes, tiles_x, tiles_y, first_warp;
     uint32_t* masks; int32_t* dirty_list; int32_t* dirty_count; int32_t* reuse_px;
-    const int32_t* alive; unsigned long long* reused_total;
+    const int32_t* alive; unsigned long long* reused_total; int32_t* status;
 };
 
-__global__ void __launch_bounds__(256) k_classify_copy_all(const ClassifyLayer* layers, int n_cached, int total_warps,
-                                                           const int32_t* n_regions, int max_regions, int S, int cur)
+__global__ void __launch_bounds__(kCopyWarps * 32) k_classify_copy_all(const ClassifyLayer* layers, int n_cached, int total_warps,
+                                                                       const int32_t* n_regions, int max_regions, int S, int cur)
 {
-    const int w = blockIdx.x * 8 + (threadIdx.x >> 5);
-    if (w >= total_warps) return;
+    extern __shared__ uint8_t copy_smem[];
+    CopyLane cl = copy_lane_setup(copy_smem);
+    const int w = blockIdx.x * kCopyWarps + (threadIdx.x >> 5);
+    if (w >= total_warps) return;                       // no copy was issued by this warp
     int lo = 0, hi = n_cached - 1;
     while (lo < hi) {
         const int mid = (lo + hi + 1) >> 1;
@@ -202,8 +311,9 @@ __global__ void __launch_bounds__(256) k_classify_copy_all(const ClassifyLayer* 
     a.prev = L.map[cur]; a.out = L.map[cur ^ 1];
     a.Ho = L.Ho; a.Wo = L.Wo; a.px_bytes = L.px_bytes; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y; a.S = S;
     a.masks = L.masks; a.dirty_list = L.dirty_list; a.dirty_count = L.dirty_count; a.reuse_px = L.reuse_px;
-    a.alive = L.alive; a.reused_total = L.reused_total;
-    classify_tile(a, w - L.first_warp, threadIdx.x & 31);
+    a.alive = L.alive; a.reused_total = L.reused_total; a.status = L.status;
+    classify_tile(a, w - L.first_warp, threadIdx.x & 31, cl);
+    rs_wait_all();
 }
 
 }  // namespace
@@ -226,6 +336,7 @@ int dc_build_classify_table(dc_cache* c)
         e.masks = L.masks; e.dirty_list = L.dirty_list; e.dirty_count = c->dirty_count + i;
         e.reuse_px = c->reuse_px + (size_t)i * c->S; e.alive = c->alive + (size_t)i * c->S;
         e.reused_total = c->reused_total + i;
+        e.status = c->status;
         warps += L.tiles_x * L.tiles_y * c->S;
     }
     c->n_cached = k; c->classify_warps = warps;
@@ -246,7 +357,10 @@ int dc_launch_classify_all(dc_cache* c, int cur)
     if (c->n_cached <= 0) return DC_OK;
     {
         dc_prof_scope ps(c, DC_ST_CLASSIFY_COPY);
-        k_classify_copy_all<<<dc_div_up(c->classify_warps, 8), 256, 0, c->stream>>>(
+        static dc_once_per_device attr_set;
+        if (attr_set.first(c->device))
+            DC_CUDA(cudaFuncSetAttribute(k_classify_copy_all, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCopySmem));
+        k_classify_copy_all<<<dc_div_up(c->classify_warps, kCopyWarps), kCopyWarps * 32, kCopySmem, c->stream>>>(
             (const ClassifyLayer*)c->classify_table, c->n_cached, c->classify_warps, c->n_regions, c->max_regions, c->S, cur);
     }
     c->launches += 1;
@@ -279,10 +393,14 @@ int dc_launch_classify_copy(dc_cache* c, int layer, const dc_region* regions, co
     a.masks = L.masks; a.dirty_list = L.dirty_list; a.dirty_count = c->dirty_count + layer;
     a.reuse_px = c->reuse_px + (size_t)layer * c->S;
     a.reused_total = c->reused_total + layer;
+    a.status = c->status;
     a.alive = (regions == c->table + (size_t)layer * c->S * c->max_regions) ? c->alive + (size_t)layer * c->S : nullptr;
     // the caller has zeroed dirty_count[layer] and reuse_px[layer][*] on the stream
     int tiles = L.tiles_x * L.tiles_y * c->S;
-    { dc_prof_scope ps(c, DC_ST_CLASSIFY_COPY); k_classify_copy<<<dc_div_up(tiles, 8), 256, 0, c->stream>>>(a); }
+    static dc_once_per_device attr_set;
+    if (attr_set.first(c->device))
+        DC_CUDA(cudaFuncSetAttribute(k_classify_copy, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCopySmem));
+    { dc_prof_scope ps(c, DC_ST_CLASSIFY_COPY); k_classify_copy<<<dc_div_up(tiles, kCopyWarps), kCopyWarps * 32, kCopySmem, c->stream>>>(a); }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;

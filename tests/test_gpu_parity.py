@@ -377,9 +377,50 @@ def test_conv_partial(dtype, hi, wi, cin, cout, k, s, p, relu):
             want, reused = orc.conv_reuse(xq[s_], L, wq, bias, quant, pq[s_], per_stream[s_])
             U.assert_map_close(full[s_], want_full, bf16, "full")
             U.assert_map_close(part[s_], want, bf16, "partial")
+            if bf16:
+                U.assert_map_close_per_element(full[s_], want_full, "full, per element")
             m = reused.astype(bool)
             got = part[s_].float().cpu().numpy().astype(np.float64)
             assert m.any() and np.array_equal(got[m], want[m]), "reused pixels must be bit-equal copies of the cached map"
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
+
+
+def test_conv_partial_ignores_rectangles_outside_the_map():
+    """A caller's rectangle that leaves the map on either side, or a count beyond max_regions, must not become an
+    out-of-bounds access: such rectangles are not reused (their pixels are convolved) and the status word says so."""
+    g = rng(77)
+    hi, wi, cout = 37, 45, 16
+    b = nets.NetBuilder(hi, wi, 3)
+    b.conv(-1, cout, 3, 1, 1, 1)
+    L = b.layers[0]
+    wts = g.normal(0, 0.2, size=(cout, 3, 3, 3)).astype(np.float32)
+    bias = g.normal(0, 0.1, size=cout).astype(np.float32)
+    x = g.normal(size=(1, hi, wi, 3)).astype(np.float32).astype(np.float64)
+    prev = g.normal(size=(1, hi, wi, cout)).astype(np.float32).astype(np.float64)
+    dc = DeepCache(wi, hi, [dict(L)], [wts], [bias], n_streams=1, block=16, search_range=4, dtype=B.DC_FP32, max_regions=8)
+    try:
+        good = (4, 5, 10, 9, 7, 2)
+        bad = [(30, 3, 10, 6, 40, 3),            # cached side leaves the map on the right
+               (2, 30, 5, 6, 2, -1),             # cached side starts above the map
+               (-3, 20, 8, 4, 0, 20),            # current side starts left of the map
+               (20, 20, 100, 4, 0, 0),           # wider than the map
+               (10, 25, 2 ** 30, 2 ** 30, 5, 5),  # sizes that would overflow a sum
+               (12, 12, -4, 3, 1, 1)]            # negative width: an empty slot, not an error
+        regs = torch.zeros((1, dc.max_regions, 6), dtype=torch.int32)
+        for i, r in enumerate([good] + bad):
+            regs[0, i] = torch.tensor(r, dtype=torch.int32)
+        xin, pin = torch.from_numpy(x).float().cuda(), torch.from_numpy(prev).float().cuda()
+        # a count far beyond the table: cut to max_regions (the eighth slot is all zeros)
+        part = dc.conv_partial(0, xin, pin, regs.cuda(), torch.tensor([1000], dtype=torch.int32).cuda())
+        only_good = np.zeros(1, orc.REGION_DTYPE); only_good[0] = good
+        want, reused = orc.conv_reuse(x[0], L, wts, bias, orc.QUANT_NONE, prev[0], only_good)
+        U.assert_map_close(part[0], want, False, "bad rectangles ignored")
+        m = reused.astype(bool)
+        assert np.array_equal(part[0].cpu().numpy().astype(np.float64)[m], want[m])
+        assert dc.status() == B.DC_ERR_ARG
+        dc.reset()
         assert dc.status() == B.DC_OK
     finally:
         dc.close()
@@ -532,6 +573,50 @@ def test_region_overflow_sets_the_status_word():
         assert dc.status() == B.DC_ERR_OVERFLOW
         dc.reset()
         assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("cin,k", [(64, 3), (32, 1), (3, 3)])      # column-slab / patch kernels, tap-by-tap kernel, few-channel kernel
+def test_bounded_device_waits_run_out_and_the_cache_stays_usable(cin, k):
+    """Failure detection without a fault: one convolution launch is armed so that its producer issues no copy.  The
+    other roles' waits then run out after a few milliseconds instead of spinning for ever: the kernel returns, the
+    status word reads DC_ERR_TIMEOUT, tensor memory is free again, and the next launch on the same cache is correct."""
+    import ctypes
+    g = rng(90 + cin)
+    hi = wi = 40
+    cout = 64
+    nb = nets.NetBuilder(hi, wi)
+    if cin == 3:
+        nb.conv(-1, cout, k, 1, k // 2, 1)
+        li = 0
+        ws = [g.normal(0, 0.2, size=(cout, k, k, 3)).astype(np.float32)]
+        bs = [g.normal(0, 0.1, size=cout).astype(np.float32)]
+    else:
+        a = nb.conv(-1, cin, 1, 1, 0)
+        nb.conv(a, cout, k, 1, k // 2, 1)
+        li = 1
+        ws = [np.zeros((cin, 1, 1, 3), np.float32), g.normal(0, 0.1, size=(cout, k, k, cin)).astype(np.float32)]
+        bs = [np.zeros(cin, np.float32), g.normal(0, 0.1, size=cout).astype(np.float32)]
+    L = nb.layers[li]
+    x = orc.quant_array(g.normal(size=(hi, wi, cin)), orc.QUANT_BF16)
+    want, _ = orc.conv_reuse(x, L, orc.quant_array(ws[li], orc.QUANT_BF16), bs[li], orc.QUANT_BF16)
+    dc = DeepCache(wi, hi, nb.layers, ws, bs, n_streams=1, block=16, search_range=4, dtype=B.DC_BF16)
+    try:
+        stall = B.load().dc_debug_stall_next_conv
+        stall.restype = ctypes.c_int
+        stall.argtypes = [ctypes.c_void_p, ctypes.c_int]
+        xin = torch.from_numpy(x[None]).to(torch.bfloat16).cuda()
+        U.assert_map_close(dc.conv_partial(li, xin)[0], want, True, "before")
+        assert dc.status() == B.DC_OK
+        assert stall(dc.handle, 5) == B.DC_OK
+        dc.conv_partial(li, xin)                                   # returns normally; its output is not valid
+        assert dc.status() == B.DC_ERR_TIMEOUT
+        dc.reset()                                                 # clears the status word
+        assert dc.status() == B.DC_OK
+        U.assert_map_close(dc.conv_partial(li, xin)[0], want, True, "after")
+        assert dc.status() == B.DC_OK
+        assert stall(dc.handle, 0) == B.DC_ERR_ARG and stall(None, 5) == B.DC_ERR_ARG
     finally:
         dc.close()
 
