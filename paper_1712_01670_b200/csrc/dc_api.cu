@@ -73,7 +73,7 @@ bool layer_executable(const dc_layer_desc& L, int in_h, int in_w)
 
 int validate(const dc_config* cfg, const dc_layer_desc* layers, int n)
 {
-    if (cfg->channels != 3 || cfg->width < 1 || cfg->height < 1 || cfg->n_streams < 1) return DC_ERR_CONFIG;
+    if (cfg->channels != 3 || cfg->width < 1 || cfg->height < 1 || cfg->n_streams < 1 || cfg->n_streams > 65535) return DC_ERR_CONFIG;
     if (cfg->block < 4 || cfg->block > 32 || cfg->range < 0 || cfg->range > 64) return DC_ERR_CONFIG;
     if (cfg->search < DC_SEARCH_EXHAUSTIVE || cfg->search > DC_SEARCH_THREE_STEP) return DC_ERR_CONFIG;
     if (cfg->cache_pool != 0 && cfg->cache_pool != 1) return DC_ERR_CONFIG;

@@ -5,11 +5,12 @@
 //              (two aligned loads + funnel shift), |a-b| per byte by vabsdiff4, squares summed
 //              by dp4a, warp-reduced.  Candidates are ordered by (SSE, |dx|+|dy|, dy, dx).
 //              Blocks that pass the PSNR bound add their vector to the Step 3 sums.
-//   k_search_ds16q  Step 2 for 16-pixel blocks with diamond search (the common case): one CTA per 8 x 4
-//              blocks, the previous frame's window (+-10 px) staged once in shared memory; a warp walks
-//              8 blocks in lockstep, 4 lanes per block with 4 block rows each in registers, one candidate
-//              per block and pass; points already scored by the previous diamond are skipped (they cannot
-//              win).  Walks that leave the window continue in k_search_ds16q_long with private windows.
+//   k_search_dsw  Step 2 for 16-pixel blocks with diamond search (the common case): one CTA per 8 x 2
+//              blocks, the previous frame's window staged once in shared memory as one word per pixel; one
+//              warp per block, lane 2r + h scoring every other pixel of block row r, so that loads are free of
+//              bank conflicts and of byte realignment; points already scored by the previous diamond are
+//              skipped (they cannot win).  Walks that leave the window continue in k_search_dsw_long with
+//              private windows.
 //   k_search_tss16q  Step 2 for 16-pixel blocks with three step search: the same lane layout, one window that
 //              covers the whole reach of the search.
 //   k_verify   Steps 3-4: rounds the mean vector M, scores every block at M (reusing the Step 2
@@ -351,10 +352,6 @@ __global__ void __launch_bounds__(1024) k_merge(const uint16_t* run_end, const i
 // ---------------------------------------------------------------------------------------------
 // Fast Steps 2 and 4: 16-pixel blocks, diamond search
 // ---------------------------------------------------------------------------------------------
-constexpr int F_WR = 10;                       // reach of a block's private window, pixels
-constexpr int F_ROWS = 16 + 2 * F_WR;          // window rows
-constexpr int L_WORDS = 32;                    // private window row: (16 + 2 * 10) px * 3 B = 108 B + slack
-constexpr int L_PITCH = 33;
 
 // NR rows (48 bytes each) of the current block per lane, masked for clipped edge blocks.
 template <int NR>
@@ -439,23 +436,29 @@ __device__ __forceinline__ void publish_block(const MatchArgs& a, int s, size_t 
 }
 
 // ---------------------------------------------------------------------------------------------
-// Step 2 for 16-pixel blocks, diamond search, several blocks per warp
+// Step 2 for 16-pixel blocks, diamond search: one warp per block
 // ---------------------------------------------------------------------------------------------
-// A warp walks 32 / LPB blocks in lockstep: LPB lanes share a block, each owning 16 / LPB of its rows
-// (kept in registers), and every pass scores ONE candidate per block.  The per-pass bookkeeping
-// (next point, bounds, addresses, best-so-far) is then paid once for 32 / LPB candidates instead of
-// once for two, and the sum over a candidate's rows needs log2(LPB) shuffles.  The search points and
-// the new-point masks are packed into immediates, so lanes that look up different entries do not
-// serialise on the constant cache.
-constexpr int kPX[13] = {0, -1, 1, -2, 2, -1, 1, 0, 0, 0, -1, 1, 0};
-constexpr int kPY[13] = {-2, -1, -1, 0, 0, 1, 1, 2, 0, -1, 0, 0, 1};
-constexpr int kNP[25] = {0, 0, 31, 0, 0, 0, 11, 0, 21, 0, 171, 0, 0, 0, 213, 0, 168, 0, 208, 0, 0, 0, 248, 0, 0};
-constexpr unsigned long long pack_nibbles(const int (&v)[13])
+// The previous frame's window is staged in shared memory with one 32-bit word per pixel (R, G, B, 0), so a candidate
+// displaced by (dx, dy) starts at a word whatever dx is: no byte realignment, and a candidate's address is the lane's
+// base plus dy * pitch + dx.  Lane 2 r + h scores pixels h, h + 2, ..., h + 14 of block row r: its 8 pixels of the
+// current block stay in registers, a candidate costs 8 loads at fixed offsets, 8 absolute differences, 8 multiply-
+// accumulates and one warp sum.  With a row pitch of p words, p = 2 (mod 4), the 32 lanes of a load fall in 32
+// different banks for every displacement (bank = r p + h + const, and r p / 2 runs through all residues mod 16),
+// so shared memory is read without conflicts, and all lanes of a warp follow the same walk, so no lane waits for
+// another block.  The points of the two diamonds sit at compile-time offsets from the centre's address.
+//
+// Points: 0-7 the large diamond, 8 its centre, 9-12 the small diamond.
+__host__ __device__ constexpr int point_x(int i)
 {
-    unsigned long long r = 0;
-    for (int i = 0; i < 13; ++i) r |= (unsigned long long)(v[i] + 2) << (4 * i);
-    return r;
+    constexpr int t[13] = {0, -1, 1, -2, 2, -1, 1, 0, 0, 0, -1, 1, 0};
+    return t[i];
 }
+__host__ __device__ constexpr int point_y(int i)
+{
+    constexpr int t[13] = {-2, -1, -1, 0, 0, 1, 1, 2, 0, -1, 0, 0, 1};
+    return t[i];
+}
+constexpr int kNP[25] = {0, 0, 31, 0, 0, 0, 11, 0, 21, 0, 171, 0, 0, 0, 213, 0, 168, 0, 208, 0, 0, 0, 248, 0, 0};
 // new-point masks of the 8 possible moves; a move's table index (my + 2) * 5 + (mx + 2) is always even
 constexpr unsigned long long pack_moves(int first)
 {
@@ -463,7 +466,6 @@ constexpr unsigned long long pack_moves(int first)
     for (int h = first; h < first + 8 && 2 * h < 25; ++h) r |= (unsigned long long)kNP[2 * h] << (8 * (h - first));
     return r;
 }
-constexpr unsigned long long kPackX = pack_nibbles(kPX), kPackY = pack_nibbles(kPY);
 constexpr unsigned long long kMovesLo = pack_moves(0), kMovesHi = pack_moves(8);
 
 // st: 0 walking, 1 finished, 2 the walk left the staged window (resume elsewhere), 3 no block
@@ -482,158 +484,319 @@ __device__ __forceinline__ uint32_t new_points(int mx, int my)
     const int h = ((my + 2) * 5 + (mx + 2)) >> 1;
     return (uint32_t)((h < 8 ? kMovesLo >> (8 * h) : kMovesHi >> (8 * (h - 8))) & 0xffu);
 }
-// A walk that stopped with st = 2 had chosen its next centre (the best point so far) but not moved yet:
-// make that move now, exactly as the uninterrupted walk would have.
-__device__ __forceinline__ void walk_resume(WalkState& w)
-{
-    const int nx = (int)(w.bt & 0xff) - 128, ny = (int)((w.bt >> 8) & 0xff) - 128;
-    w.mask = new_points(nx - w.cx, ny - w.cy);
-    w.cx = nx; w.cy = ny;
-    w.phase = 0; w.st = 0;
-}
 
-// The walks of all blocks of a warp, until every one has finished or left its window.
-//   win.reach(cx, cy)      true when every point around centre (cx, cy) is staged
-//   win.row(r, dx, dy, sh) words holding row r of the candidate displaced by (dx, dy)
-// (dx_lo, dx_span), (dy_lo, dy_span): displacements that keep the block inside the previous frame and the range.
-// QUIT: a walk that is about to move while at most QUIT blocks of the warp are still walking gives up its
-//       place (st = 2, as if it had left the window), so that a few long walks do not hold the whole warp; 0 = never.
-template <int LPB, int QUIT, typename Win>
-__device__ __forceinline__ void lockstep_walk(const MatchArgs& a, const RowCtx<16 / LPB>& rc, const Win& win, int q,
-                                              int dx_lo, unsigned dx_span, int dy_lo, unsigned dy_span, WalkState& w)
+// The same points for look-ups with a run-time index (the same in all lanes of a warp: one constant-cache access).
+__constant__ int c_point_x[13] = {0, -1, 1, -2, 2, -1, 1, 0, 0, 0, -1, 1, 0};
+__constant__ int c_point_y[13] = {-2, -1, -1, 0, 0, 1, 1, 2, 0, -1, 0, 0, 1};
+// Per point and window pitch: byte offset of the point's candidate from the centre's, << 16, | the low 16 bits of the
+// point's tie-key offset (py << 8) + px taken modulo 2^16.
+__host__ __device__ constexpr int point_word(int i, int pitch)
 {
-    constexpr int NR = 16 / LPB;
-    const int max_passes = 16 + 5 * (2 * a.R + 1) * (2 * a.R + 1);   // every move strictly lowers the key
+    return (int)(((unsigned)((point_y(i) * pitch + point_x(i)) * 4) << 16) | ((unsigned)(point_y(i) * 256 + point_x(i)) & 0xffffu));
+}
+#define DC_POINT_ROW(p) {point_word(0, p), point_word(1, p), point_word(2, p), point_word(3, p), point_word(4, p), point_word(5, p), \
+                         point_word(6, p), point_word(7, p), point_word(8, p), point_word(9, p), point_word(10, p), point_word(11, p), point_word(12, p)}
+
+// displacements that keep the block inside the previous frame and the search range
+struct WalkBounds { int dx_lo, dx_hi, dy_lo, dy_hi; };
+
+__device__ __forceinline__ WalkBounds walk_bounds(const MatchArgs& a, int x0, int y0, int bw, int bh)
+{
+    WalkBounds b = {max(-a.R, -x0), min(a.R, a.W - bw - x0), max(-a.R, -y0), min(a.R, a.H - bh - y0)};
+    return b;
+}
+// which of the 13 points around (cx, cy) are valid candidates
+__device__ __forceinline__ uint32_t valid_points(int cx, int cy, const WalkBounds& b)
+{
+    if (cx - 2 >= b.dx_lo && cx + 2 <= b.dx_hi && cy - 2 >= b.dy_lo && cy + 2 <= b.dy_hi) return 0x1fffu;
+    // near the frame's edge or the range limit (rare): a real loop, so that it is not merged into the path above
+    uint32_t m = 0;
 #pragma unroll 1
-    for (int pass = 0; pass < max_passes; ++pass) {
-        const unsigned walking = __ballot_sync(0xffffffffu, w.st == 0);
-        if (!walking) break;
-        if (w.st == 0 && w.mask == 0) {
-            if (w.phase == 0) {
-                const int nx = (int)(w.bt & 0xff) - 128, ny = (int)((w.bt >> 8) & 0xff) - 128;
-                if (nx == w.cx && ny == w.cy) { w.phase = 1; w.mask = 0x1e00u; }    // centre won: small diamond
-                else if (!win.reach(nx, ny) || (QUIT > 0 && __popc(walking) <= QUIT * LPB)) w.st = 2;
-                else {
-                    w.mask = new_points(nx - w.cx, ny - w.cy);
-                    w.cx = nx; w.cy = ny;
-                }
-            } else w.st = 1;
-        }
-        const bool run = w.st == 0;
-        const int i = run ? __ffs(w.mask) - 1 : 8;
-        w.mask &= w.mask - 1;
-        const int dx = w.cx + (int)((kPackX >> (4 * i)) & 7) - 2, dy = w.cy + (int)((kPackY >> (4 * i)) & 7) - 2;
-        const bool ok = run && (unsigned)(dx - dx_lo) <= dx_span && (unsigned)(dy - dy_lo) <= dy_span;
-        uint32_t ks = 0;
-        if (ok) {
-            // rows below a clipped block's last row hold zeros and are scored against staged words, then dropped:
-            // no branch between the rows, so their load / difference / accumulate chains interleave
-            uint32_t sh;
-#pragma unroll
-            for (int k = 0; k < NR; ++k) {
-                const uint32_t* p = win.row(q + k * LPB, dx, dy, sh);
-                const uint32_t v = rc.template sse<false>(k, p, sh);
-                ks += rc.row_on[k] ? v : 0u;
-            }
-        }
-#pragma unroll
-        for (int off = LPB / 2; off > 0; off >>= 1) ks += __shfl_xor_sync(0xffffffffu, ks, off);
-        const uint32_t kt = ((uint32_t)(abs(dx) + abs(dy)) << 16) | ((uint32_t)(dy + 128) << 8) | (uint32_t)(dx + 128);
-        if (ok && (ks < w.bs || (ks == w.bs && kt < w.bt))) { w.bs = ks; w.bt = kt; }
+    for (int i = 0; i < 13; ++i) {
+        const int dx = cx + c_point_x[i], dy = cy + c_point_y[i];
+        if (dx >= b.dx_lo && dx <= b.dx_hi && dy >= b.dy_lo && dy <= b.dy_hi) m |= 1u << i;
     }
-    // Every move strictly lowers the key, so a walk ends long before max_passes.  Should the limit ever end one, its
-    // result is not the walk's: the status word says so.
-    if (w.st == 0) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
+    return m;
+}
+__device__ __forceinline__ uint32_t tie_key(int dx, int dy)
+{
+    return ((uint32_t)(abs(dx) + abs(dy)) << 16) | ((uint32_t)(dy + 128) << 8) | (uint32_t)(dx + 128);
 }
 
-// Window shared by the VS x 8 blocks of a CTA; every block may move WR pixels from zero motion inside it.
-// Row length: a candidate starts at most (112 + 2 WR) * 3 + 15 bytes into the row (15 = alignment of the
-// window's origin) and reads 13 words from the word that holds its first byte.
-template <int WR>
-struct StackWin {
-    static constexpr int WORDS = ((((112 + 2 * WR) * 3 + 15) >> 2) + 13 + 3) & ~3;   // staged in 16-byte chunks
-    static constexpr int PITCH = WORDS | 1;                    // odd: the rows of a block's lanes fall in different banks
-    const uint32_t* win; int x0, wx0, row0;
-    __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx) + 2 <= WR && abs(cy) + 2 <= WR; }
-    __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
-    {
-        const int off = (x0 + dx) * 3 - wx0;
-        sh = (off & 3) * 8;
-        return win + (row0 + r + dy + WR) * PITCH + (off >> 2);
+// The 8 pixels of row r (48 bytes at `row`, 16-byte aligned) that lane parity h scores, one word each.
+__device__ __forceinline__ void load_lane_pixels(const uint8_t* row, int h, bool on, uint32_t (&cw)[8])
+{
+    uint32_t w[12];
+    const uint4* p = (const uint4*)row;
+    uint4 v0 = make_uint4(0, 0, 0, 0), v1 = v0, v2 = v0;
+    if (on) { v0 = __ldg(p); v1 = __ldg(p + 1); v2 = __ldg(p + 2); }
+    w[0] = v0.x; w[1] = v0.y; w[2] = v0.z; w[3] = v0.w; w[4] = v1.x; w[5] = v1.y; w[6] = v1.z; w[7] = v1.w;
+    w[8] = v2.x; w[9] = v2.y; w[10] = v2.z; w[11] = v2.w;
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+        uint32_t px[2];
+#pragma unroll
+        for (int q = 0; q < 2; ++q) {
+            const int k = 2 * j + q, wi = (3 * k) >> 2, sh = ((3 * k) & 3) * 8;      // pixel k: bytes 3k .. 3k + 2
+            px[q] = (sh == 0 ? w[wi] : sh == 8 ? w[wi] >> 8 : __funnelshift_r(w[wi], w[wi + 1 < 12 ? wi + 1 : wi], sh)) & 0x00ffffffu;
+        }
+        cw[j] = h ? px[1] : px[0];
     }
+}
+
+// Expands 4 packed pixels (12 bytes in a, b, c) to 4 words and stores them at dst (8-byte aligned).
+__device__ __forceinline__ void store_pixels4(uint32_t* dst, uint32_t a, uint32_t b, uint32_t c)
+{
+    const uint32_t m = 0x00ffffffu;
+    *(uint2*)dst = make_uint2(a & m, __funnelshift_r(a, b, 24) & m);
+    *(uint2*)(dst + 2) = make_uint2(__funnelshift_r(b, c, 16) & m, c >> 8);
+}
+// 4 pixels starting at pixel px0 (a multiple of 4) of frame row gy, zeros outside the frame copy
+__device__ __forceinline__ void load_pixels4(const uint8_t* prev, size_t pitch, int H, int gy, int px0, uint32_t& a, uint32_t& b, uint32_t& c)
+{
+    a = b = c = 0;
+    if (gy >= 0 && gy < H && px0 >= 0 && (size_t)px0 * 3 + 12 <= pitch) {
+        const uint32_t* q = (const uint32_t*)(prev + (size_t)gy * pitch + (size_t)px0 * 3);     // px0 * 3 is a multiple of 12
+        a = __ldg(q); b = __ldg(q + 1); c = __ldg(q + 2);
+    }
+}
+
+// SSE of this lane's 8 pixels against the candidate whose first word for this lane is at shared-memory address p,
+// summed over the warp.  Explicit shared-space loads at fixed offsets from one address register.
+template <int OFF>
+__device__ __forceinline__ uint32_t lds_at(uint32_t p)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(p), "n"(OFF) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t score_at(uint32_t p, const uint32_t (&cw)[8], bool row_on)
+{
+    const uint32_t w0 = lds_at<0>(p), w1 = lds_at<8>(p), w2 = lds_at<16>(p), w3 = lds_at<24>(p);
+    const uint32_t w4 = lds_at<32>(p), w5 = lds_at<40>(p), w6 = lds_at<48>(p), w7 = lds_at<56>(p);
+    uint32_t a0 = 0, a1 = 0, d;
+    d = __vabsdiffu4(cw[0], w0); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[1], w1); a1 = __dp4a(d, d, a1);
+    d = __vabsdiffu4(cw[2], w2); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[3], w3); a1 = __dp4a(d, d, a1);
+    d = __vabsdiffu4(cw[4], w4); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[5], w5); a1 = __dp4a(d, d, a1);
+    d = __vabsdiffu4(cw[6], w6); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[7], w7); a1 = __dp4a(d, d, a1);
+    const uint32_t mine = row_on ? a0 + a1 : 0u;
+    uint32_t sum;
+    asm volatile("redux.sync.add.u32 %0, %1, 0xffffffff;" : "=r"(sum) : "r"(mine));
+    return sum;
+}
+
+// The same with the candidate's offset from p known at compile time: the eight loads need no address arithmetic.
+template <int OFF>
+__device__ __forceinline__ uint32_t score_at_fixed(uint32_t p, const uint32_t (&cw)[8], bool row_on)
+{
+    const uint32_t w0 = lds_at<OFF>(p), w1 = lds_at<OFF + 8>(p), w2 = lds_at<OFF + 16>(p), w3 = lds_at<OFF + 24>(p);
+    const uint32_t w4 = lds_at<OFF + 32>(p), w5 = lds_at<OFF + 40>(p), w6 = lds_at<OFF + 48>(p), w7 = lds_at<OFF + 56>(p);
+    uint32_t a0 = 0, a1 = 0, d;
+    d = __vabsdiffu4(cw[0], w0); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[1], w1); a1 = __dp4a(d, d, a1);
+    d = __vabsdiffu4(cw[2], w2); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[3], w3); a1 = __dp4a(d, d, a1);
+    d = __vabsdiffu4(cw[4], w4); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[5], w5); a1 = __dp4a(d, d, a1);
+    d = __vabsdiffu4(cw[6], w6); a0 = __dp4a(d, d, a0);
+    d = __vabsdiffu4(cw[7], w7); a1 = __dp4a(d, d, a1);
+    const uint32_t mine = row_on ? a0 + a1 : 0u;
+    uint32_t sum;
+    asm volatile("redux.sync.add.u32 %0, %1, 0xffffffff;" : "=r"(sum) : "r"(mine));
+    return sum;
+}
+
+// Scores the points of the compile-time set MASK around the centre whose candidate starts at pc: straight-line code,
+// every load at a fixed offset.  Tracks the smallest SSE (ms), the point that gave it (mi) and whether two of
+// the scores that mattered were equal (tie): the caller settles the rare ties with the exact order.
+template <uint32_t MASK, int PITCH, int I = 0>
+__device__ __forceinline__ void score_fixed_set(uint32_t pc, const uint32_t (&cw)[8], bool row_on, uint32_t& ms, int& mi, bool& tie)
+{
+    if constexpr (I < 13) {
+        if constexpr (((MASK >> I) & 1u) != 0) {
+            const uint32_t s = score_at_fixed<(point_y(I) * PITCH + point_x(I)) * 4>(pc, cw, row_on);
+            tie |= s == ms;                                   // selects, no branches: the code stays straight
+            mi = s < ms ? I : mi;
+            ms = min(ms, s);
+        }
+        score_fixed_set<MASK, PITCH, I + 1>(pc, cw, row_on, ms, mi, tie);
+    }
+}
+
+// One block's walk, by one warp, for as long as it stays inside the staged window.
+//
+// A round scores one of ten point sets around the current centre: kind 0-7, the points of the large diamond that are
+// new after the move along diamond point `kind` (the others lost to the new centre already and cannot win); kind 8,
+// the first round (centre and all eight points); kind 9, the small diamond.  Outside the first round the centre is
+// the best point so far and bs its SSE.  When all 13 points around the centre are valid candidates the round runs
+// as straight-line code for its set and decides by SSE alone: a point that beats the centre becomes the next centre
+// and names the next round's kind.  Should two SSEs that matter be equal, or the frame edge or the range limit cut
+// the set, the round is (re)done point by point under the full order (SSE, |dx| + |dy|, dy, dx): same result.
+constexpr int KIND_FIRST = 8, KIND_SMALL = 9;
+__constant__ uint32_t c_kind_mask[10] = {31u, 11u, 21u, 171u, 213u, 168u, 208u, 248u, 0x1ffu, 0x1e00u};
+// diamond point of a move (mx, my), indexed by ((my + 2) * 5 + (mx + 2)) >> 1
+__constant__ int c_kind_of_move[13] = {0, 0, 0, 1, 2, 3, 0, 4, 5, 6, 0, 7, 0};
+
+struct WalkW {
+    int cx, cy, kind;           // centre, and how it was reached
+    uint32_t bs;                // SSE of the best point so far (the centre, after the first round)
+    int nx, ny; uint32_t ns;    // on return 2: the centre the walk has chosen and not yet moved to, and its SSE
 };
 
-// Phase 1: one CTA per 8 x VS blocks (VS strips stacked vertically share window rows), 32 / LPB blocks per
-// warp.  A walk that leaves the window is handed to phase 2.  Blocks clipped in width are left to the
-// generic kernel.  Launched without k-skip only (every block is searched).
-template <int LPB, int VS, int WR, int QUIT, int MINB>
-__global__ void __launch_bounds__(LPB * 8 * VS, MINB) k_search_ds16q(MatchArgs a, uint4* long_list, int32_t* long_count)
+//   lane_base  shared-memory address of this lane's first word of the candidate at displacement (0, 0);
+//              (dx, dy) is at lane_base + (dy * PITCH + dx) * 4
+//   reach(x, y)  true when every point around centre (x, y) is staged
+// Returns 1 when the walk has finished (result: w.cx, w.cy, w.bs), 2 when the next centre is out of reach.
+template <int PITCH, typename Reach>
+__device__ __forceinline__ int warp_walk(const MatchArgs& a, uint32_t lane_base, const uint32_t (&cw)[8], bool row_on,
+                                         const WalkBounds& wb, WalkW& w, const Reach& reach)
 {
-    using Win = StackWin<WR>;
-    constexpr int THREADS = LPB * 8 * VS, ROWS = 16 * VS + 2 * WR, CPR = Win::WORDS / 4, CHUNKS = ROWS * CPR;
-    __shared__ uint32_t win[ROWS * Win::PITCH];
-    const int strips = (a.Gx + 7) >> 3, vgroups = (a.Gy + VS - 1) / VS;
-    const int strip = blockIdx.x % strips, vg = (blockIdx.x / strips) % vgroups, s = blockIdx.x / (strips * vgroups);
-    const int xs = strip * 128, yb = vg * 16 * VS;
-    const int wx0 = ((xs - WR) * 3) & ~15;                  // byte column of the window origin (may be < 0)
-    // this lane's block: LPB lanes per block, 8 blocks per strip, VS strips
-    const int lane = threadIdx.x & 31, q = lane % LPB;
-    const int blk = threadIdx.x / LPB, by = vg * VS + (blk >> 3), bx = strip * 8 + (blk & 7);
-    const bool in_grid = bx < a.Gx && by < a.Gy;
-    const int x0 = bx * 16, y0 = by * 16;
-    const bool searched = in_grid && a.W - x0 >= 16;
-    const int bw = searched ? 16 : 0, bh = searched ? min(16, a.H - y0) : 0;
-    RowCtx<16 / LPB> rc;                                      // issued first: in flight while the window is staged
-    rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)(searched ? y0 : 0) * a.cur_pitch + (size_t)(searched ? x0 : 0) * 3,
-                  a.cur_pitch, q, LPB, bw, bh);
-    const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
-    constexpr int UNR = 4;                                    // 16-byte chunks; wx0 and the pitch are 16-byte multiples
-    for (int i0 = threadIdx.x; i0 < CHUNKS; i0 += THREADS * UNR) {
-        uint4 v[UNR];
-#pragma unroll
-        for (int u = 0; u < UNR; ++u) {
-            const int i = i0 + u * THREADS, row = i / CPR, ci = i - row * CPR;
-            const int gy = yb - WR + row, gb = wx0 + ci * 16;
-            v[u] = make_uint4(0, 0, 0, 0);
-            if (i < CHUNKS && gy >= 0 && gy < a.H && gb >= 0 && gb + 16 <= (int)a.prev_pitch)
-                v[u] = __ldg((const uint4*)(prev + (size_t)gy * a.prev_pitch + gb));
-        }
-#pragma unroll
-        for (int u = 0; u < UNR; ++u) {
-            const int i = i0 + u * THREADS, row = i / CPR, ci = i - row * CPR;
-            if (i < CHUNKS) {
-                uint32_t* d = win + row * Win::PITCH + ci * 4;
-                d[0] = v[u].x; d[1] = v[u].y; d[2] = v[u].z; d[3] = v[u].w;
+    static __constant__ int c_points[13] = DC_POINT_ROW(PITCH);
+    const int max_moves = (2 * a.R + 1) * (2 * a.R + 1);          // every move strictly lowers the key: never reached
+    // all 13 points valid  <=>  cx in [dx_lo + 2, dx_hi - 2] and cy likewise: one unsigned compare per axis
+    const int ix_lo = wb.dx_lo + 2, iy_lo = wb.dy_lo + 2;
+    const unsigned ix_span = (unsigned)max(wb.dx_hi - 2 - ix_lo, -1), iy_span = (unsigned)max(wb.dy_hi - 2 - iy_lo, -1);
+    uint32_t pc = lane_base + (uint32_t)((w.cy * PITCH + w.cx) * 4);
+#pragma unroll 1
+    for (int move = 0;; ++move) {
+        const bool interior = wb.dx_hi - 2 >= ix_lo && wb.dy_hi - 2 >= iy_lo &&
+                              (unsigned)(w.cx - ix_lo) <= ix_span && (unsigned)(w.cy - iy_lo) <= iy_span;
+        uint32_t ms = 0xffffffffu; int mi = 8; bool tie = !interior;
+        if (interior) {
+            switch (w.kind) {
+            case 0: score_fixed_set<31u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case 1: score_fixed_set<11u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case 2: score_fixed_set<21u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case 3: score_fixed_set<171u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case 4: score_fixed_set<213u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case 5: score_fixed_set<168u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case 6: score_fixed_set<208u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case 7: score_fixed_set<248u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            case KIND_FIRST: score_fixed_set<0x1ffu, PITCH>(pc, cw, row_on, ms, mi, tie); break;
+            default: score_fixed_set<0x1e00u, PITCH>(pc, cw, row_on, ms, mi, tie); break;
             }
+            tie |= ms == w.bs;
+        }
+        int nx = w.cx, ny = w.cy;                                 // the best point after this round
+        uint32_t ns = w.bs;
+        if (!tie) {
+            if (ms < w.bs) { ns = ms; nx = w.cx + c_point_x[mi]; ny = w.cy + c_point_y[mi]; }
+        } else {
+            // the exact order, point by point
+            uint32_t m = c_kind_mask[w.kind] & valid_points(w.cx, w.cy, wb);
+            uint32_t bt = w.kind == KIND_FIRST ? 0xffffffffu : tie_key(w.cx, w.cy);
+            const uint32_t kc = ((uint32_t)(w.cy + 128) << 8) | (uint32_t)(w.cx + 128);  // low half of the centre's tie key
+#pragma unroll 1
+            while (m) {                                           // one candidate per turn; m is the same in all lanes
+                const int i = __ffs(m) - 1;
+                m &= m - 1;
+                const int pw = c_points[i];
+                const uint32_t s = score_at(pc + (uint32_t)(pw >> 16), cw, row_on);
+                if (s <= ns) {
+                    const uint32_t lo = (kc + (uint32_t)pw) & 0xffffu;               // ((dy + 128) << 8) | (dx + 128)
+                    const int dx = (int)(lo & 0xff) - 128, dy = (int)(lo >> 8) - 128;
+                    const uint32_t kt = ((uint32_t)(abs(dx) + abs(dy)) << 16) | lo;
+                    if (s < ns || kt < bt) { ns = s; bt = kt; nx = dx; ny = dy; }
+                }
+            }
+        }
+        if (w.kind == KIND_SMALL) { w.cx = nx; w.cy = ny; w.bs = ns; return 1; }       // the small diamond's best is the result
+        if (nx == w.cx && ny == w.cy) { w.bs = ns; w.kind = KIND_SMALL; continue; }    // centre won: small diamond, then done
+        if (move >= max_moves) {                                  // a walk cut here is not valid: say so
+            if ((threadIdx.x & 31) == 0) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
+            w.bs = ns;
+            return 1;
+        }
+        if (!reach(nx, ny)) { w.nx = nx; w.ny = ny; w.ns = ns; return 2; }
+        const int mx = nx - w.cx, my = ny - w.cy;
+        w.kind = c_kind_of_move[((my + 2) * 5 + (mx + 2)) >> 1];
+        pc += (uint32_t)((my * PITCH + mx) * 4);
+        w.cx = nx; w.cy = ny; w.bs = ns;
+    }
+}
+
+// Phase 1: one CTA per 8 x W_VS blocks, one warp per block.  The window reaches W_WRY rows above and below the tile
+// and 12 pixels to its left and right (its left edge stays a multiple of 4 pixels, so that 4 pixels are 12 aligned
+// bytes of the packed frame).  A walk whose next centre is out of reach is handed to phase 2.  Blocks clipped in
+// width are left to the generic kernel.  Launched without k-skip only (every block is searched).
+constexpr int W_VS = 2, W_WRY = 10, W_SIDE = 12;
+constexpr int W_COLS = 128 + 2 * W_SIDE;                    // staged pixels per window row
+constexpr int W_PITCH = 154;                                // words per window row
+constexpr int W_ROWS = 16 * W_VS + 2 * W_WRY;
+static_assert(W_PITCH % 4 == 2 && W_PITCH >= W_COLS && W_COLS % 4 == 0, "conflict-free pitch, whole groups of 4 pixels");
+
+struct TileReach {
+    __device__ __forceinline__ bool operator()(int cx, int cy) const { return abs(cx) + 2 <= W_SIDE && abs(cy) + 2 <= W_WRY; }
+};
+
+__global__ void __launch_bounds__(W_VS * 8 * 32, 3) k_search_dsw(MatchArgs a, uint4* long_list, int32_t* long_count)
+{
+    constexpr int THREADS = W_VS * 8 * 32, GROUPS = W_COLS / 4;
+    constexpr int ROWS_PER_PASS = THREADS / GROUPS, PASSES = W_ROWS / ROWS_PER_PASS;      // 13 rows of 38 groups per pass
+    static_assert(W_ROWS % ROWS_PER_PASS == 0, "whole passes");
+    __shared__ __align__(16) uint32_t win[W_ROWS * W_PITCH];
+    __shared__ int32_t sums[3];
+    const int strip = blockIdx.x, vg = blockIdx.y, s = blockIdx.z;        // grid: strips of 8 blocks x groups of W_VS block rows x streams
+    const int xs = strip * 128, yb = vg * 16 * W_VS;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, r = lane >> 1, h = lane & 1;
+    const int by = vg * W_VS + (warp >> 3), bx = strip * 8 + (warp & 7);
+    const int x0 = bx * 16, y0 = by * 16;
+    const bool searched = bx < a.Gx && by < a.Gy && a.W - x0 >= 16;
+    const int bh = searched ? min(16, a.H - y0) : 0;
+    const bool row_on = r < bh;
+    uint32_t cw[8];                                            // issued first: in flight while the window is staged
+    load_lane_pixels(a.cur + (size_t)s * a.cur_stream + (size_t)(row_on ? y0 + r : 0) * a.cur_pitch + (size_t)(row_on ? x0 : 0) * 3,
+                     h, row_on, cw);
+    if (threadIdx.x < 3) sums[threadIdx.x] = 0;
+    {   // the window: a thread keeps its group of 4 pixels (one column position) and goes down the rows, 13 rows apart
+        const int gq = threadIdx.x % GROUPS, row0 = threadIdx.x / GROUPS, px0 = xs - W_SIDE + 4 * gq;
+        const bool col_ok = row0 < ROWS_PER_PASS && px0 >= 0 && (size_t)px0 * 3 + 12 <= a.prev_pitch;
+        const uint8_t* src = a.prev + (size_t)s * a.prev_stream + (size_t)px0 * 3;       // px0 * 3 is a multiple of 12
+        uint32_t* dst = win + row0 * W_PITCH + 4 * gq;
+        uint32_t pa[PASSES], pb[PASSES], pc[PASSES];
+#pragma unroll
+        for (int k = 0; k < PASSES; ++k) {                         // all loads first
+            const int gy = yb - W_WRY + row0 + k * ROWS_PER_PASS;
+            pa[k] = pb[k] = pc[k] = 0;
+            if (col_ok && gy >= 0 && gy < a.H) {
+                const uint32_t* q = (const uint32_t*)(src + (size_t)gy * a.prev_pitch);
+                pa[k] = __ldg(q); pb[k] = __ldg(q + 1); pc[k] = __ldg(q + 2);
+            }
+        }
+        if (row0 < ROWS_PER_PASS) {
+#pragma unroll
+            for (int k = 0; k < PASSES; ++k) store_pixels4(dst + k * ROWS_PER_PASS * W_PITCH, pa[k], pb[k], pc[k]);
         }
     }
     __syncthreads();
     const size_t g = (size_t)s * a.Gx * a.Gy + (size_t)by * a.Gx + bx;
-    const int dx_lo = max(-a.R, -x0), dy_lo = max(-a.R, -y0);
-    const unsigned dx_span = (unsigned)(min(a.R, a.W - bw - x0) - dx_lo), dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
-    const Win sw = {win, x0, wx0, (blk >> 3) * 16};
-    WalkState w;
-    walk_begin(w, searched);
-    lockstep_walk<LPB, QUIT>(a, rc, sw, q, dx_lo, dx_span, dy_lo, dy_span, w);
-    // finished blocks: results, and Step 3's sums once per warp (all blocks of a CTA belong to one stream)
-    const int fx = (int)(w.bt & 0xff) - 128, fy = (int)((w.bt >> 8) & 0xff) - 128;
-    const bool fin = searched && q == 0 && w.st != 2;
-    if (fin) { a.mv[2 * g] = (int16_t)fx; a.mv[2 * g + 1] = (int16_t)fy; a.sse[g] = w.bs; }
-    const bool pass = fin && w.bs <= a.limit[limit_index(a, bw, bh)];     // PSNR > T: member of Step 3's set S
-    const int n_pass = __popc(__ballot_sync(0xffffffffu, pass));
-    const int sum_x = __reduce_add_sync(0xffffffffu, pass ? fx : 0), sum_y = __reduce_add_sync(0xffffffffu, pass ? fy : 0);
-    if (lane == 0 && n_pass) {
-        atomicAdd(&a.acc[4 * s + 0], sum_x);
-        atomicAdd(&a.acc[4 * s + 1], sum_y);
-        atomicAdd(&a.acc[4 * s + 2], n_pass);
+    if (searched) {
+        const WalkBounds wb = walk_bounds(a, x0, y0, 16, bh);
+        const uint32_t lane_base = (uint32_t)__cvta_generic_to_shared(win) +
+                                   (uint32_t)((((warp >> 3) * 16 + r + W_WRY) * W_PITCH + (x0 - xs + W_SIDE) + h) * 4);
+        WalkW w = {0, 0, KIND_FIRST, 0xffffffffu, 0, 0, 0u};
+        const int st = warp_walk<W_PITCH>(a, lane_base, cw, row_on, wb, w, TileReach());
+        if (lane == 0) {
+            if (st == 1) {
+                a.mv[2 * g] = (int16_t)w.cx; a.mv[2 * g + 1] = (int16_t)w.cy; a.sse[g] = w.bs;
+                if (w.bs <= a.limit[limit_index(a, 16, bh)]) {        // PSNR > T: member of Step 3's set S
+                    atomicAdd(&sums[0], w.cx); atomicAdd(&sums[1], w.cy); atomicAdd(&sums[2], 1);
+                }
+            } else {                                                  // block, chosen next centre, its SSE, centre it was found from
+                const int slot = atomicAdd(long_count, 1);
+                long_list[slot] = make_uint4((uint32_t)g, tie_key(w.nx, w.ny), w.ns, (uint32_t)(w.cx + 128) | ((uint32_t)(w.cy + 128) << 8));
+            }
+        }
     }
-    const bool far = searched && q == 0 && w.st == 2;
-    const unsigned fm = __ballot_sync(0xffffffffu, far);
-    if (fm) {
-        int base = 0;
-        if (lane == 0) base = atomicAdd(long_count, __popc(fm));
-        base = __shfl_sync(0xffffffffu, base, 0);
-        if (far) long_list[base + __popc(fm & ((1u << lane) - 1u))] = make_uint4((uint32_t)g, w.bt, w.bs, (uint32_t)(w.cx + 128) | ((uint32_t)(w.cy + 128) << 8));   // block, best point, centre it was found from
+    __syncthreads();
+    if (threadIdx.x == 0 && sums[2]) {                                // Step 3's sums once per CTA (one stream per CTA)
+        atomicAdd(&a.acc[4 * s + 0], sums[0]);
+        atomicAdd(&a.acc[4 * s + 1], sums[1]);
+        atomicAdd(&a.acc[4 * s + 2], sums[2]);
     }
 }
 
@@ -774,123 +937,87 @@ __global__ void k_mark_unsearched(MatchArgs a)
     if (bx % a.skip_k != 0 || by % a.skip_k != 0) { a.mv[2 * gi] = 0; a.mv[2 * gi + 1] = 0; a.sse[gi] = 0xffffffffu; }
 }
 
-constexpr int P1_LPB = 4, P1_VS = 4;           // phase 1: 4 lanes per block (8 blocks per warp), 4 strips per CTA
-constexpr int P1_WR = 10;                      // phase 1 follows a walk up to 8 px from zero motion
-constexpr int P1_QUIT = 2;                     // ... and hands over the last two walks of a warp at their next move
-constexpr int P2_LPB = 16;                     // phase 2: 16 lanes per block; its 8 windows per CTA limit the resident warps,
-                                               // so fewer lanes per block would leave the SM short of warps
-
-// Private window of one block, centred on (wcx, wcy) relative to the block.
-struct BlockWin {
-    uint32_t* win; const uint8_t* prev; size_t pitch; int H, x0, y0, wcx, wcy, wx0;
-    __device__ __forceinline__ bool reach(int cx, int cy) const { return abs(cx - wcx) + 2 <= F_WR && abs(cy - wcy) + 2 <= F_WR; }
-    __device__ __forceinline__ const uint32_t* row(int r, int dx, int dy, uint32_t& sh) const
-    {
-        const int off = (x0 + dx) * 3 - wx0;
-        sh = (off & 3) * 8;
-        return win + (r + dy - wcy + F_WR) * L_PITCH + (off >> 2);
-    }
-    // the block's LPB lanes fill the window around (cx, cy)
-    template <int LPB>
-    __device__ __forceinline__ void stage(int cx, int cy, int q)
-    {
-        wcx = cx; wcy = cy;
-        wx0 = ((x0 + cx - F_WR) * 3) & ~15;
-        static_assert(L_WORDS == 32, "8 chunks of 16 bytes per window row");
-        for (int i0 = q; i0 < F_ROWS * 8; i0 += LPB * 4) {            // wx0 and the pitch are 16-byte multiples
-            uint4 v[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u * LPB, row = i >> 3, ci = i & 7;
-                const int gy = y0 + cy - F_WR + row, gb = wx0 + ci * 16;
-                v[u] = make_uint4(0, 0, 0, 0);
-                if (i < F_ROWS * 8 && gy >= 0 && gy < H && gb >= 0 && gb + 16 <= (int)pitch)
-                    v[u] = __ldg((const uint4*)(prev + (size_t)gy * pitch + gb));
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int i = i0 + u * LPB, row = i >> 3, ci = i & 7;
-                uint32_t* d = win + row * L_PITCH + ci * 4;
-                if (i < F_ROWS * 8) { d[0] = v[u].x; d[1] = v[u].y; d[2] = v[u].z; d[3] = v[u].w; }
-            }
-        }
-    }
-};
-
-// Phase 2: the walks that left their window.  Each group of LPB lanes takes walks off the list one after the
-// other; a walk's private window is re-staged around its centre whenever it nears the window's edge.
-// 8 walks per CTA (LPB / 4 warps).
+// Phase 2: the walks that left their tile's window.  A warp takes walks off the list one after the other (atomic
+// cursor); the walk gets a private window of P_ROWS x P_COLS pixels around its centre, re-staged around the next
+// centre whenever that is out of reach.  A continued walk makes exactly the move it had chosen (new points only),
+// so the sequence of scored candidates is the uninterrupted walk's.
 // With k-skip (Section 4) the searched blocks lie k blocks apart and share no window: there is no phase 1 then,
 // and this kernel walks every searched full-width block from its start (long_list == nullptr; item i is the
 // i-th searched block in stream / row / column order).
-template <int LPB, int MINB>
-__global__ void __launch_bounds__(LPB * 8, MINB) k_search_ds16q_long(MatchArgs a, const uint4* long_list, const int32_t* long_count, int32_t* cursor)
+constexpr int P_WARPS = 8;
+constexpr int P_REACH = 8;                                  // staged pixels above and left of the block at the window's centre
+constexpr int P_ROWS = 16 + 2 * P_REACH, P_COLS = 36, P_PITCH = 38;
+static_assert(P_PITCH % 4 == 2 && P_PITCH >= P_COLS && P_COLS % 4 == 0 && P_COLS >= 16 + 2 * P_REACH + 3, "window of a walk");
+
+struct PrivateReach {
+    int wcx, wcy;
+    __device__ __forceinline__ bool operator()(int cx, int cy) const { return abs(cx - wcx) + 2 <= P_REACH && abs(cy - wcy) + 2 <= P_REACH; }
+};
+
+__global__ void __launch_bounds__(P_WARPS * 32, 5) k_search_dsw_long(MatchArgs a, const uint4* long_list, const int32_t* long_count, int32_t* cursor)
 {
-    __shared__ uint32_t win_all[8][F_ROWS * L_PITCH];
-    const int lane = threadIdx.x & 31, q = lane % LPB, qb = lane / LPB;
+    __shared__ __align__(16) uint32_t win_all[P_WARPS][P_ROWS * P_PITCH];
+    const int lane = threadIdx.x & 31, r = lane >> 1, h = lane & 1;
+    uint32_t* win = win_all[threadIdx.x >> 5];
     const int per = a.Gx * a.Gy;
     const bool direct = long_list == nullptr;
     const int sgx = (a.W / 16 + a.skip_k - 1) / a.skip_k, sgy = (a.Gy + a.skip_k - 1) / a.skip_k;   // searched columns (full width only), rows
     const int n = direct ? a.S * sgx * sgy : *long_count;
-    bool fresh = false;
-    const int limit = 4 * a.R + 8;                                    // each re-staging moves the centre >= 8 px
-    WalkState w; walk_begin(w, false); w.st = 1;
-    RowCtx<16 / LPB> rc; rc.clipped = false; rc.row_bytes = 48;
-#pragma unroll
-    for (int k = 0; k < 16 / LPB; ++k) {
-        rc.row_on[k] = false;
-#pragma unroll
-        for (int j = 0; j < 12; ++j) rc.cw[k][j] = 0;
-    }
-    BlockWin bw_ = {win_all[threadIdx.x / LPB], nullptr, a.prev_pitch, a.H, 0, 0, 0, 0, 0};
-    int s = 0, bh = 16, rounds = 0, dx_lo = 0, dy_lo = 0; unsigned dx_span = 0, dy_span = 0; size_t g = 0;
+    const int max_rounds = 4 * a.R + 8;                               // each re-staging moves the centre by more than 4 px
 #pragma unroll 1
     for (;;) {
-        const bool need = w.st == 1;
-        const unsigned m = __ballot_sync(0xffffffffu, need && q == 0);
-        if (m) {
-            const int leader = __ffs(m) - 1;
-            int base = 0;
-            if (lane == leader) base = atomicAdd(cursor, __popc(m));
-            base = __shfl_sync(0xffffffffu, base, leader);
-            const int idx = base + __popc(m & ((1u << (qb * LPB)) - 1u));
-            if (need) {
-                if (idx < n) {
-                    if (direct) {
-                        const int ss = idx / (sgx * sgy), r = idx - ss * sgx * sgy, sby = r / sgx, sbx = r - sby * sgx;
-                        g = (size_t)ss * per + (size_t)(sby * a.skip_k) * a.Gx + sbx * a.skip_k;
-                        fresh = true;
-                    } else {
-                        const uint4 e = long_list[idx];
-                        g = e.x; w.bt = e.y; w.bs = e.z;
-                        w.cx = (int)(e.w & 0xff) - 128; w.cy = (int)((e.w >> 8) & 0xff) - 128;
-                    }
-                    s = (int)(g / per);
-                    const int b = (int)(g - (size_t)s * per), by = b / a.Gx, bx = b - by * a.Gx;
-                    const int x0 = bx * 16, y0 = by * 16;
-                    bh = min(16, a.H - y0);
-                    rc.load_block(a.cur + (size_t)s * a.cur_stream + (size_t)y0 * a.cur_pitch + (size_t)x0 * 3, a.cur_pitch, q, LPB, 16, bh);
-                    bw_.prev = a.prev + (size_t)s * a.prev_stream; bw_.x0 = x0; bw_.y0 = y0;
-                    dx_lo = max(-a.R, -x0); dy_lo = max(-a.R, -y0);
-                    dx_span = (unsigned)(min(a.R, a.W - 16 - x0) - dx_lo); dy_span = (unsigned)(min(a.R, a.H - bh - y0) - dy_lo);
-                    rounds = 0; w.st = 2;
-                } else w.st = 3;
+        int idx = 0;
+        if (lane == 0) idx = atomicAdd(cursor, 1);
+        idx = __shfl_sync(0xffffffffu, idx, 0);
+        if (idx >= n) break;
+        size_t g;
+        WalkW w = {0, 0, KIND_FIRST, 0xffffffffu, 0, 0, 0u};
+        if (direct) {
+            const int ss = idx / (sgx * sgy), q = idx - ss * sgx * sgy, sby = q / sgx, sbx = q - sby * sgx;
+            g = (size_t)ss * per + (size_t)(sby * a.skip_k) * a.Gx + sbx * a.skip_k;
+        } else {
+            const uint4 e = long_list[idx];
+            g = e.x; w.bs = e.z;
+            const int ox = (int)(e.w & 0xff) - 128, oy = (int)((e.w >> 8) & 0xff) - 128;      // the centre the walk stopped at
+            w.cx = (int)(e.y & 0xff) - 128; w.cy = (int)((e.y >> 8) & 0xff) - 128;            // the move it had chosen: make it
+            w.kind = c_kind_of_move[((w.cy - oy + 2) * 5 + (w.cx - ox + 2)) >> 1];
+        }
+        const int s = (int)(g / per), b = (int)(g - (size_t)s * per), by = b / a.Gx, bx = b - by * a.Gx;
+        const int x0 = bx * 16, y0 = by * 16, bh = min(16, a.H - y0);
+        const bool row_on = r < bh;
+        uint32_t cw[8];
+        load_lane_pixels(a.cur + (size_t)s * a.cur_stream + (size_t)(row_on ? y0 + r : y0) * a.cur_pitch + (size_t)x0 * 3, h, row_on, cw);
+        const uint8_t* prev = a.prev + (size_t)s * a.prev_stream;
+        const WalkBounds wb = walk_bounds(a, x0, y0, 16, bh);
+#pragma unroll 1
+        for (int round = 0;; ++round) {
+            // the window around the centre that is scored next
+            const PrivateReach reach = {w.cx, w.cy};
+            const int wx0 = (x0 + w.cx - P_REACH) & ~3, wy0 = y0 + w.cy - P_REACH;
+            constexpr int GROUPS = P_COLS / 4, ITEMS = P_ROWS * GROUPS;
+#pragma unroll 3
+            for (int it = lane; it < ITEMS; it += 32) {
+                const int row = it / GROUPS, gq = it - row * GROUPS;
+                uint32_t pa, pb, pc;
+                load_pixels4(prev, a.prev_pitch, a.H, wy0 + row, wx0 + 4 * gq, pa, pb, pc);
+                store_pixels4(win + row * P_PITCH + 4 * gq, pa, pb, pc);
             }
+            __syncwarp();
+            // this lane's first word at displacement (0, 0): frame row y0 + r, pixel x0 + h, relative to the window's
+            // origin (it may lie outside the window; only displacements near the centre are ever addressed)
+            const uint32_t lane_base = (uint32_t)__cvta_generic_to_shared(win) + (uint32_t)(((r + y0 - wy0) * P_PITCH + (x0 - wx0) + h) * 4);
+            const int st = warp_walk<P_PITCH>(a, lane_base, cw, row_on, wb, w, reach);
+            if (st == 1) break;
+            if (round >= max_rounds) {                                   // never reached; a walk cut here is not valid
+                if (lane == 0) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
+                break;
+            }
+            // make the chosen move; the next round scores its new points in a window around the new centre
+            w.kind = c_kind_of_move[((w.ny - w.cy + 2) * 5 + (w.nx - w.cx + 2)) >> 1];
+            w.cx = w.nx; w.cy = w.ny; w.bs = w.ns;
+            __syncwarp();                                                // every lane has finished reading the old window
         }
-        if (!__any_sync(0xffffffffu, w.st == 2)) break;
-        __syncwarp();
-        if (w.st == 2) {
-            if (fresh) { bw_.stage<LPB>(0, 0, q); walk_begin(w, true); fresh = false; }
-            else { bw_.stage<LPB>((int)(w.bt & 0xff) - 128, (int)((w.bt >> 8) & 0xff) - 128, q); walk_resume(w); }
-            ++rounds;
-        }
-        __syncwarp();
-        lockstep_walk<LPB, 0>(a, rc, bw_, q, dx_lo, dx_span, dy_lo, dy_span, w);
-        if (w.st == 2 && rounds >= limit) {                          // never reached; a walk cut here is not valid
-            w.st = 1;
-            if (q == 0) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
-        }
-        if (w.st == 1 && q == 0) publish_block(a, s, g, 16, bh, ((unsigned long long)w.bs << 32) | w.bt);
+        if (lane == 0) publish_block(a, s, g, 16, bh, ((unsigned long long)w.bs << 32) | tie_key(w.cx, w.cy));
     }
 }
 
@@ -1199,12 +1326,12 @@ int dc_launch_match(dc_cache* c, const uint8_t* cur_key, const uint8_t* prev_key
         {
             dc_prof_scope ps(c, DC_ST_SEARCH);
             if (a.skip_k <= 1) {
-                const int ctas = ((a.Gx + 7) / 8) * ((a.Gy + P1_VS - 1) / P1_VS) * a.S;
-                k_search_ds16q<P1_LPB, P1_VS, P1_WR, P1_QUIT, 4><<<ctas, P1_LPB * 8 * P1_VS, 0, c->stream>>>(a, c->long_list, long_count);
-                k_search_ds16q_long<P2_LPB, 5><<<c->num_sms * 5, P2_LPB * 8, 0, c->stream>>>(a, c->long_list, long_count, long_count + 1);
+                const dim3 tiles((a.Gx + 7) / 8, (a.Gy + W_VS - 1) / W_VS, a.S);
+                k_search_dsw<<<tiles, W_VS * 8 * 32, 0, c->stream>>>(a, c->long_list, long_count);
+                k_search_dsw_long<<<c->num_sms * 5, P_WARPS * 32, 0, c->stream>>>(a, c->long_list, long_count, long_count + 1);
             } else {
                 k_mark_unsearched<<<dc_div_up(a.S * a.Gx * a.Gy, 256), 256, 0, c->stream>>>(a);
-                k_search_ds16q_long<P2_LPB, 5><<<c->num_sms * 5, P2_LPB * 8, 0, c->stream>>>(a, nullptr, long_count, long_count + 1);
+                k_search_dsw_long<<<c->num_sms * 5, P_WARPS * 32, 0, c->stream>>>(a, nullptr, long_count, long_count + 1);
             }
             c->launches += 1;
         }

@@ -100,8 +100,14 @@ __global__ void k_propagate(const dc_layer_desc* layers, const int32_t* in_hw, i
 }
 
 // ---- bulk copies (cp.async.bulk) for the reuse copy ----
-constexpr int kCopyWarps = 4;                    // warps per CTA
-constexpr int kSeg = 512;                        // bytes one lane moves per round; a row span is cut into such segments
+#ifndef DC_COPY_WARPS
+#define DC_COPY_WARPS 8
+#endif
+#ifndef DC_COPY_SEG
+#define DC_COPY_SEG 256
+#endif
+constexpr int kCopyWarps = DC_COPY_WARPS;        // warps per CTA
+constexpr int kSeg = DC_COPY_SEG;                // bytes one lane moves per round; a row span is cut into such segments
 constexpr int kStageBytes = 32 * kSeg;           // staging of one warp: one segment per lane
 constexpr size_t kCopySmem = (size_t)kCopyWarps * kStageBytes + 128 + kCopyWarps * sizeof(unsigned long long);
 constexpr unsigned long long kCopyWaitNs = 2000000000ull;   // a warp gives up on its staging barrier after 2 s (far beyond any copy)
@@ -152,7 +158,7 @@ __device__ __forceinline__ void rs_commit() { asm volatile("cp.async.bulk.commit
 __device__ __forceinline__ void rs_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 __device__ __forceinline__ void rs_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 
-// What a warp needs for its bulk copies: 16 KB of staging, one mbarrier and its phase.
+// What a warp needs for its bulk copies: its staging (32 segments), one mbarrier and its phase.
 struct CopyLane { uint8_t* stage; unsigned long long* bar; uint32_t phase; bool dead; };
 
 struct ClassifyArgs {
