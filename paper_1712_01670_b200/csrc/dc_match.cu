@@ -994,13 +994,30 @@ __global__ void __launch_bounds__(P_WARPS * 32, 5) k_search_dsw_long(MatchArgs a
             // the window around the centre that is scored next
             const PrivateReach reach = {w.cx, w.cy};
             const int wx0 = (x0 + w.cx - P_REACH) & ~3, wy0 = y0 + w.cy - P_REACH;
-            constexpr int GROUPS = P_COLS / 4, ITEMS = P_ROWS * GROUPS;
-#pragma unroll 3
-            for (int it = lane; it < ITEMS; it += 32) {
-                const int row = it / GROUPS, gq = it - row * GROUPS;
-                uint32_t pa, pb, pc;
-                load_pixels4(prev, a.prev_pitch, a.H, wy0 + row, wx0 + 4 * gq, pa, pb, pc);
-                store_pixels4(win + row * P_PITCH + 4 * gq, pa, pb, pc);
+            {   // a lane keeps its group of 4 pixels (one column position) and goes down the rows, 3 rows apart
+                constexpr int GROUPS = P_COLS / 4, RPP = 32 / GROUPS, PASSES = (P_ROWS + RPP - 1) / RPP, HALF = (PASSES + 1) / 2;
+                const int gq = lane % GROUPS, row0 = lane / GROUPS, px0 = wx0 + 4 * gq;
+                const bool col_ok = row0 < RPP && px0 >= 0 && (size_t)px0 * 3 + 12 <= a.prev_pitch;
+                const uint8_t* src = prev + (size_t)px0 * 3;                          // px0 * 3 is a multiple of 12
+                uint32_t* dst = win + row0 * P_PITCH + 4 * gq;
+#pragma unroll
+                for (int half = 0; half < 2; ++half) {                               // loads of half the passes, then their stores
+                    uint32_t pa[HALF], pb[HALF], pc[HALF];
+#pragma unroll
+                    for (int k = 0; k < HALF; ++k) {
+                        const int row = row0 + (half * HALF + k) * RPP, gy = wy0 + row;
+                        pa[k] = pb[k] = pc[k] = 0;
+                        if (col_ok && row < P_ROWS && gy >= 0 && gy < a.H) {
+                            const uint32_t* q = (const uint32_t*)(src + (size_t)gy * a.prev_pitch);
+                            pa[k] = __ldg(q); pb[k] = __ldg(q + 1); pc[k] = __ldg(q + 2);
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < HALF; ++k) {
+                        const int row = row0 + (half * HALF + k) * RPP;
+                        if (row0 < RPP && row < P_ROWS) store_pixels4(dst + (half * HALF + k) * RPP * P_PITCH, pa[k], pb[k], pc[k]);
+                    }
+                }
             }
             __syncwarp();
             // this lane's first word at displacement (0, 0): frame row y0 + r, pixel x0 + h, relative to the window's
