@@ -74,6 +74,11 @@ __device__ __forceinline__ void mbar_arrive_relaxed(void* bar)
 {
     asm volatile("mbarrier.arrive.relaxed.cta.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
+// Arrival on a barrier in the other CTA of a pair (addr: shared::cluster address from mapa).
+__device__ __forceinline__ void mbar_arrive_remote(uint32_t addr)
+{
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(addr) : "memory");
+}
 __device__ __forceinline__ bool mbar_try(void* bar, uint32_t parity)
 {
     uint32_t ok;
@@ -161,7 +166,12 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
 // Epilogue warps (4 warps = 128 TMEM lanes = the 128 pixels of a tile): for every work item wait
 // for its accumulator, read it 32 columns at a time, add the bias, apply ReLU, round to bf16 and
 // store the pixel's channels unless the reuse bitmap says the pixel was filled from the cache.
-__device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uint32_t tmem_base, int n_items, int n_tiles, int warp, int lane)
+// first_item / item_stride: the items this CTA (or CTA pair) takes.  tiles_per_group / tile_sub: a group of the tile list
+// holds tiles_per_group tiles and this CTA's first one is number tile_sub in it (a pair: 2 and its rank, with a.MT = 1).
+// remote_empty: 0, or the shared::cluster address of the pair leader's tmem_empty[0], on which this CTA's epilogue
+// threads arrive instead of on their own.
+__device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uint32_t tmem_base, int n_items, int n_tiles, int warp, int lane,
+                                              int first_item, int item_stride, int tiles_per_group, int tile_sub, uint32_t remote_empty)
 {
     const int per_stream = a.tiles_x * a.tiles_y;
     const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
@@ -174,18 +184,18 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
     int tile_n0 = -1, tile_n1 = -1; uint32_t mask_n0 = 0, mask_n1 = 0;       // scalars: indexed arrays would live in local memory
     auto fetch = [&](int item) {
         if (item >= n_items) return;
-        const int idx = (item / a.NB) * a.MT;
-        tile_n0 = a.tile_list[idx];
-        mask_n0 = a.masks[(size_t)tile_n0 * 4 + mword_i];
+        const int idx = (item / a.NB) * tiles_per_group + tile_sub;
+        tile_n0 = idx < n_tiles ? a.tile_list[idx] : -1;                           // a pair's second CTA may have no tile in the last group
+        mask_n0 = tile_n0 >= 0 ? a.masks[(size_t)tile_n0 * 4 + mword_i] : 0u;
         tile_n1 = (a.MT > 1 && idx + 1 < n_tiles) ? a.tile_list[idx + 1] : -1;     // odd tile count: the last item has one tile
         mask_n1 = tile_n1 >= 0 ? a.masks[(size_t)tile_n1 * 4 + mword_i] : 0u;
     };
-    fetch(blockIdx.x);
-    for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
+    fetch(first_item);
+    for (int item = first_item; item < n_items && ok; item += item_stride) {
         const int nb = item % a.NB;
         const int tile_c0 = tile_n0, tile_c1 = tile_n1;
         const uint32_t mask_c0 = mask_n0, mask_c1 = mask_n1;
-        fetch(item + gridDim.x);
+        fetch(item + item_stride);
         ok = mbar_wait(&ctl->tmem_full[acc], acc_ph, ctl, a.status);
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
@@ -240,7 +250,8 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
             }
         }
         tc_fence_before();
-        mbar_arrive_relaxed(&ctl->tmem_empty[acc]);
+        if (remote_empty) mbar_arrive_remote(remote_empty + acc * 8u);
+        else mbar_arrive_relaxed(&ctl->tmem_empty[acc]);
         if (++acc == (uint32_t)a.nbuf) { acc = 0; acc_ph ^= 1u; }
     }
 }
@@ -358,7 +369,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         __syncwarp();
     } else {
         // ---------------- epilogue ----------------
-        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane, blockIdx.x, gridDim.x, a.MT, 0, 0u);
     }
     tc_fence_before();
     __syncthreads();
@@ -480,7 +491,7 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
         }
         __syncwarp();
     } else {
-        epilogue_loop(a, ctl, tmem_base, n_items, n_items, warp, lane);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_items, warp, lane, blockIdx.x, gridDim.x, 1, 0, 0u);
     }
     tc_fence_before();
     __syncthreads();
@@ -666,13 +677,206 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
         }
         __syncwarp();
     } else {
-        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane, blockIdx.x, gridDim.x, a.MT, 0, 0u);
     }
     tc_fence_before();
     __syncthreads();
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(a.tmem_cols) : "memory");
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// CTA pairs (tcgen05.mma.cta_group::2): the column-slab scheme with one 256-row tile pair per work item.
+// Wide layers are bound by their weights: per 64-channel chunk a tile needs 54 KB of input slabs but 288 KB of
+// weights at 256 output channels.  Here the two CTAs of a cluster (two SMs of one TPC) take one tile each and HALF of
+// the item's output channels' weights each; one MMA instruction, issued by the leader (rank 0), reads both CTAs'
+// operands (M = 256: 128 rows from each CTA's slab; N = BN: BN / 2 columns from each CTA's weight tile) and
+// accumulates into both CTAs' tensor memory (each holds its own tile's 128 rows x BN columns).  Per tile the weight
+// traffic into an SM halves, and the accumulators stay double buffered (2 x BN <= 512 columns per CTA).
+//
+// Every load is a plain per-CTA TMA load into the CTA's own shared memory (no multicast anywhere); the loads of the
+// second CTA report their bytes to the leader's barrier (cta_group::2 form of the load), because the leader's MMA
+// thread is the only consumer.  Barriers: full / a_full / tmem_empty live in the leader and collect both CTAs;
+// empty / a_empty / tmem_full exist in each CTA and are signalled in both by the leader's tcgen05.commit.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ uint32_t map_to_cta(const void* p, uint32_t rank)      // shared::cluster address of p in CTA `rank`
+{
+    uint32_t out;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(out) : "r"(smem_u32(p)), "r"(rank));
+    return out;
+}
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// loads into this CTA's shared memory whose bytes are counted on the barrier at shared::cluster address `bar` (the leader's)
+__device__ __forceinline__ void tma_load_4d_pair(void* dst, const CUtensorMap* tm, int c0, int c1, int c2, int c3, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const CUtensorMap* tm, int c0, int c1, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+                 ::"r"(smem_u32(dst)), "l"(tm), "r"(bar), "r"(c0), "r"(c1) : "memory");
+}
+__device__ __forceinline__ void umma_f16_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                 "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                 ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// arrives, once the MMAs issued so far have retired, on the barrier at this offset in both CTAs of the pair
+__device__ __forceinline__ void umma_commit_pair(void* bar)
+{
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"((uint16_t)3) : "memory");
+}
+
+// ha.t.BN: output channels per item (both CTAs together); ha.t.b_bytes: one CTA's weight tile (BN / 2 rows of 128 bytes);
+// tmW: the packed weights [2 NB][taps][kchunks][8][BN / 2][8] seen as rows of 128 bytes.
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+k_conv_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmW, const TcHaloArgs ha)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const TcArgs& a = ha.t;
+    const int n_tiles = *a.tile_count;
+    const int n_items = (n_tiles + 1) / 2 * a.NB;
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+    if (pair >= n_items) return;                              // both CTAs of a pair leave together
+    const uint32_t rank = cluster_rank();
+    const bool leader = rank == 0;
+    uint8_t* aring = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    const int a_slot = ha.patch_bytes;                        // one slab
+    uint8_t* bring = aring + (size_t)ha.a_stages * a_slot;
+    SmemCtl* ctl = (SmemCtl*)(bring + (size_t)a.stages * a.b_bytes);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int per_stream = a.tiles_x * a.tiles_y;
+    const int taps = a.kh * a.kw;
+
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < a.stages; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 256); }
+        for (int i = 0; i < 4; ++i) { mbar_init(&ctl->a_full[i], 1); mbar_init(&ctl->a_empty[i], 1); }
+        ctl->abort_flag = 0;
+        ctl->wait_ns = a.wait_ns;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
+        asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
+    }
+    if (warp == 1) {                                          // the same warp in both CTAs: tensor memory of the pair
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                       // both CTAs' barriers exist before either is signalled from outside
+    tc_fence_after();
+    const uint32_t tmem_base = ctl->tmem_base;
+
+    if (warp == 0) {
+        // ---------------- producer: this CTA's slab and its half of the weights ----------------
+        const uint32_t a_full0 = map_to_cta(&ctl->a_full[0], 0), full0 = map_to_cta(&ctl->full[0], 0);   // the leader's barriers
+        int sa = 0, sb = 0; uint32_t pa = 0, pb = 0;
+        bool ok = true;
+        const int rows_per_tile = a.b_bytes >> 7;             // weight rows of 128 bytes in one CTA's tile
+        for (int item = pair; item < n_items && ok; item += n_pairs) {
+            const int group = item / a.NB, nb = item % a.NB;
+            const int idx = group * 2 + (int)rank;
+            const int tile = a.tile_list[idx < n_tiles ? idx : group * 2];      // an absent second tile repeats the first (never stored)
+            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+            const int xb = tx * DC_TILE_W - a.pw, yb = ty * DC_TILE_H - a.ph;
+            for (int cc = 0; cc < a.kchunks && ok; ++cc) {
+                for (int kx = 0; kx < a.kw && ok; ++kx) {
+                    if (lane == 0) {
+                        ok = mbar_wait(&ctl->a_empty[sa], pa ^ 1u, ctl, a.status);
+                        if (ok && !a.skip_loads) {
+                            if (leader) mbar_expect_tx(&ctl->a_full[sa], (uint32_t)(2 * ha.patch_bytes));
+                            tma_load_4d_pair(aring + (size_t)sa * a_slot, &tmA, cc * 64, xb + kx, yb, s, a_full0 + (uint32_t)sa * 8u);
+                        }
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
+                    for (int t2 = 0; t2 < a.kh && ok; ++t2) {
+                        const int tap = t2 * a.kw + kx;
+                        if (lane == 0) {
+                            ok = mbar_wait(&ctl->empty[sb], pb ^ 1u, ctl, a.status);
+                            if (ok && !a.skip_loads) {
+                                if (leader) mbar_expect_tx(&ctl->full[sb], (uint32_t)(2 * a.b_bytes));
+                                const int row = (((nb * 2 + (int)rank) * taps + tap) * a.kchunks + cc) * rows_per_tile;
+                                tma_load_2d_pair(bring + (size_t)sb * a.b_bytes, &tmW, 0, row, full0 + (uint32_t)sb * 8u);
+                            }
+                        }
+                        ok = __shfl_sync(0xffffffffu, ok, 0);
+                        if (++sb == a.stages) { sb = 0; pb ^= 1u; }
+                    }
+                }
+            }
+        }
+        if (!ok && lane == 0) { const unsigned long long t0 = now_ns(); while (now_ns() - t0 < 2000000ull) { } }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer: the leader's lane 0 issues for both CTAs ----------------
+        if (leader && lane == 0) {
+            const uint32_t b_lbo = (uint32_t)(a.BN / 2) * 16u;
+            const uint64_t aconst = umma_desc(0, 1024, 2);
+            const uint64_t bconst = umma_desc(0, 128, 0, b_lbo);
+            const uint32_t aring_lo = smem_u32(aring) >> 4, bring_lo = smem_u32(bring) >> 4;
+            const uint32_t a_slot_lo = (uint32_t)a_slot >> 4;
+            const uint32_t b_kstep = (2 * b_lbo) >> 4, b_lo = (uint32_t)a.b_bytes >> 4;
+            int sa = 0, sb = 0; uint32_t pa = 0, pb = 0, acc = 0, acc_ph = 0;
+            bool ok = true;
+            for (int item = pair; item < n_items && ok; item += n_pairs) {
+                const uint32_t d_tmem = tmem_base + acc * (uint32_t)a.BN;
+                ok = mbar_wait(&ctl->tmem_empty[acc], acc_ph ^ 1u, ctl, a.status);
+                tc_fence_after();
+                uint32_t accumulate = 0;
+                for (int cc = 0; cc < a.kchunks && ok; ++cc) {
+                    for (int ax = 0; ax < a.kw && ok; ++ax) {
+                        ok = mbar_wait(&ctl->a_full[sa], pa, ctl, a.status);
+                        const uint64_t aslab = aconst + (aring_lo + (uint32_t)sa * a_slot_lo);
+                        for (int t = 0; t < a.kh && ok; ++t) {               // tap (t, ax): the slab from swizzle atom t on
+                            ok = mbar_wait(&ctl->full[sb], pb, ctl, a.status);
+                            if (!ok) break;
+                            tc_fence_after();
+                            const uint64_t bdesc = bconst + (bring_lo + (uint32_t)sb * b_lo);
+                            const uint64_t adesc = aslab + (uint32_t)t * 64u;
+#pragma unroll
+                            for (int kk = 0; kk < 4; ++kk) {                 // K = 16 per instruction, 64 channels per chunk
+                                umma_f16_pair(d_tmem, adesc + kk * 2u, bdesc + kk * b_kstep, a.idesc, accumulate);
+                                accumulate = 1;
+                            }
+                            umma_commit_pair(&ctl->empty[sb]);
+                            if (++sb == a.stages) { sb = 0; pb ^= 1u; }
+                        }
+                        if (ok) umma_commit_pair(&ctl->a_empty[sa]);
+                        if (++sa == ha.a_stages) { sa = 0; pa ^= 1u; }
+                    }
+                }
+                if (ok) umma_commit_pair(&ctl->tmem_full[acc]);
+                if (++acc == 2u) { acc = 0; acc_ph ^= 1u; }
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---------------- epilogue: this CTA's tile; the accumulator is handed back on the leader's barrier ----------------
+        const uint32_t remote_empty = map_to_cta(&ctl->tmem_empty[0], 0);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane, pair, n_pairs, 2, (int)rank, remote_empty);
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();                                       // neither CTA frees tensor memory or leaves while the other may still use it
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(a.tmem_cols) : "memory");
     }
 }
 
@@ -1066,10 +1270,101 @@ static int launch_halo(dc_cache* c, int layer, int mt, bool slab, const void* in
     return DC_OK;
 }
 
+// The CTA-pair kernel takes stride-1 layers with cin a multiple of 64 (the column-slab conditions) whose output
+// channels divide into blocks of 256 or 128 (half a block per CTA).
+static bool pair_ok(const dc_layer_desc& d, int& bn)
+{
+    HaloPlan h;
+    if (!halo_ok(d, h)) return false;
+    bn = d.cout % 256 == 0 ? 256 : (d.cout % 128 == 0 ? 128 : 0);
+    return bn != 0;
+}
+
+static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
+                       const int32_t* tile_count, const uint32_t* masks, int max_tiles)
+{
+    dc_layer_rt& L = c->L[layer];
+    const dc_layer_desc& d = L.d;
+    EncodeTiledFn enc = encode_fn();
+    int bn = 0;
+    if (!enc || !L.weight_halo || !pair_ok(d, bn)) return DC_ERR_CONFIG;
+    const int half = bn / 2, taps = d.kh * d.kw, kchunks = d.cin / 64;
+    if (L.halo_bn != half) {                                     // weights grouped by half blocks: [2 NB][taps][kchunks][8][half][8]
+        const size_t n = (size_t)d.cout * taps * d.cin;
+        int pgrid = (int)((n + 255) / 256); if (pgrid > c->num_sms * 8) pgrid = c->num_sms * 8;
+        k_pack_halo<<<pgrid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, d.cout, taps, d.cin, half, (__nv_bfloat16*)L.weight_halo);
+        L.halo_bn = half;
+    }
+    const int PH = DC_TILE_H + d.kh - 1;
+    bool hit_a, hit_b;
+    CUtensorMap* tmAp = tm_find(L.tm_a, 2, &L.tm_next, in, 5, 0, &hit_a);     // the column-slab map of the single-CTA kernel
+    if (!hit_a) {
+        cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
+        cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
+        cuuint32_t box[4] = {64, DC_TILE_W, (cuuint32_t)PH, 1};
+        cuuint32_t estr[4] = {1, 1, 1, 1};
+        if (enc(tmAp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            tm_drop(L.tm_a, 2, tmAp);
+            return DC_ERR_CUDA;
+        }
+    }
+    const int b_bytes = half * 128;                              // one CTA's weight tile: half rows of 64 channels
+    CUtensorMap* tmWp = tm_find(&L.tm_b, 1, nullptr, L.weight_halo, 7, half, &hit_b);
+    if (!hit_b) {                                                // the packed weights as rows of 128 bytes; a box is one tile
+        const cuuint64_t rows = (cuuint64_t)d.cout * taps * d.cin * 2 / 128;
+        cuuint64_t dims[2] = {64, rows};
+        cuuint64_t strides[1] = {128};
+        cuuint32_t box[2] = {64, (cuuint32_t)(b_bytes / 128)};
+        cuuint32_t estr[2] = {1, 1};
+        if (enc(tmWp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, L.weight_halo, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+            tm_drop(&L.tm_b, 1, tmWp);
+            return DC_ERR_CUDA;
+        }
+    }
+    TcHaloArgs ha;
+    TcArgs& a = ha.t;
+    a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
+    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
+    a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
+    a.BN = bn; a.NB = d.cout / bn; a.BK = 64; a.kchunks = kchunks; a.MT = 1; a.nbuf = 2;
+    a.a_bytes = 0; a.b_bytes = b_bytes; a.sbo = 128; a.layout_type = 0;
+    // instruction descriptor: D = f32, A = B = bf16, both K-major, N = bn, M = 256 (128 rows in each CTA)
+    a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+    a.status = c->status;
+    set_wait_limit(c, a);
+    a.tmem_cols = tmem_cols_for(2, 1, bn);
+    ha.wpacked = (const __nv_bfloat16*)L.weight_halo;
+    ha.PW = DC_TILE_W; ha.PH = PH; ha.plane_bytes = 0;
+    ha.patch_bytes = PH * DC_TILE_W * 128;                       // one slab
+    const int budget = ring_budget(1);
+    ha.a_stages = 2;
+    for (int as = 4; as > 2; --as)
+        if (budget - as * ha.patch_bytes >= 4 * b_bytes) { ha.a_stages = as; break; }
+    int st = (budget - ha.a_stages * ha.patch_bytes) / b_bytes;
+    a.stages = st > kMaxStages ? kMaxStages : st;
+    if (a.stages < 2) return DC_ERR_CONFIG;
+    const size_t smem = (size_t)ha.a_stages * ha.patch_bytes + (size_t)a.stages * b_bytes + sizeof(SmemCtl) + 1280;
+    if (smem > 227 * 1024) return DC_ERR_CONFIG;
+    static dc_once_per_device attr_set;
+    if (attr_set.first(c->device))
+        DC_CUDA(cudaFuncSetAttribute(k_conv_tc_pair, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
+    const long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + 1) / 2) * a.NB;
+    const int max_pairs = c->num_sms / 2;                        // one CTA per SM, a pair per TPC
+    const int pairs = items > max_pairs ? max_pairs : (int)items;
+    dc_prof_scope ps(c, DC_ST_CONV);
+    k_conv_tc_pair<<<2 * pairs, kThreads, smem, c->stream>>>(*tmAp, *tmWp, ha);
+    c->launches += 1;
+    DC_CUDA(cudaGetLastError());
+    return DC_OK;
+}
+
 int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
+    if (L.tc_mt == 7) return launch_pair(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
     if (L.tc_mt >= 5) return launch_halo(c, layer, L.tc_mt - 4, true, in, out, tile_list, tile_count, masks, max_tiles);
     if (L.tc_mt >= 3) return launch_halo(c, layer, L.tc_mt - 2, false, in, out, tile_list, tile_count, masks, max_tiles);
     const bool pad16 = pad16_ok(L.d) && L.weight_packed && L.in_padded;
@@ -1170,7 +1465,8 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
     const bool verbose = getenv("DC_VERBOSE") != nullptr;
     // times the launch the current L.tc_* fields select; keeps it when it is the fastest so far
     // DC_CONV_SCHEME=<code> (diagnostics, tests): only candidates of that operand scheme are timed, so the scheme runs
-    // wherever it can (1, 2 tap by tap; 3, 4 patch; 5, 6 column slabs; the second of each pair with two tiles per item)
+    // wherever it can (1, 2 tap by tap; 3, 4 patch; 5, 6 column slabs; the second of each pair with two tiles per item;
+    // 7 column slabs on CTA pairs)
     const int only = getenv("DC_CONV_SCHEME") ? atoi(getenv("DC_CONV_SCHEME")) : 0;
     auto trial = [&](const char* what) {
         if (only > 0 && generic && L.tc_mt != only) return;
@@ -1217,6 +1513,13 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
                     trial("column-slab kernel");
                 }
             }
+        }
+    }
+    {
+        int pbn = 0;
+        if (generic && L.weight_halo && pair_ok(L.d, pbn)) {          // tc_mt 7: a CTA pair per two tiles (cta_group::2)
+            L.tc_mt = 7; L.tc_bn = pbn; L.tc_ctas = 1;
+            trial("CTA-pair kernel");
         }
     }
     L.tc_mt = best_mt; L.tc_bn = best_bn; L.tc_ctas = best_ctas;

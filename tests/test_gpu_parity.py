@@ -426,10 +426,11 @@ def test_conv_partial_ignores_rectangles_outside_the_map():
         dc.close()
 
 
-@pytest.mark.parametrize("scheme", [1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("scheme", [1, 2, 3, 4, 5, 6, 7])
 def test_conv_schemes_forced(scheme, monkeypatch):
     """Every operand scheme of the tensor-core convolution (tap by tap, patch, column slabs; one or two tiles per
-    item) on layers it can take: VGG-shaped 3x3 layers, a 5x5 layer and odd map sizes, through cached frames."""
+    item; column slabs on CTA pairs) on layers it can take: VGG-shaped 3x3 layers, a 5x5 layer and odd map sizes,
+    through cached frames."""
     monkeypatch.setenv("DC_CONV_SCHEME", str(scheme))
     b = nets.NetBuilder(45, 53)
     x = b.conv(-1, 64, 3, 1, 1)
@@ -577,8 +578,55 @@ def test_region_overflow_sets_the_status_word():
         dc.close()
 
 
-@pytest.mark.parametrize("cin,k", [(64, 3), (32, 1), (3, 3)])      # column-slab / patch kernels, tap-by-tap kernel, few-channel kernel
-def test_bounded_device_waits_run_out_and_the_cache_stays_usable(cin, k):
+@pytest.mark.parametrize("scheme", [5, 7])
+@pytest.mark.parametrize("hi,wi,cin,cout,k,p", [(14, 14, 256, 512, 3, 1), (28, 28, 128, 256, 3, 1), (17, 23, 64, 128, 5, 2), (9, 40, 128, 256, 1, 0)])
+def test_conv_wide_layers_on_cta_pairs(scheme, hi, wi, cin, cout, k, p, monkeypatch):
+    """The wide layers (128 - 512 output channels) forced onto the CTA-pair kernel (7), and onto the single-CTA column-slab
+    kernel (5) for comparison: full convolution and partial convolution with an odd number of dirty tiles."""
+    monkeypatch.setenv("DC_CONV_SCHEME", str(scheme))
+    g = rng(hi * 7 + cout)
+    S = 3
+    nb = nets.NetBuilder(hi, wi)
+    a = nb.conv(-1, cin, 1, 1, 0)
+    nb.conv(a, cout, k, 1, p, 1)
+    L = nb.layers[1]
+    wts = g.normal(0, np.sqrt(2.0 / (k * k * cin)), size=(cout, k, k, cin)).astype(np.float32)
+    bias = g.normal(0, 0.1, size=cout).astype(np.float32)
+    ws = [np.zeros((cin, 1, 1, 3), np.float32), wts]
+    bs = [np.zeros(cin, np.float32), bias]
+    xq = np.stack([orc.quant_array(g.normal(size=(hi, wi, cin)), orc.QUANT_BF16) for _ in range(S)])
+    pq = np.stack([orc.quant_array(g.normal(size=(L["out_h"], L["out_w"], cout)), orc.QUANT_BF16) for _ in range(S)])
+    dc = DeepCache(wi, hi, nb.layers, ws, bs, n_streams=S, block=16, search_range=4, dtype=B.DC_BF16, max_regions=4)
+    try:
+        xin = torch.from_numpy(xq).to(torch.bfloat16).cuda()
+        pin = torch.from_numpy(pq).to(torch.bfloat16).cuda()
+        full = dc.conv_partial(1, xin)
+        # one rectangle that covers the whole map of stream 1 (its tiles are clean: the dirty count becomes odd for
+        # most shapes) and a small one in stream 0
+        regs = torch.zeros((S, dc.max_regions, 6), dtype=torch.int32)
+        regs[1, 0] = torch.tensor([0, 0, L["out_w"], L["out_h"], 0, 0], dtype=torch.int32)
+        regs[0, 0] = torch.tensor([1, 2, 5, 4, 2, 1], dtype=torch.int32)
+        counts = torch.tensor([1, 1, 0], dtype=torch.int32)
+        part = dc.conv_partial(1, xin, pin, regs.cuda(), counts.cuda())
+        wq = orc.quant_array(wts, orc.QUANT_BF16)
+        for s_ in range(S):
+            r = np.zeros(1, orc.REGION_DTYPE)
+            r[0] = tuple(int(v) for v in regs[s_, 0])
+            want_full, _ = orc.conv_reuse(xq[s_], L, wq, bias, orc.QUANT_BF16)
+            want, reused = orc.conv_reuse(xq[s_], L, wq, bias, orc.QUANT_BF16, pq[s_], r[:int(counts[s_])])
+            U.assert_map_close(full[s_], want_full, True, f"full, stream {s_}")
+            U.assert_map_close_per_element(full[s_], want_full, f"full, per element, stream {s_}")
+            U.assert_map_close(part[s_], want, True, f"partial, stream {s_}")
+            m = reused.astype(bool)
+            got = part[s_].float().cpu().numpy().astype(np.float64)
+            assert np.array_equal(got[m], want[m])
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
+
+
+@pytest.mark.parametrize("cin,k", [(64, 3), (32, 1), (3, 3), (128, 7)])      # column-slab / patch kernels, tap-by-tap kernel, few-channel kernel, CTA pairs
+def test_bounded_device_waits_run_out_and_the_cache_stays_usable(cin, k, monkeypatch):
     """Failure detection without a fault: one convolution launch is armed so that its producer issues no copy.  The
     other roles' waits then run out after a few milliseconds instead of spinning for ever: the kernel returns, the
     status word reads DC_ERR_TIMEOUT, tensor memory is free again, and the next launch on the same cache is correct."""
@@ -586,6 +634,9 @@ def test_bounded_device_waits_run_out_and_the_cache_stays_usable(cin, k):
     g = rng(90 + cin)
     hi = wi = 40
     cout = 64
+    if k == 7:                                                     # stands for: a 3x3 layer of 128 -> 256 channels forced onto CTA pairs
+        k, cout = 3, 256
+        monkeypatch.setenv("DC_CONV_SCHEME", "7")
     nb = nets.NetBuilder(hi, wi)
     if cin == 3:
         nb.conv(-1, cout, k, 1, k // 2, 1)
