@@ -54,6 +54,9 @@ def parse_args():
     ap.add_argument("--reuse-copy", action="store_true",
                     help="time the reuse copy alone (Section 5 'Reuse', step 1) on one 64-channel 224x224 bf16 layer with "
                          "rectangles covering most of the map, through dc_conv_partial; prints a short JSON line")
+    ap.add_argument("--conv-layer", default="",
+                    help="CIN,COUT,HW[,K]: time one bf16 convolution layer alone (all tiles computed, --streams maps of HW x HW, K x K "
+                         "kernel, default 3) through dc_conv_partial and print a short JSON line; DC_CONV_SCHEME selects the operand scheme")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -280,10 +283,47 @@ def reuse_copy_bench(args, B, DeepCache, rank, dev):
                           "conv_ms_per_launch": prof["conv"][0] / max(1, prof["conv"][1]), "status": status}))
 
 
+def conv_layer_bench(args, B, DeepCache, rank, dev):
+    """One convolution layer alone, every tile computed: CIN -> COUT channels on HW x HW maps, bf16, S streams."""
+    import torch
+    from paper_1712_01670_b200.synth import nets
+    parts = [int(v) for v in args.conv_layer.split(",")]
+    cin, cout, hw = parts[:3]
+    k = parts[3] if len(parts) > 3 else 3
+    S = args.streams or 32
+    nb = nets.NetBuilder(hw, hw)
+    first = nb.conv(-1, cin, 1, 1, 0)                    # stands in for the producer of the layer's input
+    nb.conv(first, cout, k, 1, k // 2, 1)
+    ws, bs = nets.random_weights(nb.layers, 9)
+    dc = DeepCache(hw, hw, nb.layers, ws, bs, n_streams=S, block=16, search_range=4, dtype=B.DC_BF16)
+    x = torch.randn((S, hw, hw, cin), device=dev).to(torch.bfloat16)
+    out = torch.empty((S, hw, hw, cout), device=dev, dtype=torch.bfloat16)
+    for _ in range(args.warmup):
+        B.dc_conv_partial(dc.handle, 1, x, None, None, None, out)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        B.dc_conv_partial(dc.handle, 1, x, None, None, None, out)
+    e1.record()
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / args.steps
+    status = dc.status()
+    dc.close()
+    flops = 2.0 * S * hw * hw * cout * cin * k * k
+    peaks = measured_peaks()
+    tf = flops / (ms * 1e-3) / 1e12
+    if rank == 0:
+        print(json.dumps({"stage": f"convolution {cin} -> {cout}, {k}x{k}, {hw}x{hw} maps, bf16, all tiles", "streams": S,
+                          "scheme": os.environ.get("DC_CONV_SCHEME", "tuned"), "ms_per_launch": ms, "tflops": tf,
+                          "frac_burst": tf / peaks["bf16_tflops"], "frac_sustained": tf / peaks["bf16_tflops_sustained"],
+                          "status": status}))
+
+
 def gpu_arm_on_stream(args, w, B, sharding, DeepCache, dist, rank, world, local, dev):
     import torch
-    if args.reuse_copy:
-        reuse_copy_bench(args, B, DeepCache, rank, dev)
+    if args.reuse_copy or args.conv_layer:
+        (reuse_copy_bench if args.reuse_copy else conv_layer_bench)(args, B, DeepCache, rank, dev)
         if world > 1:
             dist.destroy_process_group()
         return

@@ -239,6 +239,12 @@ int dc_cache_layer_map(dc_cache* cache, int layer, void** map_dev, size_t* bytes
  * `layer` ([S][max_regions]) and of their per-stream count ([S]). */
 int dc_cache_layer_regions(dc_cache* cache, int layer, dc_region** regions_dev, int32_t** n_dev);
 
+/* Which kernel family runs convolution layer `layer` (chosen at creation): -1 not an executable convolution,
+ * 0 the CUDA-core kernel (fp32 caches, channel counts the tensor-core kernels cannot take), 1-7 a tensor-core
+ * operand scheme (1, 2 tap by tap; 3, 4 input patch; 5, 6 column slabs; 7 column slabs on CTA pairs; grouped
+ * layers run their scheme once per group).  For inspection and tests.  Errors: DC_ERR_ARG. */
+int dc_cache_layer_conv_scheme(const dc_cache* cache, int layer, int32_t* scheme);
+
 /* Waits for the stream and returns the device status word: DC_OK, or what a kernel recorded since the
  * last reset: DC_ERR_OVERFLOW (Step 5 found more rectangles than max_regions), DC_ERR_TIMEOUT (a bounded
  * device-side wait or walk ran out; the affected results are not valid), DC_ERR_ARG (a caller's rectangle

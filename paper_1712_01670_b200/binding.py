@@ -52,7 +52,7 @@ REGION_DTYPE = np.dtype([(n, "<i4") for n in ("x", "y", "w", "h", "sx", "sy")])
 EXPORTS = ["dc_cache_create", "dc_cache_destroy", "dc_cache_reset", "dc_cache_bytes", "dc_cache_set_key",
            "dc_match_blocks", "dc_propagate_regions", "dc_conv_partial", "dc_infer_frame", "dc_infer_frame_host",
            "dc_prefetch_frame_host", "dc_lookahead_frame",
-           "dc_cache_layer_map", "dc_cache_layer_regions", "dc_get_status", "dc_cache_launches",
+           "dc_cache_layer_map", "dc_cache_layer_regions", "dc_cache_layer_conv_scheme", "dc_get_status", "dc_cache_launches",
            "dc_cache_set_profiling", "dc_cache_profile", "dc_cache_counters", "dc_search_blocks_noalloc", "dc_strerror"]
 PROFILE_STAGES = ["search", "verify", "merge", "propagate", "classify_copy", "conv", "input", "pointwise", "key_update"]
 
@@ -88,6 +88,7 @@ def load():
         L.dc_lookahead_frame.argtypes = [vp, vp, sz]
         L.dc_cache_layer_map.argtypes = [vp, i, C.POINTER(vp), C.POINTER(sz)]
         L.dc_cache_layer_regions.argtypes = [vp, i, C.POINTER(vp), C.POINTER(vp)]
+        L.dc_cache_layer_conv_scheme.argtypes = [vp, i, C.POINTER(C.c_int32)]
         L.dc_get_status.argtypes = [vp, C.POINTER(C.c_int32)]
         L.dc_cache_launches.argtypes = [vp, C.POINTER(C.c_int64)]
         L.dc_cache_set_profiling.argtypes = [vp, i]
@@ -213,6 +214,12 @@ def dc_cache_layer_regions(cache, layer):
     p, n = C.c_void_p(), C.c_void_p()
     _check(load().dc_cache_layer_regions(cache, layer, C.byref(p), C.byref(n)), "dc_cache_layer_regions")
     return p.value, n.value
+
+
+def dc_cache_layer_conv_scheme(cache, layer: int) -> int:
+    v = C.c_int32(0)
+    _check(load().dc_cache_layer_conv_scheme(cache, layer, C.byref(v)), "dc_cache_layer_conv_scheme")
+    return v.value
 
 
 def dc_get_status(cache) -> int:

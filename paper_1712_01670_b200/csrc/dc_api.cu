@@ -679,6 +679,16 @@ int dc_cache_layer_map(dc_cache* c, int layer, void** map_dev, size_t* bytes)
     return DC_OK;
 }
 
+int dc_cache_layer_conv_scheme(const dc_cache* c, int layer, int32_t* scheme)
+{
+    if (!c || layer < 0 || layer >= c->n_layers || !scheme) return DC_ERR_ARG;
+    const dc_layer_rt& L = c->L[layer];
+    if (L.d.kind != DC_CONV || !c->executable) { *scheme = -1; return DC_OK; }
+    if (!dc_conv_bf16_supported(c, layer)) { *scheme = 0; return DC_OK; }
+    *scheme = L.tc_mt > 0 ? L.tc_mt : 1;
+    return DC_OK;
+}
+
 int dc_cache_layer_regions(dc_cache* c, int layer, dc_region** regions_dev, int32_t** n_dev)
 {
     if (!c || layer < -1 || layer >= c->n_layers || !regions_dev) return DC_ERR_ARG;

@@ -54,7 +54,7 @@ struct dc_layer_rt {
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation
     int32_t* all_list;              // conv: every tile (used by full frames)
-    dc_tm_slot tm_a[2], tm_b;       // conv, bf16: tensor maps of the input (two bases) and of the weights
+    dc_tm_slot tm_a[4], tm_b;       // conv, bf16: tensor maps of the input (two bases, two channel groups) and of the weights
     int tm_next;                    // which of tm_a[] a new input base replaces
 };
 
@@ -168,3 +168,4 @@ bool dc_layer_cached(const dc_cache* c, int layer);
 int dc_build_classify_table(dc_cache* c);
 int dc_launch_classify_all(dc_cache* c, int cur);
 int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in);
+int dc_conv_bf16_supported(const dc_cache* c, int layer);    // 1 when the layer runs on the tensor-core kernels

@@ -35,6 +35,7 @@ struct TcArgs {
     const int32_t* tile_list; const int32_t* tile_count; const uint32_t* masks;
     int Ho, Wo, Co, Ci, kh, kw, sh, sw, ph, pw, relu, tiles_x, tiles_y;
     int BN, NB, BK, kchunks, stages, a_bytes, b_bytes;
+    int nb_off;                   // grouped convolution: first channel block of the group this launch computes
     int MT, nbuf;                 // tiles per work item (1 or 2, sharing one B tile); TMEM accumulator sets (2, or 1 when MT * BN = 512)
     uint32_t idesc, sbo, layout_type;
     uint32_t tmem_cols;           // TMEM columns this CTA allocates: a power of two >= nbuf * MT * BN (256 at most when two CTAs share an SM)
@@ -200,7 +201,7 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         tc_fence_after();
-        const float* bias = a.bias + nb * a.BN;
+        const float* bias = a.bias + (nb + a.nb_off) * a.BN;
         for (int j = 0; j < a.MT; ++j) {
             const int tile = j == 0 ? tile_c0 : tile_c1;
             if (tile < 0) break;
@@ -219,7 +220,7 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
             // tile row q * 4 + k, column lane >> 2 (the warp's 32 pixels are 4 tile rows of 8)
             const size_t row_stride = (size_t)a.Wo * a.Co;
             __nv_bfloat16* const wb = a.out + ((size_t)s * a.Ho + ty * DC_TILE_H + q * 4) * row_stride +
-                                      (size_t)(tx * DC_TILE_W + (lane >> 2)) * a.Co + nb * a.BN + (lane & 3) * 8;
+                                      (size_t)(tx * DC_TILE_W + (lane >> 2)) * a.Co + (nb + a.nb_off) * a.BN + (lane & 3) * 8;
             const uint8_t* const rd = stg + (lane >> 2) * 80 + (lane & 3) * 16;
             for (int c = 0; c < a.BN / 32; ++c) {
                 uint32_t r[32];
@@ -316,7 +317,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 #pragma unroll
                             for (int j = 0; j < MT; ++j)
                                 tma_load_4d(sa + j * a.a_bytes, &tmA, cc * a.BK, xb[j] + kx, yb[j] + ky, sN[j], &ctl->full[st]);
-                            tma_load_2d(sa + MT * a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, nb * a.BN, &ctl->full[st]);
+                            tma_load_2d(sa + MT * a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, (nb + a.nb_off) * a.BN, &ctl->full[st]);
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -612,7 +613,7 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
                             ok = mbar_wait(&ctl->empty[sb], pb ^ 1u, ctl, a.status);
                             if (ok && !a.skip_loads) {
                                 mbar_expect_tx(&ctl->full[sb], (uint32_t)a.b_bytes);
-                                const uint8_t* src = (const uint8_t*)ha.wpacked + ((size_t)(nb * taps + tap) * a.kchunks + cc) * a.b_bytes;
+                                const uint8_t* src = (const uint8_t*)ha.wpacked + ((size_t)((nb + a.nb_off) * taps + tap) * a.kchunks + cc) * a.b_bytes;
                                 bulk_copy_g2s(bring + (size_t)sb * a.b_bytes, src, (uint32_t)a.b_bytes, &ctl->full[sb]);
                             }
                         }
@@ -1007,6 +1008,19 @@ static void set_wait_limit(dc_cache* c, TcArgs& a)
     }
 }
 
+// A grouped convolution (AlexNet's layers 2, 4, 5) is `groups` independent convolutions, each from its own slice of
+// the input channels to its own slice of the output channels.  One launch per group: the input tensor map starts at
+// the group's first channel and spans the group's channels only (pixels keep the full layer's pitch), the weights
+// [cout][kh][kw][cin / groups] need no slicing, and the kernel adds the group's first channel block (nb_off) to the
+// channel blocks it reads weights for and writes.  This is the layer as one group sees it.
+static int n_groups(const dc_layer_desc& d) { return d.groups > 1 ? d.groups : 1; }
+static dc_layer_desc group_view(const dc_layer_desc& d)
+{
+    dc_layer_desc g = d;
+    g.cin = d.cin / n_groups(d); g.cout = d.cout / n_groups(d); g.groups = 1;
+    return g;
+}
+
 struct TcPlan { int BK, BN, NB, MT, nbuf, stages, a_bytes, b_bytes; CUtensorMapSwizzle swz; uint32_t layout_type, sbo; size_t smem; };
 
 bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn = 0, int ctas = 1)
@@ -1084,7 +1098,10 @@ int dc_conv_bf16_supported(const dc_cache* c, int layer)
     TcPlan p;
     if (getenv("DC_NO_TENSOR_CORES")) return 0;
     if (c->cfg.dtype != DC_BF16 || encode_fn() == nullptr) return 0;
-    if (c->L[layer].d.groups > 1) return 0;                       // grouped layers run on the CUDA-core kernel
+    if (n_groups(c->L[layer].d) > 1) {                            // per group: the tap-by-tap kernel or the patch / slab kernels
+        const dc_layer_desc g = group_view(c->L[layer].d);
+        return make_plan(g, p) && (g.cin * 2) % 16 == 0;          // a group's first channel must be 16-byte aligned for its tensor map
+    }
     return make_plan(c->L[layer].d, p) || smallc_ok(c->L[layer].d) || pad16_ok(c->L[layer].d);
 }
 
@@ -1095,16 +1112,19 @@ int dc_pack_weights_bf16(dc_cache* c, int layer)
     dc_layer_rt& L = c->L[layer];
     TcPlan p;
     HaloPlan h;
-    if (halo_ok(L.d, h)) {
-        const size_t n = (size_t)L.d.cout * L.d.kh * L.d.kw * L.d.cin;
+    const dc_layer_desc dg = group_view(L.d);                     // the layer itself when it is not grouped
+    if (halo_ok(dg, h)) {
+        // [cout][taps][cin / groups]: channel blocks never straddle a group (BN divides cout / groups)
+        const size_t n = (size_t)L.d.cout * L.d.kh * L.d.kw * dg.cin;
         DC_CUDA(cudaMalloc(&L.weight_halo, n * 2));
         c->bytes += n * 2;
         int grid = (int)((n + 255) / 256); if (grid > c->num_sms * 8) grid = c->num_sms * 8;
-        k_pack_halo<<<grid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, L.d.cout, L.d.kh * L.d.kw, L.d.cin, h.BN,
+        k_pack_halo<<<grid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, L.d.cout, L.d.kh * L.d.kw, dg.cin, h.BN,
                                                  (__nv_bfloat16*)L.weight_halo);
         L.halo_bn = h.BN;
         DC_CUDA(cudaGetLastError());
     }
+    if (n_groups(L.d) > 1) return DC_OK;                          // grouped layers use the kernels above only
     if (pad16_ok(L.d)) {
         const size_t cout_taps = (size_t)L.d.cout * L.d.kh * L.d.kw;
         const size_t wbytes = cout_taps * 16 * 2, pbytes = (size_t)c->S * L.in_h * L.in_w * 32;
@@ -1140,7 +1160,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     const size_t pixels = (size_t)c->S * L.in_h * L.in_w;
     const int PW = DC_TILE_W + d.kw - 1, PH = DC_TILE_H + d.kh - 1;
     bool hit;
-    CUtensorMap* tmAp = tm_find(L.tm_a, 2, &L.tm_next, L.in_padded, 7, 0, &hit);
+    CUtensorMap* tmAp = tm_find(L.tm_a, 4, &L.tm_next, L.in_padded, 7, 0, &hit);
     if (!hit) {
         cuuint64_t dims[4] = {8, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
         cuuint64_t strides[3] = {16, (cuuint64_t)L.in_w * 16, (cuuint64_t)L.in_h * L.in_w * 16};
@@ -1148,7 +1168,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
         cuuint32_t estr[4] = {1, 1, 1, 1};
         if (enc(tmAp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, L.in_padded, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
-            tm_drop(L.tm_a, 2, tmAp);
+            tm_drop(L.tm_a, 4, tmAp);
             return DC_ERR_CUDA;
         }
     }
@@ -1158,7 +1178,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
     a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
     a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
-    a.BN = d.cout; a.NB = 1; a.MT = 1; a.nbuf = 2; a.BK = 16; a.kchunks = 1; a.a_bytes = 0; a.b_bytes = 0; a.sbo = 128; a.layout_type = 0;
+    a.BN = d.cout; a.NB = 1; a.nb_off = 0; a.MT = 1; a.nbuf = 2; a.BK = 16; a.kchunks = 1; a.a_bytes = 0; a.b_bytes = 0; a.sbo = 128; a.layout_type = 0;
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(d.cout >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
     set_wait_limit(c, a);
@@ -1189,35 +1209,37 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     return DC_OK;
 }
 
-static int launch_halo(dc_cache* c, int layer, int mt, bool slab, const void* in, void* out, const int32_t* tile_list,
+static int launch_halo(dc_cache* c, int layer, int grp, int mt, bool slab, const void* in, void* out, const int32_t* tile_list,
                        const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
-    const dc_layer_desc& d = L.d;
+    const dc_layer_desc d = group_view(L.d);                      // what one group computes; L.d itself when ungrouped
+    const int cin_all = L.d.cin, cout_all = L.d.cout;
     HaloPlan h;
     EncodeTiledFn enc = encode_fn();
     if (!enc || !L.weight_halo || !halo_ok(d, h, L.tc_bn)) return DC_ERR_CONFIG;
     if (L.halo_bn != h.BN) {
         // the packed weights are grouped by channel block: another block width needs another packing (same size).
         // Happens while the tuner tries widths and once more for its final choice, never in steady state.
-        const size_t n = (size_t)d.cout * d.kh * d.kw * d.cin;
+        const size_t n = (size_t)cout_all * d.kh * d.kw * d.cin;
         int pgrid = (int)((n + 255) / 256); if (pgrid > c->num_sms * 8) pgrid = c->num_sms * 8;
-        k_pack_halo<<<pgrid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, d.cout, d.kh * d.kw, d.cin, h.BN,
+        k_pack_halo<<<pgrid, 256, 0, c->stream>>>((const __nv_bfloat16*)L.weight, cout_all, d.kh * d.kw, d.cin, h.BN,
                                                   (__nv_bfloat16*)L.weight_halo);
         L.halo_bn = h.BN;
     }
+    in = (const uint8_t*)in + (size_t)grp * d.cin * 2;            // the group's first input channel
     bool hit;
-    CUtensorMap* tmAp = tm_find(L.tm_a, 2, &L.tm_next, in, slab ? 5 : 3, 0, &hit);
+    CUtensorMap* tmAp = tm_find(L.tm_a, 4, &L.tm_next, in, slab ? 5 : 3, 0, &hit);
     if (!hit) {
         cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
-        cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
+        cuuint64_t strides[3] = {(cuuint64_t)cin_all * 2, (cuuint64_t)L.in_w * cin_all * 2, (cuuint64_t)L.in_h * L.in_w * cin_all * 2};
         cuuint32_t box[4] = {8, (cuuint32_t)h.PW, (cuuint32_t)h.PH, 1};
         if (slab) { box[0] = 64; box[1] = DC_TILE_W; }            // a column slab: 64 channels x 8 pixels x PH rows
         cuuint32_t estr[4] = {1, 1, 1, 1};
         if (enc(tmAp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, slab ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_NONE,
                 CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
-            tm_drop(L.tm_a, 2, tmAp);
+            tm_drop(L.tm_a, 4, tmAp);
             return DC_ERR_CUDA;
         }
     }
@@ -1225,9 +1247,9 @@ static int launch_halo(dc_cache* c, int layer, int mt, bool slab, const void* in
     TcHaloArgs ha;
     TcArgs& a = ha.t;
     a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
-    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
+    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = cout_all; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
     a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
-    a.BN = h.BN; a.NB = h.NB; a.BK = 64; a.kchunks = d.cin / 64; a.MT = mt; a.nbuf = mt * h.BN * 2 <= 512 ? 2 : 1;
+    a.BN = h.BN; a.NB = h.NB; a.nb_off = grp * h.NB; a.BK = 64; a.kchunks = d.cin / 64; a.MT = mt; a.nbuf = mt * h.BN * 2 <= 512 ? 2 : 1;
     a.a_bytes = 0; a.b_bytes = h.b_bytes; a.sbo = 128; a.layout_type = 0;
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(h.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
@@ -1275,7 +1297,7 @@ static int launch_halo(dc_cache* c, int layer, int mt, bool slab, const void* in
 static bool pair_ok(const dc_layer_desc& d, int& bn)
 {
     HaloPlan h;
-    if (!halo_ok(d, h)) return false;
+    if (n_groups(d) > 1 || !halo_ok(d, h)) return false;
     bn = d.cout % 256 == 0 ? 256 : (d.cout % 128 == 0 ? 128 : 0);
     return bn != 0;
 }
@@ -1297,7 +1319,7 @@ static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const 
     }
     const int PH = DC_TILE_H + d.kh - 1;
     bool hit_a, hit_b;
-    CUtensorMap* tmAp = tm_find(L.tm_a, 2, &L.tm_next, in, 5, 0, &hit_a);     // the column-slab map of the single-CTA kernel
+    CUtensorMap* tmAp = tm_find(L.tm_a, 4, &L.tm_next, in, 5, 0, &hit_a);     // the column-slab map of the single-CTA kernel
     if (!hit_a) {
         cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
         cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
@@ -1305,7 +1327,7 @@ static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const 
         cuuint32_t estr[4] = {1, 1, 1, 1};
         if (enc(tmAp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
                 CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
-            tm_drop(L.tm_a, 2, tmAp);
+            tm_drop(L.tm_a, 4, tmAp);
             return DC_ERR_CUDA;
         }
     }
@@ -1328,7 +1350,7 @@ static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const 
     a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
     a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = 1; a.sw = 1;
     a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
-    a.BN = bn; a.NB = d.cout / bn; a.BK = 64; a.kchunks = kchunks; a.MT = 1; a.nbuf = 2;
+    a.BN = bn; a.NB = d.cout / bn; a.nb_off = 0; a.BK = 64; a.kchunks = kchunks; a.MT = 1; a.nbuf = 2;
     a.a_bytes = 0; a.b_bytes = b_bytes; a.sbo = 128; a.layout_type = 0;
     // instruction descriptor: D = f32, A = B = bf16, both K-major, N = bn, M = 256 (128 rows in each CTA)
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(bn >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
@@ -1360,15 +1382,31 @@ static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const 
     return DC_OK;
 }
 
+static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* out, const int32_t* tile_list,
+                        const int32_t* tile_count, const uint32_t* masks, int max_tiles);
+
 int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const int32_t* tile_list,
+                        const int32_t* tile_count, const uint32_t* masks, int max_tiles)
+{
+    const int G = n_groups(c->L[layer].d);
+    for (int grp = 0; grp < G; ++grp) {                           // a grouped layer: one launch per group
+        const int rc = launch_group(c, layer, grp, in, out, tile_list, tile_count, masks, max_tiles);
+        if (rc != DC_OK) return rc;
+    }
+    return DC_OK;
+}
+
+static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* out, const int32_t* tile_list,
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
     if (L.tc_mt == 7) return launch_pair(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
-    if (L.tc_mt >= 5) return launch_halo(c, layer, L.tc_mt - 4, true, in, out, tile_list, tile_count, masks, max_tiles);
-    if (L.tc_mt >= 3) return launch_halo(c, layer, L.tc_mt - 2, false, in, out, tile_list, tile_count, masks, max_tiles);
-    const bool pad16 = pad16_ok(L.d) && L.weight_packed && L.in_padded;
-    const dc_layer_desc d = pad16 ? padded16(L.d) : L.d;
+    if (L.tc_mt >= 5) return launch_halo(c, layer, grp, L.tc_mt - 4, true, in, out, tile_list, tile_count, masks, max_tiles);
+    if (L.tc_mt >= 3) return launch_halo(c, layer, grp, L.tc_mt - 2, false, in, out, tile_list, tile_count, masks, max_tiles);
+    const bool grouped = n_groups(L.d) > 1;
+    const bool pad16 = !grouped && pad16_ok(L.d) && L.weight_packed && L.in_padded;
+    const dc_layer_desc d = pad16 ? padded16(L.d) : group_view(L.d);
+    const int cin_all = pad16 ? 16 : L.d.cin, cout_all = L.d.cout;
     const void* weights = pad16 ? L.weight_packed : L.weight;
     if (pad16) {
         const size_t pixels = (size_t)c->S * L.in_h * L.in_w;
@@ -1378,6 +1416,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
         c->launches += 1;
         in = L.in_padded;
     }
+    in = (const uint8_t*)in + (size_t)grp * d.cin * 2;            // the group's first input channel (grp = 0 when ungrouped)
     TcPlan p;
     int ctas = L.tc_ctas == 2 ? 2 : 1;
     if (ctas == 2 && !make_plan(d, p, L.tc_mt, L.tc_bn, 2)) ctas = 1;
@@ -1388,22 +1427,22 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     EncodeTiledFn enc = encode_fn();
     if (!enc) return DC_ERR_CUDA;
     bool hit_a, hit_b;
-    CUtensorMap* tmAp = tm_find(L.tm_a, 2, &L.tm_next, in, 1, 0, &hit_a);
+    CUtensorMap* tmAp = tm_find(L.tm_a, 4, &L.tm_next, in, 1, 0, &hit_a);
     CUtensorMap* tmBp = tm_find(&L.tm_b, 1, nullptr, weights, 1, p.BN, &hit_b);
     if (!hit_a) {   // input map [S][Hi][Wi][Ci] bf16; box = BK channels x 16 columns x 8 rows x 1 stream
         cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
-        cuuint64_t strides[3] = {(cuuint64_t)d.cin * 2, (cuuint64_t)L.in_w * d.cin * 2, (cuuint64_t)L.in_h * L.in_w * d.cin * 2};
+        cuuint64_t strides[3] = {(cuuint64_t)cin_all * 2, (cuuint64_t)L.in_w * cin_all * 2, (cuuint64_t)L.in_h * L.in_w * cin_all * 2};
         // a strided convolution reads every sw-th column / sh-th row: the box spans TW * sw x TH * sh input
         // pixels and the traversal strides pick TW x TH of them
         cuuint32_t box[4] = {(cuuint32_t)p.BK, (cuuint32_t)(DC_TILE_W * d.sw), (cuuint32_t)(DC_TILE_H * d.sh), 1};
         cuuint32_t estr[4] = {1, (cuuint32_t)d.sw, (cuuint32_t)d.sh, 1};
         if (enc(tmAp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, p.swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) { tm_drop(L.tm_a, 2, tmAp); tm_drop(&L.tm_b, 1, tmBp); return DC_ERR_CUDA; }
+                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) { tm_drop(L.tm_a, 4, tmAp); tm_drop(&L.tm_b, 1, tmBp); return DC_ERR_CUDA; }
     }
     if (!hit_b) {   // weights [cout][K] bf16, K = kh * kw * cin
         const cuuint64_t K = (cuuint64_t)d.kh * d.kw * d.cin;
-        cuuint64_t dims[2] = {K, (cuuint64_t)d.cout};
+        cuuint64_t dims[2] = {K, (cuuint64_t)cout_all};               // every group's rows; a launch reads its own (nb_off)
         cuuint64_t strides[1] = {K * 2};
         cuuint32_t box[2] = {(cuuint32_t)p.BK, (cuuint32_t)p.BN};
         cuuint32_t estr[2] = {1, 1};
@@ -1415,9 +1454,9 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     const CUtensorMap& tmB = *tmBp;
     TcArgs a;
     a.bias = L.bias; a.out = (__nv_bfloat16*)out; a.tile_list = tile_list; a.tile_count = tile_count; a.masks = masks;
-    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = d.cout; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = d.sh; a.sw = d.sw;
+    a.Ho = d.out_h; a.Wo = d.out_w; a.Co = cout_all; a.Ci = d.cin; a.kh = d.kh; a.kw = d.kw; a.sh = d.sh; a.sw = d.sw;
     a.ph = d.ph; a.pw = d.pw; a.relu = d.relu; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y;
-    a.BN = p.BN; a.NB = p.NB; a.BK = p.BK; a.kchunks = d.cin / p.BK; a.stages = p.stages; a.MT = p.MT; a.nbuf = p.nbuf;
+    a.BN = p.BN; a.NB = p.NB; a.nb_off = grp * p.NB; a.BK = p.BK; a.kchunks = d.cin / p.BK; a.stages = p.stages; a.MT = p.MT; a.nbuf = p.nbuf;
     a.a_bytes = p.a_bytes; a.b_bytes = p.b_bytes; a.sbo = p.sbo; a.layout_type = p.layout_type;
     a.tmem_cols = tmem_cols_for(p.nbuf, p.MT, p.BN);
     // instruction descriptor: D = f32, A = B = bf16, both K-major, N = BN, M = 128
@@ -1448,10 +1487,12 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
 {
     dc_layer_rt& L = c->L[layer];
     TcPlan p;
-    if (c->cfg.dtype != DC_BF16 || !encode_fn() || getenv("DC_NO_TENSOR_CORES") || L.d.groups > 1) return DC_OK;
-    const dc_layer_desc de = pad16_ok(L.d) ? padded16(L.d) : L.d;
+    if (c->cfg.dtype != DC_BF16 || !encode_fn() || getenv("DC_NO_TENSOR_CORES")) return DC_OK;
+    const bool grouped = n_groups(L.d) > 1;
+    if (grouped && !dc_conv_bf16_supported(c, layer)) return DC_OK;
+    const dc_layer_desc de = grouped ? group_view(L.d) : (pad16_ok(L.d) ? padded16(L.d) : L.d);
     const bool generic = make_plan(de, p);
-    if (!generic && !smallc_ok(L.d)) return DC_OK;
+    if (!generic && (grouped || !smallc_ok(L.d))) return DC_OK;
     if (getenv("DC_CONV_NO_TUNE")) return DC_OK;
     const int tiles = L.tiles_x * L.tiles_y * c->S;
     cudaEvent_t e0, e1;
@@ -1492,7 +1533,7 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
         }
         const int default_bn = p.BN;
         for (int bn = default_bn; bn >= 64 && bn >= default_bn / 2; bn -= 32) {
-            if (L.d.cout % bn != 0) continue;
+            if (de.cout % bn != 0) continue;
             for (int mt = 1; mt <= 2; ++mt) {
                 TcPlan q;
                 if (!make_plan(de, q, mt, bn, ctas)) continue;
@@ -1501,10 +1542,10 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
             }
         }
         HaloPlan h0;
-        if (L.weight_halo && halo_ok(L.d, h0)) {
+        if (L.weight_halo && halo_ok(de, h0)) {
             for (int bn = h0.BN; bn >= 64 && bn >= h0.BN / 2; bn -= 32) {
                 HaloPlan h;
-                if (!halo_ok(L.d, h, bn)) continue;
+                if (!halo_ok(de, h, bn)) continue;
                 for (int mt = 1; mt <= 2; ++mt) {                      // tc_mt 3 / 4: patch-reuse kernel with 1 / 2 tiles per item
                     if (ctas == 2 && tmem_cols_for(mt * h.BN * 2 <= 512 ? 2 : 1, mt, h.BN) > 256) continue;
                     L.tc_bn = bn;

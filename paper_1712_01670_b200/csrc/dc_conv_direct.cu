@@ -159,6 +159,6 @@ int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_d
     else k_convert_weights<float><<<grid, 256, 0, c->stream>>>(w_dev, n, (float*)L.weight);
     DC_CUDA(cudaGetLastError());
     DC_CUDA(cudaMemcpyAsync(L.bias, b_dev, sizeof(float) * L.d.cout, cudaMemcpyDeviceToDevice, c->stream));
-    if (c->cfg.dtype == DC_BF16 && L.d.groups <= 1) return dc_pack_weights_bf16(c, layer);   // grouped: no tensor-core packing
+    if (c->cfg.dtype == DC_BF16) return dc_pack_weights_bf16(c, layer);
     return DC_OK;
 }

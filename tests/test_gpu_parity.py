@@ -463,7 +463,16 @@ def test_infer_workload_3_alexnet_bf16():
 def test_infer_alexnet_with_grouped_convolutions(dtype):
     """The AlexNet trunk with two channel groups in its second, fourth and fifth convolutions: every layer's
     rectangles, reuse ratios and maps against the oracle, cached frames included."""
-    U.run_stream_parity(configs.alexnet_stream(grouped=True, dtype=dtype), 1, list(range(4)))
+    w = configs.alexnet_stream(grouped=True, dtype=dtype)
+    U.run_stream_parity(w, 1, list(range(4)))
+    # in bfloat16 every convolution, the grouped ones included, runs on the tensor-core kernels (one launch per group)
+    dc = DeepCache.from_workload(w, n_streams=1)
+    try:
+        schemes = [B.dc_cache_layer_conv_scheme(dc.handle, i) for i, l in enumerate(w.layers) if l["kind"] == 0]
+        assert len(schemes) == 5 and any(l.get("groups", 1) > 1 for l in w.layers)
+        assert all(v >= 1 for v in schemes) if dtype == configs.DTYPE_BF16 else all(v == 0 for v in schemes)
+    finally:
+        dc.close()
 
 
 def test_infer_workload_4_resnet50_bf16():
