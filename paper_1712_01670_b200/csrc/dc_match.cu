@@ -736,8 +736,7 @@ struct TileReach {
 __global__ void __launch_bounds__(W_VS * 8 * 32, 3) k_search_dsw(MatchArgs a, uint4* long_list, int32_t* long_count)
 {
     constexpr int THREADS = W_VS * 8 * 32, GROUPS = W_COLS / 4;
-    constexpr int ROWS_PER_PASS = THREADS / GROUPS, PASSES = W_ROWS / ROWS_PER_PASS;      // 13 rows of 38 groups per pass
-    static_assert(W_ROWS % ROWS_PER_PASS == 0, "whole passes");
+    constexpr int ROWS_PER_PASS = THREADS / GROUPS, PASSES = (W_ROWS + ROWS_PER_PASS - 1) / ROWS_PER_PASS;
     __shared__ __align__(16) uint32_t win[W_ROWS * W_PITCH];
     __shared__ int32_t sums[3];
     const int strip = blockIdx.x, vg = blockIdx.y, s = blockIdx.z;        // grid: strips of 8 blocks x groups of W_VS block rows x streams
@@ -760,16 +759,17 @@ __global__ void __launch_bounds__(W_VS * 8 * 32, 3) k_search_dsw(MatchArgs a, ui
         uint32_t pa[PASSES], pb[PASSES], pc[PASSES];
 #pragma unroll
         for (int k = 0; k < PASSES; ++k) {                         // all loads first
-            const int gy = yb - W_WRY + row0 + k * ROWS_PER_PASS;
+            const int row = row0 + k * ROWS_PER_PASS, gy = yb - W_WRY + row;
             pa[k] = pb[k] = pc[k] = 0;
-            if (col_ok && gy >= 0 && gy < a.H) {
+            if (col_ok && row < W_ROWS && gy >= 0 && gy < a.H) {
                 const uint32_t* q = (const uint32_t*)(src + (size_t)gy * a.prev_pitch);
                 pa[k] = __ldg(q); pb[k] = __ldg(q + 1); pc[k] = __ldg(q + 2);
             }
         }
         if (row0 < ROWS_PER_PASS) {
 #pragma unroll
-            for (int k = 0; k < PASSES; ++k) store_pixels4(dst + k * ROWS_PER_PASS * W_PITCH, pa[k], pb[k], pc[k]);
+            for (int k = 0; k < PASSES; ++k)
+                if (row0 + k * ROWS_PER_PASS < W_ROWS) store_pixels4(dst + k * ROWS_PER_PASS * W_PITCH, pa[k], pb[k], pc[k]);
         }
     }
     __syncthreads();
