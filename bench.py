@@ -45,6 +45,7 @@ def parse_args():
     ap.add_argument("--skip-k", type=int, default=1, help="Step 2 on every k-th block row / column only (Section 4); default 1 = all blocks")
     ap.add_argument("--search", default="", choices=["", "exhaustive", "diamond", "three_step"],
                     help="Step 2 search unit; default: the workload's (diamond)")
+    ap.add_argument("--grouped", action="store_true", help="workload 3 with the cited AlexNet's two channel groups in layers 2, 4, 5")
     ap.add_argument("--cache-pool", action="store_true", help="also cache and reuse max-pooling outputs (Section 5's extension)")
     ap.add_argument("--per-block-regions", action="store_true", help="rectangles carry their blocks' own vectors (extension)")
     ap.add_argument("--no-lookahead", action="store_true", help="do not overlap the next frame's matching with this frame's inference")
@@ -585,6 +586,10 @@ def main():
     args = parse_args()
     from paper_1712_01670_b200.synth import configs
     w = configs.WORKLOADS[args.workload]()
+    if args.grouped:
+        if args.workload != 3:
+            raise SystemExit("--grouped applies to workload 3 (the AlexNet trunk)")
+        w = configs.alexnet_stream(grouped=True)
     if args.search:
         w.search = {"exhaustive": configs.SEARCH_ES, "diamond": configs.SEARCH_DS, "three_step": configs.SEARCH_TSS}[args.search]
     if args.impl == "reference":
