@@ -474,6 +474,7 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
     // the library's own aligned copy of the frame: matched now, the cache key of the next frame (Section 3)
     uint8_t* frame_copy = c->key[(c->key_cur + 1) % 3];
     const bool looked_ahead = c->la_frame == frame_dev && c->la_pitch == pitch && c->key_valid;
+    c->overlap_mode = looked_ahead;                   // a caller that looks ahead keeps doing so: see ring_budget()
     if (looked_ahead) {
         // dc_lookahead_frame already copied this frame in and (unless it is a full frame) matched it
         DC_CUDA(cudaStreamWaitEvent(c->stream, c->ev_match, 0));

@@ -86,6 +86,7 @@ struct dc_cache {
     cudaEvent_t ev_key, ev_match;   // main stream: frame copied in; side stream: lookahead finished
     const uint8_t* la_frame; size_t la_pitch; bool la_matched;
     bool last_refreshed;
+    bool overlap_mode;              // the last frame was looked ahead: the next one's matching will run beside this inference
     void* classify_table; int n_cached, classify_warps;   // all cached layers' classification in one launch (dc_regions.cu)
     size_t key_pitch;
     int num_sms;

@@ -994,7 +994,12 @@ static uint32_t tmem_cols_for(int nbuf, int mt, int bn)
     while (cols < need) cols <<= 1;
     return cols;
 }
-static int ring_budget(int ctas) { return 200 * 1024 / (ctas == 2 ? 2 : 1); }
+// Operand-ring bytes of a CTA that has its SM alone: 200 KB, or 182 KB while the cache's matcher runs beside the
+// inference (dc_lookahead_frame): with 182 KB a convolution CTA leaves room for one CTA of the block search (32 KB) on
+// its SM, which then works in the tensor-core kernel's idle issue slots instead of waiting for a free SM.  Set per
+// launch from the cache's state.
+static thread_local int t_ring_kb = 200;
+static int ring_budget(int ctas) { return t_ring_kb * 1024 / (ctas == 2 ? 2 : 1); }
 
 // Every launch waits at most kWaitLimitNs on the device.  dc_debug_stall_next_conv (below) arms the next launch
 // only: its producer issues no copy and its waits run out after the given time.
@@ -1389,6 +1394,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     const int G = n_groups(c->L[layer].d);
+    t_ring_kb = c->overlap_mode ? 182 : 200;
     for (int grp = 0; grp < G; ++grp) {                           // a grouped layer: one launch per group
         const int rc = launch_group(c, layer, grp, in, out, tile_list, tile_count, masks, max_tiles);
         if (rc != DC_OK) return rc;
