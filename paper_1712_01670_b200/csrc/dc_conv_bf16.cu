@@ -1396,7 +1396,11 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     const int G = n_groups(c->L[layer].d);
     t_ring_kb = c->overlap_mode ? 182 : 200;
     for (int grp = 0; grp < G; ++grp) {                           // a grouped layer: one launch per group
-        const int rc = launch_group(c, layer, grp, in, out, tile_list, tile_count, masks, max_tiles);
+        int rc = launch_group(c, layer, grp, in, out, tile_list, tile_count, masks, max_tiles);
+        if (rc == DC_ERR_CONFIG && t_ring_kb != 200) {            // the layer's tuned shape needs the full rings: it gets them
+            t_ring_kb = 200;
+            rc = launch_group(c, layer, grp, in, out, tile_list, tile_count, masks, max_tiles);
+        }
         if (rc != DC_OK) return rc;
     }
     return DC_OK;
