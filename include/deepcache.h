@@ -240,9 +240,10 @@ int dc_cache_layer_map(dc_cache* cache, int layer, void** map_dev, size_t* bytes
 int dc_cache_layer_regions(dc_cache* cache, int layer, dc_region** regions_dev, int32_t** n_dev);
 
 /* Which kernel family runs convolution layer `layer` (chosen at creation): -1 not an executable convolution,
- * 0 the CUDA-core kernel (fp32 caches, channel counts the tensor-core kernels cannot take), 1-7 a tensor-core
- * operand scheme (1, 2 tap by tap; 3, 4 input patch; 5, 6 column slabs; 7 column slabs on CTA pairs; grouped
- * layers run their scheme once per group).  For inspection and tests.  Errors: DC_ERR_ARG. */
+ * 0 the CUDA-core kernel (fp32 caches, channel counts the tensor-core kernels cannot take), 1-9 a tensor-core
+ * operand scheme (1, 2 tap by tap; 3, 4 input patch; 5, 6 column slabs; 7 column slabs on CTA pairs; 8, 9 tap by
+ * tap on tiles made of 16 row pieces of 8 pixels taken across rows and streams, for small maps; grouped layers
+ * run their scheme once per group).  For inspection and tests.  Errors: DC_ERR_ARG. */
 int dc_cache_layer_conv_scheme(const dc_cache* cache, int layer, int32_t* scheme);
 
 /* Waits for the stream and returns the device status word: DC_OK, or what a kernel recorded since the

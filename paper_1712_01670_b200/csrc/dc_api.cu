@@ -168,7 +168,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     DC_TRY(dev_alloc(c, &c->layers_dev, (size_t)n));
     DC_TRY(dev_alloc(c, &c->in_hw_dev, (size_t)n * 2));
     DC_TRY(dev_alloc(c, &c->dirty_count, (size_t)n));
-    DC_TRY(dev_alloc(c, &c->all_count, (size_t)n));
+    DC_TRY(dev_alloc(c, &c->all_count, (size_t)n * 2));
     DC_TRY(dev_alloc(c, &c->reuse_px, (size_t)n * S * 2));
     c->alive = c->reuse_px + (size_t)n * S;
     DC_TRY(dev_alloc(c, &c->status, (size_t)1));
@@ -199,7 +199,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
         DC_CUDA(cudaMemcpy(c->pix_lut, lut, sizeof(lut), cudaMemcpyHostToDevice));
     }
 
-    int32_t in_hw[DC_MAX_LAYERS * 2], all_count[DC_MAX_LAYERS];
+    int32_t in_hw[DC_MAX_LAYERS * 2], all_count[DC_MAX_LAYERS * 2];
     size_t max_tiles = 1;
     bool need_input_map = false;
     for (int i = 0; i < n; ++i) {
@@ -211,7 +211,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
         L.in_h = L.d.in0 < 0 ? cfg.height : layers[L.d.in0].out_h;
         L.in_w = L.d.in0 < 0 ? cfg.width : layers[L.d.in0].out_w;
         in_hw[2 * i] = L.in_h; in_hw[2 * i + 1] = L.in_w;
-        all_count[i] = 0;
+        all_count[i] = 0; all_count[n + i] = 0;
         if (!c->executable) continue;
         if (L.d.in0 < 0 && L.d.kind != DC_RESIZE_AREA) need_input_map = true;
         if ((L.d.kind == DC_ADD || L.d.kind == DC_CONCAT) && L.d.in1 < 0) need_input_map = true;
@@ -225,9 +225,11 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
         if (cached) {
             L.tiles_x = dc_div_up(L.d.out_w, DC_TILE_W);
             L.tiles_y = dc_div_up(L.d.out_h, DC_TILE_H);
-            size_t tiles = (size_t)L.tiles_x * L.tiles_y * S;
+            L.gpr = dc_div_up(L.d.out_w, DC_TILE_W);
+            L.tiles_flat = (int)(((size_t)S * L.d.out_h * L.gpr + DC_TILE_H - 1) / DC_TILE_H);
+            size_t tiles = (size_t)L.tiles_x * L.tiles_y * S;             // never fewer than the flat tiles
             if (tiles > max_tiles) max_tiles = tiles;
-            all_count[i] = (int32_t)tiles;
+            all_count[i] = (int32_t)tiles; all_count[n + i] = L.tiles_flat;
             DC_TRY(dev_alloc(c, &L.masks, tiles * 4));
             DC_TRY(dev_alloc(c, &L.dirty_list, tiles));
             DC_TRY(dev_alloc(c, &L.all_list, tiles));
@@ -244,13 +246,12 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
         }
     }
     DC_CUDA(cudaMemcpyAsync(c->in_hw_dev, in_hw, sizeof(int32_t) * 2 * n, cudaMemcpyHostToDevice, c->stream));
-    DC_CUDA(cudaMemcpyAsync(c->all_count, all_count, sizeof(int32_t) * n, cudaMemcpyHostToDevice, c->stream));
+    DC_CUDA(cudaMemcpyAsync(c->all_count, all_count, sizeof(int32_t) * 2 * n, cudaMemcpyHostToDevice, c->stream));
     DC_TRY(dev_alloc(c, &c->zero_masks, max_tiles * 4));
     DC_CUDA(cudaMemsetAsync(c->zero_masks, 0, max_tiles * 4 * sizeof(uint32_t), c->stream));
     if (need_input_map)
         DC_TRY(dev_alloc(c, (uint8_t**)&c->input_map, (size_t)S * cfg.height * cfg.width * 3 * c->elt));
     size_t stat_ints = (size_t)S * (3 + 4 + 1) + (size_t)n * S;
-    if (c->executable) DC_TRY(dc_build_classify_table(c));
     if (cudaMallocHost(&c->stats_pinned, stat_ints * sizeof(int32_t)) != cudaSuccess) { cudaGetLastError(); return DC_ERR_ALLOC; }
     DC_CUDA(cudaStreamSynchronize(c->stream));      // layers / in_hw / all_count live on this stack frame
     for (int i = 0; i < n; ++i)
@@ -258,6 +259,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
             const void* in = c->L[i].d.in0 < 0 ? c->input_map : c->L[c->L[i].d.in0].map[0];
             DC_TRY(dc_conv_bf16_autotune(c, i, in));
         }
+    if (c->executable) DC_TRY(dc_build_classify_table(c));       // after the tuner: it decides each layer's tile geometry
     DC_CUDA(cudaStreamSynchronize(c->stream));
     return DC_OK;
 }
@@ -453,7 +455,7 @@ int dc_conv_partial(dc_cache* c, int layer, const void* in_map_dev, const void* 
     if (!c || !in_map_dev || !out_map_dev || layer < 0 || layer >= c->n_layers) return DC_ERR_ARG;
     if (!c->executable || c->L[layer].d.kind != DC_CONV) return DC_ERR_CONFIG;
     dc_layer_rt& L = c->L[layer];
-    const int tiles = L.tiles_x * L.tiles_y * c->S;
+    const int tiles = dc_layer_tiles(c, L);
     if (regions_dev || n_regions_dev) {
         if (!regions_dev || !n_regions_dev || !prev_out_dev || prev_out_dev == out_map_dev) return DC_ERR_ARG;
         DC_CUDA(cudaMemsetAsync(c->dirty_count + layer, 0, sizeof(int32_t), c->stream));
@@ -461,7 +463,7 @@ int dc_conv_partial(dc_cache* c, int layer, const void* in_map_dev, const void* 
         DC_TRY(dc_launch_classify_copy(c, layer, regions_dev, n_regions_dev, prev_out_dev, out_map_dev));
         return dc_launch_conv(c, layer, in_map_dev, out_map_dev, L.dirty_list, c->dirty_count + layer, L.masks, tiles);
     }
-    return dc_launch_conv(c, layer, in_map_dev, out_map_dev, L.all_list, c->all_count + layer, c->zero_masks, tiles);
+    return dc_launch_conv(c, layer, in_map_dev, out_map_dev, L.all_list, dc_all_count(c, layer), c->zero_masks, tiles);
 }
 
 int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* out_map_dev, dc_frame_stats* stats)
@@ -507,13 +509,13 @@ int dc_infer_frame(dc_cache* c, const uint8_t* frame_dev, size_t pitch, void* ou
         const void* in = layer_input(c, L.d.in0);
         switch (L.d.kind) {
         case DC_CONV: {
-            const int tiles = L.tiles_x * L.tiles_y * S;
+            const int tiles = dc_layer_tiles(c, L);
             void* prev = L.map[L.cur]; void* out = L.map[L.cur ^ 1];
             if (!refresh) {
                 if (!classified) DC_TRY(dc_launch_classify_copy(c, i, c->table + per_layer * i, c->n_regions, prev, out));
                 DC_TRY(dc_launch_conv(c, i, in, out, L.dirty_list, c->dirty_count + i, L.masks, tiles));
             } else {
-                DC_TRY(dc_launch_conv(c, i, in, out, L.all_list, c->all_count + i, c->zero_masks, tiles));
+                DC_TRY(dc_launch_conv(c, i, in, out, L.all_list, dc_all_count(c, i), c->zero_masks, tiles));
             }
             L.cur ^= 1;          // the newest output is next frame's cached value
             break;
@@ -686,7 +688,7 @@ int dc_cache_layer_conv_scheme(const dc_cache* c, int layer, int32_t* scheme)
     const dc_layer_rt& L = c->L[layer];
     if (L.d.kind != DC_CONV || !c->executable) { *scheme = -1; return DC_OK; }
     if (!dc_conv_bf16_supported(c, layer)) { *scheme = 0; return DC_OK; }
-    *scheme = L.tc_mt > 0 ? L.tc_mt : 1;
+    *scheme = (L.tc_mt > 0 ? L.tc_mt : 1) + (L.flat ? 7 : 0);
     return DC_OK;
 }
 

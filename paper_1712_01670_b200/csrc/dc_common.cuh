@@ -37,7 +37,13 @@ struct dc_tm_slot {
 struct dc_layer_rt {
     dc_layer_desc d;
     int in_h, in_w;                 // size of the input map (or of the frame)
-    int tiles_x, tiles_y;           // conv only: output tiles per stream
+    int tiles_x, tiles_y;           // cached layers: 16 x 8 output tiles per stream
+    // Flat tiles (convolutions on small or narrow maps): a tile is 16 consecutive GROUPS of 8 pixels of one image row,
+    // groups numbered through rows, then streams: (stream * out_h + y) * gpr + column group.  A tile is then full
+    // whatever the map's height, and across streams; only a row's last group can hold fewer than 8 pixels.
+    int flat;                       // 1: this layer's tile list, bitmaps and convolution use flat tiles
+    int gpr;                        // groups per image row = ceil(out_w / 8)
+    int tiles_flat;                 // ceil(S * out_h * gpr / 16)
     void* map[2];                   // conv: current / cached output (ping-pong); others: map[0]
     int cur;                        // conv: which of map[] holds the newest output
     size_t map_bytes;               // bytes of one map, all streams
@@ -132,6 +138,10 @@ struct dc_prof_scope {
 };
 
 static inline int dc_div_up(int a, int b) { return (a + b - 1) / b; }
+// number of tiles of a cached layer in the tile geometry it uses
+static inline int dc_layer_tiles(const dc_cache* c, const dc_layer_rt& L) { return L.flat ? L.tiles_flat : L.tiles_x * L.tiles_y * c->S; }
+// device counter "all tiles" for full frames: [n_layers] for 16 x 8 tiles, then [n_layers] for flat tiles
+static inline const int32_t* dc_all_count(const dc_cache* c, int layer) { return c->all_count + (c->L[layer].flat ? c->n_layers : 0) + layer; }
 
 // A kernel's opt-in to more than 48 KB of dynamic shared memory (cudaFuncSetAttribute) holds for one device only.
 // One of these per call site remembers on which devices it has been made.  Two threads may both find it unset and

@@ -42,6 +42,9 @@ struct TcArgs {
     int32_t* status;
     unsigned long long wait_ns;   // limit of every device-side wait
     int skip_loads;               // failure-detection tests: the producer issues no copy, so the other roles' waits run out
+    // flat tiles (tap-by-tap kernel only): row i of tile t is group t * 16 + i, a group being 8 output pixels of one
+    // image row, numbered (stream * Ho + y) * gpr + column group; n_groups_all = S * Ho * gpr.  0: 16 x 8 blocks.
+    int flat = 0, gpr = 0, n_groups_all = 0;
 };
 
 struct SmemCtl {
@@ -205,10 +208,30 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
         for (int j = 0; j < a.MT; ++j) {
             const int tile = j == 0 ? tile_c0 : tile_c1;
             if (tile < 0) break;
-            const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
-            const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
             const bool reused = ((j == 0 ? mask_c0 : mask_c1) >> mbit) & 1u;
-            const bool active = oy < a.Ho && ox < a.Wo && !reused;
+            bool active;
+            // write-back addressing, once per tile: piece k of this lane is the 16-byte part (lane & 3) of the pixel in
+            // tile row q * 4 + k, column lane >> 2 (the warp's 32 pixels are 4 tile rows of 8)
+            const size_t row_stride = (size_t)a.Wo * a.Co;
+            const size_t ch_off = (size_t)(nb + a.nb_off) * a.BN + (lane & 3) * 8;
+            size_t wb_off[4];                                   // element offset of piece k's pixel
+            if (a.flat) {
+                const int gps = a.Ho * a.gpr;
+                const int g = tile * DC_TILE_H + prow, s = g / gps, loc = g - s * gps, y = loc / a.gpr, gx = loc - y * a.gpr;
+                active = g < a.n_groups_all && gx * DC_TILE_W + pcol < a.Wo && !reused;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                    const int gk = tile * DC_TILE_H + q * 4 + k, sk = gk / gps, lk = gk - sk * gps, yk = lk / a.gpr, xk = lk - yk * a.gpr;
+                    wb_off[k] = (((size_t)sk * a.Ho + yk) * a.Wo + xk * DC_TILE_W + (lane >> 2)) * a.Co + ch_off;
+                }
+            } else {
+                const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+                const int oy = ty * DC_TILE_H + prow, ox = tx * DC_TILE_W + pcol;
+                active = oy < a.Ho && ox < a.Wo && !reused;
+#pragma unroll
+                for (int k = 0; k < 4; ++k)
+                    wb_off[k] = ((size_t)s * a.Ho + ty * DC_TILE_H + q * 4 + k) * row_stride + (size_t)(tx * DC_TILE_W + (lane >> 2)) * a.Co + ch_off;
+            }
             const uint32_t taddr = tmem_base + ((uint32_t)(q * 32) << 16) + (acc * (uint32_t)a.MT + (uint32_t)j) * (uint32_t)a.BN;
             // Each lane owns one pixel (TMEM lane) and gets 32 channels = 64 bytes per step.  Storing them
             // directly would make every warp store touch 32 different lines 16 bytes at a time (half-written
@@ -216,11 +239,6 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
             // 4 lanes per pixel, so each pixel's 64 bytes leave as two whole sectors.
             const unsigned act_mask = __ballot_sync(0xffffffffu, active);
             uint8_t* stg = ctl->stage[q];
-            // write-back addressing, once per tile: piece k of this lane is the 16-byte part (lane & 3) of the pixel in
-            // tile row q * 4 + k, column lane >> 2 (the warp's 32 pixels are 4 tile rows of 8)
-            const size_t row_stride = (size_t)a.Wo * a.Co;
-            __nv_bfloat16* const wb = a.out + ((size_t)s * a.Ho + ty * DC_TILE_H + q * 4) * row_stride +
-                                      (size_t)(tx * DC_TILE_W + (lane >> 2)) * a.Co + (nb + a.nb_off) * a.BN + (lane & 3) * 8;
             const uint8_t* const rd = stg + (lane >> 2) * 80 + (lane & 3) * 16;
             for (int c = 0; c < a.BN / 32; ++c) {
                 uint32_t r[32];
@@ -245,7 +263,7 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     if ((act_mask >> ((lane >> 2) + 8 * k)) & 1u)
-                        *(uint4*)(wb + k * row_stride + c * 32) = *(const uint4*)(rd + k * (8 * 80));
+                        *(uint4*)(a.out + wb_off[k] + c * 32) = *(const uint4*)(rd + k * (8 * 80));
                 }
                 __syncwarp();
             }
@@ -299,12 +317,27 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         for (int item = blockIdx.x; item < n_items && ok; item += gridDim.x) {
             const int group = item / a.NB, nb = item % a.NB;
             int sN[MT], xb[MT], yb[MT];
+            // flat tiles: lane l fetches group (l & 15) of tile (l >> 4), one box of 8 pixels per tap and chunk
+            int fs = 0, fx = 0, fy = 0; bool fon = false; uint32_t flat_tx = 0;
+            if (a.flat) {
+                const int j = lane >> 4, idx = group * MT + j;
+                if (j < MT) {
+                    const int tile = a.tile_list[idx < n_tiles ? idx : group * MT];
+                    const int gps = a.Ho * a.gpr, g = tile * DC_TILE_H + (lane & 15);
+                    fon = g < a.n_groups_all;                   // the last tile may have fewer groups: their rows stay as they are (never stored)
+                    fs = g / gps;
+                    const int loc = g - fs * gps, y = loc / a.gpr;
+                    fx = (loc - y * a.gpr) * DC_TILE_W * a.sw - a.pw; fy = y * a.sh - a.ph;
+                }
+                flat_tx = (uint32_t)__popc(__ballot_sync(0xffffffffu, fon)) * (uint32_t)(a.a_bytes / DC_TILE_H) + (uint32_t)a.b_bytes;
+            } else {
 #pragma unroll
-            for (int j = 0; j < MT; ++j) {                      // an absent second tile repeats the first (never stored)
-                const int idx = group * MT + j;
-                const int tile = a.tile_list[idx < n_tiles ? idx : group * MT];
-                const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
-                sN[j] = s; xb[j] = tx * DC_TILE_W * a.sw - a.pw; yb[j] = ty * DC_TILE_H * a.sh - a.ph;
+                for (int j = 0; j < MT; ++j) {                      // an absent second tile repeats the first (never stored)
+                    const int idx = group * MT + j;
+                    const int tile = a.tile_list[idx < n_tiles ? idx : group * MT];
+                    const int s = tile / per_stream, t = tile - s * per_stream, ty = t / a.tiles_x, tx = t - ty * a.tiles_x;
+                    sN[j] = s; xb[j] = tx * DC_TILE_W * a.sw - a.pw; yb[j] = ty * DC_TILE_H * a.sh - a.ph;
+                }
             }
             for (int tap = 0; tap < taps && ok; ++tap) {
                 const int ky = tap / a.kw, kx = tap - ky * a.kw;
@@ -313,14 +346,20 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
                         ok = mbar_wait(&ctl->empty[st], ph ^ 1u, ctl, a.status);
                         if (ok && !a.skip_loads) {
                             uint8_t* sa = ring + (size_t)st * stage_bytes;
-                            mbar_expect_tx(&ctl->full[st], (uint32_t)stage_bytes);
+                            mbar_expect_tx(&ctl->full[st], a.flat ? flat_tx : (uint32_t)stage_bytes);
+                            if (!a.flat) {
 #pragma unroll
-                            for (int j = 0; j < MT; ++j)
-                                tma_load_4d(sa + j * a.a_bytes, &tmA, cc * a.BK, xb[j] + kx, yb[j] + ky, sN[j], &ctl->full[st]);
+                                for (int j = 0; j < MT; ++j)
+                                    tma_load_4d(sa + j * a.a_bytes, &tmA, cc * a.BK, xb[j] + kx, yb[j] + ky, sN[j], &ctl->full[st]);
+                            }
                             tma_load_2d(sa + MT * a.a_bytes, &tmB, tap * a.Ci + cc * a.BK, (nb + a.nb_off) * a.BN, &ctl->full[st]);
                         }
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
+                    // the slot is free and its byte count announced (lane 0, above): every lane brings its own group
+                    if (a.flat && ok && !a.skip_loads && fon)
+                        tma_load_4d(ring + (size_t)st * stage_bytes + (size_t)lane * (a.a_bytes / DC_TILE_H), &tmA, cc * a.BK, fx + kx, fy + ky, fs,
+                                    &ctl->full[st]);
                     if (++st == a.stages) { st = 0; ph ^= 1u; }
                 }
             }
@@ -1410,6 +1449,7 @@ static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* o
                         const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
+    if (L.flat && L.tc_mt > 2) return DC_ERR_CONFIG;              // flat tiles exist in the tap-by-tap kernel only
     if (L.tc_mt == 7) return launch_pair(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
     if (L.tc_mt >= 5) return launch_halo(c, layer, grp, L.tc_mt - 4, true, in, out, tile_list, tile_count, masks, max_tiles);
     if (L.tc_mt >= 3) return launch_halo(c, layer, grp, L.tc_mt - 2, false, in, out, tile_list, tile_count, masks, max_tiles);
@@ -1437,15 +1477,16 @@ static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* o
     EncodeTiledFn enc = encode_fn();
     if (!enc) return DC_ERR_CUDA;
     bool hit_a, hit_b;
-    CUtensorMap* tmAp = tm_find(L.tm_a, 4, &L.tm_next, in, 1, 0, &hit_a);
+    CUtensorMap* tmAp = tm_find(L.tm_a, 4, &L.tm_next, in, L.flat ? 8 : 1, 0, &hit_a);
     CUtensorMap* tmBp = tm_find(&L.tm_b, 1, nullptr, weights, 1, p.BN, &hit_b);
     if (!hit_a) {   // input map [S][Hi][Wi][Ci] bf16; box = BK channels x 16 columns x 8 rows x 1 stream
         cuuint64_t dims[4] = {(cuuint64_t)d.cin, (cuuint64_t)L.in_w, (cuuint64_t)L.in_h, (cuuint64_t)c->S};
         cuuint64_t strides[3] = {(cuuint64_t)cin_all * 2, (cuuint64_t)L.in_w * cin_all * 2, (cuuint64_t)L.in_h * L.in_w * cin_all * 2};
         // a strided convolution reads every sw-th column / sh-th row: the box spans TW * sw x TH * sh input
         // pixels and the traversal strides pick TW x TH of them
-        cuuint32_t box[4] = {(cuuint32_t)p.BK, (cuuint32_t)(DC_TILE_W * d.sw), (cuuint32_t)(DC_TILE_H * d.sh), 1};
-        cuuint32_t estr[4] = {1, (cuuint32_t)d.sw, (cuuint32_t)d.sh, 1};
+        // (flat tiles: one image row of 8 pixels per box)
+        cuuint32_t box[4] = {(cuuint32_t)p.BK, (cuuint32_t)(DC_TILE_W * d.sw), (cuuint32_t)(L.flat ? 1 : DC_TILE_H * d.sh), 1};
+        cuuint32_t estr[4] = {1, (cuuint32_t)d.sw, (cuuint32_t)(L.flat ? 1 : d.sh), 1};
         if (enc(tmAp, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(in), dims, strides, box, estr,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, p.swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) { tm_drop(L.tm_a, 4, tmAp); tm_drop(&L.tm_b, 1, tmBp); return DC_ERR_CUDA; }
@@ -1472,6 +1513,7 @@ static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* o
     // instruction descriptor: D = f32, A = B = bf16, both K-major, N = BN, M = 128
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
+    a.flat = L.flat; a.gpr = L.gpr; a.n_groups_all = c->S * d.out_h * L.gpr;
     set_wait_limit(c, a);
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device)) {
@@ -1504,35 +1546,34 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
     const bool generic = make_plan(de, p);
     if (!generic && (grouped || !smallc_ok(L.d))) return DC_OK;
     if (getenv("DC_CONV_NO_TUNE")) return DC_OK;
-    const int tiles = L.tiles_x * L.tiles_y * c->S;
     cudaEvent_t e0, e1;
     DC_CUDA(cudaEventCreate(&e0));
     DC_CUDA(cudaEventCreate(&e1));
-    float best = 1e30f; int best_mt = L.tc_mt, best_bn = L.tc_bn, best_ctas = 1;
+    float best = 1e30f; int best_mt = L.tc_mt, best_bn = L.tc_bn, best_ctas = 1, best_flat = 0;
     constexpr int kTuneReps = 6;                                      // timed launches per candidate, after one untimed
     // the GPU may have been idle: bring the clocks up before the first candidate is timed
     for (int rep = 0; rep < 12; ++rep)
-        if (dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles) != DC_OK) break;
+        if (dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, dc_all_count(c, layer), c->zero_masks, dc_layer_tiles(c, L)) != DC_OK) break;
     const bool verbose = getenv("DC_VERBOSE") != nullptr;
     // times the launch the current L.tc_* fields select; keeps it when it is the fastest so far
     // DC_CONV_SCHEME=<code> (diagnostics, tests): only candidates of that operand scheme are timed, so the scheme runs
     // wherever it can (1, 2 tap by tap; 3, 4 patch; 5, 6 column slabs; the second of each pair with two tiles per item;
-    // 7 column slabs on CTA pairs)
+    // 7 column slabs on CTA pairs; 8, 9 tap by tap on flat tiles)
     const int only = getenv("DC_CONV_SCHEME") ? atoi(getenv("DC_CONV_SCHEME")) : 0;
     auto trial = [&](const char* what) {
-        if (only > 0 && generic && L.tc_mt != only) return;
+        if (only > 0 && generic && (L.flat ? L.tc_mt + 7 : L.tc_mt) != only) return;
         int rc = DC_OK;
         for (int rep = 0; rep < kTuneReps + 1 && rc == DC_OK; ++rep) {
             if (rep == 1) cudaEventRecord(e0, c->stream);
-            rc = dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, c->all_count + layer, c->zero_masks, tiles);
+            rc = dc_launch_conv_bf16(c, layer, in, L.map[0], L.all_list, dc_all_count(c, layer), c->zero_masks, dc_layer_tiles(c, L));
         }
         cudaEventRecord(e1, c->stream);
         if (rc != DC_OK || cudaEventSynchronize(e1) != cudaSuccess) { cudaGetLastError(); return; }
         float ms = 0.f;
         cudaEventElapsedTime(&ms, e0, e1);
         if (verbose) fprintf(stderr, "libdeepcache: layer %d: %s, tiles/item code %d, %d channels per block, %d CTA(s) per SM: %.3f ms\n",
-                             layer, what, L.tc_mt, L.tc_bn, L.tc_ctas, ms / kTuneReps);
-        if (ms < best) { best = ms; best_mt = L.tc_mt; best_bn = L.tc_bn; best_ctas = L.tc_ctas; }
+                             layer, what, L.flat ? L.tc_mt + 7 : L.tc_mt, L.tc_bn, L.tc_ctas, ms / kTuneReps);
+        if (ms < best) { best = ms; best_mt = L.tc_mt; best_bn = L.tc_bn; best_ctas = L.tc_ctas; best_flat = L.flat; }
     };
     for (int ctas = 1; ctas <= 2; ++ctas) {
         L.tc_ctas = ctas;
@@ -1549,6 +1590,12 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
                 if (!make_plan(de, q, mt, bn, ctas)) continue;
                 L.tc_mt = mt; L.tc_bn = bn;
                 trial("tap-by-tap kernel");
+                // flat tiles where the 16 x 8 blocks leave a good part of their pixels outside the map
+                if (L.tiles_flat * 20 <= L.tiles_x * L.tiles_y * c->S * 19 || only >= 8) {
+                    L.flat = 1;
+                    trial("tap-by-tap kernel, flat tiles");
+                    L.flat = 0;
+                }
             }
         }
         HaloPlan h0;
@@ -1573,11 +1620,11 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
             trial("CTA-pair kernel");
         }
     }
-    L.tc_mt = best_mt; L.tc_bn = best_bn; L.tc_ctas = best_ctas;
+    L.tc_mt = best_mt; L.tc_bn = best_bn; L.tc_ctas = best_ctas; L.flat = best_flat;
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     c->launches = 0;
     if (verbose) fprintf(stderr, "libdeepcache: layer %d: chose code %d, %d channels per block, %d CTA(s) per SM (%.3f ms)\n",
-                         layer, best_mt, best_bn, best_ctas, best / kTuneReps);
+                         layer, best_flat ? best_mt + 7 : best_mt, best_bn, best_ctas, best / kTuneReps);
     return DC_OK;
 }
 

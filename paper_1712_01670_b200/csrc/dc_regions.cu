@@ -166,6 +166,7 @@ struct ClassifyArgs {
     const uint8_t* prev; uint8_t* out;           // maps as bytes
     int Ho, Wo, px_bytes;                        // px_bytes = cout * element size (multiple of 16)
     int tiles_x, tiles_y, S;
+    int gpr, n_tiles;                            // gpr > 0: flat tiles of 16 groups of 8 pixels, gpr groups per image row; n_tiles: tiles in all
     uint32_t* masks; int32_t* dirty_list; int32_t* dirty_count; int32_t* reuse_px;
     const int32_t* alive;                        // per stream: rectangles alive at this layer, or NULL (unknown)
     unsigned long long* reused_total;
@@ -266,6 +267,113 @@ __device__ __forceinline__ void classify_tile(const ClassifyArgs& a, const int t
     }
 }
 
+
+// The same for a layer with flat tiles: row i of the tile's bitmap is group tile * 16 + i, a group being 8 pixels of
+// one image row, numbered (stream * Ho + y) * gpr + column group.  A tile may hold groups of several streams (small
+// maps); each stream's rectangles are tested against that stream's groups only.
+__device__ __forceinline__ void classify_tile_flat(const ClassifyArgs& a, const int tile, const int lane, CopyLane& cl)
+{
+    const int gps = a.Ho * a.gpr;                                  // groups per stream
+    const int G0 = tile * DC_TILE_H, G1 = min(G0 + DC_TILE_H, a.S * gps);
+    uint32_t m0 = 0, m1 = 0, m2 = 0, m3 = 0;
+    int in_tile;
+    {   // pixels of the tile that exist: a row's last group may be cut by the map's width
+        const int g = G0 + lane, loc = g % gps, gx = loc % a.gpr;
+        in_tile = __reduce_add_sync(0xffffffffu, (lane < DC_TILE_H && g < G1) ? min(DC_TILE_W, a.Wo - gx * DC_TILE_W) : 0);
+    }
+    const int segs_max = (DC_TILE_W * a.px_bytes + kSeg - 1) / kSeg;   // segments of a whole group's pixels
+    for (int s = G0 / gps; s * gps < G1; ++s) {
+        const int g_lo = max(G0, s * gps), g_hi = min(G1, (s + 1) * gps);     // this stream's groups in the tile
+        const int loc0 = g_lo - s * gps, y_first = loc0 / a.gpr, gx_first = loc0 - y_first * a.gpr;
+        const dc_region* regs = a.regions + (size_t)s * a.max_regions;
+        const int n = (a.alive && a.alive[s] == 0) ? 0 : min(a.n_regions[s], a.max_regions);
+        const size_t map_base = (size_t)s * a.Ho * a.Wo * a.px_bytes;
+        uint32_t s0 = 0, s1 = 0, s2 = 0, s3 = 0;                  // this stream's part of the bitmap
+        for (int base = 0; base < n; base += 32) {
+            const int i = base + lane;
+            dc_region r = empty_region();
+            uint32_t hit16 = 0;                                   // rows of the tile that the rectangle touches
+            if (i < n) {
+                r = regs[i];
+                const bool inside = r.x >= 0 && r.y >= 0 && r.sx >= 0 && r.sy >= 0 && r.w <= a.Wo && r.h <= a.Ho &&
+                                    r.x <= a.Wo - r.w && r.y <= a.Ho - r.h && r.sx <= a.Wo - r.w && r.sy <= a.Ho - r.h;
+                if (r.w <= 0 || r.h <= 0) r = empty_region();
+                else if (!inside) {                               // see classify_tile
+                    if (loc0 == 0 && a.status) atomicExch(a.status, (int)DC_ERR_ARG);
+                    r = empty_region();
+                }
+                if (r.w > 0) {
+                    int y = y_first, gx = gx_first;
+                    for (int g = g_lo; g < g_hi; ++g) {
+                        const int x0 = gx * DC_TILE_W;
+                        const int cx0 = max(r.x, x0), cx1 = min(r.x + r.w, min(x0 + DC_TILE_W, a.Wo));
+                        if (y >= r.y && y < r.y + r.h && cx1 > cx0) {
+                            const int row = g - G0;
+                            const uint32_t v = (((1u << (cx1 - x0)) - 1u) & ~((1u << (cx0 - x0)) - 1u)) << ((row & 3) * DC_TILE_W);
+                            switch (row >> 2) { case 0: s0 |= v; break; case 1: s1 |= v; break; case 2: s2 |= v; break; default: s3 |= v; }
+                            hit16 |= 1u << row;
+                        }
+                        if (++gx == a.gpr) { gx = 0; ++y; }
+                    }
+                }
+            }
+            // the warp copies every touched row's span together (Section 5 "Reuse", step 1): per round one segment per lane
+            unsigned hits = __ballot_sync(0xffffffffu, hit16 != 0);
+            while (hits) {
+                const int src_lane = __ffs(hits) - 1; hits &= hits - 1;
+                const int rx = __shfl_sync(0xffffffffu, r.x, src_lane), ry = __shfl_sync(0xffffffffu, r.y, src_lane);
+                const int rw = __shfl_sync(0xffffffffu, r.w, src_lane);
+                const int rsx = __shfl_sync(0xffffffffu, r.sx, src_lane), rsy = __shfl_sync(0xffffffffu, r.sy, src_lane);
+                const uint32_t h16 = __shfl_sync(0xffffffffu, hit16, src_lane);
+                for (int i0 = 0; i0 < DC_TILE_H * segs_max && !cl.dead; i0 += 32) {
+                    const int it = i0 + lane, row = it / segs_max, sg = it - row * segs_max;
+                    uint32_t bytes = 0;
+                    size_t src_off = 0, dst_off = 0;
+                    if (row < DC_TILE_H && ((h16 >> row) & 1u)) {
+                        const int loc = G0 + row - s * gps, y = loc / a.gpr, x0 = (loc - y * a.gpr) * DC_TILE_W;
+                        const int cx0 = max(rx, x0), cx1 = min(rx + rw, min(x0 + DC_TILE_W, a.Wo));
+                        const int span = (cx1 - cx0) * a.px_bytes - sg * kSeg;
+                        if (span > 0) {
+                            bytes = (uint32_t)min(kSeg, span);
+                            src_off = ((size_t)(y - ry + rsy) * a.Wo + (cx0 - rx + rsx)) * a.px_bytes + (size_t)sg * kSeg;
+                            dst_off = ((size_t)y * a.Wo + cx0) * a.px_bytes + (size_t)sg * kSeg;
+                        }
+                    }
+                    const uint32_t total = __reduce_add_sync(0xffffffffu, bytes);
+                    if (total == 0) continue;                     // the same in all lanes
+                    if (lane == 0) rs_expect(cl.bar, total);
+                    __syncwarp();
+                    if (bytes) rs_load(cl.stage + lane * kSeg, a.prev + map_base + src_off, bytes, cl.bar);
+                    const bool landed = rs_wait(cl.bar, cl.phase);
+                    if (!__all_sync(0xffffffffu, landed)) {
+                        if (lane == 0 && a.status) atomicExch(a.status, (int)DC_ERR_TIMEOUT);
+                        cl.dead = true;
+                        break;
+                    }
+                    cl.phase ^= 1u;
+                    if (bytes) rs_store(a.out + map_base + dst_off, cl.stage + lane * kSeg, bytes);
+                    rs_commit();
+                    rs_wait_read();
+                    __syncwarp();
+                }
+            }
+        }
+        s0 = __reduce_or_sync(0xffffffffu, s0); s1 = __reduce_or_sync(0xffffffffu, s1);
+        s2 = __reduce_or_sync(0xffffffffu, s2); s3 = __reduce_or_sync(0xffffffffu, s3);
+        const int covered_s = __popc(s0) + __popc(s1) + __popc(s2) + __popc(s3);
+        if (lane == 0 && covered_s) { atomicAdd(&a.reuse_px[s], covered_s); atomicAdd(a.reused_total, (unsigned long long)covered_s); }
+        m0 |= s0; m1 |= s1; m2 |= s2; m3 |= s3;
+    }
+    if (lane == 0) {
+        uint32_t* mk = a.masks + (size_t)tile * 4;
+        mk[0] = m0; mk[1] = m1; mk[2] = m2; mk[3] = m3;
+        if (__popc(m0) + __popc(m1) + __popc(m2) + __popc(m3) < in_tile) {
+            const int slot = atomicAdd(a.dirty_count, 1);
+            a.dirty_list[slot] = tile;
+        }
+    }
+}
+
 // Staging and barrier of this warp, carved from the CTA's dynamic shared memory.
 __device__ __forceinline__ CopyLane copy_lane_setup(uint8_t* smem_raw)
 {
@@ -285,7 +393,10 @@ __global__ void __launch_bounds__(kCopyWarps * 32) k_classify_copy(ClassifyArgs 
     extern __shared__ uint8_t copy_smem[];
     CopyLane cl = copy_lane_setup(copy_smem);
     const int tile = blockIdx.x * kCopyWarps + (threadIdx.x >> 5);
-    if (tile < a.tiles_x * a.tiles_y * a.S) classify_tile(a, tile, threadIdx.x & 31, cl);
+    if (tile < a.n_tiles) {
+        if (a.gpr > 0) classify_tile_flat(a, tile, threadIdx.x & 31, cl);
+        else classify_tile(a, tile, threadIdx.x & 31, cl);
+    }
     rs_wait_all();
 }
 
@@ -294,7 +405,7 @@ __global__ void __launch_bounds__(kCopyWarps * 32) k_classify_copy(ClassifyArgs 
 // Warps are numbered through all layers' tiles; first_warp is the running sum.
 struct ClassifyLayer {
     const dc_region* regions; uint8_t* map[2];
-    int Ho, Wo, px_bytes, tiles_x, tiles_y, first_warp;
+    int Ho, Wo, px_bytes, tiles_x, tiles_y, first_warp, gpr;
     uint32_t* masks; int32_t* dirty_list; int32_t* dirty_count; int32_t* reuse_px;
     const int32_t* alive; unsigned long long* reused_total; int32_t* status;
 };
@@ -316,9 +427,11 @@ __global__ void __launch_bounds__(kCopyWarps * 32) k_classify_copy_all(const Cla
     a.regions = L.regions; a.n_regions = n_regions; a.max_regions = max_regions;
     a.prev = L.map[cur]; a.out = L.map[cur ^ 1];
     a.Ho = L.Ho; a.Wo = L.Wo; a.px_bytes = L.px_bytes; a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y; a.S = S;
+    a.gpr = L.gpr; a.n_tiles = 0;
     a.masks = L.masks; a.dirty_list = L.dirty_list; a.dirty_count = L.dirty_count; a.reuse_px = L.reuse_px;
     a.alive = L.alive; a.reused_total = L.reused_total; a.status = L.status;
-    classify_tile(a, w - L.first_warp, threadIdx.x & 31, cl);
+    if (a.gpr > 0) classify_tile_flat(a, w - L.first_warp, threadIdx.x & 31, cl);
+    else classify_tile(a, w - L.first_warp, threadIdx.x & 31, cl);
     rs_wait_all();
 }
 
@@ -339,11 +452,12 @@ int dc_build_classify_table(dc_cache* c)
         e.map[0] = (uint8_t*)L.map[0]; e.map[1] = (uint8_t*)L.map[1];
         e.Ho = L.d.out_h; e.Wo = L.d.out_w; e.px_bytes = L.d.cout * c->elt;
         e.tiles_x = L.tiles_x; e.tiles_y = L.tiles_y; e.first_warp = warps;
+        e.gpr = L.flat ? L.gpr : 0;
         e.masks = L.masks; e.dirty_list = L.dirty_list; e.dirty_count = c->dirty_count + i;
         e.reuse_px = c->reuse_px + (size_t)i * c->S; e.alive = c->alive + (size_t)i * c->S;
         e.reused_total = c->reused_total + i;
         e.status = c->status;
-        warps += L.tiles_x * L.tiles_y * c->S;
+        warps += dc_layer_tiles(c, L);
     }
     c->n_cached = k; c->classify_warps = warps;
     int rc = DC_OK;
@@ -396,13 +510,14 @@ int dc_launch_classify_copy(dc_cache* c, int layer, const dc_region* regions, co
     a.prev = (const uint8_t*)prev_out; a.out = (uint8_t*)out;
     a.Ho = L.d.out_h; a.Wo = L.d.out_w; a.px_bytes = L.d.cout * c->elt;
     a.tiles_x = L.tiles_x; a.tiles_y = L.tiles_y; a.S = c->S;
+    a.gpr = L.flat ? L.gpr : 0; a.n_tiles = dc_layer_tiles(c, L);
     a.masks = L.masks; a.dirty_list = L.dirty_list; a.dirty_count = c->dirty_count + layer;
     a.reuse_px = c->reuse_px + (size_t)layer * c->S;
     a.reused_total = c->reused_total + layer;
     a.status = c->status;
     a.alive = (regions == c->table + (size_t)layer * c->S * c->max_regions) ? c->alive + (size_t)layer * c->S : nullptr;
     // the caller has zeroed dirty_count[layer] and reuse_px[layer][*] on the stream
-    int tiles = L.tiles_x * L.tiles_y * c->S;
+    int tiles = dc_layer_tiles(c, L);
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device))
         DC_CUDA(cudaFuncSetAttribute(k_classify_copy, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kCopySmem));

@@ -426,10 +426,10 @@ def test_conv_partial_ignores_rectangles_outside_the_map():
         dc.close()
 
 
-@pytest.mark.parametrize("scheme", [1, 2, 3, 4, 5, 6, 7])
+@pytest.mark.parametrize("scheme", [1, 2, 3, 4, 5, 6, 7, 8, 9])
 def test_conv_schemes_forced(scheme, monkeypatch):
     """Every operand scheme of the tensor-core convolution (tap by tap, patch, column slabs; one or two tiles per
-    item; column slabs on CTA pairs) on layers it can take: VGG-shaped 3x3 layers, a 5x5 layer and odd map sizes,
+    item; column slabs on CTA pairs; tap by tap on flat tiles) on layers it can take: VGG-shaped 3x3 layers, a 5x5 layer and odd map sizes,
     through cached frames."""
     monkeypatch.setenv("DC_CONV_SCHEME", str(scheme))
     b = nets.NetBuilder(45, 53)
@@ -593,11 +593,30 @@ def test_conv_wide_layers_on_cta_pairs(scheme, hi, wi, cin, cout, k, p, monkeypa
     """The wide layers (128 - 512 output channels) forced onto the CTA-pair kernel (7), and onto the single-CTA column-slab
     kernel (5) for comparison: full convolution and partial convolution with an odd number of dirty tiles."""
     monkeypatch.setenv("DC_CONV_SCHEME", str(scheme))
+    _one_layer_full_and_partial(hi, wi, cin, cout, k, 1, p, 3, scheme)
+
+
+@pytest.mark.parametrize("scheme", [8, 9])
+@pytest.mark.parametrize("hi,wi,cin,cout,k,st,p,S", [
+    (7, 7, 128, 256, 3, 1, 1, 5),        # 7 pieces per stream: every tile holds pieces of two or three streams
+    (14, 14, 256, 512, 3, 1, 1, 3),      # two pieces per row
+    (13, 13, 64, 96, 3, 1, 1, 4),        # a cut last piece in every row; 32-channel blocks
+    (27, 27, 32, 64, 5, 2, 2, 3),        # a strided layer (14 x 14 output), 64-byte operand rows
+    (9, 40, 128, 256, 1, 1, 0, 3),       # 1 x 1
+    (3, 5, 64, 64, 3, 1, 1, 1),          # one tile, mostly absent
+])
+def test_conv_flat_tiles_across_rows_and_streams(scheme, hi, wi, cin, cout, k, st, p, S, monkeypatch):
+    """Small maps on tiles made of 16 row pieces of 8 pixels that run on across rows and streams (scheme 8; 9 with two
+    tiles per item): the reuse bitmap, the dirty list and the copies then follow that numbering too."""
+    monkeypatch.setenv("DC_CONV_SCHEME", str(scheme))
+    _one_layer_full_and_partial(hi, wi, cin, cout, k, st, p, S, scheme)
+
+
+def _one_layer_full_and_partial(hi, wi, cin, cout, k, st, p, S, scheme):
     g = rng(hi * 7 + cout)
-    S = 3
     nb = nets.NetBuilder(hi, wi)
     a = nb.conv(-1, cin, 1, 1, 0)
-    nb.conv(a, cout, k, 1, p, 1)
+    nb.conv(a, cout, k, st, p, 1)
     L = nb.layers[1]
     wts = g.normal(0, np.sqrt(2.0 / (k * k * cin)), size=(cout, k, k, cin)).astype(np.float32)
     bias = g.normal(0, 0.1, size=cout).astype(np.float32)
@@ -607,15 +626,21 @@ def test_conv_wide_layers_on_cta_pairs(scheme, hi, wi, cin, cout, k, p, monkeypa
     pq = np.stack([orc.quant_array(g.normal(size=(L["out_h"], L["out_w"], cout)), orc.QUANT_BF16) for _ in range(S)])
     dc = DeepCache(wi, hi, nb.layers, ws, bs, n_streams=S, block=16, search_range=4, dtype=B.DC_BF16, max_regions=4)
     try:
+        if scheme >= 8:
+            assert B.dc_cache_layer_conv_scheme(dc.handle, 1) == scheme
         xin = torch.from_numpy(xq).to(torch.bfloat16).cuda()
         pin = torch.from_numpy(pq).to(torch.bfloat16).cuda()
         full = dc.conv_partial(1, xin)
         # one rectangle that covers the whole map of stream 1 (its tiles are clean: the dirty count becomes odd for
         # most shapes) and a small one in stream 0
         regs = torch.zeros((S, dc.max_regions, 6), dtype=torch.int32)
-        regs[1, 0] = torch.tensor([0, 0, L["out_w"], L["out_h"], 0, 0], dtype=torch.int32)
-        regs[0, 0] = torch.tensor([1, 2, 5, 4, 2, 1], dtype=torch.int32)
-        counts = torch.tensor([1, 1, 0], dtype=torch.int32)
+        counts = torch.zeros(S, dtype=torch.int32)
+        ow, oh = L["out_w"], L["out_h"]
+        regs[0, 0] = torch.tensor([1, 2, min(5, ow - 2), min(4, oh - 2), 2, 1] if oh >= 4 else [1, 1, ow - 1, oh - 1, 0, 0], dtype=torch.int32)
+        counts[0] = 1
+        if S > 1:
+            regs[1, 0] = torch.tensor([0, 0, ow, oh, 0, 0], dtype=torch.int32)
+            counts[1] = 1
         part = dc.conv_partial(1, xin, pin, regs.cuda(), counts.cuda())
         wq = orc.quant_array(wts, orc.QUANT_BF16)
         for s_ in range(S):
