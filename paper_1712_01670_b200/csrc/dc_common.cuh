@@ -52,6 +52,7 @@ struct dc_layer_rt {
     void* weight_packed;            // conv, bf16: K-major tensor-core layout (see dc_conv_bf16.cu)
     int k_packed;                   // padded reduction length of weight_packed
     int tc_ctas;                    // conv, bf16: CTAs per SM the tuned launch uses (1 or 2)
+    int tc_ew;                      // conv, bf16: epilogue warps per CTA (4, or 8 with one CTA per SM); 0 = 4
     int tc_mt, tc_bn;               // conv, bf16: tuned tiles per work item (3, 4: patch-reuse kernel with 1, 2; 5, 6: column-slab kernel) and
                                     // channels per block (0 = default)
     void* weight_halo;              // conv, bf16: weights packed for the patch-reuse and column-slab kernels

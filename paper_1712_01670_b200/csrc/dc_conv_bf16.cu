@@ -26,7 +26,9 @@
 
 namespace {
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 192;          // producer warp, MMA warp, four epilogue warps
+constexpr int kThreadsWide = 320;      // ... or eight epilogue warps
+static inline int threads_for(int epi_warps) { return 64 + 32 * epi_warps; }
 constexpr int kMaxStages = 8;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // 2 s
 
@@ -45,6 +47,7 @@ struct TcArgs {
     // flat tiles (tap-by-tap kernel only): row i of tile t is group t * 16 + i, a group being 8 output pixels of one
     // image row, numbered (stream * Ho + y) * gpr + column group; n_groups_all = S * Ho * gpr.  0: 16 x 8 blocks.
     int flat = 0, gpr = 0, n_groups_all = 0;
+    int epi_warps = 4;            // epilogue warps of the CTA: 4 (192 threads) or 8 (320 threads)
 };
 
 struct SmemCtl {
@@ -54,9 +57,13 @@ struct SmemCtl {
     volatile int abort_flag;
     unsigned long long wait_ns;
     // epilogue staging: per warp 32 pixels x 64 bytes (32 bf16 channels), rows padded to 80 bytes so
-    // 16-byte accesses of neighbouring lanes fall in different banks
-    __align__(16) uint8_t stage[4][32 * 80];
+    // 16-byte accesses of neighbouring lanes fall in different banks.  Last member: a launch with four epilogue
+    // warps asks for (and touches) the first four only, see ctl_bytes().
+    __align__(16) uint8_t stage[8][32 * 80];
 };
+constexpr int kStageBytes = 32 * 80;
+// Shared memory the control block takes with `epi_warps` epilogue warps (4 or 8).
+constexpr size_t ctl_bytes(int epi_warps) { return sizeof(SmemCtl) - (size_t)(8 - epi_warps) * kStageBytes; }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -166,19 +173,41 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// (acc0 + b0, acc1 + b1) in fp32 (one packed add), then round to nearest even into two bf16; RELU clamps negative
+// results to zero in the same conversion (rounding is monotonic, so clamping before or after it gives the same value).
+template <bool RELU>
+__device__ __forceinline__ uint32_t bias_pack_bf16(uint32_t acc0, uint32_t acc1, float b0, float b1)
+{
+    uint32_t out;
+    if (RELU)
+        asm("{\n\t.reg .b64 a, b, d;\n\t.reg .f32 x, y;\n\tmov.b64 a, {%1, %2};\n\tmov.b64 b, {%3, %4};\n\t"
+            "add.rn.f32x2 d, a, b;\n\tmov.b64 {x, y}, d;\n\tcvt.rn.relu.bf16x2.f32 %0, y, x;\n\t}"
+            : "=r"(out) : "r"(acc0), "r"(acc1), "f"(b0), "f"(b1));
+    else
+        asm("{\n\t.reg .b64 a, b, d;\n\t.reg .f32 x, y;\n\tmov.b64 a, {%1, %2};\n\tmov.b64 b, {%3, %4};\n\t"
+            "add.rn.f32x2 d, a, b;\n\tmov.b64 {x, y}, d;\n\tcvt.rn.bf16x2.f32 %0, y, x;\n\t}"
+            : "=r"(out) : "r"(acc0), "r"(acc1), "f"(b0), "f"(b1));
+    return out;
+}
 
 // Epilogue warps (4 warps = 128 TMEM lanes = the 128 pixels of a tile): for every work item wait
 // for its accumulator, read it 32 columns at a time, add the bias, apply ReLU, round to bf16 and
 // store the pixel's channels unless the reuse bitmap says the pixel was filled from the cache.
+// epi_warps = 8: two warps per TMEM lane quadrant (warps 2-5 and 6-9), each taking half of the item's channels:
+// layers with little accumulation per output (1x1, few input channels) are bound by this read-out.
 // first_item / item_stride: the items this CTA (or CTA pair) takes.  tiles_per_group / tile_sub: a group of the tile list
 // holds tiles_per_group tiles and this CTA's first one is number tile_sub in it (a pair: 2 and its rank, with a.MT = 1).
 // remote_empty: 0, or the shared::cluster address of the pair leader's tmem_empty[0], on which this CTA's epilogue
 // threads arrive instead of on their own.
 __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uint32_t tmem_base, int n_items, int n_tiles, int warp, int lane,
-                                              int first_item, int item_stride, int tiles_per_group, int tile_sub, uint32_t remote_empty)
+                                              int first_item, int item_stride, int tiles_per_group, int tile_sub, uint32_t remote_empty,
+                                              int epi_warps = 4)
 {
     const int per_stream = a.tiles_x * a.tiles_y;
     const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
+    // this warp's 32-column steps of an item: all of them, or the lower / upper half
+    const int n_steps = a.BN / 32, mid = epi_warps == 8 ? (n_steps + 1) / 2 : n_steps;
+    const int c_begin = warp >= 6 ? mid : 0, c_end = warp >= 6 ? n_steps : mid;
     const int m = q * 32 + lane, prow = m / DC_TILE_W, pcol = m % DC_TILE_W;
     const int mword_i = DC_TILE_BIT(prow, pcol) >> 5, mbit = DC_TILE_BIT(prow, pcol) & 31;
     uint32_t acc = 0, acc_ph = 0;
@@ -238,26 +267,32 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
             // sectors); instead the warp stages its 32 x 64 bytes in shared memory and writes them back with
             // 4 lanes per pixel, so each pixel's 64 bytes leave as two whole sectors.
             const unsigned act_mask = __ballot_sync(0xffffffffu, active);
-            uint8_t* stg = ctl->stage[q];
+            uint8_t* stg = ctl->stage[warp - 2];
             const uint8_t* const rd = stg + (lane >> 2) * 80 + (lane & 3) * 16;
-            for (int c = 0; c < a.BN / 32; ++c) {
+            for (int c = c_begin; c < c_end; ++c) {
                 uint32_t r[32];
                 tmem_ld32(taddr + c * 32, r);
-                tmem_ld_wait();
+                // the step's 32 bias values travel while the accumulator read is in flight
+                float4 bv[8];
                 const float4* b4 = (const float4*)(bias + c * 32);
+#pragma unroll
+                for (int v = 0; v < 8; ++v) bv[v] = __ldg(b4 + v);
+                tmem_ld_wait();
                 uint4* mine = (uint4*)(stg + lane * 80);
+                if (a.relu) {
 #pragma unroll
-                for (int v = 0; v < 4; ++v) {
-                    const float4 ba = __ldg(b4 + 2 * v), bb = __ldg(b4 + 2 * v + 1);
-                    float f[8] = {__uint_as_float(r[v * 8 + 0]) + ba.x, __uint_as_float(r[v * 8 + 1]) + ba.y,
-                                  __uint_as_float(r[v * 8 + 2]) + ba.z, __uint_as_float(r[v * 8 + 3]) + ba.w,
-                                  __uint_as_float(r[v * 8 + 4]) + bb.x, __uint_as_float(r[v * 8 + 5]) + bb.y,
-                                  __uint_as_float(r[v * 8 + 6]) + bb.z, __uint_as_float(r[v * 8 + 7]) + bb.w};
-                    if (a.relu) {
+                    for (int v = 0; v < 4; ++v)
+                        mine[v] = make_uint4(bias_pack_bf16<true>(r[v * 8 + 0], r[v * 8 + 1], bv[2 * v].x, bv[2 * v].y),
+                                             bias_pack_bf16<true>(r[v * 8 + 2], r[v * 8 + 3], bv[2 * v].z, bv[2 * v].w),
+                                             bias_pack_bf16<true>(r[v * 8 + 4], r[v * 8 + 5], bv[2 * v + 1].x, bv[2 * v + 1].y),
+                                             bias_pack_bf16<true>(r[v * 8 + 6], r[v * 8 + 7], bv[2 * v + 1].z, bv[2 * v + 1].w));
+                } else {
 #pragma unroll
-                        for (int jj = 0; jj < 8; ++jj) f[jj] = fmaxf(f[jj], 0.f);
-                    }
-                    mine[v] = make_uint4(pack_bf16(f[0], f[1]), pack_bf16(f[2], f[3]), pack_bf16(f[4], f[5]), pack_bf16(f[6], f[7]));
+                    for (int v = 0; v < 4; ++v)
+                        mine[v] = make_uint4(bias_pack_bf16<false>(r[v * 8 + 0], r[v * 8 + 1], bv[2 * v].x, bv[2 * v].y),
+                                             bias_pack_bf16<false>(r[v * 8 + 2], r[v * 8 + 3], bv[2 * v].z, bv[2 * v].w),
+                                             bias_pack_bf16<false>(r[v * 8 + 4], r[v * 8 + 5], bv[2 * v + 1].x, bv[2 * v + 1].y),
+                                             bias_pack_bf16<false>(r[v * 8 + 6], r[v * 8 + 7], bv[2 * v + 1].z, bv[2 * v + 1].w));
                 }
                 __syncwarp();
 #pragma unroll
@@ -276,7 +311,7 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
 }
 
 template <int MT>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsWide, 1)
 k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -294,7 +329,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < a.stages; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 128); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 32u * (uint32_t)a.epi_warps); }
         ctl->abort_flag = 0;
         ctl->wait_ns = a.wait_ns;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -409,7 +444,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         __syncwarp();
     } else {
         // ---------------- epilogue ----------------
-        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane, blockIdx.x, gridDim.x, a.MT, 0, 0u);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane, blockIdx.x, gridDim.x, a.MT, 0, 0u, a.epi_warps);
     }
     tc_fence_before();
     __syncthreads();
@@ -437,7 +472,7 @@ struct TcSmallArgs {
     int PW, PH, stage_bytes;      // input patch per tile: (8 + kw - 1) x (16 + kh - 1) pixels of 16 bytes, + pad
 };
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsWide, 1)
 k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -454,7 +489,7 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < a.stages; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 128); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 32u * (uint32_t)a.epi_warps); }
         ctl->abort_flag = 0;
         ctl->wait_ns = a.wait_ns;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -462,9 +497,9 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
     }
     // weights into shared memory; zero the ring once: each slot ends in a pad that no TMA box fills but
     // the last (zero-weight) K block reads, and 0 x garbage could be NaN
-    for (int i = threadIdx.x; i < sa.w_bytes / 16; i += kThreads)
+    for (int i = threadIdx.x; i < sa.w_bytes / 16; i += blockDim.x)
         ((uint4*)wsm)[i] = __ldg((const uint4*)sa.wpacked + i);
-    for (int i = threadIdx.x; i < a.stages * sa.stage_bytes / 16; i += kThreads)
+    for (int i = threadIdx.x; i < a.stages * sa.stage_bytes / 16; i += blockDim.x)
         ((uint4*)ring)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to TMA / MMA
     if (warp == 1) {
@@ -531,7 +566,7 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
         }
         __syncwarp();
     } else {
-        epilogue_loop(a, ctl, tmem_base, n_items, n_items, warp, lane, blockIdx.x, gridDim.x, 1, 0, 0u);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_items, warp, lane, blockIdx.x, gridDim.x, 1, 0, 0u, a.epi_warps);
     }
     tc_fence_before();
     __syncthreads();
@@ -573,7 +608,7 @@ __device__ __forceinline__ void bulk_copy_g2s(void* dst, const void* src, uint32
 //               K-major tile.  kw loads of whole 128-byte rows per chunk instead of kh * kw (tap by tap) or eight
 //               loads of 16-byte rows (patch).  ha.patch_bytes then holds the bytes of one slab.
 template <int MT, bool SLAB>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsWide, 1)
 k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
 {
     extern __shared__ uint8_t smem_raw[];
@@ -592,7 +627,7 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
 
     if (threadIdx.x == 0) {
         for (int i = 0; i < a.stages; ++i) { mbar_init(&ctl->full[i], 1); mbar_init(&ctl->empty[i], 1); }
-        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 128); }
+        for (int i = 0; i < 2; ++i) { mbar_init(&ctl->tmem_full[i], 1); mbar_init(&ctl->tmem_empty[i], 32u * (uint32_t)a.epi_warps); }
         for (int i = 0; i < 4; ++i) { mbar_init(&ctl->a_full[i], 1); mbar_init(&ctl->a_empty[i], 1); }
         ctl->abort_flag = 0;
         ctl->wait_ns = a.wait_ns;
@@ -717,7 +752,7 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
         }
         __syncwarp();
     } else {
-        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane, blockIdx.x, gridDim.x, a.MT, 0, 0u);
+        epilogue_loop(a, ctl, tmem_base, n_items, n_tiles, warp, lane, blockIdx.x, gridDim.x, a.MT, 0, 0u, a.epi_warps);
     }
     tc_fence_before();
     __syncthreads();
@@ -1038,7 +1073,10 @@ static uint32_t tmem_cols_for(int nbuf, int mt, int bn)
 // its SM, which then works in the tensor-core kernel's idle issue slots instead of waiting for a free SM.  Set per
 // launch from the cache's state.
 static thread_local int t_ring_kb = 200;
-static int ring_budget(int ctas) { return t_ring_kb * 1024 / (ctas == 2 ? 2 : 1); }
+static thread_local int t_epi_warps = 4;      // the layer's tuned epilogue width, honoured by launches with one CTA per SM
+static int epi_warps_for(int ctas) { return t_epi_warps == 8 && ctas != 2 ? 8 : 4; }
+// eight epilogue warps stage twice as much: the rings give that up
+static int ring_budget(int ctas) { return (t_ring_kb * 1024 - (epi_warps_for(ctas) == 8 ? 4 * kStageBytes : 0)) / (ctas == 2 ? 2 : 1); }
 
 // Every launch waits at most kWaitLimitNs on the device.  dc_debug_stall_next_conv (below) arms the next launch
 // only: its producer issues no copy and its waits run out after the given time.
@@ -1095,7 +1133,7 @@ bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn =
     int st = ring_budget(ctas) / (p.MT * p.a_bytes + p.b_bytes);
     p.stages = st > kMaxStages ? kMaxStages : st;
     if (p.stages < 2) return false;
-    p.smem = (size_t)p.stages * (p.MT * p.a_bytes + p.b_bytes) + sizeof(SmemCtl) + 1024;
+    p.smem = (size_t)p.stages * (p.MT * p.a_bytes + p.b_bytes) + ctl_bytes(epi_warps_for(ctas)) + 1024;
     return true;
 }
 
@@ -1237,7 +1275,8 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     int st = (ring_budget(ctas) - sa.w_bytes) / stage_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
-    const size_t smem = (size_t)a.stages * stage_bytes + ((sa.w_bytes + 127) & ~127) + sizeof(SmemCtl) + 256;
+    a.epi_warps = epi_warps_for(ctas);
+    const size_t smem = (size_t)a.stages * stage_bytes + ((sa.w_bytes + 127) & ~127) + ctl_bytes(a.epi_warps) + 256;
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device)) {
         DC_CUDA(cudaFuncSetAttribute(k_conv_tc_smallc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
@@ -1247,7 +1286,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     int grid = items > c->num_sms * ctas ? c->num_sms * ctas : items;
     dc_prof_scope ps(c, DC_ST_CONV);
     k_pad_channels8<<<grid_pad, 256, 0, c->stream>>>((const __nv_bfloat16*)in, pixels, d.cin, (__nv_bfloat16*)L.in_padded);
-    k_conv_tc_smallc<<<grid, kThreads, smem, c->stream>>>(tmA, sa);
+    k_conv_tc_smallc<<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, sa);
     c->launches += 2;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -1312,7 +1351,8 @@ static int launch_halo(dc_cache* c, int layer, int grp, int mt, bool slab, const
     int st = (budget - a_total) / h.b_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
-    const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + sizeof(SmemCtl) + (slab ? 1280 : 256);
+    a.epi_warps = epi_warps_for(ctas);
+    const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + ctl_bytes(a.epi_warps) + (slab ? 1280 : 256);
     if (smem > 227 * 1024) return DC_ERR_CONFIG;
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device)) {
@@ -1325,11 +1365,11 @@ static int launch_halo(dc_cache* c, int layer, int grp, int mt, bool slab, const
     int grid = items > c->num_sms * ctas ? c->num_sms * ctas : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
     if (slab) {
-        if (mt == 2) k_conv_tc_halo<2, true><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
-        else k_conv_tc_halo<1, true><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+        if (mt == 2) k_conv_tc_halo<2, true><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
+        else k_conv_tc_halo<1, true><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
     } else {
-        if (mt == 2) k_conv_tc_halo<2, false><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
-        else k_conv_tc_halo<1, false><<<grid, kThreads, smem, c->stream>>>(tmA, ha);
+        if (mt == 2) k_conv_tc_halo<2, false><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
+        else k_conv_tc_halo<1, false><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
     }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
@@ -1411,7 +1451,7 @@ static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const 
     int st = (budget - ha.a_stages * ha.patch_bytes) / b_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
-    const size_t smem = (size_t)ha.a_stages * ha.patch_bytes + (size_t)a.stages * b_bytes + sizeof(SmemCtl) + 1280;
+    const size_t smem = (size_t)ha.a_stages * ha.patch_bytes + (size_t)a.stages * b_bytes + ctl_bytes(4) + 1280;
     if (smem > 227 * 1024) return DC_ERR_CONFIG;
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device))
@@ -1434,6 +1474,9 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
 {
     const int G = n_groups(c->L[layer].d);
     t_ring_kb = c->overlap_mode ? 182 : 200;
+    // eight epilogue warps take the registers that the block search of the next frame needs to stay resident beside
+    // this kernel: while that overlap is in use the CTA keeps to four
+    t_epi_warps = c->L[layer].tc_ew == 8 && !c->overlap_mode ? 8 : 4;
     for (int grp = 0; grp < G; ++grp) {                           // a grouped layer: one launch per group
         int rc = launch_group(c, layer, grp, in, out, tile_list, tile_count, masks, max_tiles);
         if (rc == DC_ERR_CONFIG && t_ring_kb != 200) {            // the layer's tuned shape needs the full rings: it gets them
@@ -1514,6 +1557,7 @@ static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* o
     a.idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(p.BN >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
     a.status = c->status;
     a.flat = L.flat; a.gpr = L.gpr; a.n_groups_all = c->S * d.out_h * L.gpr;
+    a.epi_warps = epi_warps_for(ctas);
     set_wait_limit(c, a);
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device)) {
@@ -1523,8 +1567,8 @@ static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* o
     long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + p.MT - 1) / p.MT) * p.NB;
     int grid = items > c->num_sms * ctas ? c->num_sms * ctas : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
-    if (p.MT == 2) k_conv_tc<2><<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
-    else k_conv_tc<1><<<grid, kThreads, p.smem, c->stream>>>(tmA, tmB, a);
+    if (p.MT == 2) k_conv_tc<2><<<grid, threads_for(a.epi_warps), p.smem, c->stream>>>(tmA, tmB, a);
+    else k_conv_tc<1><<<grid, threads_for(a.epi_warps), p.smem, c->stream>>>(tmA, tmB, a);
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -1549,7 +1593,7 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
     cudaEvent_t e0, e1;
     DC_CUDA(cudaEventCreate(&e0));
     DC_CUDA(cudaEventCreate(&e1));
-    float best = 1e30f; int best_mt = L.tc_mt, best_bn = L.tc_bn, best_ctas = 1, best_flat = 0;
+    float best = 1e30f; int best_mt = L.tc_mt, best_bn = L.tc_bn, best_ctas = 1, best_flat = 0, best_ew = 4;
     constexpr int kTuneReps = 6;                                      // timed launches per candidate, after one untimed
     // the GPU may have been idle: bring the clocks up before the first candidate is timed
     for (int rep = 0; rep < 12; ++rep)
@@ -1571,12 +1615,15 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
         if (rc != DC_OK || cudaEventSynchronize(e1) != cudaSuccess) { cudaGetLastError(); return; }
         float ms = 0.f;
         cudaEventElapsedTime(&ms, e0, e1);
-        if (verbose) fprintf(stderr, "libdeepcache: layer %d: %s, tiles/item code %d, %d channels per block, %d CTA(s) per SM: %.3f ms\n",
-                             layer, what, L.flat ? L.tc_mt + 7 : L.tc_mt, L.tc_bn, L.tc_ctas, ms / kTuneReps);
-        if (ms < best) { best = ms; best_mt = L.tc_mt; best_bn = L.tc_bn; best_ctas = L.tc_ctas; best_flat = L.flat; }
+        if (verbose) fprintf(stderr, "libdeepcache: layer %d: %s, tiles/item code %d, %d channels per block, %d CTA(s) per SM, %d epilogue warps: %.3f ms\n",
+                             layer, what, L.flat ? L.tc_mt + 7 : L.tc_mt, L.tc_bn, L.tc_ctas, L.tc_ew, ms / kTuneReps);
+        if (ms < best) { best = ms; best_mt = L.tc_mt; best_bn = L.tc_bn; best_ctas = L.tc_ctas; best_flat = L.flat; best_ew = L.tc_ew; }
     };
-    for (int ctas = 1; ctas <= 2; ++ctas) {
-        L.tc_ctas = ctas;
+    // one CTA per SM with four or eight epilogue warps, or two CTAs per SM with four each
+    for (int shape = 0; shape < 3; ++shape) {
+        const int ctas = shape == 2 ? 2 : 1;
+        L.tc_ctas = ctas; L.tc_ew = shape == 1 ? 8 : 4;
+        t_epi_warps = L.tc_ew;                                        // make_plan below sizes the rings for it
         if (!generic) {                                               // few input channels: one kernel shape, 1 or 2 CTAs per SM
             if (ctas == 2 && tmem_cols_for(2, 1, L.d.cout) > 256) continue;
             trial("few-channel kernel");
@@ -1616,15 +1663,15 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
     {
         int pbn = 0;
         if (generic && L.weight_halo && pair_ok(L.d, pbn)) {          // tc_mt 7: a CTA pair per two tiles (cta_group::2)
-            L.tc_mt = 7; L.tc_bn = pbn; L.tc_ctas = 1;
+            L.tc_mt = 7; L.tc_bn = pbn; L.tc_ctas = 1; L.tc_ew = 4;
             trial("CTA-pair kernel");
         }
     }
-    L.tc_mt = best_mt; L.tc_bn = best_bn; L.tc_ctas = best_ctas; L.flat = best_flat;
+    L.tc_mt = best_mt; L.tc_bn = best_bn; L.tc_ctas = best_ctas; L.flat = best_flat; L.tc_ew = best_ew;
     cudaEventDestroy(e0); cudaEventDestroy(e1);
     c->launches = 0;
-    if (verbose) fprintf(stderr, "libdeepcache: layer %d: chose code %d, %d channels per block, %d CTA(s) per SM (%.3f ms)\n",
-                         layer, best_flat ? best_mt + 7 : best_mt, best_bn, best_ctas, best / kTuneReps);
+    if (verbose) fprintf(stderr, "libdeepcache: layer %d: chose code %d, %d channels per block, %d CTA(s) per SM, %d epilogue warps (%.3f ms)\n",
+                         layer, best_flat ? best_mt + 7 : best_mt, best_bn, best_ctas, best_ew, best / kTuneReps);
     return DC_OK;
 }
 
