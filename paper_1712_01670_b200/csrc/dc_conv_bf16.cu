@@ -67,6 +67,14 @@ constexpr size_t ctl_bytes(int epi_warps) { return sizeof(SmemCtl) - (size_t)(8 
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
+// Programmatic dependent launch: a convolution kernel is launched so that its CTAs may become resident while the
+// previous kernel of the stream is still running (on SMs that kernel has left).  Barrier set-up, tensor-memory
+// allocation and descriptor prefetch run there; pdl_wait() returns once the previous kernel has completed and its
+// writes are visible, and nothing that another kernel produces is read (or overwritten) before it.
+// pdl_release() lets the kernel after this one do the same.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void mbar_init(void* bar, uint32_t count)
 {
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
@@ -315,9 +323,6 @@ __global__ void __launch_bounds__(kThreadsWide, 1)
 k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const TcArgs a)
 {
     extern __shared__ uint8_t smem_raw[];
-    const int n_tiles = *a.tile_count;
-    const int n_items = (n_tiles + MT - 1) / MT * a.NB;     // an item: MT tiles x one block of BN channels
-    if ((int)blockIdx.x >= n_items) return;
 
     // operand ring at a 1024-byte boundary (the swizzle pattern repeats every 1024 bytes), then control words
     uint8_t* ring = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -344,6 +349,10 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    pdl_wait();                 // the previous kernel's output, the tile list and its count are read from here on
+    pdl_release();
+    const int n_tiles = *a.tile_count;
+    const int n_items = (n_tiles + MT - 1) / MT * a.NB;     // an item: MT tiles x one block of BN channels; none for this CTA: it only frees its tensor memory
 
     if (warp == 0) {
         // ---------------- TMA producer ----------------
@@ -477,8 +486,6 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
 {
     extern __shared__ uint8_t smem_raw[];
     const TcArgs& a = sa.t;
-    const int n_items = *a.tile_count;
-    if ((int)blockIdx.x >= n_items) return;
     uint8_t* base = (uint8_t*)(((uintptr_t)smem_raw + 127) & ~(uintptr_t)127);
     uint8_t* wsm = base;                                        // packed weights
     uint8_t* ring = wsm + ((sa.w_bytes + 127) & ~127);
@@ -510,6 +517,9 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    pdl_wait();                 // the previous kernel's output, the tile list and its count are read from here on
+    pdl_release();
+    const int n_items = *a.tile_count;
 
     if (warp == 0) {
         if (lane == 0) {                                        // producer: one patch per item
@@ -613,9 +623,6 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
 {
     extern __shared__ uint8_t smem_raw[];
     const TcArgs& a = ha.t;
-    const int n_tiles = *a.tile_count;
-    const int n_items = (n_tiles + MT - 1) / MT * a.NB;
-    if ((int)blockIdx.x >= n_items) return;
     constexpr uintptr_t kAlign = SLAB ? 1023 : 127;           // swizzle atoms start on 1024-byte boundaries
     uint8_t* aring = (uint8_t*)(((uintptr_t)smem_raw + kAlign) & ~kAlign);
     const int a_slot = MT * ha.patch_bytes;
@@ -642,6 +649,10 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    pdl_wait();                 // the previous kernel's output, the tile list and its count are read from here on
+    pdl_release();
+    const int n_tiles = *a.tile_count;
+    const int n_items = (n_tiles + MT - 1) / MT * a.NB;
 
     if (warp == 0) {
         // ---------------- producer: patches by TMA, weights by bulk copy ----------------
@@ -824,10 +835,7 @@ k_conv_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 {
     extern __shared__ uint8_t smem_raw[];
     const TcArgs& a = ha.t;
-    const int n_tiles = *a.tile_count;
-    const int n_items = (n_tiles + 1) / 2 * a.NB;
     const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
-    if (pair >= n_items) return;                              // both CTAs of a pair leave together
     const uint32_t rank = cluster_rank();
     const bool leader = rank == 0;
     uint8_t* aring = (uint8_t*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
@@ -857,6 +865,10 @@ k_conv_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     cluster_sync_all();                                       // both CTAs' barriers exist before either is signalled from outside
     tc_fence_after();
     const uint32_t tmem_base = ctl->tmem_base;
+    pdl_wait();                 // the previous kernel's output, the tile list and its count are read from here on
+    pdl_release();
+    const int n_tiles = *a.tile_count;
+    const int n_items = (n_tiles + 1) / 2 * a.NB;
 
     if (warp == 0) {
         // ---------------- producer: this CTA's slab and its half of the weights ----------------
@@ -1072,6 +1084,25 @@ static uint32_t tmem_cols_for(int nbuf, int mt, int bn)
 // inference (dc_lookahead_frame): with 182 KB a convolution CTA leaves room for one CTA of the block search (32 KB) on
 // its SM, which then works in the tensor-core kernel's idle issue slots instead of waiting for a free SM.  Set per
 // launch from the cache's state.
+// Launch with programmatic stream serialization allowed (see pdl_wait): the kernel may start before the previous
+// kernel of the stream has ended.  Not while the block search of the next frame runs beside the inference: there the
+// search is the longer chain, and it is the gaps between convolution kernels that let more of its CTAs in.
+// DC_NO_PDL=1 (diagnostics) always launches the ordinary way.
+static thread_local bool t_pdl = true;
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_conv_kernel(void (*kernel)(KArgs...), int grid, int threads, size_t smem, cudaStream_t stream, Args&&... args)
+{
+    static const bool pdl_env = getenv("DC_NO_PDL") == nullptr;
+    const bool pdl = pdl_env && t_pdl;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid); cfg.blockDim = dim3((unsigned)threads); cfg.dynamicSmemBytes = smem; cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = pdl ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 static thread_local int t_ring_kb = 200;
 static thread_local int t_epi_warps = 4;      // the layer's tuned epilogue width, honoured by launches with one CTA per SM
 static int epi_warps_for(int ctas) { return t_epi_warps == 8 && ctas != 2 ? 8 : 4; }
@@ -1286,7 +1317,7 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     int grid = items > c->num_sms * ctas ? c->num_sms * ctas : items;
     dc_prof_scope ps(c, DC_ST_CONV);
     k_pad_channels8<<<grid_pad, 256, 0, c->stream>>>((const __nv_bfloat16*)in, pixels, d.cin, (__nv_bfloat16*)L.in_padded);
-    k_conv_tc_smallc<<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, sa);
+    DC_CUDA(launch_conv_kernel(k_conv_tc_smallc, grid, threads_for(a.epi_warps), smem, c->stream, tmA, sa));
     c->launches += 2;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -1365,11 +1396,11 @@ static int launch_halo(dc_cache* c, int layer, int grp, int mt, bool slab, const
     int grid = items > c->num_sms * ctas ? c->num_sms * ctas : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
     if (slab) {
-        if (mt == 2) k_conv_tc_halo<2, true><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
-        else k_conv_tc_halo<1, true><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
+        if (mt == 2) DC_CUDA(launch_conv_kernel(k_conv_tc_halo<2, true>, grid, threads_for(a.epi_warps), smem, c->stream, tmA, ha));
+        else DC_CUDA(launch_conv_kernel(k_conv_tc_halo<1, true>, grid, threads_for(a.epi_warps), smem, c->stream, tmA, ha));
     } else {
-        if (mt == 2) k_conv_tc_halo<2, false><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
-        else k_conv_tc_halo<1, false><<<grid, threads_for(a.epi_warps), smem, c->stream>>>(tmA, ha);
+        if (mt == 2) DC_CUDA(launch_conv_kernel(k_conv_tc_halo<2, false>, grid, threads_for(a.epi_warps), smem, c->stream, tmA, ha));
+        else DC_CUDA(launch_conv_kernel(k_conv_tc_halo<1, false>, grid, threads_for(a.epi_warps), smem, c->stream, tmA, ha));
     }
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
@@ -1460,7 +1491,7 @@ static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const 
     const int max_pairs = c->num_sms / 2;                        // one CTA per SM, a pair per TPC
     const int pairs = items > max_pairs ? max_pairs : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
-    k_conv_tc_pair<<<2 * pairs, kThreads, smem, c->stream>>>(*tmAp, *tmWp, ha);
+    DC_CUDA(launch_conv_kernel(k_conv_tc_pair, 2 * pairs, kThreads, smem, c->stream, *tmAp, *tmWp, ha));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
@@ -1474,6 +1505,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
 {
     const int G = n_groups(c->L[layer].d);
     t_ring_kb = c->overlap_mode ? 182 : 200;
+    t_pdl = !c->overlap_mode;
     // eight epilogue warps take the registers that the block search of the next frame needs to stay resident beside
     // this kernel: while that overlap is in use the CTA keeps to four
     t_epi_warps = c->L[layer].tc_ew == 8 && !c->overlap_mode ? 8 : 4;
@@ -1567,8 +1599,8 @@ static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* o
     long long items = (long long)(((max_tiles < 1 ? 1 : max_tiles) + p.MT - 1) / p.MT) * p.NB;
     int grid = items > c->num_sms * ctas ? c->num_sms * ctas : (int)items;
     dc_prof_scope ps(c, DC_ST_CONV);
-    if (p.MT == 2) k_conv_tc<2><<<grid, threads_for(a.epi_warps), p.smem, c->stream>>>(tmA, tmB, a);
-    else k_conv_tc<1><<<grid, threads_for(a.epi_warps), p.smem, c->stream>>>(tmA, tmB, a);
+    if (p.MT == 2) DC_CUDA(launch_conv_kernel(k_conv_tc<2>, grid, threads_for(a.epi_warps), p.smem, c->stream, tmA, tmB, a));
+    else DC_CUDA(launch_conv_kernel(k_conv_tc<1>, grid, threads_for(a.epi_warps), p.smem, c->stream, tmA, tmB, a));
     c->launches += 1;
     DC_CUDA(cudaGetLastError());
     return DC_OK;
