@@ -48,6 +48,7 @@ struct TcArgs {
     // image row, numbered (stream * Ho + y) * gpr + column group; n_groups_all = S * Ho * gpr.  0: 16 x 8 blocks.
     int flat = 0, gpr = 0, n_groups_all = 0;
     int epi_warps = 4;            // epilogue warps of the CTA: 4 (192 threads) or 8 (320 threads)
+    int bias_smem = 0;            // > 0: that many bias values (the launch's NB * BN, from channel block nb_off on) are staged in shared memory behind the control block
 };
 
 struct SmemCtl {
@@ -63,7 +64,7 @@ struct SmemCtl {
 };
 constexpr int kStageBytes = 32 * 80;
 // Shared memory the control block takes with `epi_warps` epilogue warps (4 or 8).
-constexpr size_t ctl_bytes(int epi_warps) { return sizeof(SmemCtl) - (size_t)(8 - epi_warps) * kStageBytes; }
+__host__ __device__ constexpr size_t ctl_bytes(int epi_warps) { return sizeof(SmemCtl) - (size_t)(8 - epi_warps) * kStageBytes; }
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -181,6 +182,18 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b)
     __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&v);
 }
+// 16-byte accesses to the epilogue's staging by shared-space address: through a generic pointer they would be
+// generic loads and stores, which resolve the address space first and wait on the long-latency scoreboard.
+__device__ __forceinline__ void sts128(uint32_t addr, uint32_t x, uint32_t y, uint32_t z, uint32_t w)
+{
+    asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+__device__ __forceinline__ uint4 lds128(uint32_t addr)
+{
+    uint4 v;
+    asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
+    return v;
+}
 // (acc0 + b0, acc1 + b1) in fp32 (one packed add), then round to nearest even into two bf16; RELU clamps negative
 // results to zero in the same conversion (rounding is monotonic, so clamping before or after it gives the same value).
 template <bool RELU>
@@ -198,6 +211,16 @@ __device__ __forceinline__ uint32_t bias_pack_bf16(uint32_t acc0, uint32_t acc1,
     return out;
 }
 
+// Copies the launch's bias values behind the control block (all threads; before the set-up's __syncthreads).  The
+// epilogue reads 32 of them per step and lane: from shared memory that is eight short broadcast loads, through the
+// read-only cache it was a fifth of the time of the layers that the epilogue bounds.
+__device__ __forceinline__ void stage_bias(const TcArgs& a, SmemCtl* ctl, int epi_warps)
+{
+    float* dst = (float*)((uint8_t*)ctl + ctl_bytes(epi_warps));
+    const float* src = a.bias + (size_t)a.nb_off * a.BN;
+    for (int i = threadIdx.x; i < a.bias_smem; i += blockDim.x) dst[i] = __ldg(src + i);
+}
+
 // Epilogue warps (4 warps = 128 TMEM lanes = the 128 pixels of a tile): for every work item wait
 // for its accumulator, read it 32 columns at a time, add the bias, apply ReLU, round to bf16 and
 // store the pixel's channels unless the reuse bitmap says the pixel was filled from the cache.
@@ -211,6 +234,8 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
                                               int first_item, int item_stride, int tiles_per_group, int tile_sub, uint32_t remote_empty,
                                               int epi_warps = 4)
 {
+    // the launch's bias values in shared memory (stage_bias), or 0: read through the read-only cache
+    const uint32_t bias_s = a.bias_smem > 0 ? smem_u32((const uint8_t*)ctl + ctl_bytes(epi_warps)) : 0u;
     const int per_stream = a.tiles_x * a.tiles_y;
     const int q = warp & 3;                                     // TMEM lane quadrant this warp may read
     // this warp's 32-column steps of an item: all of them, or the lower / upper half
@@ -275,38 +300,46 @@ __device__ __forceinline__ void epilogue_loop(const TcArgs& a, SmemCtl* ctl, uin
             // sectors); instead the warp stages its 32 x 64 bytes in shared memory and writes them back with
             // 4 lanes per pixel, so each pixel's 64 bytes leave as two whole sectors.
             const unsigned act_mask = __ballot_sync(0xffffffffu, active);
-            uint8_t* stg = ctl->stage[warp - 2];
-            const uint8_t* const rd = stg + (lane >> 2) * 80 + (lane & 3) * 16;
+            const uint32_t stg = smem_u32(ctl->stage[warp - 2]);
+            const uint32_t rd = stg + (lane >> 2) * 80 + (lane & 3) * 16, mine = stg + lane * 80;
             for (int c = c_begin; c < c_end; ++c) {
                 uint32_t r[32];
                 tmem_ld32(taddr + c * 32, r);
                 // the step's 32 bias values travel while the accumulator read is in flight
                 float4 bv[8];
-                const float4* b4 = (const float4*)(bias + c * 32);
+                if (bias_s) {
+                    const uint32_t b4 = bias_s + (uint32_t)(nb * a.BN + c * 32) * 4u;
 #pragma unroll
-                for (int v = 0; v < 8; ++v) bv[v] = __ldg(b4 + v);
+                    for (int v = 0; v < 8; ++v) {
+                        const uint4 t = lds128(b4 + v * 16);
+                        bv[v] = make_float4(__uint_as_float(t.x), __uint_as_float(t.y), __uint_as_float(t.z), __uint_as_float(t.w));
+                    }
+                } else {
+                    const float4* b4 = (const float4*)(bias + c * 32);
+#pragma unroll
+                    for (int v = 0; v < 8; ++v) bv[v] = __ldg(b4 + v);
+                }
                 tmem_ld_wait();
-                uint4* mine = (uint4*)(stg + lane * 80);
                 if (a.relu) {
 #pragma unroll
                     for (int v = 0; v < 4; ++v)
-                        mine[v] = make_uint4(bias_pack_bf16<true>(r[v * 8 + 0], r[v * 8 + 1], bv[2 * v].x, bv[2 * v].y),
-                                             bias_pack_bf16<true>(r[v * 8 + 2], r[v * 8 + 3], bv[2 * v].z, bv[2 * v].w),
-                                             bias_pack_bf16<true>(r[v * 8 + 4], r[v * 8 + 5], bv[2 * v + 1].x, bv[2 * v + 1].y),
-                                             bias_pack_bf16<true>(r[v * 8 + 6], r[v * 8 + 7], bv[2 * v + 1].z, bv[2 * v + 1].w));
+                        sts128(mine + v * 16, bias_pack_bf16<true>(r[v * 8 + 0], r[v * 8 + 1], bv[2 * v].x, bv[2 * v].y),
+                               bias_pack_bf16<true>(r[v * 8 + 2], r[v * 8 + 3], bv[2 * v].z, bv[2 * v].w),
+                               bias_pack_bf16<true>(r[v * 8 + 4], r[v * 8 + 5], bv[2 * v + 1].x, bv[2 * v + 1].y),
+                               bias_pack_bf16<true>(r[v * 8 + 6], r[v * 8 + 7], bv[2 * v + 1].z, bv[2 * v + 1].w));
                 } else {
 #pragma unroll
                     for (int v = 0; v < 4; ++v)
-                        mine[v] = make_uint4(bias_pack_bf16<false>(r[v * 8 + 0], r[v * 8 + 1], bv[2 * v].x, bv[2 * v].y),
-                                             bias_pack_bf16<false>(r[v * 8 + 2], r[v * 8 + 3], bv[2 * v].z, bv[2 * v].w),
-                                             bias_pack_bf16<false>(r[v * 8 + 4], r[v * 8 + 5], bv[2 * v + 1].x, bv[2 * v + 1].y),
-                                             bias_pack_bf16<false>(r[v * 8 + 6], r[v * 8 + 7], bv[2 * v + 1].z, bv[2 * v + 1].w));
+                        sts128(mine + v * 16, bias_pack_bf16<false>(r[v * 8 + 0], r[v * 8 + 1], bv[2 * v].x, bv[2 * v].y),
+                               bias_pack_bf16<false>(r[v * 8 + 2], r[v * 8 + 3], bv[2 * v].z, bv[2 * v].w),
+                               bias_pack_bf16<false>(r[v * 8 + 4], r[v * 8 + 5], bv[2 * v + 1].x, bv[2 * v + 1].y),
+                               bias_pack_bf16<false>(r[v * 8 + 6], r[v * 8 + 7], bv[2 * v + 1].z, bv[2 * v + 1].w));
                 }
                 __syncwarp();
 #pragma unroll
                 for (int k = 0; k < 4; ++k) {
                     if ((act_mask >> ((lane >> 2) + 8 * k)) & 1u)
-                        *(uint4*)(a.out + wb_off[k] + c * 32) = *(const uint4*)(rd + k * (8 * 80));
+                        *(uint4*)(a.out + wb_off[k] + c * 32) = lds128(rd + k * (8 * 80));
                 }
                 __syncwarp();
             }
@@ -341,6 +374,7 @@ k_conv_tc(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUten
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmB) : "memory");
     }
+    stage_bias(a, ctl, a.epi_warps);
     if (warp == 1) {       // up to 512 columns: two accumulators of up to 256 columns
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -509,6 +543,7 @@ k_conv_tc_smallc(const __grid_constant__ CUtensorMap tmA, const TcSmallArgs sa)
     for (int i = threadIdx.x; i < a.stages * sa.stage_bytes / 16; i += blockDim.x)
         ((uint4*)ring)[i] = make_uint4(0, 0, 0, 0);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> visible to TMA / MMA
+    stage_bias(a, ctl, a.epi_warps);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -641,6 +676,7 @@ k_conv_tc_halo(const __grid_constant__ CUtensorMap tmA, const TcHaloArgs ha)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
     }
+    stage_bias(a, ctl, a.epi_warps);
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -856,6 +892,7 @@ k_conv_tc_pair(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmA) : "memory");
         asm volatile("prefetch.tensormap [%0];" ::"l"(&tmW) : "memory");
     }
+    stage_bias(a, ctl, 4);
     if (warp == 1) {                                          // the same warp in both CTAs: tensor memory of the pair
         asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&ctl->tmem_base)), "r"(a.tmem_cols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
@@ -1106,8 +1143,14 @@ static cudaError_t launch_conv_kernel(void (*kernel)(KArgs...), int grid, int th
 static thread_local int t_ring_kb = 200;
 static thread_local int t_epi_warps = 4;      // the layer's tuned epilogue width, honoured by launches with one CTA per SM
 static int epi_warps_for(int ctas) { return t_epi_warps == 8 && ctas != 2 ? 8 : 4; }
-// eight epilogue warps stage twice as much: the rings give that up
-static int ring_budget(int ctas) { return (t_ring_kb * 1024 - (epi_warps_for(ctas) == 8 ? 4 * kStageBytes : 0)) / (ctas == 2 ? 2 : 1); }
+static thread_local int t_bias_bytes = 0;     // the launch's bias values staged in shared memory (0: too many, read from global memory)
+static int bias_bytes_for(const dc_layer_desc& group) { return group.cout * 4 <= 16384 ? (group.cout * 4 + 15) & ~15 : 0; }
+// eight epilogue warps stage twice as much, and every CTA keeps its bias values: the rings give that up
+static int ring_budget(int ctas)
+{
+    const int n = ctas == 2 ? 2 : 1;
+    return (t_ring_kb * 1024 - (epi_warps_for(ctas) == 8 ? 4 * kStageBytes : 0) - n * t_bias_bytes) / n;
+}
 
 // Every launch waits at most kWaitLimitNs on the device.  dc_debug_stall_next_conv (below) arms the next launch
 // only: its producer issues no copy and its waits run out after the given time.
@@ -1164,7 +1207,7 @@ bool make_plan(const dc_layer_desc& d, TcPlan& p, int want_mt = 0, int want_bn =
     int st = ring_budget(ctas) / (p.MT * p.a_bytes + p.b_bytes);
     p.stages = st > kMaxStages ? kMaxStages : st;
     if (p.stages < 2) return false;
-    p.smem = (size_t)p.stages * (p.MT * p.a_bytes + p.b_bytes) + ctl_bytes(epi_warps_for(ctas)) + 1024;
+    p.smem = (size_t)p.stages * (p.MT * p.a_bytes + p.b_bytes) + ctl_bytes(epi_warps_for(ctas)) + t_bias_bytes + 1024;
     return true;
 }
 
@@ -1307,7 +1350,8 @@ static int launch_smallc(dc_cache* c, int layer, const void* in, void* out, cons
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
     a.epi_warps = epi_warps_for(ctas);
-    const size_t smem = (size_t)a.stages * stage_bytes + ((sa.w_bytes + 127) & ~127) + ctl_bytes(a.epi_warps) + 256;
+    a.bias_smem = t_bias_bytes ? d.cout : 0;
+    const size_t smem = (size_t)a.stages * stage_bytes + ((sa.w_bytes + 127) & ~127) + ctl_bytes(a.epi_warps) + t_bias_bytes + 256;
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device)) {
         DC_CUDA(cudaFuncSetAttribute(k_conv_tc_smallc, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024));
@@ -1383,7 +1427,8 @@ static int launch_halo(dc_cache* c, int layer, int grp, int mt, bool slab, const
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
     a.epi_warps = epi_warps_for(ctas);
-    const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + ctl_bytes(a.epi_warps) + (slab ? 1280 : 256);
+    a.bias_smem = t_bias_bytes ? d.cout : 0;
+    const size_t smem = (size_t)a_total + (size_t)a.stages * h.b_bytes + ctl_bytes(a.epi_warps) + t_bias_bytes + (slab ? 1280 : 256);
     if (smem > 227 * 1024) return DC_ERR_CONFIG;
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device)) {
@@ -1482,7 +1527,8 @@ static int launch_pair(dc_cache* c, int layer, const void* in, void* out, const 
     int st = (budget - ha.a_stages * ha.patch_bytes) / b_bytes;
     a.stages = st > kMaxStages ? kMaxStages : st;
     if (a.stages < 2) return DC_ERR_CONFIG;
-    const size_t smem = (size_t)ha.a_stages * ha.patch_bytes + (size_t)a.stages * b_bytes + ctl_bytes(4) + 1280;
+    a.bias_smem = t_bias_bytes ? d.cout : 0;
+    const size_t smem = (size_t)ha.a_stages * ha.patch_bytes + (size_t)a.stages * b_bytes + ctl_bytes(4) + t_bias_bytes + 1280;
     if (smem > 227 * 1024) return DC_ERR_CONFIG;
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device))
@@ -1506,6 +1552,7 @@ int dc_launch_conv_bf16(dc_cache* c, int layer, const void* in, void* out, const
     const int G = n_groups(c->L[layer].d);
     t_ring_kb = c->overlap_mode ? 182 : 200;
     t_pdl = !c->overlap_mode;
+    t_bias_bytes = bias_bytes_for(group_view(c->L[layer].d));
     // eight epilogue warps take the registers that the block search of the next frame needs to stay resident beside
     // this kernel: while that overlap is in use the CTA keeps to four
     t_epi_warps = c->L[layer].tc_ew == 8 && !c->overlap_mode ? 8 : 4;
@@ -1590,6 +1637,7 @@ static int launch_group(dc_cache* c, int layer, int grp, const void* in, void* o
     a.status = c->status;
     a.flat = L.flat; a.gpr = L.gpr; a.n_groups_all = c->S * d.out_h * L.gpr;
     a.epi_warps = epi_warps_for(ctas);
+    a.bias_smem = t_bias_bytes ? d.cout : 0;
     set_wait_limit(c, a);
     static dc_once_per_device attr_set;
     if (attr_set.first(c->device)) {
@@ -1656,6 +1704,7 @@ int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in)
         const int ctas = shape == 2 ? 2 : 1;
         L.tc_ctas = ctas; L.tc_ew = shape == 1 ? 8 : 4;
         t_epi_warps = L.tc_ew;                                        // make_plan below sizes the rings for it
+        t_bias_bytes = bias_bytes_for(de);
         if (!generic) {                                               // few input channels: one kernel shape, 1 or 2 CTAs per SM
             if (ctas == 2 && tmem_cols_for(2, 1, L.d.cout) > 256) continue;
             trial("few-channel kernel");
