@@ -80,7 +80,9 @@ typedef enum {
  *   whose kernel covers the whole map: weights [cout][kh][kw][cin], out 1 x 1, optional ReLU).  Table 2: nothing of
  *   its output is reusable.
  * A layer table with an LRN or FC layer of another shape is accepted for region propagation, but such a cache
- * cannot run dc_infer_frame. */
+ * cannot run dc_infer_frame.
+ * Limit: an executable cache takes DC_CONV and DC_FC kernels of at most 11 columns (kw <= 11; any kh);
+ * dc_cache_create returns DC_ERR_CONFIG for a wider one. */
 typedef struct {
     int32_t kind, kh, kw, sh, sw, ph, pw, cin, cout, relu, in0, in1, out_h, out_w;
     int32_t groups;   /* DC_CONV only: grouped convolution (the cited AlexNet's form); 0 or 1 = ordinary.  Output channel

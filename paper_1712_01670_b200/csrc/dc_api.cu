@@ -257,6 +257,7 @@ int build(dc_cache* c, const dc_layer_desc* layers, const void* const* weights_d
     for (int i = 0; i < n; ++i)
         if (c->executable && c->L[i].d.kind == DC_CONV) {
             const void* in = c->L[i].d.in0 < 0 ? c->input_map : c->L[c->L[i].d.in0].map[0];
+            if (c->L[i].s2d_s) in = c->L[i].in_s2d;               // the kernels being timed read the block map
             DC_TRY(dc_conv_bf16_autotune(c, i, in));
         }
     if (c->executable) DC_TRY(dc_build_classify_table(c));       // after the tuner: it decides each layer's tile geometry
@@ -283,7 +284,7 @@ void release(dc_cache* c)
     if (c->stats_pinned) cudaFreeHost(c->stats_pinned);
     for (int i = 0; i < c->n_layers; ++i) {
         dc_layer_rt& L = c->L[i];
-        cudaFree(L.map[0]); cudaFree(L.map[1]); cudaFree(L.weight); cudaFree(L.bias); cudaFree(L.weight_packed); cudaFree(L.in_padded); cudaFree(L.weight_halo);
+        cudaFree(L.map[0]); cudaFree(L.map[1]); cudaFree(L.weight); cudaFree(L.bias); cudaFree(L.weight_packed); cudaFree(L.in_padded); cudaFree(L.in_s2d); cudaFree(L.weight_halo);
         cudaFree(L.masks); cudaFree(L.dirty_list); cudaFree(L.all_list);
     }
     cudaGetLastError();

@@ -58,6 +58,8 @@ struct dc_layer_rt {
     void* weight_halo;              // conv, bf16: weights packed for the patch-reuse and column-slab kernels
     int halo_bn;                    // channels per block that packing is grouped by
     void* in_padded;                // conv, bf16, cin <= 8: input with channels padded to 8
+    void* in_s2d;                   // conv, bf16, strided over few channels: the space-to-depth copy of the input the rewritten layer reads (dc_conv_s2d.cu)
+    int s2d_s, s2d_py, s2d_px, s2d_cin, s2d_hi, s2d_wi;   // ... its block size (0: layer as declared), leading zero rows / columns, and the input as declared
     uint32_t* masks;                // conv: [S][tiles_y][tiles_x][4] reuse bitmap of each tile
     int32_t* dirty_list;            // conv: compacted tiles needing computation
     int32_t* all_list;              // conv: every tile (used by full frames)
@@ -180,4 +182,7 @@ bool dc_layer_cached(const dc_cache* c, int layer);
 int dc_build_classify_table(dc_cache* c);
 int dc_launch_classify_all(dc_cache* c, int cur);
 int dc_conv_bf16_autotune(dc_cache* c, int layer, const void* in);
+bool dc_s2d_eligible(const dc_cache* c, const dc_layer_desc& d);
+int dc_s2d_rewrite(dc_cache* c, int layer);
+int dc_launch_s2d(dc_cache* c, int layer, const void* in);
 int dc_conv_bf16_supported(const dc_cache* c, int layer);    // 1 when the layer runs on the tensor-core kernels

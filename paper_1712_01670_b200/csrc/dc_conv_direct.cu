@@ -121,6 +121,12 @@ int dc_launch_conv(dc_cache* c, int layer, const void* in, void* out, const int3
                    const int32_t* tile_count, const uint32_t* masks, int max_tiles)
 {
     dc_layer_rt& L = c->L[layer];
+    if (L.s2d_s) {                                                // the rewritten layer reads the block map of its input
+        dc_prof_scope ps(c, DC_ST_CONV);
+        const int rc = dc_launch_s2d(c, layer, in);
+        if (rc != DC_OK) return rc;
+        in = L.in_s2d;
+    }
     if (c->cfg.dtype == DC_BF16 && dc_conv_bf16_supported(c, layer))
         return dc_launch_conv_bf16(c, layer, in, out, tile_list, tile_count, masks, max_tiles);
     ConvArgs a;
@@ -159,6 +165,12 @@ int dc_pack_weights(dc_cache* c, int layer, const float* w_dev, const float* b_d
     else k_convert_weights<float><<<grid, 256, 0, c->stream>>>(w_dev, n, (float*)L.weight);
     DC_CUDA(cudaGetLastError());
     DC_CUDA(cudaMemcpyAsync(L.bias, b_dev, sizeof(float) * L.d.cout, cudaMemcpyDeviceToDevice, c->stream));
-    if (c->cfg.dtype == DC_BF16) return dc_pack_weights_bf16(c, layer);
+    if (c->cfg.dtype == DC_BF16) {
+        if (dc_s2d_eligible(c, L.d)) {                            // from here on the layer is the stride-1 one
+            const int rc = dc_s2d_rewrite(c, layer);
+            if (rc != DC_OK) return rc;
+        }
+        return dc_pack_weights_bf16(c, layer);
+    }
     return DC_OK;
 }

@@ -659,6 +659,54 @@ def _one_layer_full_and_partial(hi, wi, cin, cout, k, st, p, S, scheme):
         dc.close()
 
 
+@pytest.mark.parametrize("hi,wi,cout,k,st,p,S", [
+    (59, 63, 96, 11, 4, 0, 3),       # AlexNet's first layer: 4 x 4 blocks of 3 channels = 48 -> 64 channels, 3 x 3 taps
+    (45, 53, 64, 7, 2, 3, 2),        # ResNet's stem: 2 x 2 blocks = 12 -> 16 channels, 4 x 4 taps, three zero rows in front
+    (37, 41, 32, 5, 2, 2, 2),
+    (30, 34, 64, 3, 2, 1, 1),
+    (40, 43, 32, 7, 3, 2, 2),        # 3 x 3 blocks = 27 -> 32 channels
+    (33, 35, 64, 11, 4, 2, 2),       # padding that is not a multiple of the stride
+])
+def test_conv_strided_first_layers_as_space_to_depth(hi, wi, cout, k, st, p, S):
+    """Strided convolutions on RGB run as stride-1 convolutions over a space-to-depth copy of their input: full and
+    partial convolution against the oracle's strided one."""
+    g = rng(hi * 3 + k)
+    nb = nets.NetBuilder(hi, wi)
+    nb.conv(-1, cout, k, st, p, 1)
+    L = nb.layers[0]
+    oh, ow = L["out_h"], L["out_w"]
+    wts = g.normal(0, np.sqrt(2.0 / (k * k * 3)), size=(cout, k, k, 3)).astype(np.float32)
+    bias = g.normal(0, 0.1, size=cout).astype(np.float32)
+    xq = np.stack([orc.quant_array(g.uniform(0, 1, size=(hi, wi, 3)), orc.QUANT_BF16) for _ in range(S)])
+    pq = np.stack([orc.quant_array(g.normal(size=(oh, ow, cout)), orc.QUANT_BF16) for _ in range(S)])
+    dc = DeepCache(wi, hi, nb.layers, [wts], [bias], n_streams=S, block=16, search_range=4, dtype=B.DC_BF16, max_regions=4)
+    try:
+        assert B.dc_cache_layer_conv_scheme(dc.handle, 0) >= 1          # a tensor-core scheme
+        xin = torch.from_numpy(xq).to(torch.bfloat16).cuda()
+        pin = torch.from_numpy(pq).to(torch.bfloat16).cuda()
+        full = dc.conv_partial(0, xin)
+        regs = torch.zeros((S, dc.max_regions, 6), dtype=torch.int32)
+        counts = torch.zeros(S, dtype=torch.int32)
+        regs[0, 0] = torch.tensor([1, 2, min(5, ow - 2), min(4, oh - 3), 2, 1], dtype=torch.int32)
+        counts[0] = 1
+        part = dc.conv_partial(0, xin, pin, regs.cuda(), counts.cuda())
+        wq = orc.quant_array(wts, orc.QUANT_BF16)
+        for s_ in range(S):
+            r = np.zeros(1, orc.REGION_DTYPE)
+            r[0] = tuple(int(v) for v in regs[s_, 0])
+            want_full, _ = orc.conv_reuse(xq[s_], L, wq, bias, orc.QUANT_BF16)
+            want, reused = orc.conv_reuse(xq[s_], L, wq, bias, orc.QUANT_BF16, pq[s_], r[:int(counts[s_])])
+            U.assert_map_close(full[s_], want_full, True, f"full, stream {s_}")
+            U.assert_map_close_per_element(full[s_], want_full, f"full, per element, stream {s_}")
+            U.assert_map_close(part[s_], want, True, f"partial, stream {s_}")
+            m = reused.astype(bool)
+            got = part[s_].float().cpu().numpy().astype(np.float64)
+            assert np.array_equal(got[m], want[m])
+        assert dc.status() == B.DC_OK
+    finally:
+        dc.close()
+
+
 @pytest.mark.parametrize("cin,k", [(64, 3), (32, 1), (3, 3), (128, 7)])      # column-slab / patch kernels, tap-by-tap kernel, few-channel kernel, CTA pairs
 def test_bounded_device_waits_run_out_and_the_cache_stays_usable(cin, k, monkeypatch):
     """Failure detection without a fault: one convolution launch is armed so that its producer issues no copy.  The
