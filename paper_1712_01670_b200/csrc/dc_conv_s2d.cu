@@ -13,7 +13,9 @@
 // rectangles (Table 2 works on the layer as declared) and its tiles do not change.
 //
 // The rewritten layer (channels padded to 16, 32 or 64) runs on the ordinary kernels: AlexNet's first layer becomes a
-// 3 x 3 convolution over 64 channels (column slabs), ResNet's stem a 4 x 4 convolution over 16.
+// 3 x 3 convolution over 64 channels (column slabs), ResNet's stem a 4 x 4 convolution over 16.  (The same rewrite with
+// 1 x 1 blocks, padding a stride-1 layer's 96 channels to 128 so that it leaves the tap-by-tap kernel, was measured on
+// AlexNet's second layer: faster alone, slower in the trunk with the copy it needs: not kept.)
 #include "dc_common.cuh"
 
 #include <cuda_bf16.h>
@@ -76,8 +78,8 @@ __global__ void k_s2d_weights(const __nv_bfloat16* w, int cout, int kh, int kw, 
 bool dc_s2d_eligible(const dc_cache* c, const dc_layer_desc& d)
 {
     if (c->cfg.dtype != DC_BF16 || !c->executable || getenv("DC_NO_S2D") || getenv("DC_NO_TENSOR_CORES")) return false;
-    if (d.kind != DC_CONV || d.groups > 1 || d.sh != d.sw || d.sh < 2 || d.sh > 8) return false;
-    if (d.cin * d.sh * d.sw > 64 || d.cout % 32 != 0) return false;
+    if (d.kind != DC_CONV || d.groups > 1 || d.sh != d.sw || d.sh < 2 || d.sh > 8 || d.cout % 32 != 0) return false;
+    if (d.cin * d.sh * d.sw > 64) return false;
     const int s = d.sh;
     const int offy = (d.ph + s - 1) / s * s - d.ph, offx = (d.pw + s - 1) / s * s - d.pw;
     return (d.kh + offy + s - 1) / s <= 5 && (d.kw + offx + s - 1) / s <= 5;      // what every operand scheme takes
