@@ -479,6 +479,14 @@ def test_infer_workload_4_resnet50_bf16():
     U.run_stream_parity(configs.WORKLOADS[4](), 1, list(range(4)))
 
 
+@pytest.mark.parametrize("wid,frames", [(3, [0, 1, 2]), (4, [0, 1])])
+def test_infer_small_map_trunks_three_streams(wid, frames):
+    """The AlexNet and ResNet-50 trunks with three streams in one cache: tiles of their small maps may hold pixels of
+    two streams (flat tiles), and their strided first layers run on the space-to-depth copy; every layer's map of
+    every stream against the oracle."""
+    U.run_stream_parity(configs.WORKLOADS[wid](), 3, frames)
+
+
 def test_infer_workload_5_two_streams():
     """Full-HD matching, area resize to 224x224, VGG-16 trunk; 2 of the 32 streams, frames 0-2."""
     U.run_stream_parity(configs.WORKLOADS[5](), 2, [0, 1, 2])
